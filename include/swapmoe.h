@@ -1,0 +1,212 @@
+/*
+ * swapmoe.h - C ABI of the B200 (sm_100a) Virtual-Expert MoE-layer forward.
+ *
+ * The library runs ONE thing: the forward pass of a Mixture-of-Experts layer that
+ * is restricted to a small resident set of experts ("Virtual Experts", SwapMoE,
+ * arXiv 2308.15030, abstract and Section 3), plus the per-expert importance score
+ * (Eq. 1) that decides which experts should be resident next, and the
+ * asynchronous copy that brings a new expert into a spare slot (Section 3.2).
+ *
+ * Conventions that hold for every call
+ *   - every function returns an int32 status: 0 = SWAPMOE_OK, negative = error
+ *     (swapmoe_status_string() names it).  Nothing throws or aborts.
+ *   - "dev" pointers are device (HBM) addresses on the layer's GPU, "host"
+ *     pointers are host addresses; `stream` / `event` are cudaStream_t /
+ *     cudaEvent_t passed as void* (NULL = the legacy default stream).
+ *   - matrices are row-major with the contraction index innermost:
+ *     x, out [n_tokens, d_model]; router Wr [E, d_model]; expert input matrices
+ *     [d_ff, d_model]; expert output matrix [d_model, d_ff].  Elements are fp32
+ *     (SWAPMOE_F32) or bfloat16 (SWAPMOE_BF16) as fixed at create; logits, gate
+ *     values and importance are always fp32; indices are int32.
+ *   - device buffers passed in must be 16-byte aligned, are owned by the caller,
+ *     are never copied unless stated, and must stay valid while work that uses
+ *     them is in flight.  x and out must not overlap.
+ *   - a layer object may be driven from one stream at a time.
+ *   - all device work is done by this library's own kernels; there is no CPU
+ *     fallback.  If no usable GPU is present create() fails with
+ *     SWAPMOE_ERR_CUDA.
+ */
+#ifndef SWAPMOE_H_
+#define SWAPMOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct swapmoe_layer swapmoe_layer_t; /* opaque, owned by the library */
+
+enum { SWAPMOE_F32 = 0, SWAPMOE_BF16 = 1 };
+enum { SWAPMOE_ACT_RELU = 0, SWAPMOE_ACT_SWIGLU = 1 };
+
+enum {
+  SWAPMOE_OK = 0,
+  SWAPMOE_ERR_INVALID_ARG = -1,     /* null pointer, size out of range, K < top_k ...   */
+  SWAPMOE_ERR_NOT_READY = -2,       /* router or resident set not set yet               */
+  SWAPMOE_ERR_TOO_MANY_TOKENS = -3, /* n_tokens > max_tokens given at create            */
+  SWAPMOE_ERR_BAD_SLOT_TABLE = -4,  /* expert out of range / listed twice / bad phys    */
+  SWAPMOE_ERR_CUDA = -5,            /* a CUDA runtime or driver call failed             */
+  SWAPMOE_ERR_DEVICE_TIMEOUT = -6,  /* a bounded in-kernel wait gave up                 */
+  SWAPMOE_ERR_UNSUPPORTED = -7      /* shape outside what the kernels are built for     */
+};
+
+/* Limits of this build: E <= 256, K + spare_slots <= 64, top_k <= 4,
+ * d_model and d_ff multiples of 64, max_tokens * top_k < 2^24. */
+typedef struct {
+  int32_t E;           /* experts of the off-the-shelf layer (Section 2)                  */
+  int32_t d_model;     /* token width                                                     */
+  int32_t d_ff;        /* expert hidden width                                             */
+  int32_t top_k;       /* experts per token chosen by the gate (Section 2, k)             */
+  int32_t K;           /* resident budget: number of Virtual-Expert slots (#experts_l of  */
+                       /* the configuration tuple, Section 3.3); top_k <= K <= E          */
+  int32_t dtype;       /* SWAPMOE_F32 or SWAPMOE_BF16: storage type of x, out, weights    */
+  int32_t act;         /* SWAPMOE_ACT_RELU: out-proj(relu(in-proj x));                    */
+                       /* SWAPMOE_ACT_SWIGLU: out-proj(silu(W1 x) * (W3 x))               */
+  int32_t renorm_topk; /* 0: gate value = softmax probability over the allowed experts;   */
+                       /* 1: gate value = softmax over the top_k selected logits          */
+  int32_t max_tokens;  /* largest n_tokens of any forward; workspace is sized for it      */
+  int32_t spare_slots; /* extra arena entries (beyond K) that asynchronous loads may fill */
+} swapmoe_config_t;
+
+/* Selectors of swapmoe_debug_copy (intermediates of the LAST forward). */
+enum {
+  SWAPMOE_TAP_LOGITS = 0, /* fp32 [T, E]                                         */
+  SWAPMOE_TAP_UIDX = 1,   /* int32 [T, k]  unmasked top-k experts                */
+  SWAPMOE_TAP_UGATE = 2,  /* fp32 [T, k]                                         */
+  SWAPMOE_TAP_MIDX = 3,   /* int32 [T, k]  masked (resident-only) top-k experts  */
+  SWAPMOE_TAP_MGATE = 4,  /* fp32 [T, k]                                         */
+  SWAPMOE_TAP_SLOT = 5,   /* int32 [T, k]                                        */
+  SWAPMOE_TAP_COUNT = 6,  /* int32 [K]                                           */
+  SWAPMOE_TAP_OFFSET = 7, /* int32 [K+1]                                         */
+  SWAPMOE_TAP_PERM = 8,   /* int32 [T*k]   position -> flat pair index t*k+j     */
+  SWAPMOE_TAP_INV = 9,    /* int32 [T*k]   flat pair index -> position           */
+  SWAPMOE_TAP_XNORM = 10  /* fp32 [T]      L2 norm of every token                */
+};
+
+/*
+ * Section 3 (online phase): one layer object = one MoE layer served from K
+ * resident slots.  Allocates the layer's device workspace (sized for
+ * cfg->max_tokens) on the CURRENT CUDA device and zeroes the importance
+ * accumulator.  *out is written only on success.  Errors: INVALID_ARG
+ * (null, K < top_k, K > E, sizes out of the limits above), UNSUPPORTED, CUDA.
+ */
+int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg);
+
+/* Frees the workspace.  The caller must have synchronised the streams that used
+ * the layer.  NULL is accepted. */
+int32_t swapmoe_destroy(swapmoe_layer_t* layer);
+
+/*
+ * Section 2 (gate G(x)) and Eq. (1) (||E_i||).  Wr_dev: router matrix [E, d_model]
+ * on the device, in the layer's dtype, NOT copied (must outlive the layer's use).
+ * enorm_host: E fp32 values ||E_i|| on the host, copied to the device on `stream`
+ * before this call returns control (the host array may be reused at once).
+ * The norm of an expert's parameters does not depend on the tokens, and
+ * non-resident experts are not in HBM, so the caller supplies it.
+ */
+int32_t swapmoe_set_router(swapmoe_layer_t* layer, const void* Wr_dev, const float* enorm_host,
+                           void* stream);
+
+/*
+ * Abstract / Section 3: the Virtual-Expert -> actual-expert mapping, and where
+ * the resident weights live.
+ *   slot_to_expert_host [K]: expert id served by each logical slot (host, copied;
+ *       validated: 0 <= id < E, no id twice -> else BAD_SLOT_TABLE).
+ *   phys_slot_host [K]: arena entry backing each logical slot, 0 <= p < K +
+ *       spare_slots, no entry twice (host, copied); NULL means identity.
+ *   arena_in_dev : [K + spare_slots, nin, d_ff, d_model], nin = 1 (ReLU: wi) or
+ *       2 (SwiGLU: w1 then w3);  arena_out_dev: [K + spare_slots, d_model, d_ff].
+ *       Device memory, layer dtype, caller-owned, not copied.
+ * The new tables take effect for forwards enqueued on `stream` after this call;
+ * forwards enqueued earlier keep the old tables.  No host synchronisation.
+ */
+int32_t swapmoe_set_resident(swapmoe_layer_t* layer, const int32_t* slot_to_expert_host,
+                             const int32_t* phys_slot_host, const void* arena_in_dev,
+                             const void* arena_out_dev, void* stream);
+
+/*
+ * The hot path (Sections 2, 3.1; Fig. 4): for every token row of x_dev
+ *   logits = x Wr^T;  unmasked top-k gate (feeds Eq. 1);  Masked Gating over the
+ *   resident experts;  slot remap;  stable grouping of (token, j) pairs by slot;
+ *   grouped expert FFN;  out[t] = sum_j gate[t,j] * E_{slot[t,j]}(x[t]).
+ * It also adds this batch's terms of Eq. (1) to the layer's importance
+ * accumulator.  out_dev [n_tokens, d_model] is overwritten.  Everything is
+ * enqueued on `stream`; the call does not synchronise and does not allocate.
+ * n_tokens = 0 is a valid no-op.  Errors: NOT_READY, TOO_MANY_TOKENS,
+ * INVALID_ARG, CUDA (launch failure).
+ */
+int32_t swapmoe_forward(swapmoe_layer_t* layer, const void* x_dev, void* out_dev,
+                        int32_t n_tokens, void* stream);
+
+/* Same, but the router product is replaced by caller-supplied fp32 logits
+ * [n_tokens, E] on the device (test tap: lets routing be compared on identical
+ * logits).  x_dev is still needed for ||x|| and the FFN. */
+int32_t swapmoe_forward_from_logits(swapmoe_layer_t* layer, const void* x_dev,
+                                    const float* logits_dev, void* out_dev, int32_t n_tokens,
+                                    void* stream);
+
+/* End-to-end form with HOST buffers: copies x_host [n_tokens, d_model] to the
+ * device, runs swapmoe_forward, copies the result to out_host, and returns after
+ * `stream` has completed.  Pinned host memory makes the copies asynchronous
+ * with respect to other streams; pageable memory works but is slower. */
+int32_t swapmoe_forward_host(swapmoe_layer_t* layer, const void* x_host, void* out_host,
+                             int32_t n_tokens, void* stream);
+
+/*
+ * Eq. (1): importance(E_i, X) = sum_{x in X_i} ||x|| * |G(x)_i| * ||E_i||, X_i =
+ * tokens whose unmasked top-k contains i, accumulated over every forward since
+ * the last reset.  Waits for `stream`, copies E fp32 values to imp_host, and if
+ * reset != 0 zeroes the accumulator (ordered on `stream`).
+ */
+int32_t swapmoe_read_importance(swapmoe_layer_t* layer, float* imp_host, int32_t reset,
+                                void* stream);
+
+/* Sections 3.1-3.2: the K most important experts, by descending importance, ties
+ * to the lowest index.  Pure host function (E <= 256 floats). */
+int32_t swapmoe_topk_importance(const float* imp_host, int32_t E, int32_t K,
+                                int32_t* out_idx_host);
+
+/*
+ * Section 3.2 (asynchronous expert loading): enqueue on `side_stream` the copy of
+ * one expert's matrices from PINNED host memory into arena entry `phys` of the
+ * arenas last given to set_resident (in_host_pinned: [nin, d_ff, d_model],
+ * out_host_pinned: [d_model, d_ff]), then record `done_event` (may be NULL) on
+ * side_stream.  `phys` must not back any logical slot of the current table
+ * (-> BAD_SLOT_TABLE), so a running forward never reads memory being written.
+ * The caller later makes its compute stream wait on done_event and calls
+ * set_resident with a table that uses `phys`.
+ */
+int32_t swapmoe_load_slot_async(swapmoe_layer_t* layer, int32_t phys, const void* in_host_pinned,
+                                const void* out_host_pinned, void* side_stream,
+                                void* done_event);
+
+/* Copies one intermediate of the last forward to the host after waiting for
+ * `stream`.  `bytes` must equal the tap's size for the last n_tokens. */
+int32_t swapmoe_debug_copy(swapmoe_layer_t* layer, int32_t which, void* host, size_t bytes,
+                           void* stream);
+
+/* Waits for `stream` and returns the device-side status word of the layer:
+ * SWAPMOE_OK, or SWAPMOE_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel
+ * gave up since the last call.  *detail (may be NULL) receives a code naming
+ * the wait.  The word is cleared. */
+int32_t swapmoe_device_status(swapmoe_layer_t* layer, int32_t* detail, void* stream);
+
+/* Number of kernels of this library launched by the layer so far (host counter). */
+int64_t swapmoe_launch_count(const swapmoe_layer_t* layer);
+
+/* Bytes of device workspace the layer allocated at create. */
+int64_t swapmoe_workspace_bytes(const swapmoe_layer_t* layer);
+
+/* Selects the grouped-GEMM implementation for later forwards (test / benchmark
+ * hook): 0 = automatic, 1 = CUDA-core FFMA tiles, 2 = tcgen05 tensor-core tiles
+ * (bf16 only; UNSUPPORTED otherwise). */
+int32_t swapmoe_set_gemm_path(swapmoe_layer_t* layer, int32_t path);
+
+const char* swapmoe_status_string(int32_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWAPMOE_H_ */

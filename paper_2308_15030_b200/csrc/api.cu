@@ -1,0 +1,428 @@
+// C ABI of the Virtual-Expert MoE-layer forward (see include/swapmoe.h): argument
+// checks, workspace layout and kernel launches.  No host synchronisation and no
+// allocation happen inside forward().
+#include "../../include/swapmoe.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+#include "permute.cuh"
+#include "router_gate.cuh"
+
+using namespace swapmoe;
+
+struct swapmoe_layer {
+  swapmoe_config_t cfg;
+  int device;
+  int nin;
+  size_t elem;
+  // device workspace (one allocation)
+  char* ws_base;
+  size_t ws_bytes;
+  float *logits, *ugate, *mgate, *xnorm, *cta_imp, *imp, *enorm, *y;
+  int32_t *uidx, *midx, *slot, *cta_hist, *cta_base, *count, *offset, *pad_offset;
+  int32_t *perm, *inv, *inv_pad, *n_tiles, *e2s, *phys, *s2e, *status;
+  TileDesc* tiles;
+  void *xp, *h, *x_stage, *out_stage;
+  // host state
+  const void *Wr, *arena_in, *arena_out;
+  bool router_set, resident_set;
+  int32_t h_s2e[kMaxSlots], h_phys[kMaxSlots];
+  int32_t last_T;
+  int64_t launches;
+  int32_t gemm_path;
+  int32_t rows_pad_max;
+  TcState tc;
+};
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Carver {
+  size_t off = 0;
+  template <typename T>
+  size_t take(size_t n) {
+    const size_t o = off;
+    off = align_up(off + n * sizeof(T), 256);
+    return o;
+  }
+};
+
+inline bool cuda_ok(cudaError_t e) { return e == cudaSuccess; }
+
+struct EnormTable { float v[kMaxE]; };
+__global__ void set_enorm_kernel(const EnormTable t, int E, float* enorm) {
+  for (int i = threadIdx.x; i < E; i += blockDim.x) enorm[i] = t.v[i];
+}
+
+int32_t check_launch() { return cuda_ok(cudaGetLastError()) ? SWAPMOE_OK : SWAPMOE_ERR_CUDA; }
+
+template <typename DT>
+int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, void* out, int32_t T,
+                     cudaStream_t st) {
+  const swapmoe_config_t& c = L->cfg;
+  const int n_cta = (T + kTokTile - 1) / kTokTile;
+  const int n_pairs = T * c.top_k;
+  const bool use_tc = tc_selected(L->gemm_path, c, T);
+  const int tile_rows = use_tc ? kTcBM : kSimtBM;
+  const int max_tiles = (n_pairs + tile_rows - 1) / tile_rows + c.K;
+
+  RouterArgs ra;
+  ra.x = x; ra.Wr = L->Wr; ra.ext_logits = ext_logits; ra.e2s = L->e2s; ra.enorm = L->enorm;
+  ra.logits = L->logits; ra.uidx = L->uidx; ra.ugate = L->ugate; ra.midx = L->midx;
+  ra.mgate = L->mgate; ra.slot = L->slot; ra.xnorm = L->xnorm; ra.cta_hist = L->cta_hist;
+  ra.cta_imp = L->cta_imp;
+  ra.T = T; ra.d = c.d_model; ra.E = c.E; ra.k = c.top_k; ra.K = c.K; ra.renorm = c.renorm_topk;
+  router_gate_kernel<DT><<<n_cta, 256, router_smem_bytes(c.E), st>>>(ra);
+  L->launches++;
+
+  ScanArgs sa;
+  sa.cta_hist = L->cta_hist; sa.cta_imp = L->cta_imp; sa.phys_slot = L->phys;
+  sa.cta_base = L->cta_base; sa.count = L->count; sa.offset = L->offset;
+  sa.pad_offset = L->pad_offset; sa.tiles = L->tiles; sa.n_tiles = L->n_tiles; sa.imp = L->imp;
+  sa.n_cta = n_cta; sa.K = c.K; sa.E = c.E; sa.tile_rows = tile_rows;
+  scan_reduce_kernel<<<1, 1024, 0, st>>>(sa);
+  L->launches++;
+
+  PermuteArgs pa;
+  pa.x = x; pa.slot = L->slot; pa.cta_base = L->cta_base; pa.offset = L->offset;
+  pa.pad_offset = L->pad_offset; pa.perm = L->perm; pa.inv = L->inv; pa.inv_pad = L->inv_pad;
+  pa.xp = L->xp; pa.T = T; pa.d = c.d_model; pa.k = c.top_k; pa.K = c.K;
+  permute_gather_kernel<DT><<<n_cta, 256, 0, st>>>(pa);
+  L->launches++;
+
+  if (use_tc) {
+    const int32_t rc = tc_ffn(L->tc, c, L->xp, L->h, L->y, L->tiles, L->n_tiles, max_tiles,
+                              L->status, st, &L->launches);
+    if (rc != SWAPMOE_OK) return rc;
+  } else {
+    SimtGemmArgs g1;
+    g1.A = L->xp; g1.W = L->arena_in; g1.C = L->h; g1.tiles = L->tiles; g1.n_tiles = L->n_tiles;
+    g1.slot_stride = (long long)L->nin * c.d_ff * c.d_model;
+    g1.gate_offset = (long long)c.d_ff * c.d_model;
+    g1.N = c.d_ff; g1.Kdim = c.d_model;
+    const dim3 grid1(c.d_ff / kSimtBN, max_tiles);
+    if (c.act == SWAPMOE_ACT_SWIGLU)
+      gemm_simt_kernel<DT, DT, DT, kEpiSwiglu><<<grid1, 256, 0, st>>>(g1);
+    else
+      gemm_simt_kernel<DT, DT, DT, kEpiRelu><<<grid1, 256, 0, st>>>(g1);
+    L->launches++;
+    SimtGemmArgs g2;
+    g2.A = L->h; g2.W = L->arena_out; g2.C = L->y; g2.tiles = L->tiles; g2.n_tiles = L->n_tiles;
+    g2.slot_stride = (long long)c.d_ff * c.d_model;
+    g2.gate_offset = 0;
+    g2.N = c.d_model; g2.Kdim = c.d_ff;
+    const dim3 grid2(c.d_model / kSimtBN, max_tiles);
+    gemm_simt_kernel<DT, DT, float, kEpiNone><<<grid2, 256, 0, st>>>(g2);
+    L->launches++;
+  }
+
+  CombineArgs ca;
+  ca.y = L->y; ca.inv_pad = L->inv_pad; ca.mgate = L->mgate; ca.out = out;
+  ca.T = T; ca.d = c.d_model; ca.k = c.top_k;
+  const long long work = (long long)T * (c.d_model / 8);
+  combine_kernel<DT><<<(unsigned)((work + 255) / 256), 256, 0, st>>>(ca);
+  L->launches++;
+  return check_launch();
+}
+
+int32_t forward_checked(swapmoe_layer* L, const void* x, const float* ext, void* out, int32_t T,
+                        void* stream) {
+  if (!L || T < 0) return SWAPMOE_ERR_INVALID_ARG;
+  if (T == 0) { L->last_T = 0; return SWAPMOE_OK; }
+  if (!x || !out) return SWAPMOE_ERR_INVALID_ARG;
+  if (!L->router_set || !L->resident_set) return SWAPMOE_ERR_NOT_READY;
+  if (T > L->cfg.max_tokens) return SWAPMOE_ERR_TOO_MANY_TOKENS;
+  if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(out)) & 15) return SWAPMOE_ERR_INVALID_ARG;
+  L->last_T = T;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (L->cfg.dtype == SWAPMOE_BF16) return forward_impl<bf16>(L, x, ext, out, T, st);
+  return forward_impl<float>(L, x, ext, out, T, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
+  if (!out || !cfg) return SWAPMOE_ERR_INVALID_ARG;
+  const swapmoe_config_t c = *cfg;
+  if (c.E < 1 || c.K < 1 || c.top_k < 1 || c.d_model < 1 || c.d_ff < 1 || c.max_tokens < 1 ||
+      c.spare_slots < 0)
+    return SWAPMOE_ERR_INVALID_ARG;
+  if (c.K < c.top_k || c.K > c.E) return SWAPMOE_ERR_INVALID_ARG;
+  if (c.dtype != SWAPMOE_F32 && c.dtype != SWAPMOE_BF16) return SWAPMOE_ERR_INVALID_ARG;
+  if (c.act != SWAPMOE_ACT_RELU && c.act != SWAPMOE_ACT_SWIGLU) return SWAPMOE_ERR_INVALID_ARG;
+  if (c.renorm_topk != 0 && c.renorm_topk != 1) return SWAPMOE_ERR_INVALID_ARG;
+  if (c.E > kMaxE || c.K + c.spare_slots > kMaxSlots || c.top_k > kMaxTopK) return SWAPMOE_ERR_UNSUPPORTED;
+  if (c.d_model % 64 || c.d_ff % 64) return SWAPMOE_ERR_UNSUPPORTED;
+  if ((long long)c.max_tokens * c.top_k >= (1ll << 24)) return SWAPMOE_ERR_UNSUPPORTED;
+
+  int dev = 0;
+  if (!cuda_ok(cudaGetDevice(&dev))) { cudaGetLastError(); return SWAPMOE_ERR_CUDA; }
+  cudaDeviceProp prop;
+  if (!cuda_ok(cudaGetDeviceProperties(&prop, dev))) { cudaGetLastError(); return SWAPMOE_ERR_CUDA; }
+  if (prop.major != 10) return SWAPMOE_ERR_UNSUPPORTED;  // kernels are built for sm_100a only
+
+  swapmoe_layer* L = new (std::nothrow) swapmoe_layer();
+  if (!L) return SWAPMOE_ERR_INVALID_ARG;
+  std::memset(L, 0, sizeof(*L));
+  L->cfg = c;
+  L->device = dev;
+  L->nin = c.act == SWAPMOE_ACT_SWIGLU ? 2 : 1;
+  L->elem = c.dtype == SWAPMOE_BF16 ? 2 : 4;
+
+  const size_t T = (size_t)c.max_tokens, P = T * c.top_k;
+  const size_t n_cta = (T + kTokTile - 1) / kTokTile;
+  const size_t rows_pad = align_up(P + (size_t)c.K * kSegAlign, kSegAlign);
+  const size_t max_tiles = (P + kSimtBM - 1) / kSimtBM + c.K;
+  L->rows_pad_max = (int32_t)rows_pad;
+
+  Carver cv;
+  const size_t o_logits = cv.take<float>(T * c.E);
+  const size_t o_ugate = cv.take<float>(P), o_mgate = cv.take<float>(P), o_xnorm = cv.take<float>(T);
+  const size_t o_cta_imp = cv.take<float>(n_cta * c.E);
+  const size_t o_imp = cv.take<float>(c.E), o_enorm = cv.take<float>(c.E);
+  const size_t o_uidx = cv.take<int32_t>(P), o_midx = cv.take<int32_t>(P), o_slot = cv.take<int32_t>(P);
+  const size_t o_cta_hist = cv.take<int32_t>(n_cta * c.K), o_cta_base = cv.take<int32_t>(n_cta * c.K);
+  const size_t o_count = cv.take<int32_t>(c.K), o_offset = cv.take<int32_t>(c.K + 1);
+  const size_t o_pad = cv.take<int32_t>(c.K + 1);
+  const size_t o_perm = cv.take<int32_t>(P), o_inv = cv.take<int32_t>(P), o_invp = cv.take<int32_t>(P);
+  const size_t o_ntiles = cv.take<int32_t>(4), o_e2s = cv.take<int32_t>(c.E);
+  const size_t o_phys = cv.take<int32_t>(kMaxSlots), o_s2e = cv.take<int32_t>(kMaxSlots);
+  const size_t o_status = cv.take<int32_t>(4);
+  const size_t o_tiles = cv.take<TileDesc>(max_tiles);
+  const size_t o_xp = cv.take<char>(rows_pad * c.d_model * L->elem);
+  const size_t o_h = cv.take<char>(rows_pad * c.d_ff * L->elem);
+  const size_t o_y = cv.take<float>(rows_pad * c.d_model);
+  const size_t o_xs = cv.take<char>(T * c.d_model * L->elem);
+  const size_t o_os = cv.take<char>(T * c.d_model * L->elem);
+  L->ws_bytes = cv.off;
+  if (!cuda_ok(cudaMalloc(&L->ws_base, L->ws_bytes))) { cudaGetLastError(); delete L; return SWAPMOE_ERR_CUDA; }
+  char* b = L->ws_base;
+  L->logits = (float*)(b + o_logits); L->ugate = (float*)(b + o_ugate); L->mgate = (float*)(b + o_mgate);
+  L->xnorm = (float*)(b + o_xnorm); L->cta_imp = (float*)(b + o_cta_imp); L->imp = (float*)(b + o_imp);
+  L->enorm = (float*)(b + o_enorm); L->uidx = (int32_t*)(b + o_uidx); L->midx = (int32_t*)(b + o_midx);
+  L->slot = (int32_t*)(b + o_slot); L->cta_hist = (int32_t*)(b + o_cta_hist);
+  L->cta_base = (int32_t*)(b + o_cta_base); L->count = (int32_t*)(b + o_count);
+  L->offset = (int32_t*)(b + o_offset); L->pad_offset = (int32_t*)(b + o_pad);
+  L->perm = (int32_t*)(b + o_perm); L->inv = (int32_t*)(b + o_inv); L->inv_pad = (int32_t*)(b + o_invp);
+  L->n_tiles = (int32_t*)(b + o_ntiles); L->e2s = (int32_t*)(b + o_e2s); L->phys = (int32_t*)(b + o_phys);
+  L->s2e = (int32_t*)(b + o_s2e); L->status = (int32_t*)(b + o_status);
+  L->tiles = (TileDesc*)(b + o_tiles);
+  L->xp = b + o_xp; L->h = b + o_h; L->y = (float*)(b + o_y);
+  L->x_stage = b + o_xs; L->out_stage = b + o_os;
+
+  bool ok = cuda_ok(cudaMemset(L->imp, 0, sizeof(float) * c.E));
+  ok = ok && cuda_ok(cudaMemset(L->status, 0, sizeof(int32_t) * 4));
+  // Rows of the padded workspaces that no pair occupies are computed on but never
+  // read back; start them at zero so they hold finite values.
+  ok = ok && cuda_ok(cudaMemset(L->xp, 0, rows_pad * c.d_model * L->elem));
+  ok = ok && cuda_ok(cudaFuncSetAttribute(router_gate_kernel<float>,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)router_smem_bytes(kMaxE)));
+  ok = ok && cuda_ok(cudaFuncSetAttribute(router_gate_kernel<bf16>,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)router_smem_bytes(kMaxE)));
+  ok = ok && tc_init(L->tc, c, L->xp, L->h, L->y, L->rows_pad_max) == SWAPMOE_OK;
+  if (!ok) { cudaGetLastError(); cudaFree(L->ws_base); delete L; return SWAPMOE_ERR_CUDA; }
+  *out = L;
+  return SWAPMOE_OK;
+}
+
+int32_t swapmoe_destroy(swapmoe_layer_t* L) {
+  if (!L) return SWAPMOE_OK;
+  cudaFree(L->ws_base);
+  delete L;
+  return SWAPMOE_OK;
+}
+
+int32_t swapmoe_set_router(swapmoe_layer_t* L, const void* Wr_dev, const float* enorm_host, void* stream) {
+  if (!L || !Wr_dev || !enorm_host) return SWAPMOE_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(Wr_dev) & 15) return SWAPMOE_ERR_INVALID_ARG;
+  EnormTable t;
+  std::memset(&t, 0, sizeof(t));
+  for (int i = 0; i < L->cfg.E; ++i) t.v[i] = enorm_host[i];
+  set_enorm_kernel<<<1, 256, 0, static_cast<cudaStream_t>(stream)>>>(t, L->cfg.E, L->enorm);
+  L->launches++;
+  L->Wr = Wr_dev;
+  L->router_set = true;
+  return check_launch();
+}
+
+int32_t swapmoe_set_resident(swapmoe_layer_t* L, const int32_t* s2e, const int32_t* phys,
+                             const void* arena_in, const void* arena_out, void* stream) {
+  if (!L || !s2e || !arena_in || !arena_out) return SWAPMOE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(arena_in) | reinterpret_cast<uintptr_t>(arena_out)) & 15)
+    return SWAPMOE_ERR_INVALID_ARG;
+  const swapmoe_config_t& c = L->cfg;
+  const int P = c.K + c.spare_slots;
+  SlotTables t;
+  for (int e = 0; e < kMaxE; ++e) t.e2s[e] = -1;
+  bool used[kMaxSlots];
+  for (int p = 0; p < kMaxSlots; ++p) { used[p] = false; t.phys[p] = 0; t.s2e[p] = -1; }
+  for (int s = 0; s < c.K; ++s) {
+    const int e = s2e[s];
+    if (e < 0 || e >= c.E || t.e2s[e] != -1) return SWAPMOE_ERR_BAD_SLOT_TABLE;
+    t.e2s[e] = s;
+    t.s2e[s] = e;
+    const int p = phys ? phys[s] : s;
+    if (p < 0 || p >= P || used[p]) return SWAPMOE_ERR_BAD_SLOT_TABLE;
+    used[p] = true;
+    t.phys[s] = p;
+  }
+  if (arena_in != L->arena_in || arena_out != L->arena_out) {
+    const int32_t rc = tc_bind_arena(L->tc, c, arena_in, arena_out);
+    if (rc != SWAPMOE_OK) return rc;
+  }
+  set_tables_kernel<<<1, 256, 0, static_cast<cudaStream_t>(stream)>>>(t, c.E, c.K, L->e2s, L->phys, L->s2e);
+  L->launches++;
+  for (int s = 0; s < c.K; ++s) { L->h_s2e[s] = t.s2e[s]; L->h_phys[s] = t.phys[s]; }
+  L->arena_in = arena_in;
+  L->arena_out = arena_out;
+  L->resident_set = true;
+  return check_launch();
+}
+
+int32_t swapmoe_forward(swapmoe_layer_t* L, const void* x, void* out, int32_t T, void* stream) {
+  return forward_checked(L, x, nullptr, out, T, stream);
+}
+
+int32_t swapmoe_forward_from_logits(swapmoe_layer_t* L, const void* x, const float* logits, void* out,
+                                    int32_t T, void* stream) {
+  if (!logits && T > 0) return SWAPMOE_ERR_INVALID_ARG;
+  return forward_checked(L, x, logits, out, T, stream);
+}
+
+int32_t swapmoe_forward_host(swapmoe_layer_t* L, const void* x_host, void* out_host, int32_t T,
+                             void* stream) {
+  if (!L || T < 0) return SWAPMOE_ERR_INVALID_ARG;
+  if (T == 0) return SWAPMOE_OK;
+  if (!x_host || !out_host) return SWAPMOE_ERR_INVALID_ARG;
+  if (T > L->cfg.max_tokens) return SWAPMOE_ERR_TOO_MANY_TOKENS;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)T * L->cfg.d_model * L->elem;
+  if (!cuda_ok(cudaMemcpyAsync(L->x_stage, x_host, bytes, cudaMemcpyHostToDevice, st))) return SWAPMOE_ERR_CUDA;
+  const int32_t rc = forward_checked(L, L->x_stage, nullptr, L->out_stage, T, stream);
+  if (rc != SWAPMOE_OK) return rc;
+  if (!cuda_ok(cudaMemcpyAsync(out_host, L->out_stage, bytes, cudaMemcpyDeviceToHost, st))) return SWAPMOE_ERR_CUDA;
+  if (!cuda_ok(cudaStreamSynchronize(st))) return SWAPMOE_ERR_CUDA;
+  return SWAPMOE_OK;
+}
+
+int32_t swapmoe_read_importance(swapmoe_layer_t* L, float* imp_host, int32_t reset, void* stream) {
+  if (!L || !imp_host) return SWAPMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!cuda_ok(cudaMemcpyAsync(imp_host, L->imp, sizeof(float) * L->cfg.E, cudaMemcpyDeviceToHost, st)))
+    return SWAPMOE_ERR_CUDA;
+  if (reset && !cuda_ok(cudaMemsetAsync(L->imp, 0, sizeof(float) * L->cfg.E, st))) return SWAPMOE_ERR_CUDA;
+  if (!cuda_ok(cudaStreamSynchronize(st))) return SWAPMOE_ERR_CUDA;
+  return SWAPMOE_OK;
+}
+
+int32_t swapmoe_topk_importance(const float* imp, int32_t E, int32_t K, int32_t* out_idx) {
+  if (!imp || !out_idx || E < 1 || K < 1 || K > E || E > kMaxE) return SWAPMOE_ERR_INVALID_ARG;
+  bool taken[kMaxE];
+  for (int e = 0; e < E; ++e) taken[e] = false;
+  for (int j = 0; j < K; ++j) {
+    int best = -1;
+    for (int e = 0; e < E; ++e) {
+      if (taken[e]) continue;
+      if (best < 0 || imp[e] > imp[best]) best = e;
+    }
+    taken[best] = true;
+    out_idx[j] = best;
+  }
+  return SWAPMOE_OK;
+}
+
+int32_t swapmoe_load_slot_async(swapmoe_layer_t* L, int32_t phys, const void* in_host, const void* out_host,
+                                void* side_stream, void* done_event) {
+  if (!L || !in_host || !out_host) return SWAPMOE_ERR_INVALID_ARG;
+  if (!L->resident_set) return SWAPMOE_ERR_NOT_READY;
+  const swapmoe_config_t& c = L->cfg;
+  if (phys < 0 || phys >= c.K + c.spare_slots) return SWAPMOE_ERR_INVALID_ARG;
+  for (int s = 0; s < c.K; ++s)
+    if (L->h_phys[s] == phys) return SWAPMOE_ERR_BAD_SLOT_TABLE;
+  cudaStream_t st = static_cast<cudaStream_t>(side_stream);
+  const size_t in_bytes = (size_t)L->nin * c.d_ff * c.d_model * L->elem;
+  const size_t out_bytes = (size_t)c.d_ff * c.d_model * L->elem;
+  char* din = static_cast<char*>(const_cast<void*>(L->arena_in)) + (size_t)phys * in_bytes;
+  char* dout = static_cast<char*>(const_cast<void*>(L->arena_out)) + (size_t)phys * out_bytes;
+  if (!cuda_ok(cudaMemcpyAsync(din, in_host, in_bytes, cudaMemcpyHostToDevice, st))) return SWAPMOE_ERR_CUDA;
+  if (!cuda_ok(cudaMemcpyAsync(dout, out_host, out_bytes, cudaMemcpyHostToDevice, st))) return SWAPMOE_ERR_CUDA;
+  if (done_event && !cuda_ok(cudaEventRecord(static_cast<cudaEvent_t>(done_event), st))) return SWAPMOE_ERR_CUDA;
+  return SWAPMOE_OK;
+}
+
+int32_t swapmoe_debug_copy(swapmoe_layer_t* L, int32_t which, void* host, size_t bytes, void* stream) {
+  if (!L || !host) return SWAPMOE_ERR_INVALID_ARG;
+  const swapmoe_config_t& c = L->cfg;
+  const size_t T = (size_t)L->last_T, P = T * c.top_k;
+  const void* src = nullptr;
+  size_t need = 0;
+  switch (which) {
+    case SWAPMOE_TAP_LOGITS: src = L->logits; need = T * c.E * 4; break;
+    case SWAPMOE_TAP_UIDX: src = L->uidx; need = P * 4; break;
+    case SWAPMOE_TAP_UGATE: src = L->ugate; need = P * 4; break;
+    case SWAPMOE_TAP_MIDX: src = L->midx; need = P * 4; break;
+    case SWAPMOE_TAP_MGATE: src = L->mgate; need = P * 4; break;
+    case SWAPMOE_TAP_SLOT: src = L->slot; need = P * 4; break;
+    case SWAPMOE_TAP_COUNT: src = L->count; need = (size_t)c.K * 4; break;
+    case SWAPMOE_TAP_OFFSET: src = L->offset; need = (size_t)(c.K + 1) * 4; break;
+    case SWAPMOE_TAP_PERM: src = L->perm; need = P * 4; break;
+    case SWAPMOE_TAP_INV: src = L->inv; need = P * 4; break;
+    case SWAPMOE_TAP_XNORM: src = L->xnorm; need = T * 4; break;
+    default: return SWAPMOE_ERR_INVALID_ARG;
+  }
+  if (bytes != need) return SWAPMOE_ERR_INVALID_ARG;
+  if (need == 0) return SWAPMOE_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!cuda_ok(cudaMemcpyAsync(host, src, need, cudaMemcpyDeviceToHost, st))) return SWAPMOE_ERR_CUDA;
+  if (!cuda_ok(cudaStreamSynchronize(st))) return SWAPMOE_ERR_CUDA;
+  return SWAPMOE_OK;
+}
+
+int32_t swapmoe_device_status(swapmoe_layer_t* L, int32_t* detail, void* stream) {
+  if (!L) return SWAPMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t w[4] = {0, 0, 0, 0};
+  if (!cuda_ok(cudaMemcpyAsync(w, L->status, sizeof(w), cudaMemcpyDeviceToHost, st))) return SWAPMOE_ERR_CUDA;
+  if (!cuda_ok(cudaMemsetAsync(L->status, 0, sizeof(w), st))) return SWAPMOE_ERR_CUDA;
+  if (!cuda_ok(cudaStreamSynchronize(st))) return SWAPMOE_ERR_CUDA;
+  if (detail) *detail = w[1];
+  return w[0] != 0 ? SWAPMOE_ERR_DEVICE_TIMEOUT : SWAPMOE_OK;
+}
+
+int64_t swapmoe_launch_count(const swapmoe_layer_t* L) { return L ? L->launches : 0; }
+int64_t swapmoe_workspace_bytes(const swapmoe_layer_t* L) { return L ? (int64_t)L->ws_bytes : 0; }
+
+int32_t swapmoe_set_gemm_path(swapmoe_layer_t* L, int32_t path) {
+  if (!L || path < 0 || path > 2) return SWAPMOE_ERR_INVALID_ARG;
+  if (path == 2 && !tc_supported(L->cfg)) return SWAPMOE_ERR_UNSUPPORTED;
+  L->gemm_path = path;
+  return SWAPMOE_OK;
+}
+
+const char* swapmoe_status_string(int32_t s) {
+  switch (s) {
+    case SWAPMOE_OK: return "ok";
+    case SWAPMOE_ERR_INVALID_ARG: return "invalid argument";
+    case SWAPMOE_ERR_NOT_READY: return "router or resident set not set";
+    case SWAPMOE_ERR_TOO_MANY_TOKENS: return "n_tokens exceeds max_tokens";
+    case SWAPMOE_ERR_BAD_SLOT_TABLE: return "bad slot table";
+    case SWAPMOE_ERR_CUDA: return "CUDA error";
+    case SWAPMOE_ERR_DEVICE_TIMEOUT: return "bounded device wait timed out";
+    case SWAPMOE_ERR_UNSUPPORTED: return "unsupported shape or device";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,462 @@
+// Grouped expert-FFN GEMM on the 5th-generation tensor cores (tcgen05 / TMEM / TMA),
+// bf16 operands, fp32 accumulation.  SwapMoE Section 2: E_i(x) = W_out * act(W_in * x),
+// evaluated per Virtual-Expert slot segment of the permuted token matrix.
+//
+// One persistent CTA per SM walks a list of 128-row output tiles:
+//   warp 0   : TMA producer  (cp.async.bulk.tensor 2D, 128-byte swizzle, mbarrier tx)
+//   warp 1   : MMA issuer    (one thread, tcgen05.mma kind::f16, M=128, N=BN, K=16)
+//   warp 2   : TMEM allocator
+//   warps 4-7: epilogue      (tcgen05.ld -> activation -> global stores), overlapped with
+//                             the next tile's MMAs through two TMEM accumulator buffers.
+// No load uses cluster multicast.  Every mbarrier wait is bounded: on expiry the
+// kernel records a status word, stops issuing work, drains and frees its TMEM.
+#pragma once
+#include <cuda.h>
+
+#include "../../include/swapmoe.h"
+#include "common.cuh"
+
+namespace swapmoe {
+
+constexpr int kTcBM = 128;   // rows per tile (TMEM lanes)
+constexpr int kTcBK = 64;    // bf16 elements per k-block = one 128-byte swizzle row
+constexpr int kTcUmmaK = 16;
+constexpr int kTcThreads = 256;
+constexpr int kTcSmemBudget = 200 * 1024;
+
+enum { kTcEpiReluBf16 = 0, kTcEpiSwigluBf16 = 1, kTcEpiF32 = 2 };
+
+struct TcGemmArgs {
+  void* C;                  // [rows_pad, ldc]
+  const TileDesc* tiles;
+  const int32_t* n_tiles;   // number of row tiles (device)
+  int32_t* status;          // [0] = error flag, [1] = code of the wait that gave up
+  int32_t ldc;              // columns of C
+  int32_t n_col_tiles;      // column tiles per row tile
+  int32_t k_blocks;         // contraction length / 64
+  int32_t b_rows_per_phys;  // rows of the flattened weight map per arena entry
+  int32_t b_rows_gate;      // row offset of the second input matrix (SwiGLU), else 0
+};
+
+// ----------------------------------------------------------------------------- PTX wrappers
+namespace ptx {
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
+               "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(tmem_d),
+      "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+}  // namespace ptx
+
+// Shared-memory operand descriptor: K-major tile whose rows are 128 bytes, written by
+// TMA with 128-byte swizzle; 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);  // start address
+  d |= (uint64_t)(1024u >> 4) << 32;             // stride between 8-row groups
+  d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                        // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
+__host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// Bounded wait: polls the barrier, and every 256 polls checks a 2-second deadline.
+// Returns false (after recording `code`) when the wait gave up or another role aborted.
+__device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                             int32_t* status, int code) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = ptx::globaltimer_ns();
+  for (uint32_t spin = 1;; ++spin) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((spin & 255u) == 0) {
+      if (*abort_flag) return false;
+      if (ptx::globaltimer_ns() - t0 > 2000000000ull) {
+        *abort_flag = 1;
+        if (atomicCAS(status, 0, 1) == 0) status[1] = code;
+        return false;
+      }
+    }
+  }
+}
+
+template <int BN>
+struct TcSmem {
+  static constexpr int kABytes = kTcBM * kTcBK * 2;
+  static constexpr int kBBytes = BN * kTcBK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = (kTcSmemBudget - 2048) / kStageBytes;
+  static constexpr int kBytes = kStages * kStageBytes + 2048;  // + alignment slack and barriers
+};
+
+// C tile [128, BN (or BN/2 for SwiGLU)] = epi(A[row0:row0+128, :] * B[brow:brow+BN, :]^T)
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kTcThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const TcGemmArgs a) {
+  using S = TcSmem<BN>;
+  constexpr int kStages = S::kStages;
+  constexpr int kNB = (EPI == kTcEpiSwigluBf16) ? 2 : 1;   // weight boxes per stage
+  constexpr int kBoxRows = BN / kNB;
+  constexpr int kOutCols = BN / kNB;                        // output columns per tile
+  constexpr uint32_t kTmemCols = 2 * BN;                    // two accumulator buffers
+  constexpr uint32_t kIdesc = make_idesc_bf16(kTcBM, BN);
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  unsigned char* sA = smem;                                   // [stages][128][64] bf16
+  unsigned char* sB = smem + kStages * S::kABytes;            // [stages][BN][64] bf16
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * S::kStageBytes);
+  uint64_t* full = bars;                    // [stages]
+  uint64_t* empty = bars + kStages;         // [stages]
+  uint64_t* acc_full = bars + 2 * kStages;  // [2]
+  uint64_t* acc_empty = acc_full + 2;       // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 128); }
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmA);
+    ptx::prefetch_tmap(&tmB);
+  }
+  if (warp == 2) {
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int n_row_tiles = *a.n_tiles;
+  const int total = n_row_tiles * a.n_col_tiles;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ------------------------------------------------------------------ TMA producer
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        const int ct = t / n_row_tiles, rt = t - ct * n_row_tiles;   // row tiles vary fastest
+        const TileDesc td = a.tiles[rt];
+        const int brow = td.phys * a.b_rows_per_phys + ct * kBoxRows;
+        for (int kb = 0; kb < a.k_blocks; ++kb) {
+          ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 1);
+          if (!ok) break;
+          ptx::mbar_expect_tx(&full[stage], S::kStageBytes);
+          ptx::tma_load_2d(sA + stage * S::kABytes, &tmA, &full[stage], kb * kTcBK, td.row0);
+#pragma unroll
+          for (int j = 0; j < kNB; ++j)
+            ptx::tma_load_2d(sB + stage * S::kBBytes + j * kBoxRows * kTcBK * 2, &tmB, &full[stage],
+                             kb * kTcBK, brow + j * a.b_rows_gate);
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // Give copies that are still in flight time to land before shared memory is released.
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ptx::globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ------------------------------------------------------------------ MMA issuer
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        ok = bounded_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, a.status, 2);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < a.k_blocks; ++kb) {
+          ok = bounded_wait(&full[stage], phase, abort_flag, a.status, 3);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          const uint64_t da = make_kmajor_sw128_desc(ptx::smem_u32(sA + stage * S::kABytes));
+          const uint64_t db = make_kmajor_sw128_desc(ptx::smem_u32(sB + stage * S::kBBytes));
+#pragma unroll
+          for (int k = 0; k < kTcBK / kTcUmmaK; ++k) {
+            // advancing 16 elements along K inside the swizzled row = +32 bytes = +2 in the address field
+            ptx::umma_bf16(tmem_d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), kIdesc,
+                           (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          ptx::umma_commit(&empty[stage]);   // frees the stage once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::umma_commit(&acc_full[acc]);    // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else if (warp >= 4) {
+    // -------------------------------------------------------------------- epilogue
+    const int q = warp - 4;                    // TMEM lane quarter this warp may read
+    const int r = q * 32 + lane;               // row of the tile owned by this thread
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+      const int ct = t / n_row_tiles, rt = t - ct * n_row_tiles;
+      const TileDesc td = a.tiles[rt];
+      ok = bounded_wait(&acc_full[acc], acc_phase, abort_flag, a.status, 4);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+      const bool row_ok = r < td.rows;
+      const size_t crow = (size_t)(td.row0 + r) * a.ldc + (size_t)ct * kOutCols;
+#pragma unroll 1
+      for (int c0 = 0; c0 < kOutCols; c0 += 32) {
+        uint32_t v[32];
+        ptx::tmem_ld32(taddr + (uint32_t)c0, v);
+        if (EPI == kTcEpiSwigluBf16) {
+          uint32_t g[32];
+          ptx::tmem_ld32(taddr + (uint32_t)(c0 + kOutCols), g);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float x1 = __uint_as_float(v[i]);
+            v[i] = __float_as_uint(x1 / (1.f + __expf(-x1)) * __uint_as_float(g[i]));
+          }
+        } else {
+          ptx::tmem_ld_wait();
+        }
+        if (row_ok) {
+          if (EPI == kTcEpiF32) {
+            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(a.C) + crow + c0);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                   __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+          } else {
+            uint4* dst = reinterpret_cast<uint4*>(static_cast<bf16*>(a.C) + crow + c0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              float f[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                f[j] = __uint_as_float(v[8 * i + j]);
+                if (EPI == kTcEpiReluBf16) f[j] = fmaxf(f[j], 0.f);
+              }
+              dst[i] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]),
+                                  pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+            }
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&acc_empty[acc]);       // 128 arrivals hand the buffer back to the MMA warp
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ----------------------------------------------------------------------------- host side
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                    CUtensorMapFloatOOBfill);
+
+struct TcState {
+  bool enabled;
+  int sm_count;
+  PFN_encodeTiled encode;
+  CUtensorMap map_xp, map_h;          // activations: [rows_pad, d], [rows_pad, f], box 64 x 128
+  CUtensorMap map_win, map_wout;      // weights flattened to 2D, box 64 x (rows per load)
+  int bn2;                            // column tile of the second GEMM
+  bool arena_bound;
+};
+
+inline bool tc_supported(const swapmoe_config_t& c) {
+  return c.dtype == SWAPMOE_BF16 && c.d_model % 128 == 0 && c.d_ff % 256 == 0;
+}
+
+// Automatic choice: tensor cores whenever the shape allows it.
+inline bool tc_selected(int path, const swapmoe_config_t& c, int /*T*/) {
+  if (path == 1) return false;
+  return tc_supported(c);
+}
+
+inline bool tc_encode_2d(PFN_encodeTiled enc, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                         uint32_t box_rows) {
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kTcBK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, int EPI>
+inline bool tc_set_smem_attr() {
+  return cudaFuncSetAttribute(tc_gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              TcSmem<BN>::kBytes) == cudaSuccess;
+}
+
+inline int32_t tc_init(TcState& s, const swapmoe_config_t& c, void* xp, void* h, float* /*y*/, int rows_pad) {
+  s.enabled = false;
+  s.arena_bound = false;
+  if (!tc_supported(c)) return SWAPMOE_OK;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SWAPMOE_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&s.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SWAPMOE_ERR_CUDA;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres) !=
+          cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
+    return SWAPMOE_ERR_CUDA;
+  s.encode = reinterpret_cast<PFN_encodeTiled>(fn);
+  if (!tc_encode_2d(s.encode, &s.map_xp, xp, (uint64_t)rows_pad, (uint64_t)c.d_model, kTcBM)) return SWAPMOE_ERR_CUDA;
+  if (!tc_encode_2d(s.encode, &s.map_h, h, (uint64_t)rows_pad, (uint64_t)c.d_ff, kTcBM)) return SWAPMOE_ERR_CUDA;
+  bool ok = tc_set_smem_attr<256, kTcEpiReluBf16>() && tc_set_smem_attr<256, kTcEpiSwigluBf16>() &&
+            tc_set_smem_attr<256, kTcEpiF32>() && tc_set_smem_attr<128, kTcEpiF32>();
+  if (!ok) return SWAPMOE_ERR_CUDA;
+  s.bn2 = (c.d_model % 256 == 0 && c.d_model >= 2048) ? 256 : 128;
+  s.enabled = true;
+  return SWAPMOE_OK;
+}
+
+inline int32_t tc_bind_arena(TcState& s, const swapmoe_config_t& c, const void* arena_in, const void* arena_out) {
+  if (!s.enabled) return SWAPMOE_OK;
+  const int P = c.K + c.spare_slots;
+  const int nin = c.act == SWAPMOE_ACT_SWIGLU ? 2 : 1;
+  const uint32_t box_in = nin == 2 ? 128 : 256;
+  if (!tc_encode_2d(s.encode, &s.map_win, arena_in, (uint64_t)P * nin * c.d_ff, (uint64_t)c.d_model, box_in))
+    return SWAPMOE_ERR_CUDA;
+  if (!tc_encode_2d(s.encode, &s.map_wout, arena_out, (uint64_t)P * c.d_model, (uint64_t)c.d_ff, (uint32_t)s.bn2))
+    return SWAPMOE_ERR_CUDA;
+  s.arena_bound = true;
+  return SWAPMOE_OK;
+}
+
+inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* /*xp*/, void* h, float* y, const TileDesc* tiles,
+                      const int32_t* n_tiles, int max_tiles, int32_t* status, cudaStream_t st, int64_t* launches) {
+  if (!s.enabled || !s.arena_bound) return SWAPMOE_ERR_NOT_READY;
+  const bool swiglu = c.act == SWAPMOE_ACT_SWIGLU;
+  TcGemmArgs g1;
+  g1.C = h; g1.tiles = tiles; g1.n_tiles = n_tiles; g1.status = status; g1.ldc = c.d_ff;
+  g1.n_col_tiles = swiglu ? c.d_ff / 128 : c.d_ff / 256;
+  g1.k_blocks = c.d_model / kTcBK;
+  g1.b_rows_per_phys = swiglu ? 2 * c.d_ff : c.d_ff;
+  g1.b_rows_gate = swiglu ? c.d_ff : 0;
+  int grid = max_tiles * g1.n_col_tiles;
+  if (grid > s.sm_count) grid = s.sm_count;
+  if (swiglu)
+    tc_gemm_kernel<256, kTcEpiSwigluBf16><<<grid, kTcThreads, TcSmem<256>::kBytes, st>>>(s.map_xp, s.map_win, g1);
+  else
+    tc_gemm_kernel<256, kTcEpiReluBf16><<<grid, kTcThreads, TcSmem<256>::kBytes, st>>>(s.map_xp, s.map_win, g1);
+  ++*launches;
+
+  TcGemmArgs g2;
+  g2.C = y; g2.tiles = tiles; g2.n_tiles = n_tiles; g2.status = status; g2.ldc = c.d_model;
+  g2.n_col_tiles = c.d_model / s.bn2;
+  g2.k_blocks = c.d_ff / kTcBK;
+  g2.b_rows_per_phys = c.d_model;
+  g2.b_rows_gate = 0;
+  grid = max_tiles * g2.n_col_tiles;
+  if (grid > s.sm_count) grid = s.sm_count;
+  if (s.bn2 == 256)
+    tc_gemm_kernel<256, kTcEpiF32><<<grid, kTcThreads, TcSmem<256>::kBytes, st>>>(s.map_h, s.map_wout, g2);
+  else
+    tc_gemm_kernel<128, kTcEpiF32><<<grid, kTcThreads, TcSmem<128>::kBytes, st>>>(s.map_h, s.map_wout, g2);
+  ++*launches;
+  return cudaGetLastError() == cudaSuccess ? SWAPMOE_OK : SWAPMOE_ERR_CUDA;
+}
+
+}  // namespace swapmoe

@@ -1,0 +1,196 @@
+// Slot histogram scan, stable token permutation, row gather and the importance
+// reduction (SwapMoE Section 2: every token may pick a different expert; Eq. 1).
+#pragma once
+#include "common.cuh"
+
+namespace swapmoe {
+
+struct ScanArgs {
+  const int32_t* cta_hist;   // [n_cta, K]
+  const float* cta_imp;      // [n_cta, E]
+  const int32_t* phys_slot;  // [K]
+  int32_t* cta_base;         // [n_cta, K] pairs of the same slot in earlier CTAs
+  int32_t* count;            // [K]
+  int32_t* offset;           // [K+1]  exclusive scan of count
+  int32_t* pad_offset;       // [K+1]  same with every segment rounded up to kSegAlign rows
+  TileDesc* tiles;           // GEMM work list
+  int32_t* n_tiles;          // [1]
+  float* imp;                // [E] accumulator of Eq. (1)
+  int32_t n_cta, K, E, tile_rows;
+};
+
+// One CTA of 1024 threads.  Warp w scans slot w, w+32, ... over the CTAs in order;
+// then thread s lays out slot s (offsets, padded offsets, tile list); warps also
+// reduce the per-CTA importance partials in a fixed order.
+__global__ void __launch_bounds__(1024) scan_reduce_kernel(const ScanArgs a) {
+  __shared__ int32_t s_count[kMaxSlots];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  for (int s = warp; s < a.K; s += 32) {
+    int running = 0;
+    for (int c0 = 0; c0 < a.n_cta; c0 += 32) {
+      const int c = c0 + lane;
+      const int v = (c < a.n_cta) ? a.cta_hist[(size_t)c * a.K + s] : 0;
+      int incl = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      if (c < a.n_cta) a.cta_base[(size_t)c * a.K + s] = running + incl - v;
+      running += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) s_count[s] = running;
+  }
+  // Eq. (1): add this batch's per-CTA partial sums, CTA order fixed by the lane
+  // stride and the shuffle tree, so repeated runs give identical bits.
+  for (int e = warp; e < a.E; e += 32) {
+    float acc = 0.f;
+    for (int c = lane; c < a.n_cta; c += 32) acc += a.cta_imp[(size_t)c * a.E + e];
+    acc = warp_sum(acc);
+    if (lane == 0) a.imp[e] += acc;
+  }
+  __syncthreads();
+  if (tid < a.K) {
+    int off = 0, pad = 0, t0 = 0;
+    for (int s = 0; s < tid; ++s) {
+      const int c = s_count[s];
+      off += c;
+      pad += (c + kSegAlign - 1) / kSegAlign * kSegAlign;
+      t0 += (c + a.tile_rows - 1) / a.tile_rows;
+    }
+    const int c = s_count[tid];
+    a.count[tid] = c;
+    a.offset[tid] = off;
+    a.pad_offset[tid] = pad;
+    const int nt = (c + a.tile_rows - 1) / a.tile_rows;
+    const int ph = a.phys_slot[tid];
+    for (int i = 0; i < nt; ++i) {
+      TileDesc td;
+      td.phys = ph;
+      td.row0 = pad + i * a.tile_rows;
+      td.rows = min(a.tile_rows, c - i * a.tile_rows);
+      td.slot = tid;
+      a.tiles[t0 + i] = td;
+    }
+    if (tid == a.K - 1) {
+      a.offset[a.K] = off + c;
+      a.pad_offset[a.K] = pad + (c + kSegAlign - 1) / kSegAlign * kSegAlign;
+      *a.n_tiles = t0 + nt;
+    }
+  }
+}
+
+struct PermuteArgs {
+  const void* x;              // [T, d]
+  const int32_t* slot;        // [T*k]
+  const int32_t* cta_base;    // [n_cta, K]
+  const int32_t* offset;      // [K+1]
+  const int32_t* pad_offset;  // [K+1]
+  int32_t* perm;              // [T*k]
+  int32_t* inv;               // [T*k]
+  int32_t* inv_pad;           // [T*k] row of the pair in the padded workspace
+  void* xp;                   // [rows_pad, d]
+  int32_t T, d, k, K;
+};
+
+// One CTA = the pairs of kTokTile tokens in flat order p = t*k + j.  The rank of a
+// pair among the pairs of the same slot is: pairs in earlier CTAs (cta_base) +
+// pairs in earlier warps of this CTA + earlier lanes of this warp (match + popc),
+// which is exactly a stable counting sort.
+template <typename T>
+__global__ void __launch_bounds__(256) permute_gather_kernel(const PermuteArgs a) {
+  __shared__ int32_t wcount[kMaxTopK][kMaxSlots];
+  __shared__ int32_t dst_row[kTokTile * kMaxTopK];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int npair = kTokTile * a.k;            // <= 128
+  const int nwarp_p = (npair + 31) >> 5;
+  const int p0 = blockIdx.x * npair;
+  const int n_total = a.T * a.k;
+
+  for (int i = tid; i < kMaxTopK * kMaxSlots; i += 256) (&wcount[0][0])[i] = 0;
+  __syncthreads();
+  int s = -1, rank = 0;
+  const int p = p0 + tid;
+  if (warp < nwarp_p) {
+    if (tid < npair && p < n_total) s = a.slot[p];
+    const uint32_t same = __match_any_sync(0xffffffffu, s);
+    rank = __popc(same & ((1u << lane) - 1u));
+    if (s >= 0 && rank == 0) wcount[warp][s] = __popc(same);
+  }
+  __syncthreads();
+  if (s >= 0) {
+    int before = a.cta_base[(size_t)blockIdx.x * a.K + s];
+    for (int w = 0; w < warp; ++w) before += wcount[w][s];
+    const int within = before + rank;
+    const int pos = a.offset[s] + within;
+    a.perm[pos] = p;
+    a.inv[p] = pos;
+    const int row = a.pad_offset[s] + within;
+    a.inv_pad[p] = row;
+    dst_row[tid] = row;
+  } else if (tid < npair) {
+    dst_row[tid] = -1;
+  }
+  __syncthreads();
+  // Gather: copy each pair's token row into its slot segment, 16 bytes per access.
+  const int vec_per_row = a.d * (int)sizeof(T) / 16;
+  const uint4* src = static_cast<const uint4*>(a.x);
+  uint4* dst = static_cast<uint4*>(a.xp);
+  for (int i = tid; i < npair * vec_per_row; i += 256) {
+    const int pl = i / vec_per_row, v = i - pl * vec_per_row;
+    const int row = dst_row[pl];
+    if (row >= 0) {
+      const int t = (p0 + pl) / a.k;
+      dst[(size_t)row * vec_per_row + v] = src[(size_t)t * vec_per_row + v];
+    }
+  }
+}
+
+struct CombineArgs {
+  const float* y;            // [rows_pad, d] fp32 expert outputs
+  const int32_t* inv_pad;    // [T*k]
+  const float* mgate;        // [T*k]
+  void* out;                 // [T, d]
+  int32_t T, d, k;
+};
+
+// out[t, c] = sum_j mgate[t,j] * y[inv_pad[t,j], c]; each thread owns 8 columns.
+template <typename T>
+__global__ void __launch_bounds__(256) combine_kernel(const CombineArgs a) {
+  const int c8n = a.d >> 3;
+  const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= (long long)a.T * c8n) return;
+  const int t = (int)(idx / c8n), c = (int)(idx - (long long)t * c8n) * 8;
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int j = 0; j < a.k; ++j) {
+    const float g = a.mgate[(size_t)t * a.k + j];
+    const float* yr = a.y + (size_t)a.inv_pad[(size_t)t * a.k + j] * a.d + c;
+    const float4 y0 = reinterpret_cast<const float4*>(yr)[0];
+    const float4 y1 = reinterpret_cast<const float4*>(yr)[1];
+    acc[0] = fmaf(g, y0.x, acc[0]); acc[1] = fmaf(g, y0.y, acc[1]);
+    acc[2] = fmaf(g, y0.z, acc[2]); acc[3] = fmaf(g, y0.w, acc[3]);
+    acc[4] = fmaf(g, y1.x, acc[4]); acc[5] = fmaf(g, y1.y, acc[5]);
+    acc[6] = fmaf(g, y1.z, acc[6]); acc[7] = fmaf(g, y1.w, acc[7]);
+  }
+  store8(static_cast<T*>(a.out) + (size_t)t * a.d + c, acc);
+}
+
+// Installs the slot tables (arguments travel by value in the launch, so the host
+// arrays may be reused immediately and earlier forwards keep the old tables).
+struct SlotTables {
+  int32_t e2s[kMaxE];
+  int32_t phys[kMaxSlots];
+  int32_t s2e[kMaxSlots];
+};
+__global__ void set_tables_kernel(const SlotTables t, int E, int K, int32_t* e2s, int32_t* phys,
+                                  int32_t* s2e) {
+  for (int i = threadIdx.x; i < E; i += blockDim.x) e2s[i] = t.e2s[i];
+  for (int i = threadIdx.x; i < K; i += blockDim.x) { phys[i] = t.phys[i]; s2e[i] = t.s2e[i]; }
+}
+
+__global__ void zero_f32_kernel(float* p, int n) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) p[i] = 0.f;
+}
+
+}  // namespace swapmoe
