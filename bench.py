@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the Virtual-Expert MoE-layer forward on B200.
+
+One "step" is one pass of the whole hot path (router+gate, scan, permute, grouped
+FFN GEMMs, combine, importance) over one batch of synthetic tokens.  The default
+workload is the Switch-base-64-shaped layer (bf16, d_model 768, d_ff 3072, E 64,
+top-1, K 16 resident slots, 2048 tokens with Zipf(1.1) expert popularity and
+runs of 32 tokens sharing a preferred expert set).
+
+    python bench.py --gpus 1 --steps 50 --warmup 10
+    python bench.py --impl reference            # the CPU oracle on the host cores
+
+Prints ONE JSON line.  With --gpus N > 1 (under torchrun) every rank runs an
+independent replica on its own tokens ("replicas only": the path has no
+exchange step), rank 0 prints the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2308_15030_b200 import inputs as I  # noqa: E402
+
+METRIC = "moe_layer_tokens_per_s_at_budget_K"
+UNIT = "tokens/s"
+L2_BYTES = 126e6
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+def workload_string(cfg):
+    return ("%s: %s d_model=%d d_ff=%d E=%d top%d K=%d resident T=%d tokens %s, zipf_s=%.1f "
+            "runs of %d" % (cfg.name, "bf16" if cfg.dtype == I.BF16 else "fp32", cfg.d, cfg.f, cfg.E,
+                            cfg.k, cfg.K, cfg.T, "SwiGLU" if cfg.act else "ReLU", cfg.zipf_s,
+                            cfg.run_len))
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [s.strip() for s in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- the CUDA arm
+def algorithmic_bytes(cfg, touched):
+    """Method's own traffic of one forward: resident weights that received >= 1 token,
+    x in, out out, router matrix (implementation round trips of xp/h/y are excluded)."""
+    return touched * cfg.nmat * cfg.d * cfg.f * cfg.nb + 2 * cfg.T * cfg.d * cfg.nb + cfg.E * cfg.d * cfg.nb
+
+
+def gemm_algorithmic(cfg, touched):
+    """Bytes and flops of the two grouped-GEMM launches of one forward: the touched
+    slots' weights, the permuted tokens in and the expert outputs out; the hidden
+    activations between the two GEMMs are an implementation round trip."""
+    pairs = cfg.T * cfg.k
+    nbytes = touched * cfg.nmat * cfg.d * cfg.f * cfg.nb + 2 * pairs * cfg.d * cfg.nb
+    flops = 2.0 * pairs * cfg.d * cfg.f * cfg.nmat
+    return nbytes, flops
+
+
+def run_cuda(args, cfg):
+    import torch
+    import torch.distributed as dist
+    from paper_2308_15030_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit("--gpus %d but WORLD_SIZE=%d (launch with torch.distributed.run)" % (args.gpus, world))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    tdt = torch.bfloat16 if cfg.dtype == I.BF16 else torch.float32
+
+    def dev(a):
+        a = np.ascontiguousarray(a, dtype=np.float32)
+        if cfg.dtype == I.BF16:
+            return torch.from_numpy(I.bf16_bits(a).view(np.int16)).view(torch.bfloat16).cuda()
+        return torch.from_numpy(a).cuda()
+
+    Wr = I.make_router(cfg)
+    enorm = I.make_enorm(cfg)
+    # every rank draws its own tokens (replicas on different batches)
+    x_host = I.make_tokens(cfg, Wr, seed=cfg.seed + 1000 * rank)
+    d_Wr = dev(Wr)
+    weight_bytes = cfg.K * cfg.nmat * cfg.d * cfg.f * cfg.nb
+    copies = max(1, int(np.ceil(4 * L2_BYTES / weight_bytes)))   # rotation spans > 4x L2
+    stream = torch.cuda.Stream()
+
+    # Resident set chosen the product's own way: one pass with an arbitrary set to
+    # collect Eq. (1) importance, then the top-K experts become resident.
+    d_x = [dev(x_host) for _ in range(copies)]
+    d_out = [torch.empty((cfg.T, cfg.d), dtype=tdt, device="cuda") for _ in range(copies)]
+    with torch.cuda.stream(stream):
+        first = list(range(cfg.K))
+        a_in, a_out = I.build_arena(cfg, first)
+        arenas = [(dev(a_in), dev(a_out))]
+        layers = [binding.Layer(cfg.E, cfg.d, cfg.f, cfg.k, cfg.K, cfg.dtype, cfg.act, cfg.renorm,
+                                max_tokens=cfg.T) for _ in range(copies)]
+        layers[0].set_router(d_Wr, enorm)
+        layers[0].set_resident(first, *arenas[0])
+        layers[0].forward(d_x[0], d_out[0])
+        imp = layers[0].read_importance(reset=True)
+        s2e = binding.topk_importance(imp, cfg.K)
+        a_in, a_out = I.build_arena(cfg, s2e)
+        arenas = [(dev(a_in), dev(a_out)) for _ in range(copies)]
+        del a_in, a_out
+        for L, ar in zip(layers, arenas):
+            L.set_router(d_Wr, enorm)
+            L.set_resident(s2e, *ar)
+        layers[0].forward(d_x[0], d_out[0])
+        count = layers[0].tap("count")
+        uidx = layers[0].tap("uidx")
+        for L in layers:
+            L.read_importance(reset=True)
+    touched = int(np.count_nonzero(count))
+    hit = float(np.mean(np.isin(uidx, s2e)))
+
+    def step(i):
+        j = i % copies
+        layers[j].forward(d_x[j], d_out[j], stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region 1: device-resident inputs
+    with torch.cuda.stream(stream):
+        for i in range(args.warmup):
+            step(i)
+    barrier()
+    l0 = sum(L.launch_count for L in layers)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for i in range(args.steps):
+            step(i)
+        e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    launches = sum(L.launch_count for L in layers) - l0
+
+    # ---- timed region 2: same steps with events at the stage boundaries (per-kernel times)
+    nst = binding.N_STAGES
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nst + 1)] for _ in range(args.steps)]
+    with torch.cuda.stream(stream):
+        for i in range(args.steps):
+            j = i % copies
+            layers[j].forward_timed(d_x[j], d_out[j], evs[i], stream=stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    stage_ms = np.array([[evs[i][s].elapsed_time(evs[i][s + 1]) for s in range(nst)]
+                         for i in range(args.steps)])
+    stage_avg = stage_ms.mean(axis=0)
+
+    # ---- timed region 3: end to end through the host-buffer entry point
+    xh = torch.from_numpy(I.bf16_bits(x_host).view(np.int16)).view(torch.bfloat16) \
+        if cfg.dtype == I.BF16 else torch.from_numpy(x_host)
+    xh = xh.pin_memory()
+    oh = torch.empty((cfg.T, cfg.d), dtype=tdt).pin_memory()
+    for i in range(min(3, args.warmup)):
+        layers[i % copies].forward_host(xh, oh, stream=stream)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        layers[i % copies].forward_host(xh, oh, stream=stream)
+    barrier()
+    e2e_s = time.perf_counter() - t0
+
+    st = [L.device_status() for L in layers]
+    if any(s[0] != 0 for s in st):
+        raise SystemExit("device status error: %r" % (st,))
+
+    times = torch.tensor([ms_total, e2e_s * 1e3], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = float(times[0]), float(times[1])
+    if world > 1:
+        dist.barrier()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return None
+
+    peaks = load_peaks()
+    ms_step = ms_total / args.steps
+    value = world * cfg.T * args.steps / (ms_total * 1e-3)
+    g_bytes, g_flops = gemm_algorithmic(cfg, touched)
+    g_ms = float(stage_avg[3] + stage_avg[4]) / 2.0          # average duration of one GEMM launch
+    t_hbm = g_bytes / (peaks["hbm_gbs"] * 1e9)
+    t_tc = g_flops / (peaks["bf16_tflops"] * 1e12) if cfg.dtype == I.BF16 else 0.0
+    if cfg.dtype != I.BF16:
+        bound, peak, ach, unit = "alu", 74.4, g_flops / 2 / (g_ms * 1e-3) / 1e12, "TFLOP/s"
+    elif t_hbm >= t_tc:
+        bound, peak, ach, unit = "hbm", peaks["hbm_gbs"], g_bytes / 2 / (g_ms * 1e-3) / 1e9, "GB/s"
+    else:
+        bound, peak, ach, unit = "tensor", peaks["bf16_tflops"], g_flops / 2 / (g_ms * 1e-3) / 1e12, "TFLOP/s"
+    layer_bytes = algorithmic_bytes(cfg, touched)
+    layer_flops = 2.0 * cfg.T * cfg.d * cfg.E + g_flops
+    t_roof = max(layer_bytes / (peaks["hbm_gbs"] * 1e9),
+                 layer_flops / (peaks["bf16_tflops"] * 1e12) if cfg.dtype == I.BF16
+                 else layer_flops / 74.4e12)
+    res = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg.dtype == I.BF16 else "f32", "data": "synthetic",
+        "config": {"workload": workload_string(cfg),
+                   "l2": "inputs rotate over %d copies of tokens+weights (%.0f MB > 126 MB L2)"
+                         % (copies, copies * weight_bytes / 1e6),
+                   "resident_set": "top-K by Eq.(1) importance of the batch",
+                   "touched_slots": touched, "slot_counts": [int(c) for c in count],
+                   "unmasked_hit_rate": hit, "multi_gpu": "replicas only"},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "e2e": {"value": world * cfg.T * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": cfg.T * cfg.d * cfg.nb, "d2h_bytes_per_step": cfg.T * cfg.d * cfg.nb,
+                "ms_per_step": e2e_ms / args.steps},
+        "roofline": {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                     "traffic": None, "peak_source": peaks["source"],
+                     "kernel": "tc_gemm_kernel (grouped FFN GEMM, 2 launches per step: GEMM-1+act, GEMM-2)"
+                               if cfg.dtype == I.BF16 else "gemm_simt_kernel (2 launches per step)",
+                     "algorithmic_bytes_per_launch": g_bytes / 2, "flops_per_launch": g_flops / 2,
+                     "avg_launch_ms": g_ms,
+                     "tensor_tflops": g_flops / 2 / (g_ms * 1e-3) / 1e12},
+        "layer_roofline": {"t_roof_us": t_roof * 1e6, "frac": t_roof * 1e3 / ms_step,
+                           "algorithmic_bytes": layer_bytes, "flops": layer_flops},
+        "stage_us": {n: float(v * 1e3) for n, v in zip(binding.STAGE_NAMES, stage_avg)},
+        "stage_pass_ms_per_step": float(stage_ms.sum(axis=1).mean()),
+    }
+    if world > 1:
+        dist.destroy_process_group()
+    return res
+
+
+# ----------------------------------------------------------------------------- the oracle arm
+def oracle_sample(cfg, steps=1, warmup=0):
+    """Times the CPU oracle, as it stands, on the workload's batch (host cores)."""
+    import oracle
+    Wr = I.make_router(cfg)
+    enorm = I.make_enorm(cfg)
+    x = I.make_tokens(cfg, Wr)
+    lg = oracle.logits(x, Wr)
+    uidx, ugate = oracle.gate(lg, cfg.k, cfg.renorm)
+    s2e = oracle.topk_importance(oracle.importance(x, uidx, ugate, enorm), cfg.K)
+    a_in, a_out = I.build_arena(cfg, s2e)
+    # bound the work to roughly 10-30 s: the FFN of a token subset, routing over all tokens
+    flops_tok = 2.0 * cfg.k * cfg.d * cfg.f * cfg.nmat
+    n_sub = int(min(cfg.T, max(16, 40e9 / flops_tok)))
+    sub = None if n_sub >= cfg.T else np.sort(
+        np.random.default_rng(0).choice(cfg.T, n_sub, replace=False)).astype(np.int32)
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle.forward(x, Wr, enorm, s2e, a_in, a_out, k=cfg.k, act=cfg.act, renorm=cfg.renorm,
+                       token_subset=sub)
+        if i >= warmup:
+            times.append(time.perf_counter() - t0)
+    n_tok = cfg.T if sub is None else n_sub
+    sample = ("full %d-token batch" % cfg.T) if sub is None else \
+        ("routing on all %d tokens, expert FFN on a seeded %d-token subset; tokens/s counts the subset"
+         % (cfg.T, n_sub))
+    return n_tok, times, oracle.num_threads(), sample
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return None
+    n_tok, times, cores, sample = oracle_sample(cfg, steps=args.steps, warmup=min(args.warmup, 1))
+    total = float(np.sum(times))
+    value = n_tok * len(times) / total
+    return {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": total / len(times) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": workload_string(cfg)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg5"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = I.CONFIGS[args.workload]
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else min(args.steps, 5)
+        args.warmup = 1 if args.warmup is None else args.warmup
+        res = run_reference(args, cfg)
+        if res is not None:
+            print(json.dumps(res), flush=True)
+        return
+    args.steps = 200 if args.steps is None else args.steps
+    args.warmup = 20 if args.warmup is None else max(3, args.warmup)
+    res = run_cuda(args, cfg)
+    if res is None:
+        return
+    if args.gpus == 1 and not args.no_cpu_baseline:
+        n_tok, times, cores, sample = oracle_sample(cfg, steps=3, warmup=0)
+        res["cpu_baseline"] = {"value": n_tok / float(np.min(times)), "unit": UNIT, "cores": cores,
+                               "kind": "oracle", "sample": sample}
+    print(json.dumps(res), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -147,6 +147,17 @@ int32_t swapmoe_forward_from_logits(swapmoe_layer_t* layer, const void* x_dev,
                                     const float* logits_dev, void* out_dev, int32_t n_tokens,
                                     void* stream);
 
+/* Measurement form of swapmoe_forward: identical work, but records the
+ * SWAPMOE_N_STAGES + 1 caller-owned cudaEvent_t of `events` on `stream` at the
+ * stage boundaries (event i before stage i, the last one after the final
+ * stage), so a caller can time each kernel of the path with
+ * cudaEventElapsedTime.  Stages: 0 router+gate, 1 scan+importance reduce,
+ * 2 permute+gather, 3 grouped GEMM-1 (+activation), 4 grouped GEMM-2,
+ * 5 combine. */
+#define SWAPMOE_N_STAGES 6
+int32_t swapmoe_forward_timed(swapmoe_layer_t* layer, const void* x_dev, void* out_dev,
+                              int32_t n_tokens, void* stream, void* const* events);
+
 /* End-to-end form with HOST buffers: copies x_host [n_tokens, d_model] to the
  * device, runs swapmoe_forward, copies the result to out_host, and returns after
  * `stream` has completed.  Pinned host memory makes the copies asynchronous

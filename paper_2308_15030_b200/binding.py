@@ -16,6 +16,8 @@ import numpy as np
 from . import build as _build
 
 F32, BF16 = 0, 1
+N_STAGES = 6
+STAGE_NAMES = ("router_gate", "scan_reduce", "permute_gather", "gemm1_act", "gemm2", "combine")
 ACT_RELU, ACT_SWIGLU = 0, 1
 
 TAPS = {
@@ -27,7 +29,7 @@ TAPS = {
 
 EXPORTS = [
     "swapmoe_create", "swapmoe_destroy", "swapmoe_set_router", "swapmoe_set_resident",
-    "swapmoe_forward", "swapmoe_forward_from_logits", "swapmoe_forward_host",
+    "swapmoe_forward", "swapmoe_forward_timed", "swapmoe_forward_from_logits", "swapmoe_forward_host",
     "swapmoe_read_importance", "swapmoe_topk_importance", "swapmoe_load_slot_async",
     "swapmoe_debug_copy", "swapmoe_device_status", "swapmoe_launch_count",
     "swapmoe_workspace_bytes", "swapmoe_set_gemm_path", "swapmoe_status_string",
@@ -62,6 +64,7 @@ def lib() -> ctypes.CDLL:
         L.swapmoe_set_router.argtypes = [vp, vp, vp, vp]
         L.swapmoe_set_resident.argtypes = [vp, vp, vp, vp, vp, vp]
         L.swapmoe_forward.argtypes = [vp, vp, vp, i32, vp]
+        L.swapmoe_forward_timed.argtypes = [vp, vp, vp, i32, vp, ctypes.POINTER(vp)]
         L.swapmoe_forward_from_logits.argtypes = [vp, vp, vp, vp, i32, vp]
         L.swapmoe_forward_host.argtypes = [vp, vp, vp, i32, vp]
         L.swapmoe_read_importance.argtypes = [vp, vp, i32, vp]
@@ -165,6 +168,18 @@ class Layer:
         self.last_T = T
         _check(lib().swapmoe_forward(self._h, x.data_ptr(), out.data_ptr(), T, _stream_ptr(stream)),
                "swapmoe_forward")
+
+    def forward_timed(self, x, out, events, n_tokens: Optional[int] = None, stream=None) -> None:
+        """Like forward, recording the N_STAGES + 1 torch.cuda.Event objects at stage boundaries."""
+        T = int(x.shape[0]) if n_tokens is None else int(n_tokens)
+        self.last_T = T
+        assert len(events) == N_STAGES + 1
+        for e in events:              # torch creates the CUDA event lazily, on its first record
+            if not e.cuda_event:
+                e.record()
+        arr = (ctypes.c_void_p * (N_STAGES + 1))(*[e.cuda_event for e in events])
+        _check(lib().swapmoe_forward_timed(self._h, x.data_ptr(), out.data_ptr(), T,
+                                           _stream_ptr(stream), arr), "swapmoe_forward_timed")
 
     def forward_from_logits(self, x, logits, out, stream=None) -> None:
         T = int(x.shape[0])

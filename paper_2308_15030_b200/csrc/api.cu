@@ -38,6 +38,7 @@ struct swapmoe_layer {
   int64_t launches;
   int32_t gemm_path;
   int32_t rows_pad_max;
+  void* const* stage_events;   // 7 cudaEvent_t of the forward being enqueued, or nullptr
   TcState tc;
 };
 
@@ -62,6 +63,10 @@ __global__ void set_enorm_kernel(const EnormTable t, int E, float* enorm) {
   for (int i = threadIdx.x; i < E; i += blockDim.x) enorm[i] = t.v[i];
 }
 
+inline void mark(swapmoe_layer* L, int i, cudaStream_t st) {
+  if (L->stage_events) cudaEventRecord(static_cast<cudaEvent_t>(L->stage_events[i]), st);
+}
+
 int32_t check_launch() { return cuda_ok(cudaGetLastError()) ? SWAPMOE_OK : SWAPMOE_ERR_CUDA; }
 
 template <typename DT>
@@ -80,6 +85,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   ra.mgate = L->mgate; ra.slot = L->slot; ra.xnorm = L->xnorm; ra.cta_hist = L->cta_hist;
   ra.cta_imp = L->cta_imp;
   ra.T = T; ra.d = c.d_model; ra.E = c.E; ra.k = c.top_k; ra.K = c.K; ra.renorm = c.renorm_topk;
+  mark(L, 0, st);
   router_gate_kernel<DT><<<n_cta, 256, router_smem_bytes(c.E), st>>>(ra);
   L->launches++;
 
@@ -88,6 +94,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   sa.cta_base = L->cta_base; sa.count = L->count; sa.offset = L->offset;
   sa.pad_offset = L->pad_offset; sa.tiles = L->tiles; sa.n_tiles = L->n_tiles; sa.imp = L->imp;
   sa.n_cta = n_cta; sa.K = c.K; sa.E = c.E; sa.tile_rows = tile_rows;
+  mark(L, 1, st);
   scan_reduce_kernel<<<1, 1024, 0, st>>>(sa);
   L->launches++;
 
@@ -95,12 +102,15 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   pa.x = x; pa.slot = L->slot; pa.cta_base = L->cta_base; pa.offset = L->offset;
   pa.pad_offset = L->pad_offset; pa.perm = L->perm; pa.inv = L->inv; pa.inv_pad = L->inv_pad;
   pa.xp = L->xp; pa.T = T; pa.d = c.d_model; pa.k = c.top_k; pa.K = c.K;
+  mark(L, 2, st);
   permute_gather_kernel<DT><<<n_cta, 256, 0, st>>>(pa);
   L->launches++;
 
+  mark(L, 3, st);
   if (use_tc) {
+    cudaEvent_t mid = L->stage_events ? static_cast<cudaEvent_t>(L->stage_events[4]) : nullptr;
     const int32_t rc = tc_ffn(L->tc, c, L->xp, L->h, L->y, L->tiles, L->n_tiles, max_tiles,
-                              L->status, st, &L->launches);
+                              L->status, st, &L->launches, mid);
     if (rc != SWAPMOE_OK) return rc;
   } else {
     SimtGemmArgs g1;
@@ -114,6 +124,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     else
       gemm_simt_kernel<DT, DT, DT, kEpiRelu><<<grid1, 256, 0, st>>>(g1);
     L->launches++;
+    mark(L, 4, st);
     SimtGemmArgs g2;
     g2.A = L->h; g2.W = L->arena_out; g2.C = L->y; g2.tiles = L->tiles; g2.n_tiles = L->n_tiles;
     g2.slot_stride = (long long)c.d_ff * c.d_model;
@@ -128,8 +139,10 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   ca.y = L->y; ca.inv_pad = L->inv_pad; ca.mgate = L->mgate; ca.out = out;
   ca.T = T; ca.d = c.d_model; ca.k = c.top_k;
   const long long work = (long long)T * (c.d_model / 8);
+  mark(L, 5, st);
   combine_kernel<DT><<<(unsigned)((work + 255) / 256), 256, 0, st>>>(ca);
   L->launches++;
+  mark(L, 6, st);
   return check_launch();
 }
 
@@ -293,6 +306,17 @@ int32_t swapmoe_set_resident(swapmoe_layer_t* L, const int32_t* s2e, const int32
 
 int32_t swapmoe_forward(swapmoe_layer_t* L, const void* x, void* out, int32_t T, void* stream) {
   return forward_checked(L, x, nullptr, out, T, stream);
+}
+
+int32_t swapmoe_forward_timed(swapmoe_layer_t* L, const void* x, void* out, int32_t T, void* stream,
+                              void* const* events) {
+  if (!L || !events) return SWAPMOE_ERR_INVALID_ARG;
+  for (int i = 0; i < SWAPMOE_N_STAGES + 1; ++i)
+    if (!events[i]) return SWAPMOE_ERR_INVALID_ARG;
+  L->stage_events = events;
+  const int32_t rc = forward_checked(L, x, nullptr, out, T, stream);
+  L->stage_events = nullptr;
+  return rc;
 }
 
 int32_t swapmoe_forward_from_logits(swapmoe_layer_t* L, const void* x, const float* logits, void* out,

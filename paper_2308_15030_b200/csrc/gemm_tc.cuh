@@ -426,7 +426,8 @@ inline int32_t tc_bind_arena(TcState& s, const swapmoe_config_t& c, const void* 
 }
 
 inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* /*xp*/, void* h, float* y, const TileDesc* tiles,
-                      const int32_t* n_tiles, int max_tiles, int32_t* status, cudaStream_t st, int64_t* launches) {
+                      const int32_t* n_tiles, int max_tiles, int32_t* status, cudaStream_t st, int64_t* launches,
+                      cudaEvent_t between = nullptr) {
   if (!s.enabled || !s.arena_bound) return SWAPMOE_ERR_NOT_READY;
   const bool swiglu = c.act == SWAPMOE_ACT_SWIGLU;
   TcGemmArgs g1;
@@ -442,6 +443,7 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* /*xp*/, void*
   else
     tc_gemm_kernel<256, kTcEpiReluBf16><<<grid, kTcThreads, TcSmem<256>::kBytes, st>>>(s.map_xp, s.map_win, g1);
   ++*launches;
+  if (between) cudaEventRecord(between, st);
 
   TcGemmArgs g2;
   g2.C = y; g2.tiles = tiles; g2.n_tiles = n_tiles; g2.status = status; g2.ldc = c.d_model;
