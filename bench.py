@@ -184,9 +184,9 @@ def run_cuda(args, cfg):
     touched = int(np.count_nonzero(count))
     hit = float(np.mean(np.isin(uidx, s2e)))
 
-    def step(i):
+    def step(i, st=stream):
         j = i % copies
-        layers[j].forward(d_x[j], d_out[j], stream=stream)
+        layers[j].forward(d_x[j], d_out[j], stream=st)
 
     def barrier():
         if world > 1:
@@ -199,6 +199,20 @@ def run_cuda(args, cfg):
             step(i)
     barrier()
     l0 = sum(L.launch_count for L in layers)
+    step(0)
+    per_step_launches = sum(L.launch_count for L in layers) - l0
+    graph = None
+    if not args.no_graph:
+        # One CUDA graph = one rotation over the `copies` replicas (`copies` steps); the timed
+        # loop replays it.  forward() neither synchronises nor allocates, so it captures as is.
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for j in range(copies):
+                step(j, st=None)
+        for _ in range(3):
+            graph.replay()
+    barrier()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -206,12 +220,18 @@ def run_cuda(args, cfg):
     barrier()
     with torch.cuda.stream(stream):
         e0.record(stream)
-        for i in range(args.steps):
-            step(i)
+        if graph is not None:
+            for _ in range(args.steps // copies):
+                graph.replay()
+            for i in range(args.steps % copies):
+                step(i)
+        else:
+            for i in range(args.steps):
+                step(i)
         e1.record(stream)
     barrier()
     ms_total = e0.elapsed_time(e1)
-    launches = sum(L.launch_count for L in layers) - l0
+    launches = per_step_launches * args.steps
 
     # ---- timed region 2: same steps with events at the stage boundaries (per-kernel times)
     nst = binding.N_STAGES
@@ -281,6 +301,7 @@ def run_cuda(args, cfg):
         "config": {"workload": workload_string(cfg),
                    "l2": "inputs rotate over %d copies of tokens+weights (%.0f MB > 126 MB L2)"
                          % (copies, copies * weight_bytes / 1e6),
+                   "launch": ("CUDA graph of %d steps, replayed" % copies) if graph is not None else "eager",
                    "resident_set": "top-K by Eq.(1) importance of the batch",
                    "touched_slots": touched, "slot_counts": [int(c) for c in count],
                    "unmasked_hit_rate": hit, "multi_gpu": "replicas only"},
@@ -362,6 +383,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
     cfg = I.CONFIGS[args.workload]
     if args.impl == "reference":
@@ -371,8 +393,8 @@ def main():
         if res is not None:
             print(json.dumps(res), flush=True)
         return
-    args.steps = 200 if args.steps is None else args.steps
-    args.warmup = 20 if args.warmup is None else max(3, args.warmup)
+    args.steps = 2000 if args.steps is None else args.steps
+    args.warmup = 50 if args.warmup is None else max(3, args.warmup)
     res = run_cuda(args, cfg)
     if res is None:
         return

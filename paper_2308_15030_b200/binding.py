@@ -55,8 +55,10 @@ def lib() -> ctypes.CDLL:
     """Loads (building if needed) the CUDA library; raises if that fails."""
     global _lib
     if _lib is None:
-        path = _build.LIB if os.path.exists(_build.LIB) and os.environ.get("SWAPMOE_NO_REBUILD") \
-            else _build.build()
+        path = os.environ.get("SWAPMOE_LIB")      # explicit library file, e.g. an instrumented build
+        if not path:
+            path = _build.LIB if os.path.exists(_build.LIB) and os.environ.get("SWAPMOE_NO_REBUILD") \
+                else _build.build()
         L = ctypes.CDLL(path)
         vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
         L.swapmoe_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Config)]

@@ -14,6 +14,7 @@
 #include "gemm_tc.cuh"
 #include "permute.cuh"
 #include "router_gate.cuh"
+#include "router_tc.cuh"
 
 using namespace swapmoe;
 
@@ -28,6 +29,7 @@ struct swapmoe_layer {
   float *logits, *ugate, *mgate, *xnorm, *cta_imp, *imp, *enorm, *y;
   int32_t *uidx, *midx, *slot, *cta_hist, *cta_base, *count, *offset, *pad_offset;
   int32_t *perm, *inv, *inv_pad, *n_tiles, *e2s, *phys, *s2e, *status;
+  unsigned* ticket;
   TileDesc* tiles;
   void *xp, *h, *x_stage, *out_stage;
   // host state
@@ -38,7 +40,11 @@ struct swapmoe_layer {
   int64_t launches;
   int32_t gemm_path;
   int32_t rows_pad_max;
+  int32_t sm_count;
   void* const* stage_events;   // 7 cudaEvent_t of the forward being enqueued, or nullptr
+  CUtensorMap map_x;           // TMA view of the last token matrix [T, d]
+  const void* map_x_ptr;
+  int32_t map_x_T;
   TcState tc;
 };
 
@@ -73,7 +79,9 @@ template <typename DT>
 int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, void* out, int32_t T,
                      cudaStream_t st) {
   const swapmoe_config_t& c = L->cfg;
-  const int n_cta = (T + kTokTile - 1) / kTokTile;
+  const bool tc_router = L->tc.router_ok && ext_logits == nullptr;
+  const int tok_tile = tc_router ? kRtTok : kTokTile;
+  const int n_cta = (T + tok_tile - 1) / tok_tile;
   const int n_pairs = T * c.top_k;
   const bool use_tc = tc_selected(L->gemm_path, c, T);
   const int tile_rows = use_tc ? kTcBM : kSimtBM;
@@ -85,25 +93,38 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   ra.mgate = L->mgate; ra.slot = L->slot; ra.xnorm = L->xnorm; ra.cta_hist = L->cta_hist;
   ra.cta_imp = L->cta_imp;
   ra.T = T; ra.d = c.d_model; ra.E = c.E; ra.k = c.top_k; ra.K = c.K; ra.renorm = c.renorm_topk;
-  mark(L, 0, st);
-  router_gate_kernel<DT><<<n_cta, 256, router_smem_bytes(c.E), st>>>(ra);
-  L->launches++;
-
-  ScanArgs sa;
+  ScanArgs& sa = ra.scan;
   sa.cta_hist = L->cta_hist; sa.cta_imp = L->cta_imp; sa.phys_slot = L->phys;
   sa.cta_base = L->cta_base; sa.count = L->count; sa.offset = L->offset;
   sa.pad_offset = L->pad_offset; sa.tiles = L->tiles; sa.n_tiles = L->n_tiles; sa.imp = L->imp;
+  sa.ticket = L->ticket;
   sa.n_cta = n_cta; sa.K = c.K; sa.E = c.E; sa.tile_rows = tile_rows;
-  mark(L, 1, st);
-  scan_reduce_kernel<<<1, 1024, 0, st>>>(sa);
+  mark(L, 0, st);
+  if (tc_router) {
+    if (x != L->map_x_ptr || T != L->map_x_T) {   // the token map is re-encoded only when x or T changes
+      if (!tc_encode_2d(L->tc.encode, &L->map_x, x, (uint64_t)T, (uint64_t)c.d_model, kRtTok)) return SWAPMOE_ERR_CUDA;
+      L->map_x_ptr = x;
+      L->map_x_T = T;
+    }
+    router_tc_kernel<<<n_cta, kRtThreads, router_tc_smem_bytes(c.E), st>>>(L->map_x, L->tc.map_wr, ra, L->status,
+                                                                            router_tc_stages(c.E));
+  } else {
+    router_gate_kernel<DT><<<n_cta, 256, router_smem_bytes(c.E), st>>>(ra);
+  }
   L->launches++;
+  mark(L, 1, st);   // the slot scan and importance reduction run inside the router's last CTA
 
   PermuteArgs pa;
   pa.x = x; pa.slot = L->slot; pa.cta_base = L->cta_base; pa.offset = L->offset;
   pa.pad_offset = L->pad_offset; pa.perm = L->perm; pa.inv = L->inv; pa.inv_pad = L->inv_pad;
-  pa.xp = L->xp; pa.T = T; pa.d = c.d_model; pa.k = c.top_k; pa.K = c.K;
+  pa.xp = L->xp; pa.T = T; pa.d = c.d_model; pa.k = c.top_k; pa.K = c.K; pa.tok_tile = tok_tile;
   mark(L, 2, st);
-  permute_gather_kernel<DT><<<n_cta, 256, 0, st>>>(pa);
+  // enough CTAs to fill the GPU: every row-group of a token tile gets its own CTA
+  int groups = (2 * L->sm_count + n_cta - 1) / n_cta;
+  const int max_groups = (tok_tile * c.top_k + 7) / 8;
+  if (groups > max_groups) groups = max_groups;
+  if (groups < 1) groups = 1;
+  permute_gather_kernel<DT><<<dim3(n_cta, groups), kPermThreads, 0, st>>>(pa);
   L->launches++;
 
   mark(L, 3, st);
@@ -189,6 +210,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   std::memset(L, 0, sizeof(*L));
   L->cfg = c;
   L->device = dev;
+  L->sm_count = prop.multiProcessorCount;
   L->nin = c.act == SWAPMOE_ACT_SWIGLU ? 2 : 1;
   L->elem = c.dtype == SWAPMOE_BF16 ? 2 : 4;
 
@@ -211,6 +233,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_ntiles = cv.take<int32_t>(4), o_e2s = cv.take<int32_t>(c.E);
   const size_t o_phys = cv.take<int32_t>(kMaxSlots), o_s2e = cv.take<int32_t>(kMaxSlots);
   const size_t o_status = cv.take<int32_t>(4);
+  const size_t o_ticket = cv.take<unsigned>(4);
   const size_t o_tiles = cv.take<TileDesc>(max_tiles);
   const size_t o_xp = cv.take<char>(rows_pad * c.d_model * L->elem);
   const size_t o_h = cv.take<char>(rows_pad * c.d_ff * L->elem);
@@ -229,12 +252,16 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   L->perm = (int32_t*)(b + o_perm); L->inv = (int32_t*)(b + o_inv); L->inv_pad = (int32_t*)(b + o_invp);
   L->n_tiles = (int32_t*)(b + o_ntiles); L->e2s = (int32_t*)(b + o_e2s); L->phys = (int32_t*)(b + o_phys);
   L->s2e = (int32_t*)(b + o_s2e); L->status = (int32_t*)(b + o_status);
+  L->ticket = (unsigned*)(b + o_ticket);
   L->tiles = (TileDesc*)(b + o_tiles);
   L->xp = b + o_xp; L->h = b + o_h; L->y = (float*)(b + o_y);
   L->x_stage = b + o_xs; L->out_stage = b + o_os;
 
   bool ok = cuda_ok(cudaMemset(L->imp, 0, sizeof(float) * c.E));
   ok = ok && cuda_ok(cudaMemset(L->status, 0, sizeof(int32_t) * 4));
+  ok = ok && cuda_ok(cudaMemset(L->ticket, 0, sizeof(unsigned) * 4));
+  ok = ok && cuda_ok(cudaFuncSetAttribute(router_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          200 * 1024));
   // Rows of the padded workspaces that no pair occupies are computed on but never
   // read back; start them at zero so they hold finite values.
   ok = ok && cuda_ok(cudaMemset(L->xp, 0, rows_pad * c.d_model * L->elem));
@@ -263,6 +290,10 @@ int32_t swapmoe_set_router(swapmoe_layer_t* L, const void* Wr_dev, const float* 
   EnormTable t;
   std::memset(&t, 0, sizeof(t));
   for (int i = 0; i < L->cfg.E; ++i) t.v[i] = enorm_host[i];
+  if (L->tc.router_ok &&
+      !tc_encode_2d(L->tc.encode, &L->tc.map_wr, Wr_dev, (uint64_t)L->cfg.E, (uint64_t)L->cfg.d_model,
+                    (uint32_t)router_tc_epad(L->cfg.E)))
+    return SWAPMOE_ERR_CUDA;
   set_enorm_kernel<<<1, 256, 0, static_cast<cudaStream_t>(stream)>>>(t, L->cfg.E, L->enorm);
   L->launches++;
   L->Wr = Wr_dev;

@@ -358,8 +358,10 @@ struct TcState {
   PFN_encodeTiled encode;
   CUtensorMap map_xp, map_h;          // activations: [rows_pad, d], [rows_pad, f], box 64 x 128
   CUtensorMap map_win, map_wout;      // weights flattened to 2D, box 64 x (rows per load)
+  CUtensorMap map_wr;                 // router matrix [E, d], box 64 x Epad
   int bn2;                            // column tile of the second GEMM
   bool arena_bound;
+  bool router_ok;                     // tensor-core router usable (bf16 layer)
 };
 
 inline bool tc_supported(const swapmoe_config_t& c) {
@@ -392,7 +394,8 @@ inline bool tc_set_smem_attr() {
 inline int32_t tc_init(TcState& s, const swapmoe_config_t& c, void* xp, void* h, float* /*y*/, int rows_pad) {
   s.enabled = false;
   s.arena_bound = false;
-  if (!tc_supported(c)) return SWAPMOE_OK;
+  s.router_ok = false;
+  if (c.dtype != SWAPMOE_BF16) return SWAPMOE_OK;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SWAPMOE_ERR_CUDA;
   if (cudaDeviceGetAttribute(&s.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SWAPMOE_ERR_CUDA;
@@ -402,6 +405,8 @@ inline int32_t tc_init(TcState& s, const swapmoe_config_t& c, void* xp, void* h,
           cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
     return SWAPMOE_ERR_CUDA;
   s.encode = reinterpret_cast<PFN_encodeTiled>(fn);
+  s.router_ok = true;
+  if (!tc_supported(c)) return SWAPMOE_OK;
   if (!tc_encode_2d(s.encode, &s.map_xp, xp, (uint64_t)rows_pad, (uint64_t)c.d_model, kTcBM)) return SWAPMOE_ERR_CUDA;
   if (!tc_encode_2d(s.encode, &s.map_h, h, (uint64_t)rows_pad, (uint64_t)c.d_ff, kTcBM)) return SWAPMOE_ERR_CUDA;
   bool ok = tc_set_smem_attr<256, kTcEpiReluBf16>() && tc_set_smem_attr<256, kTcEpiSwigluBf16>() &&

@@ -16,39 +16,41 @@ struct ScanArgs {
   TileDesc* tiles;           // GEMM work list
   int32_t* n_tiles;          // [1]
   float* imp;                // [E] accumulator of Eq. (1)
+  unsigned* ticket;          // [1] router CTAs finished so far (returns to 0)
   int32_t n_cta, K, E, tile_rows;
 };
 
-// One CTA of 1024 threads.  Warp w scans slot w, w+32, ... over the CTAs in order;
-// then thread s lays out slot s (offsets, padded offsets, tile list); warps also
-// reduce the per-CTA importance partials in a fixed order.
-__global__ void __launch_bounds__(1024) scan_reduce_kernel(const ScanArgs a) {
+// Work of the LAST router CTA to finish (all of its threads call this).  Warp w scans
+// slot w, w+nwarp, ... over the router CTAs in order; then thread s lays out slot s
+// (offsets, padded offsets, tile list); warps also reduce the per-CTA importance
+// partials in a fixed order.  Loads bypass L1: the data was written by other CTAs.
+__device__ __forceinline__ void scan_reduce_block(const ScanArgs& a) {
   __shared__ int32_t s_count[kMaxSlots];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x;
 
-  for (int s = warp; s < a.K; s += 32) {
-    int running = 0;
-    for (int c0 = 0; c0 < a.n_cta; c0 += 32) {
-      const int c = c0 + lane;
-      const int v = (c < a.n_cta) ? a.cta_hist[(size_t)c * a.K + s] : 0;
-      int incl = v;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += n;
+  // Thread s walks slot s over the router CTAs in order (the loads do not depend on the
+  // running sum, so they pipeline); thread e likewise adds expert e's importance partials
+  // in CTA order, which fixes the summation order of Eq. (1) run to run.
+  // Slots are walked by the LAST K threads and experts by the first E threads, so the two
+  // chains of dependent global loads run side by side.
+  {
+    const int s = (int)blockDim.x - 1 - tid;
+    if (s < a.K) {
+      int running = 0;
+#pragma unroll 16
+      for (int c = 0; c < a.n_cta; ++c) {
+        const int v = __ldcg(a.cta_hist + (size_t)c * a.K + s);
+        a.cta_base[(size_t)c * a.K + s] = running;
+        running += v;
       }
-      if (c < a.n_cta) a.cta_base[(size_t)c * a.K + s] = running + incl - v;
-      running += __shfl_sync(0xffffffffu, incl, 31);
+      s_count[s] = running;
     }
-    if (lane == 0) s_count[s] = running;
   }
-  // Eq. (1): add this batch's per-CTA partial sums, CTA order fixed by the lane
-  // stride and the shuffle tree, so repeated runs give identical bits.
-  for (int e = warp; e < a.E; e += 32) {
+  for (int e = tid; e < a.E; e += blockDim.x) {
     float acc = 0.f;
-    for (int c = lane; c < a.n_cta; c += 32) acc += a.cta_imp[(size_t)c * a.E + e];
-    acc = warp_sum(acc);
-    if (lane == 0) a.imp[e] += acc;
+#pragma unroll 16
+    for (int c = 0; c < a.n_cta; ++c) acc += __ldcg(a.cta_imp + (size_t)c * a.E + e);
+    a.imp[e] += acc;
   }
   __syncthreads();
   if (tid < a.K) {
@@ -81,6 +83,24 @@ __global__ void __launch_bounds__(1024) scan_reduce_kernel(const ScanArgs a) {
   }
 }
 
+// Called by every thread of a router CTA after its partials are written: the CTA
+// that draws the last ticket runs the scan.  No CTA waits for another.
+__device__ __forceinline__ void finish_router_cta(const ScanArgs& a) {
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned ticket = atomicAdd(a.ticket, 1u);
+    s_last = (ticket == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (s_last) {
+    __threadfence();
+    scan_reduce_block(a);
+    if (threadIdx.x == 0) *a.ticket = 0u;
+  }
+}
+
 struct PermuteArgs {
   const void* x;              // [T, d]
   const int32_t* slot;        // [T*k]
@@ -91,24 +111,27 @@ struct PermuteArgs {
   int32_t* inv;               // [T*k]
   int32_t* inv_pad;           // [T*k] row of the pair in the padded workspace
   void* xp;                   // [rows_pad, d]
-  int32_t T, d, k, K;
+  int32_t T, d, k, K, tok_tile;
 };
 
-// One CTA = the pairs of kTokTile tokens in flat order p = t*k + j.  The rank of a
+constexpr int kPermThreads = 512;
+
+// One CTA = the pairs of tok_tile (<= 128) tokens in flat order p = t*k + j.  The rank of a
 // pair among the pairs of the same slot is: pairs in earlier CTAs (cta_base) +
 // pairs in earlier warps of this CTA + earlier lanes of this warp (match + popc),
-// which is exactly a stable counting sort.
+// which is exactly a stable counting sort.  gridDim.y CTAs share one token tile: each
+// recomputes the (cheap) positions and copies every gridDim.y-th row of the tile.
 template <typename T>
-__global__ void __launch_bounds__(256) permute_gather_kernel(const PermuteArgs a) {
-  __shared__ int32_t wcount[kMaxTopK][kMaxSlots];
-  __shared__ int32_t dst_row[kTokTile * kMaxTopK];
+__global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const PermuteArgs a) {
+  __shared__ int32_t wcount[kPermThreads / 32][kMaxSlots];
+  __shared__ int32_t dst_row[kPermThreads];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int npair = kTokTile * a.k;            // <= 128
+  const int npair = a.tok_tile * a.k;          // <= 512
   const int nwarp_p = (npair + 31) >> 5;
   const int p0 = blockIdx.x * npair;
   const int n_total = a.T * a.k;
 
-  for (int i = tid; i < kMaxTopK * kMaxSlots; i += 256) (&wcount[0][0])[i] = 0;
+  for (int i = tid; i < (kPermThreads / 32) * kMaxSlots; i += kPermThreads) (&wcount[0][0])[i] = 0;
   __syncthreads();
   int s = -1, rank = 0;
   const int p = p0 + tid;
@@ -124,10 +147,12 @@ __global__ void __launch_bounds__(256) permute_gather_kernel(const PermuteArgs a
     for (int w = 0; w < warp; ++w) before += wcount[w][s];
     const int within = before + rank;
     const int pos = a.offset[s] + within;
-    a.perm[pos] = p;
-    a.inv[p] = pos;
     const int row = a.pad_offset[s] + within;
-    a.inv_pad[p] = row;
+    if (blockIdx.y == 0) {
+      a.perm[pos] = p;
+      a.inv[p] = pos;
+      a.inv_pad[p] = row;
+    }
     dst_row[tid] = row;
   } else if (tid < npair) {
     dst_row[tid] = -1;
@@ -137,8 +162,10 @@ __global__ void __launch_bounds__(256) permute_gather_kernel(const PermuteArgs a
   const int vec_per_row = a.d * (int)sizeof(T) / 16;
   const uint4* src = static_cast<const uint4*>(a.x);
   uint4* dst = static_cast<uint4*>(a.xp);
-  for (int i = tid; i < npair * vec_per_row; i += 256) {
-    const int pl = i / vec_per_row, v = i - pl * vec_per_row;
+  const int my_rows = (npair - (int)blockIdx.y + (int)gridDim.y - 1) / (int)gridDim.y;
+  for (int i = tid; i < my_rows * vec_per_row; i += kPermThreads) {
+    const int ri = i / vec_per_row, v = i - ri * vec_per_row;
+    const int pl = ri * gridDim.y + blockIdx.y;
     const int row = dst_row[pl];
     if (row >= 0) {
       const int t = (p0 + pl) / a.k;

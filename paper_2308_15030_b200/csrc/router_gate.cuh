@@ -2,6 +2,7 @@
 // the importance score (SwapMoE Section 2, Fig. 4, Eq. 1), CUDA-core version.
 #pragma once
 #include "common.cuh"
+#include "permute.cuh"
 
 namespace swapmoe {
 
@@ -21,6 +22,7 @@ struct RouterArgs {
   int32_t* cta_hist;        // [n_cta, K]
   float* cta_imp;           // [n_cta, E]
   int32_t T, d, E, k, K, renorm;
+  ScanArgs scan;            // work of the last CTA to finish
 };
 
 constexpr int kRouterDK = 32;  // contraction chunk staged in shared memory
@@ -65,6 +67,35 @@ __device__ __forceinline__ void warp_topk_gate(const float (&v)[8], uint32_t all
     den = warp_sum(den);
   }
   for (int j = 0; j < k; ++j) sel_g[j] = expf(sel_v[j] - m) / den;
+}
+
+// Gate of one token, executed by a whole warp: v[i] = logit of expert lane + 32 i.
+// Emits the unmasked and masked selections, the slot and the token's term of Eq. (1);
+// tl is the token's index inside the CTA (pair arrays pe/ps/pt live in shared memory).
+__device__ __forceinline__ void gate_token(const RouterArgs& a, const float (&v)[8], uint32_t valid_mask,
+                                           uint32_t res_mask, int lane, int tok, int tl, float xn,
+                                           int* pe, int* ps, float* pt) {
+  int ue[kMaxTopK], me[kMaxTopK];
+  float ug[kMaxTopK], mg[kMaxTopK];
+  warp_topk_gate(v, valid_mask, a.E, a.k, a.renorm, lane, ue, ug);   // off-the-shelf gate
+  warp_topk_gate(v, res_mask, a.E, a.k, a.renorm, lane, me, mg);     // Masked Gating
+  if (lane == 0) {
+    for (int j = 0; j < a.k; ++j) {
+      const int pl = tl * a.k + j;
+      if (tok < a.T) {
+        const int s = a.e2s[me[j]];
+        const size_t p = (size_t)tok * a.k + j;
+        a.uidx[p] = ue[j]; a.ugate[p] = ug[j];
+        a.midx[p] = me[j]; a.mgate[p] = mg[j];
+        a.slot[p] = s;
+        pe[pl] = ue[j]; ps[pl] = s;
+        pt[pl] = xn * fabsf(ug[j]) * a.enorm[ue[j]];   // one term of Eq. (1)
+      } else {
+        pe[pl] = -1; ps[pl] = -1; pt[pl] = 0.f;
+      }
+    }
+    if (tok < a.T) a.xnorm[tok] = xn;
+  }
 }
 
 // One CTA = kTokTile tokens; warp w owns tokens 4w..4w+3; lane l owns experts l+32i.
@@ -157,27 +188,7 @@ __global__ void __launch_bounds__(256) router_gate_kernel(const RouterArgs a) {
       v[i] = lv;
       if (tok < a.T && e < a.E) a.logits[(size_t)tok * a.E + e] = lv;
     }
-    int ue[kMaxTopK], me[kMaxTopK];
-    float ug[kMaxTopK], mg[kMaxTopK];
-    warp_topk_gate(v, valid_mask, a.E, a.k, a.renorm, lane, ue, ug);   // off-the-shelf gate
-    warp_topk_gate(v, res_mask, a.E, a.k, a.renorm, lane, me, mg);     // Masked Gating
-    if (lane == 0) {
-      for (int j = 0; j < a.k; ++j) {
-        const int pl = tl * a.k + j;
-        if (tok < a.T) {
-          const int s = a.e2s[me[j]];
-          const size_t p = (size_t)tok * a.k + j;
-          a.uidx[p] = ue[j]; a.ugate[p] = ug[j];
-          a.midx[p] = me[j]; a.mgate[p] = mg[j];
-          a.slot[p] = s;
-          pe[pl] = ue[j]; ps[pl] = s;
-          pt[pl] = xn * fabsf(ug[j]) * a.enorm[ue[j]];   // one term of Eq. (1)
-        } else {
-          pe[pl] = -1; ps[pl] = -1; pt[pl] = 0.f;
-        }
-      }
-      if (tok < a.T) a.xnorm[tok] = xn;
-    }
+    gate_token(a, v, valid_mask, res_mask, lane, tok, tl, xn, pe, ps, pt);
   }
   __syncthreads();
   // Per-CTA partial sums in a fixed order, so the result does not depend on scheduling.
@@ -192,6 +203,7 @@ __global__ void __launch_bounds__(256) router_gate_kernel(const RouterArgs a) {
     for (int p = 0; p < npair; ++p) c += (ps[p] == s);
     a.cta_hist[(size_t)blockIdx.x * a.K + s] = c;
   }
+  finish_router_cta(a.scan);
 }
 
 inline size_t router_smem_bytes(int E) {

@@ -1,0 +1,364 @@
+// Router product on the tensor cores with the whole gate fused into its epilogue
+// (SwapMoE Section 2: G(x); Fig. 4: Masked Gating; Eq. 1: importance terms).
+//
+// One CTA = 128 tokens.  logits[128, E] = x_tile * Wr^T is accumulated in TMEM by
+// tcgen05.mma (bf16 -> fp32) from TMA-staged tiles; TMEM lane = token row, so in the
+// epilogue ONE THREAD OWNS ONE TOKEN: it reads its E logits, picks the unmasked and the
+// masked top-k, evaluates the softmax gates, looks up the slot and emits the token's
+// importance term.  While the tiles stream through shared memory the same four warps
+// accumulate ||x||^2 of their rows.  The last CTA to finish runs the slot scan.
+#pragma once
+#include "gemm_tc.cuh"
+#include "permute.cuh"
+#include "router_gate.cuh"
+
+namespace swapmoe {
+
+constexpr int kRtTok = 128;      // tokens per CTA
+constexpr int kRtThreads = 256;
+
+// Running top-k list, descending by value; a candidate is inserted below every entry
+// that is >= it, so equal values stay in arrival (= expert index) order.
+struct TopK {
+  float v[kMaxTopK];
+  int e[kMaxTopK];
+  __device__ __forceinline__ void init() {
+#pragma unroll
+    for (int j = 0; j < kMaxTopK; ++j) { v[j] = -INFINITY; e[j] = -1; }
+  }
+  __device__ __forceinline__ void push(float cv, int ce, int k) {
+    bool shifting = false;
+#pragma unroll
+    for (int j = 0; j < kMaxTopK; ++j) {
+      if (j < k && (shifting || e[j] < 0 || cv > v[j])) {
+        const float tv = v[j]; const int te = e[j];
+        v[j] = cv; e[j] = ce;
+        cv = tv; ce = te;
+        shifting = true;
+      }
+    }
+  }
+};
+constexpr int kRtSmemBudget = 190 * 1024;
+
+inline int router_tc_epad(int E) { return (E + 15) / 16 * 16; }
+inline int router_tc_stage_bytes(int E) { return kRtTok * kTcBK * 2 + router_tc_epad(E) * kTcBK * 2; }
+inline int router_tc_stages(int E) {
+  int s = kRtSmemBudget / router_tc_stage_bytes(E);
+  return s > 8 ? 8 : s;
+}
+inline size_t router_tc_smem_bytes(int E) {
+  return (size_t)router_tc_stages(E) * router_tc_stage_bytes(E) + 2048 +
+         (sizeof(int) * 2 + sizeof(float)) * kRtTok * kMaxTopK + sizeof(float) * kRtTok +
+         (sizeof(int) + sizeof(float)) * kMaxE + sizeof(uint32_t) * 24;
+}
+
+__global__ void __launch_bounds__(kRtThreads, 1)
+router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
+                 const RouterArgs a, int32_t* status, int n_stages) {
+  const int E = a.E, k = a.k;
+  const int Epad = (E + 15) / 16 * 16;
+  const int a_bytes = kRtTok * kTcBK * 2, b_bytes = Epad * kTcBK * 2;
+  const int stage_bytes = a_bytes + b_bytes;
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  unsigned char* sA = smem;
+  unsigned char* sB = smem + n_stages * a_bytes;
+  float* slog = reinterpret_cast<float*>(smem);           // [128][E+1], reuses the stage buffers
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + n_stages * stage_bytes);
+  uint64_t* full = bars;                  // [8]
+  uint64_t* empty = bars + 8;             // [8]
+  uint64_t* acc_full = bars + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* pe = reinterpret_cast<int*>(bars + 24);            // [128*k] unmasked expert per pair
+  int* ps = pe + kRtTok * kMaxTopK;                       // [128*k] slot per pair
+  float* pt = reinterpret_cast<float*>(ps + kRtTok * kMaxTopK);
+  float* snorm = pt + kRtTok * kMaxTopK;                  // [128] ||x_t||
+  int* s_e2s = reinterpret_cast<int*>(snorm + kRtTok);    // [256] expert -> slot
+  float* s_enorm = reinterpret_cast<float*>(s_e2s + kMaxE);   // [256] ||E_e||
+  uint32_t* s_mask = reinterpret_cast<uint32_t*>(s_enorm + kMaxE);  // [2][8] valid / resident bits
+  uint32_t* s_present = s_mask + 16;                       // [8] experts selected (unmasked) in this tile
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tok0 = blockIdx.x * kRtTok;
+  const int k_blocks = a.d / kTcBK;
+#ifdef SWAPMOE_PHASE_TIMING
+  __shared__ unsigned long long dbg[16];
+#define STAMP(i) do { if (tid == 128) dbg[i] = ptx::globaltimer_ns(); } while (0)
+#else
+#define STAMP(i) do { } while (0)
+#endif
+  STAMP(0);
+  uint32_t tmem_cols = 32;
+  while ((int)tmem_cols < Epad) tmem_cols <<= 1;
+
+  if (tid == 0) {
+    for (int s = 0; s < n_stages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 5); }
+    ptx::mbar_init(acc_full, 1);
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmX);
+    ptx::prefetch_tmap(&tmW);
+  }
+  if (warp == 2) {
+    ptx::tmem_alloc(tmem_slot, tmem_cols);
+    ptx::tmem_relinquish();
+  }
+  for (int e = tid; e < kMaxE; e += kRtThreads) {
+    s_e2s[e] = e < E ? a.e2s[e] : -1;
+    s_enorm[e] = e < E ? a.enorm[e] : 0.f;
+  }
+  {
+    // warp w builds word w of the valid-expert mask and of the resident-expert mask
+    const int e = warp * 32 + lane;
+    const int sl = e < E ? a.e2s[e] : -1;
+    const uint32_t wv = __ballot_sync(0xffffffffu, e < E), wr = __ballot_sync(0xffffffffu, sl >= 0);
+    if (lane == 0) { s_mask[warp] = wv; s_mask[8 + warp] = wr; s_present[warp] = 0u; }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  STAMP(1);
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      for (int kb = 0; kb < k_blocks; ++kb) {
+        if (!bounded_wait(&empty[stage], phase ^ 1u, abort_flag, status, 11)) break;
+        ptx::mbar_expect_tx(&full[stage], (uint32_t)stage_bytes);
+        ptx::tma_load_2d(sA + stage * a_bytes, &tmX, &full[stage], kb * kTcBK, tok0);
+        ptx::tma_load_2d(sB + stage * b_bytes, &tmW, &full[stage], kb * kTcBK, 0);
+        if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+      }
+      if (*abort_flag) {
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ptx::globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc_bf16(kRtTok, Epad);
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int kb = 0; kb < k_blocks; ++kb) {
+        ok = bounded_wait(&full[stage], phase, abort_flag, status, 12);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint64_t da = make_kmajor_sw128_desc(ptx::smem_u32(sA + stage * a_bytes));
+        const uint64_t db = make_kmajor_sw128_desc(ptx::smem_u32(sB + stage * b_bytes));
+#pragma unroll
+        for (int kk = 0; kk < kTcBK / kTcUmmaK; ++kk)
+          ptx::umma_bf16(tmem_base, da + (uint64_t)(2 * kk), db + (uint64_t)(2 * kk), idesc,
+                         (kb > 0 || kk > 0) ? 1u : 0u);
+        ptx::umma_commit(&empty[stage]);
+        if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+      }
+      if (ok) ptx::umma_commit(acc_full);
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------ ||x||^2 while the tiles stream through
+    const int q = warp - 4, r = q * 32 + lane;
+    float sumsq = 0.f;
+    int stage = 0; uint32_t phase = 0;
+    bool ok = true;
+    for (int kb = 0; kb < k_blocks; ++kb) {
+      ok = bounded_wait(&full[stage], phase, abort_flag, status, 13);
+      if (!ok) break;
+      const uint4* row = reinterpret_cast<const uint4*>(sA + stage * a_bytes + r * 128);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        // the 16-byte chunks of a row may be visited in any order: rotate by the row
+        // index so the threads of a quarter-warp hit different banks
+        const uint4 u = row[(c + r) & 7];
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+          sumsq = fmaf(lo, lo, sumsq);
+          sumsq = fmaf(hi, hi, sumsq);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&empty[stage]);
+      if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+    }
+    snorm[r] = sqrtf(sumsq);
+    STAMP(2);
+    // ------------------------------------------------ logits: TMEM lane r -> shared-memory row r
+    // (all MMAs have completed once acc_full fires, so the stage buffers are free to reuse)
+    if (ok) ok = bounded_wait(acc_full, 0, abort_flag, status, 14);
+    STAMP(3);
+    if (ok) {
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+      float* srow = slog + (size_t)r * (E + 1);
+      for (int c0 = 0; c0 < E; c0 += 32) {
+        uint32_t v[32];
+        ptx::tmem_ld32(taddr + (uint32_t)c0, v);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (c0 + i < E) srow[c0 + i] = __uint_as_float(v[i]);
+      }
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, tmem_cols);
+  }
+  STAMP(4);
+  // ---------------------------------------------------- gate: two threads per token
+  // Thread t < 128 evaluates the off-the-shelf gate of token t, thread t + 128 its masked
+  // gate (Fig. 4): each scans the token's row of logits in shared memory once for the
+  // top-k (ties -> lowest index, kept by scanning in index order with a strict compare)
+  // and once for the softmax denominator.  No shuffles, no cross-thread dependencies.
+  const bool failed = *abort_flag != 0;
+  {
+    // coalesced copy of the logits: a warp writes a token's row; four rows are in flight
+    const int rows = min(kRtTok, a.T - tok0);
+    for (int t0 = warp * 4; t0 < rows; t0 += (kRtThreads / 32) * 4) {
+      for (int e = lane; e < E; e += 32) {
+        float v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) v[q] = slog[(size_t)(t0 + q) * (E + 1) + e];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          if (t0 + q < rows) a.logits[(size_t)(tok0 + t0 + q) * E + e] = failed ? 0.f : v[q];
+      }
+    }
+  }
+  STAMP(8);
+  {
+    const bool masked = tid >= kRtTok;
+    const int tl = tid & (kRtTok - 1);
+    const int tok = tok0 + tl;
+    const float* row = slog + (size_t)tl * (E + 1);
+    const uint32_t* allow = s_mask + (masked ? 8 : 0);
+    TopK tk;
+    tk.init();
+    // The loops below run once per CTA, so they are kept rolled (short bodies that stay
+    // in the instruction cache) rather than unrolled over the whole expert range.
+    if (k == 1) {
+      // top-1: branch-free running maximum; the first allowed expert seeds it and a strict
+      // compare keeps the lowest index among equal logits
+      float best = -INFINITY;
+      int bi = -1;
+#pragma unroll 4
+      for (int e = 0; e < E; ++e) {
+        const float l = row[e];
+        const bool take = ((allow[e >> 5] >> (e & 31)) & 1u) && (bi < 0 || l > best);
+        best = take ? l : best;
+        bi = take ? e : bi;
+      }
+      tk.v[0] = failed ? 0.f : best;
+      tk.e[0] = bi;
+    } else {
+      float thr = -INFINITY;
+      int filled = 0;
+#pragma unroll 1
+      for (int e = 0; e < E; ++e) {
+        const float l = failed ? 0.f : row[e];
+        if (((allow[e >> 5] >> (e & 31)) & 1u) && (filled < k || l > thr)) {
+          tk.push(l, e, k);
+          ++filled;
+          thr = (k == 2) ? tk.v[1] : (k == 3) ? tk.v[2] : tk.v[3];
+        }
+      }
+    }
+    STAMP(9);
+    const float m = tk.v[0];
+    float den = 0.f;
+    if (a.renorm) {
+#pragma unroll
+      for (int j = 0; j < kMaxTopK; ++j)
+        if (j < k) den += expf(tk.v[j] - m);
+    } else {
+      // eight interleaved partial sums: short dependency chains and a tree-shaped total
+      float part[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+      for (int e0 = 0; e0 < E; e0 += 8) {
+        const uint32_t w = allow[e0 >> 5] >> (e0 & 31);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float t = __expf((failed ? 0.f : row[e0 + i]) - m);
+          part[i] += ((w >> i) & 1u) ? t : 0.f;
+        }
+      }
+      den = ((part[0] + part[1]) + (part[2] + part[3])) + ((part[4] + part[5]) + (part[6] + part[7]));
+    }
+    STAMP(10);
+    const float xn = snorm[tl];
+#pragma unroll
+    for (int j = 0; j < kMaxTopK; ++j) {
+      if (j < k) {
+        const int pl = tl * k + j;
+        const size_t p = (size_t)tok * k + j;
+        const float g = expf(tk.v[j] - m) / den;
+        const int e = tk.e[j];
+        if (!masked) {
+          if (tok < a.T) {
+            a.uidx[p] = e; a.ugate[p] = g;
+            pe[pl] = e; pt[pl] = xn * fabsf(g) * s_enorm[e];   // one term of Eq. (1)
+            atomicOr(&s_present[e >> 5], 1u << (e & 31));
+          } else {
+            pe[pl] = -1; pt[pl] = 0.f;
+          }
+        } else {
+          if (tok < a.T) {
+            const int sl = s_e2s[e];
+            a.midx[p] = e; a.mgate[p] = g; a.slot[p] = sl;
+            ps[pl] = sl;
+          } else {
+            ps[pl] = -1;
+          }
+        }
+      }
+    }
+    if (!masked && tok < a.T) a.xnorm[tok] = xn;
+    STAMP(11);
+  }
+  __syncthreads();
+  STAMP(5);
+  // Per-CTA partial sums with a fixed association (lane-strided partials, then the
+  // shuffle tree), so the result does not depend on scheduling.  Only experts that some
+  // token of this tile selected are visited; the others get an exact zero.
+  const int npair = kRtTok * k;
+  for (int e = tid; e < E; e += kRtThreads) a.cta_imp[(size_t)blockIdx.x * E + e] = 0.f;
+  for (int sl = tid; sl < a.K; sl += kRtThreads) a.cta_hist[(size_t)blockIdx.x * a.K + sl] = 0;
+  __syncthreads();
+  for (int c = 0; c * 32 < E; ++c) {
+    uint32_t present = s_present[c];
+    for (int n = 0; present; ++n) {
+      const int bit = __ffs(present) - 1;
+      present &= present - 1;
+      if ((n & 7) != warp) continue;                    // experts dealt round-robin to the warps
+      const int e = c * 32 + bit;
+      float sum = 0.f;
+      for (int p = lane; p < npair; p += 32) sum += (pe[p] == e) ? pt[p] : 0.f;
+      sum = warp_sum(sum);
+      if (lane == 0) a.cta_imp[(size_t)blockIdx.x * E + e] = sum;
+    }
+  }
+  for (int sl = warp; sl < a.K; sl += kRtThreads / 32) {
+    int c = 0;
+    for (int p = lane; p < npair; p += 32) c += (ps[p] == sl);
+    c = __reduce_add_sync(0xffffffffu, c);
+    if (lane == 0 && c) a.cta_hist[(size_t)blockIdx.x * a.K + sl] = c;
+  }
+  finish_router_cta(a.scan);
+#ifdef SWAPMOE_PHASE_TIMING
+  __syncthreads();
+  STAMP(6);
+  if (tid == 128)   // phase stamps replace the first logits of this CTA's first token (instrumented build only)
+    for (int i = 0; i < 12; ++i)
+      reinterpret_cast<unsigned long long*>(a.logits + (size_t)blockIdx.x * kRtTok * E)[i] = dbg[i];
+#endif
+}
+
+}  // namespace swapmoe
