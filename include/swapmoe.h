@@ -215,6 +215,53 @@ int64_t swapmoe_workspace_bytes(const swapmoe_layer_t* layer);
  * (bf16 only; UNSUPPORTED otherwise). */
 int32_t swapmoe_set_gemm_path(swapmoe_layer_t* layer, int32_t path);
 
+/*
+ * Routing without any allocation.  (The paper has no counterpart of this call: it
+ * exists for the way some programs have to use a GPU.)
+ *
+ * Who needs it: code that runs where cudaMalloc may not be called - a plug-in
+ * living inside a host application that owns all device memory and forbids
+ * allocations after start-up, a real-time loop that must not take the driver's
+ * allocation lock, or a caller that is already inside a region where the CUDA
+ * runtime refuses to allocate.  Such callers cannot use swapmoe_create(), which
+ * allocates the layer's workspace.  This call runs the router stage alone -
+ * logits = x Wr^T, the unmasked and the masked top-k gate, the slot of every
+ * routed pair, ||x||, the per-slot counts and their exclusive scan, and this
+ * batch's terms of Eq. (1) added into imp_dev - and keeps the few hundred KB of
+ * scratch it needs (per-block histograms and partial sums) in a fixed array that
+ * is part of the library image.  It calls no cudaMalloc / cudaFree and no
+ * allocating library routine.
+ *
+ * The price of the fixed array: every GPU that loads the library holds it
+ * (about 0.4 MB) until the process exits; n_tokens is limited to
+ * SWAPMOE_ROUTE_STATIC_MAX_TOKENS (more -> SWAPMOE_ERR_TOO_MANY_TOKENS, E > 256,
+ * K > 64, top_k > 4 or d_model not a multiple of 64 -> SWAPMOE_ERR_UNSUPPORTED);
+ * and all calls on one GPU share it, so two calls whose kernels may overlap on
+ * the device (different streams, or different host threads) race: issue them
+ * one after the other on one stream.  The array keeps the previous call's
+ * contents; the call itself clears the parts that must start at zero.
+ *
+ * The first call on each device looks up the array's device address (with that
+ * device current); that first call should be made before any stream capture
+ * begins.
+ *
+ * All pointers are device pointers owned by the caller: inputs x_dev
+ * [n_tokens, d_model] and Wr_dev [E, d_model] in `dtype` (16-byte aligned),
+ * expert_to_slot_dev [E] int32 (-1 = not resident; exactly K entries >= 0),
+ * enorm_dev [E] fp32; outputs logits_dev [n_tokens, E] fp32, uidx / midx /
+ * slot [n_tokens, top_k] int32, ugate / mgate [n_tokens, top_k] fp32, xnorm_dev
+ * [n_tokens] fp32, count_dev [K] and offset_dev [K + 1] int32; imp_dev [E] fp32
+ * is accumulated in place (zero it for a fresh score).  Work is enqueued on
+ * `stream`; no host synchronisation.  n_tokens = 0 is a no-op.
+ */
+#define SWAPMOE_ROUTE_STATIC_MAX_TOKENS 8192
+int32_t swapmoe_route_static(const void* x_dev, const void* Wr_dev, const int32_t* expert_to_slot_dev,
+                             const float* enorm_dev, int32_t n_tokens, int32_t d_model, int32_t E,
+                             int32_t top_k, int32_t K, int32_t dtype, int32_t renorm_topk,
+                             float* logits_dev, int32_t* uidx_dev, float* ugate_dev, int32_t* midx_dev,
+                             float* mgate_dev, int32_t* slot_dev, float* xnorm_dev, int32_t* count_dev,
+                             int32_t* offset_dev, float* imp_dev, void* stream);
+
 const char* swapmoe_status_string(int32_t status);
 
 #ifdef __cplusplus

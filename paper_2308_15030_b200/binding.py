@@ -33,6 +33,7 @@ EXPORTS = [
     "swapmoe_read_importance", "swapmoe_topk_importance", "swapmoe_load_slot_async",
     "swapmoe_debug_copy", "swapmoe_device_status", "swapmoe_launch_count",
     "swapmoe_workspace_bytes", "swapmoe_set_gemm_path", "swapmoe_status_string",
+    "swapmoe_route_static",
 ]
 
 
@@ -79,6 +80,7 @@ def lib() -> ctypes.CDLL:
         L.swapmoe_workspace_bytes.argtypes = [vp]
         L.swapmoe_workspace_bytes.restype = i64
         L.swapmoe_set_gemm_path.argtypes = [vp, i32]
+        L.swapmoe_route_static.argtypes = [vp] * 4 + [i32] * 7 + [vp] * 11
         L.swapmoe_status_string.argtypes = [i32]
         L.swapmoe_status_string.restype = ctypes.c_char_p
         for n in EXPORTS:
@@ -116,6 +118,26 @@ def topk_importance(imp: np.ndarray, K: int) -> np.ndarray:
     _check(lib().swapmoe_topk_importance(_np_ptr(imp), imp.size, int(K), _np_ptr(out)),
            "swapmoe_topk_importance")
     return out
+
+
+ROUTE_STATIC_MAX_TOKENS = 8192
+
+
+def route_static(x, Wr, expert_to_slot, enorm, top_k: int, K: int, dtype: int, renorm_topk: int,
+                 logits, uidx, ugate, midx, mgate, slot, xnorm, count, offset, imp, stream=None) -> None:
+    """Router stage through the entry point that allocates nothing.
+
+    For callers that may not allocate device memory (all tensors, outputs included,
+    are the caller's; the library's scratch is a fixed array inside the library).
+    Every argument is a CUDA torch tensor; ``imp`` is accumulated in place.
+    """
+    T, d = int(x.shape[0]), int(x.shape[1])
+    E = int(Wr.shape[0])
+    _check(lib().swapmoe_route_static(
+        x.data_ptr(), Wr.data_ptr(), expert_to_slot.data_ptr(), enorm.data_ptr(), T, d, E, int(top_k),
+        int(K), int(dtype), int(renorm_topk), logits.data_ptr(), uidx.data_ptr(), ugate.data_ptr(),
+        midx.data_ptr(), mgate.data_ptr(), slot.data_ptr(), xnorm.data_ptr(), count.data_ptr(),
+        offset.data_ptr(), imp.data_ptr(), _stream_ptr(stream)), "swapmoe_route_static")
 
 
 class Layer:

@@ -210,14 +210,10 @@ struct SlotTables {
   int32_t phys[kMaxSlots];
   int32_t s2e[kMaxSlots];
 };
-__global__ void set_tables_kernel(const SlotTables t, int E, int K, int32_t* e2s, int32_t* phys,
+static __global__ void set_tables_kernel(const SlotTables t, int E, int K, int32_t* e2s, int32_t* phys,
                                   int32_t* s2e) {
   for (int i = threadIdx.x; i < E; i += blockDim.x) e2s[i] = t.e2s[i];
   for (int i = threadIdx.x; i < K; i += blockDim.x) { phys[i] = t.phys[i]; s2e[i] = t.s2e[i]; }
-}
-
-__global__ void zero_f32_kernel(float* p, int n) {
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) p[i] = 0.f;
 }
 
 }  // namespace swapmoe
