@@ -264,10 +264,8 @@ def run_cuda(args, cfg):
     if any(s[0] != 0 for s in st):
         raise SystemExit("device status error: %r" % (st,))
 
-    times = torch.tensor([ms_total, e2e_s * 1e3], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = float(times[0]), float(times[1])
+    from paper_2308_15030_b200.replicas import max_over_ranks
+    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_s * 1e3], device="cuda")
     if world > 1:
         dist.barrier()
     if rank != 0:

@@ -230,6 +230,8 @@ class Layer:
 
     def load_slot_async(self, phys: int, in_host_pinned, out_host_pinned, side_stream,
                         done_event=None) -> None:
+        if done_event is not None and not done_event.cuda_event:
+            done_event.record(side_stream)      # torch creates the CUDA event on its first record
         ev = None if done_event is None else done_event.cuda_event
         _check(lib().swapmoe_load_slot_async(self._h, int(phys), in_host_pinned.data_ptr(),
                                              out_host_pinned.data_ptr(), _stream_ptr(side_stream),
