@@ -17,7 +17,7 @@ from . import build as _build
 
 F32, BF16 = 0, 1
 N_STAGES = 6
-STAGE_NAMES = ("router_gate", "scan_reduce", "permute_gather", "gemm1_act", "gemm2", "combine")
+STAGE_NAMES = ("router_gate_scan", "(scan: fused into router)", "permute_gather", "gemm1_act", "gemm2", "combine")
 ACT_RELU, ACT_SWIGLU = 0, 1
 
 TAPS = {

@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -28,7 +29,7 @@ struct swapmoe_layer {
   size_t ws_bytes;
   float *logits, *ugate, *mgate, *xnorm, *cta_imp, *imp, *enorm, *y;
   int32_t *uidx, *midx, *slot, *cta_hist, *cta_base, *count, *offset, *pad_offset;
-  int32_t *perm, *inv, *inv_pad, *n_tiles, *e2s, *phys, *s2e, *status;
+  int32_t *perm, *inv, *inv_pad, *row_pair, *n_tiles, *e2s, *phys, *s2e, *status;
   unsigned* ticket;
   TileDesc* tiles;
   void *xp, *h, *x_stage, *out_stage;
@@ -41,6 +42,9 @@ struct swapmoe_layer {
   int32_t gemm_path;
   int32_t rows_pad_max;
   int32_t sm_count;
+  bool use_pdl;                // programmatic dependent launch between the kernels of a forward
+  bool prefetch;               // pull resident weights into L2 from the router kernel
+  long long l2_prefetch_bytes; // how much of them (L2 capacity minus head room)
   void* const* stage_events;   // 7 cudaEvent_t of the forward being enqueued, or nullptr
   CUtensorMap map_x;           // TMA view of the last token matrix [T, d]
   const void* map_x_ptr;
@@ -79,6 +83,7 @@ template <typename DT>
 int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, void* out, int32_t T,
                      cudaStream_t st) {
   const swapmoe_config_t& c = L->cfg;
+  const bool pdl = L->use_pdl && L->stage_events == nullptr;
   const bool tc_router = L->tc.router_ok && ext_logits == nullptr;
   const int tok_tile = tc_router ? kRtTok : kTokTile;
   const int n_cta = (T + tok_tile - 1) / tok_tile;
@@ -99,6 +104,29 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   sa.pad_offset = L->pad_offset; sa.tiles = L->tiles; sa.n_tiles = L->n_tiles; sa.imp = L->imp;
   sa.ticket = L->ticket;
   sa.n_cta = n_cta; sa.K = c.K; sa.E = c.E; sa.tile_rows = tile_rows;
+  ra.pf_base[0] = ra.pf_base[1] = nullptr;
+  ra.pf_slot_bytes[0] = ra.pf_slot_bytes[1] = 16384;
+  ra.pf_total_bytes[0] = ra.pf_total_bytes[1] = 0;
+  ra.pf_phys = L->phys;
+  int pf_ctas = 0;
+  if (tc_router && use_tc && L->prefetch && n_pairs >= 8 * c.K) {
+    // Every slot will most likely be touched: pull the resident weights towards L2 now, while the
+    // router and the permutation leave HBM idle.  GEMM-1's matrices first, then as much of GEMM-2's
+    // as the L2 budget allows.
+    const long long in_slot = (long long)L->nin * c.d_ff * c.d_model * L->elem;
+    const long long out_slot = (long long)c.d_ff * c.d_model * L->elem;
+    const long long budget = L->l2_prefetch_bytes;
+    long long in_total = in_slot * c.K, out_total = out_slot * c.K;
+    if (in_total > budget) in_total = budget / 16384 * 16384;
+    if (out_total > budget - in_total) out_total = (budget - in_total) / 16384 * 16384;
+    ra.pf_base[0] = static_cast<const char*>(L->arena_in);
+    ra.pf_base[1] = static_cast<const char*>(L->arena_out);
+    ra.pf_slot_bytes[0] = in_slot; ra.pf_slot_bytes[1] = out_slot;
+    ra.pf_total_bytes[0] = in_total; ra.pf_total_bytes[1] = out_total;
+    pf_ctas = L->sm_count - n_cta;
+    if (pf_ctas < 0) pf_ctas = 0;
+    if (pf_ctas > 64) pf_ctas = 64;
+  }
   mark(L, 0, st);
   if (tc_router) {
     if (x != L->map_x_ptr || T != L->map_x_T) {   // the token map is re-encoded only when x or T changes
@@ -106,10 +134,13 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
       L->map_x_ptr = x;
       L->map_x_T = T;
     }
-    router_tc_kernel<<<n_cta, kRtThreads, router_tc_smem_bytes(c.E), st>>>(L->map_x, L->tc.map_wr, ra, L->status,
-                                                                            router_tc_stages(c.E));
+    if (launch_kernel(router_tc_kernel, dim3(n_cta + pf_ctas), dim3(kRtThreads), router_tc_smem_bytes(c.E), st, pdl,
+                      L->map_x, L->tc.map_wr, ra, L->status, router_tc_stages(c.E)) != cudaSuccess)
+      return SWAPMOE_ERR_CUDA;
   } else {
-    router_gate_kernel<DT><<<n_cta, 256, router_smem_bytes(c.E), st>>>(ra);
+    if (launch_kernel(router_gate_kernel<DT>, dim3(n_cta), dim3(256), router_smem_bytes(c.E), st, pdl, ra) !=
+        cudaSuccess)
+      return SWAPMOE_ERR_CUDA;
   }
   L->launches++;
   mark(L, 1, st);   // the slot scan and importance reduction run inside the router's last CTA
@@ -117,6 +148,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   PermuteArgs pa;
   pa.x = x; pa.slot = L->slot; pa.cta_base = L->cta_base; pa.offset = L->offset;
   pa.pad_offset = L->pad_offset; pa.perm = L->perm; pa.inv = L->inv; pa.inv_pad = L->inv_pad;
+  pa.row_pair = L->row_pair;
   pa.xp = L->xp; pa.T = T; pa.d = c.d_model; pa.k = c.top_k; pa.K = c.K; pa.tok_tile = tok_tile;
   mark(L, 2, st);
   // enough CTAs to fill the GPU: every row-group of a token tile gets its own CTA
@@ -124,14 +156,17 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   const int max_groups = (tok_tile * c.top_k + 7) / 8;
   if (groups > max_groups) groups = max_groups;
   if (groups < 1) groups = 1;
-  permute_gather_kernel<DT><<<dim3(n_cta, groups), kPermThreads, 0, st>>>(pa);
+  if (launch_kernel(permute_gather_kernel<DT>, dim3(n_cta, groups), dim3(kPermThreads), 0, st, pdl, pa) !=
+      cudaSuccess)
+    return SWAPMOE_ERR_CUDA;
   L->launches++;
 
   mark(L, 3, st);
+  bool combined = false;
   if (use_tc) {
     cudaEvent_t mid = L->stage_events ? static_cast<cudaEvent_t>(L->stage_events[4]) : nullptr;
-    const int32_t rc = tc_ffn(L->tc, c, L->xp, L->h, L->y, L->tiles, L->n_tiles, max_tiles,
-                              L->status, st, &L->launches, mid);
+    const int32_t rc = tc_ffn(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->row_pair, L->mgate, max_tiles,
+                              L->status, st, pdl, &L->launches, &combined, mid);
     if (rc != SWAPMOE_OK) return rc;
   } else {
     SimtGemmArgs g1;
@@ -140,10 +175,12 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     g1.gate_offset = (long long)c.d_ff * c.d_model;
     g1.N = c.d_ff; g1.Kdim = c.d_model;
     const dim3 grid1(c.d_ff / kSimtBN, max_tiles);
+    cudaError_t e;
     if (c.act == SWAPMOE_ACT_SWIGLU)
-      gemm_simt_kernel<DT, DT, DT, kEpiSwiglu><<<grid1, 256, 0, st>>>(g1);
+      e = launch_kernel(gemm_simt_kernel<DT, DT, DT, kEpiSwiglu>, grid1, dim3(256), 0, st, pdl, g1);
     else
-      gemm_simt_kernel<DT, DT, DT, kEpiRelu><<<grid1, 256, 0, st>>>(g1);
+      e = launch_kernel(gemm_simt_kernel<DT, DT, DT, kEpiRelu>, grid1, dim3(256), 0, st, pdl, g1);
+    if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
     L->launches++;
     mark(L, 4, st);
     SimtGemmArgs g2;
@@ -152,7 +189,8 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     g2.gate_offset = 0;
     g2.N = c.d_model; g2.Kdim = c.d_ff;
     const dim3 grid2(c.d_model / kSimtBN, max_tiles);
-    gemm_simt_kernel<DT, DT, float, kEpiNone><<<grid2, 256, 0, st>>>(g2);
+    if (launch_kernel(gemm_simt_kernel<DT, DT, float, kEpiNone>, grid2, dim3(256), 0, st, pdl, g2) != cudaSuccess)
+      return SWAPMOE_ERR_CUDA;
     L->launches++;
   }
 
@@ -161,8 +199,12 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   ca.T = T; ca.d = c.d_model; ca.k = c.top_k;
   const long long work = (long long)T * (c.d_model / 8);
   mark(L, 5, st);
-  combine_kernel<DT><<<(unsigned)((work + 255) / 256), 256, 0, st>>>(ca);
-  L->launches++;
+  if (!combined) {
+    if (launch_kernel(combine_kernel<DT>, dim3((unsigned)((work + 255) / 256)), dim3(256), 0, st, pdl, ca) !=
+        cudaSuccess)
+      return SWAPMOE_ERR_CUDA;
+    L->launches++;
+  }
   mark(L, 6, st);
   return check_launch();
 }
@@ -211,6 +253,19 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   L->cfg = c;
   L->device = dev;
   L->sm_count = prop.multiProcessorCount;
+  {
+    const char* env = std::getenv("SWAPMOE_PDL");      // SWAPMOE_PDL=0 launches every kernel fully serialised
+    L->use_pdl = !(env && env[0] == '0');
+    env = std::getenv("SWAPMOE_PREFETCH");              // SWAPMOE_PREFETCH=0 disables the L2 weight prefetch
+    L->prefetch = !(env && env[0] == '0');
+    // The prefetch must drain while the router runs (about 15 us on 16-64 SMs): what HBM delivers
+    // in that time, and well under the L2 capacity.  Measured on B200: 56 MB hides fully, 76 MB
+    // stretches the router kernel.
+    const long long l2 = prop.l2CacheSize;
+    L->l2_prefetch_bytes = l2 > (80ll << 20) ? (56ll << 20) : 0;
+    env = std::getenv("SWAPMOE_PREFETCH_MB");
+    if (env) L->l2_prefetch_bytes = std::atoll(env) << 20;
+  }
   L->nin = c.act == SWAPMOE_ACT_SWIGLU ? 2 : 1;
   L->elem = c.dtype == SWAPMOE_BF16 ? 2 : 4;
 
@@ -230,6 +285,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_count = cv.take<int32_t>(c.K), o_offset = cv.take<int32_t>(c.K + 1);
   const size_t o_pad = cv.take<int32_t>(c.K + 1);
   const size_t o_perm = cv.take<int32_t>(P), o_inv = cv.take<int32_t>(P), o_invp = cv.take<int32_t>(P);
+  const size_t o_rowpair = cv.take<int32_t>(rows_pad);
   const size_t o_ntiles = cv.take<int32_t>(4), o_e2s = cv.take<int32_t>(c.E);
   const size_t o_phys = cv.take<int32_t>(kMaxSlots), o_s2e = cv.take<int32_t>(kMaxSlots);
   const size_t o_status = cv.take<int32_t>(4);
@@ -250,6 +306,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   L->cta_base = (int32_t*)(b + o_cta_base); L->count = (int32_t*)(b + o_count);
   L->offset = (int32_t*)(b + o_offset); L->pad_offset = (int32_t*)(b + o_pad);
   L->perm = (int32_t*)(b + o_perm); L->inv = (int32_t*)(b + o_inv); L->inv_pad = (int32_t*)(b + o_invp);
+  L->row_pair = (int32_t*)(b + o_rowpair);
   L->n_tiles = (int32_t*)(b + o_ntiles); L->e2s = (int32_t*)(b + o_e2s); L->phys = (int32_t*)(b + o_phys);
   L->s2e = (int32_t*)(b + o_s2e); L->status = (int32_t*)(b + o_status);
   L->ticket = (unsigned*)(b + o_ticket);

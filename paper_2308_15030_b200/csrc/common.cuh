@@ -52,6 +52,13 @@ __device__ __forceinline__ void store8(bf16* p, const float v[8]) {
                                             pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may
+// start while its predecessor is still running; it must execute pdl_wait() before it reads or
+// writes any global memory the predecessors touch.  pdl_trigger() lets the NEXT kernel's
+// blocks be scheduled (they stop at their own pdl_wait()).  Both are no-ops otherwise.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

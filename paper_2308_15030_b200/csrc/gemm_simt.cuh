@@ -25,6 +25,8 @@ enum { kEpiNone = 0, kEpiRelu = 1, kEpiSwiglu = 2 };
 // C[tile rows, 64 cols] = epi(A[tile rows, :] * W[phys][n0:n0+64, :]^T); grid = (N/64, max tiles).
 template <typename TA, typename TW, typename TC, int EPI>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const SimtGemmArgs a) {
+  pdl_wait();
+  pdl_trigger();
   if ((int)blockIdx.y >= *a.n_tiles) return;
   const TileDesc td = a.tiles[blockIdx.y];
   constexpr int LD = kSimtBM + 4;

@@ -24,7 +24,9 @@ constexpr int kTcUmmaK = 16;
 constexpr int kTcThreads = 256;
 constexpr int kTcSmemBudget = 200 * 1024;
 
-enum { kTcEpiReluBf16 = 0, kTcEpiSwigluBf16 = 1, kTcEpiF32 = 2 };
+// Epilogues: ReLU -> bf16 h; silu(a)*b -> bf16 h; plain fp32 y; and, for top-1 layers, the
+// scatter-combine fused in: out[token(row)] = gate(row) * acc, written once per row in bf16.
+enum { kTcEpiReluBf16 = 0, kTcEpiSwigluBf16 = 1, kTcEpiF32 = 2, kTcEpiScatterBf16 = 3 };
 
 struct TcGemmArgs {
   void* C;                  // [rows_pad, ldc]
@@ -36,6 +38,9 @@ struct TcGemmArgs {
   int32_t k_blocks;         // contraction length / 64
   int32_t b_rows_per_phys;  // rows of the flattened weight map per arena entry
   int32_t b_rows_gate;      // row offset of the second input matrix (SwiGLU), else 0
+  const int32_t* row_pair;  // [rows_pad] pair index of each padded row (scatter epilogue)
+  const float* gate;        // [T*k] masked gate values (scatter epilogue)
+  int32_t top_k;
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -216,6 +221,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  pdl_wait();      // the tile list and the operands come from the preceding kernels
+  pdl_trigger();
   const int n_row_tiles = *a.n_tiles;
   const int total = n_row_tiles * a.n_col_tiles;
 
@@ -226,7 +233,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t phase = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
-        const int ct = t / n_row_tiles, rt = t - ct * n_row_tiles;   // row tiles vary fastest
+        const int rt = t / a.n_col_tiles, ct = t - rt * a.n_col_tiles;   // column tiles vary fastest
         const TileDesc td = a.tiles[rt];
         const int brow = td.phys * a.b_rows_per_phys + ct * kBoxRows;
         for (int kb = 0; kb < a.k_blocks; ++kb) {
@@ -286,14 +293,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
-      const int ct = t / n_row_tiles, rt = t - ct * n_row_tiles;
+      const int rt = t / a.n_col_tiles, ct = t - rt * a.n_col_tiles;
       const TileDesc td = a.tiles[rt];
       ok = bounded_wait(&acc_full[acc], acc_phase, abort_flag, a.status, 4);
       if (!ok) break;
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
       const bool row_ok = r < td.rows;
-      const size_t crow = (size_t)(td.row0 + r) * a.ldc + (size_t)ct * kOutCols;
+      size_t crow = (size_t)(td.row0 + r) * a.ldc + (size_t)ct * kOutCols;
+      float gate = 1.f;
+      if (EPI == kTcEpiScatterBf16 && row_ok) {
+        const int p = a.row_pair[td.row0 + r];
+        gate = a.gate[p];
+        crow = (size_t)(p / a.top_k) * a.ldc + (size_t)ct * kOutCols;
+      }
 #pragma unroll 1
       for (int c0 = 0; c0 < kOutCols; c0 += 32) {
         uint32_t v[32];
@@ -326,6 +339,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               for (int j = 0; j < 8; ++j) {
                 f[j] = __uint_as_float(v[8 * i + j]);
                 if (EPI == kTcEpiReluBf16) f[j] = fmaxf(f[j], 0.f);
+                if (EPI == kTcEpiScatterBf16) f[j] *= gate;
               }
               dst[i] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]),
                                   pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
@@ -410,7 +424,8 @@ inline int32_t tc_init(TcState& s, const swapmoe_config_t& c, void* xp, void* h,
   if (!tc_encode_2d(s.encode, &s.map_xp, xp, (uint64_t)rows_pad, (uint64_t)c.d_model, kTcBM)) return SWAPMOE_ERR_CUDA;
   if (!tc_encode_2d(s.encode, &s.map_h, h, (uint64_t)rows_pad, (uint64_t)c.d_ff, kTcBM)) return SWAPMOE_ERR_CUDA;
   bool ok = tc_set_smem_attr<256, kTcEpiReluBf16>() && tc_set_smem_attr<256, kTcEpiSwigluBf16>() &&
-            tc_set_smem_attr<256, kTcEpiF32>() && tc_set_smem_attr<128, kTcEpiF32>();
+            tc_set_smem_attr<256, kTcEpiF32>() && tc_set_smem_attr<128, kTcEpiF32>() &&
+            tc_set_smem_attr<256, kTcEpiScatterBf16>() && tc_set_smem_attr<128, kTcEpiScatterBf16>();
   if (!ok) return SWAPMOE_ERR_CUDA;
   s.bn2 = (c.d_model % 256 == 0 && c.d_model >= 2048) ? 256 : 128;
   s.enabled = true;
@@ -430,8 +445,26 @@ inline int32_t tc_bind_arena(TcState& s, const swapmoe_config_t& c, const void* 
   return SWAPMOE_OK;
 }
 
-inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* /*xp*/, void* h, float* y, const TileDesc* tiles,
-                      const int32_t* n_tiles, int max_tiles, int32_t* status, cudaStream_t st, int64_t* launches,
+// Launch helper: programmatic dependent launch lets the kernel's prologue overlap the tail of
+// the kernel before it on the stream.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                 bool pdl, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// Runs both grouped GEMMs.  With top_k == 1 the second GEMM writes gate * y straight into
+// `out` (*combined = true) and no combine kernel is needed.
+inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, void* out, const TileDesc* tiles,
+                      const int32_t* n_tiles, const int32_t* row_pair, const float* mgate, int max_tiles,
+                      int32_t* status, cudaStream_t st, bool pdl, int64_t* launches, bool* combined,
                       cudaEvent_t between = nullptr) {
   if (!s.enabled || !s.arena_bound) return SWAPMOE_ERR_NOT_READY;
   const bool swiglu = c.act == SWAPMOE_ACT_SWIGLU;
@@ -441,29 +474,51 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* /*xp*/, void*
   g1.k_blocks = c.d_model / kTcBK;
   g1.b_rows_per_phys = swiglu ? 2 * c.d_ff : c.d_ff;
   g1.b_rows_gate = swiglu ? c.d_ff : 0;
+  g1.row_pair = nullptr; g1.gate = nullptr; g1.top_k = c.top_k;
   int grid = max_tiles * g1.n_col_tiles;
   if (grid > s.sm_count) grid = s.sm_count;
+  cudaError_t e;
   if (swiglu)
-    tc_gemm_kernel<256, kTcEpiSwigluBf16><<<grid, kTcThreads, TcSmem<256>::kBytes, st>>>(s.map_xp, s.map_win, g1);
+    e = launch_kernel(tc_gemm_kernel<256, kTcEpiSwigluBf16>, dim3(grid), dim3(kTcThreads), TcSmem<256>::kBytes, st, pdl,
+                      s.map_xp, s.map_win, g1);
   else
-    tc_gemm_kernel<256, kTcEpiReluBf16><<<grid, kTcThreads, TcSmem<256>::kBytes, st>>>(s.map_xp, s.map_win, g1);
+    e = launch_kernel(tc_gemm_kernel<256, kTcEpiReluBf16>, dim3(grid), dim3(kTcThreads), TcSmem<256>::kBytes, st, pdl,
+                      s.map_xp, s.map_win, g1);
+  if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
   ++*launches;
   if (between) cudaEventRecord(between, st);
 
+  const bool scatter = c.top_k == 1;
   TcGemmArgs g2;
-  g2.C = y; g2.tiles = tiles; g2.n_tiles = n_tiles; g2.status = status; g2.ldc = c.d_model;
+  g2.C = scatter ? out : static_cast<void*>(y);
+  g2.tiles = tiles; g2.n_tiles = n_tiles; g2.status = status; g2.ldc = c.d_model;
   g2.n_col_tiles = c.d_model / s.bn2;
   g2.k_blocks = c.d_ff / kTcBK;
   g2.b_rows_per_phys = c.d_model;
   g2.b_rows_gate = 0;
+  g2.row_pair = row_pair; g2.gate = mgate; g2.top_k = c.top_k;
   grid = max_tiles * g2.n_col_tiles;
   if (grid > s.sm_count) grid = s.sm_count;
-  if (s.bn2 == 256)
-    tc_gemm_kernel<256, kTcEpiF32><<<grid, kTcThreads, TcSmem<256>::kBytes, st>>>(s.map_h, s.map_wout, g2);
-  else
-    tc_gemm_kernel<128, kTcEpiF32><<<grid, kTcThreads, TcSmem<128>::kBytes, st>>>(s.map_h, s.map_wout, g2);
+  const bool pdl2 = pdl && between == nullptr;
+  if (s.bn2 == 256) {
+    if (scatter)
+      e = launch_kernel(tc_gemm_kernel<256, kTcEpiScatterBf16>, dim3(grid), dim3(kTcThreads), TcSmem<256>::kBytes, st,
+                        pdl2, s.map_h, s.map_wout, g2);
+    else
+      e = launch_kernel(tc_gemm_kernel<256, kTcEpiF32>, dim3(grid), dim3(kTcThreads), TcSmem<256>::kBytes, st, pdl2,
+                        s.map_h, s.map_wout, g2);
+  } else {
+    if (scatter)
+      e = launch_kernel(tc_gemm_kernel<128, kTcEpiScatterBf16>, dim3(grid), dim3(kTcThreads), TcSmem<128>::kBytes, st,
+                        pdl2, s.map_h, s.map_wout, g2);
+    else
+      e = launch_kernel(tc_gemm_kernel<128, kTcEpiF32>, dim3(grid), dim3(kTcThreads), TcSmem<128>::kBytes, st, pdl2,
+                        s.map_h, s.map_wout, g2);
+  }
+  if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
   ++*launches;
-  return cudaGetLastError() == cudaSuccess ? SWAPMOE_OK : SWAPMOE_ERR_CUDA;
+  *combined = scatter;
+  return SWAPMOE_OK;
 }
 
 }  // namespace swapmoe

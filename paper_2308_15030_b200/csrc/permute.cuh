@@ -91,7 +91,7 @@ __device__ __forceinline__ void finish_router_cta(const ScanArgs& a) {
   __syncthreads();
   if (threadIdx.x == 0) {
     const unsigned ticket = atomicAdd(a.ticket, 1u);
-    s_last = (ticket == gridDim.x - 1);
+    s_last = (ticket == (unsigned)a.n_cta - 1);
   }
   __syncthreads();
   if (s_last) {
@@ -110,6 +110,7 @@ struct PermuteArgs {
   int32_t* perm;              // [T*k]
   int32_t* inv;               // [T*k]
   int32_t* inv_pad;           // [T*k] row of the pair in the padded workspace
+  int32_t* row_pair;          // [rows_pad] flat pair index stored in each occupied padded row
   void* xp;                   // [rows_pad, d]
   int32_t T, d, k, K, tok_tile;
 };
@@ -132,6 +133,8 @@ __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const Perm
   const int n_total = a.T * a.k;
 
   for (int i = tid; i < (kPermThreads / 32) * kMaxSlots; i += kPermThreads) (&wcount[0][0])[i] = 0;
+  pdl_wait();
+  pdl_trigger();
   __syncthreads();
   int s = -1, rank = 0;
   const int p = p0 + tid;
@@ -152,6 +155,7 @@ __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const Perm
       a.perm[pos] = p;
       a.inv[p] = pos;
       a.inv_pad[p] = row;
+      a.row_pair[row] = p;
     }
     dst_row[tid] = row;
   } else if (tid < npair) {
@@ -185,6 +189,8 @@ struct CombineArgs {
 // out[t, c] = sum_j mgate[t,j] * y[inv_pad[t,j], c]; each thread owns 8 columns.
 template <typename T>
 __global__ void __launch_bounds__(256) combine_kernel(const CombineArgs a) {
+  pdl_wait();
+  pdl_trigger();
   const int c8n = a.d >> 3;
   const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
   if (idx >= (long long)a.T * c8n) return;

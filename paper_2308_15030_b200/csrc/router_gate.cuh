@@ -23,6 +23,12 @@ struct RouterArgs {
   float* cta_imp;           // [n_cta, E]
   int32_t T, d, E, k, K, renorm;
   ScanArgs scan;            // work of the last CTA to finish
+  // Weight prefetch (tensor-core router only): blocks beyond the token tiles pull the resident
+  // experts' matrices into L2 while the router runs, when HBM is otherwise idle.
+  const char* pf_base[2];       // arena_in, arena_out
+  long long pf_slot_bytes[2];   // bytes of one arena entry
+  long long pf_total_bytes[2];  // bytes to prefetch, counted over logical slots 0..K-1 in order
+  const int32_t* pf_phys;       // [K] arena entry of each logical slot
 };
 
 constexpr int kRouterDK = 32;  // contraction chunk staged in shared memory
@@ -121,6 +127,8 @@ __global__ void __launch_bounds__(256) router_gate_kernel(const RouterArgs a) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[t][i] = 0.f;
   float sumsq = 0.f;
+  pdl_wait();
+  pdl_trigger();
 
   const int lrow = tid >> 3;         // token row this thread stages (0..31); == warp*4 + lane/8
   const int lcol = (tid & 7) * 4;    // 4 consecutive contraction indices

@@ -56,6 +56,25 @@ inline size_t router_tc_smem_bytes(int E) {
 __global__ void __launch_bounds__(kRtThreads, 1)
 router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
                  const RouterArgs a, int32_t* status, int n_stages) {
+  if ((int)blockIdx.x >= a.scan.n_cta) {
+    // ---------------------------------------------------- weight-prefetch blocks
+    pdl_wait();
+    pdl_trigger();
+    constexpr long long kChunk = 16384;
+    const long long n_pf = (long long)(gridDim.x - a.scan.n_cta) * kRtThreads;
+    const long long me = (long long)(blockIdx.x - a.scan.n_cta) * kRtThreads + threadIdx.x;
+#pragma unroll 1
+    for (int m = 0; m < 2; ++m) {
+      const long long per_slot = a.pf_slot_bytes[m] / kChunk;
+      const long long n_chunks = a.pf_total_bytes[m] / kChunk;
+      for (long long c = me; c < n_chunks; c += n_pf) {
+        const long long s = c / per_slot, o = c - s * per_slot;
+        const char* src = a.pf_base[m] + (long long)a.pf_phys[s] * a.pf_slot_bytes[m] + o * kChunk;
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"((unsigned)kChunk) : "memory");
+      }
+    }
+    return;
+  }
   const int E = a.E, k = a.k;
   const int Epad = (E + 15) / 16 * 16;
   const int a_bytes = kRtTok * kTcBK * 2, b_bytes = Epad * kTcBK * 2;
@@ -107,6 +126,8 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     ptx::tmem_alloc(tmem_slot, tmem_cols);
     ptx::tmem_relinquish();
   }
+  pdl_wait();      // everything above touched only shared memory, TMEM and kernel parameters
+  pdl_trigger();
   for (int e = tid; e < kMaxE; e += kRtThreads) {
     s_e2s[e] = e < E ? a.e2s[e] : -1;
     s_enorm[e] = e < E ? a.enorm[e] : 0.f;
