@@ -325,6 +325,148 @@ def run_cuda(args, cfg):
     return res
 
 
+# ----------------------------------------------------------------------------- decode loop (cfg4)
+def run_decode(args, cfg):
+    """12-layer decode loop with asynchronous expert swapping; B tokens per step, 256 steps.
+    Reports tokens/s through the whole stack for each batch size, the achieved host->device
+    rate of the expert copies against a PCIe peak probed in the same run, and the stalls."""
+    import torch
+    from paper_2308_15030_b200 import binding
+    from paper_2308_15030_b200.decode import DecodeStack, LayerState
+    torch.cuda.set_device(0)
+    L, steps, spare = cfg.n_layers, (args.steps or cfg.n_steps), 2
+    peaks = load_peaks()
+
+    def dev(a):
+        return torch.from_numpy(I.bf16_bits(np.ascontiguousarray(a, np.float32)).view(np.int16)).view(torch.bfloat16).cuda()
+
+    # PCIe probe: 1 GiB pinned -> device, best of 10
+    probe_h = torch.empty(1 << 30, dtype=torch.uint8).pin_memory()
+    probe_d = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+    best = 1e9
+    for _ in range(10):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); probe_d.copy_(probe_h, non_blocking=True); b.record(); b.synchronize()
+        best = min(best, a.elapsed_time(b))
+    pcie_gbs = (1 << 30) / (best * 1e-3) / 1e9
+    del probe_h, probe_d
+
+    # One bank of E experts (values shared by the layers: only timing is measured here), one
+    # pinned copy per layer so every layer's loads come from its own host memory.
+    w_in = np.empty((cfg.E, cfg.nin, cfg.f, cfg.d), np.float32)
+    w_out = np.empty((cfg.E, cfg.d, cfg.f), np.float32)
+    for e in range(cfg.E):
+        w_in[e], w_out[e] = I.make_expert(cfg, e)
+    bank_in = torch.from_numpy(I.bf16_bits(w_in).view(np.int16)).view(torch.bfloat16)
+    bank_out = torch.from_numpy(I.bf16_bits(w_out).view(np.int16)).view(torch.bfloat16)
+    del w_in, w_out
+    host_in = [bank_in.clone().pin_memory() for _ in range(L)]
+    host_out = [bank_out.clone().pin_memory() for _ in range(L)]
+    Wr = [I.make_router(cfg.scaled(seed=1000 + l)) for l in range(L)]
+    enorm = [I.make_enorm(cfg.scaled(seed=1000 + l)) for l in range(L)]
+    d_Wr = [dev(w) for w in Wr]
+    expert_bytes = cfg.nmat * cfg.d * cfg.f * cfg.nb
+
+    results = {}
+    for B in args.batches:
+        x = I.make_decode_tokens(cfg, Wr, B, steps)
+        d_x = dev(x.reshape(-1, cfg.d)).reshape(steps, L, B, cfg.d)
+        outs = torch.empty((L, B, cfg.d), dtype=torch.bfloat16, device="cuda")
+
+        def make_stack(time_loads, frequency=8):
+            states = []
+            for l in range(L):
+                P = cfg.K + spare
+                a_in = torch.empty((P, cfg.nin, cfg.f, cfg.d), dtype=torch.bfloat16, device="cuda")
+                a_out = torch.empty((P, cfg.d, cfg.f), dtype=torch.bfloat16, device="cuda")
+                a_in[: cfg.K].copy_(host_in[l][: cfg.K]); a_out[: cfg.K].copy_(host_out[l][: cfg.K])
+                layer = binding.Layer(cfg.E, cfg.d, cfg.f, cfg.k, cfg.K, cfg.dtype, cfg.act, cfg.renorm,
+                                      max_tokens=B, spare_slots=spare)
+                layer.set_router(d_Wr[l], enorm[l])
+                states.append(LayerState(layer, np.arange(cfg.K, dtype=np.int32), np.arange(cfg.K, dtype=np.int32),
+                                         list(range(cfg.K, P)), a_in, a_out, host_in[l], host_out[l]))
+            torch.cuda.synchronize()
+            return DecodeStack(states, frequency=frequency, loads_per_step=1, lag=2, time_loads=time_loads)
+
+        # pass 1: timed, nothing read back except the importance every 8 steps
+        stack = make_stack(True)
+        for s in range(min(8, steps)):            # warm-up steps (tables evolve; they are part of the loop)
+            stack.step([d_x[s, l] for l in range(L)], [outs[l] for l in range(L)], record=False)
+        torch.cuda.synchronize()
+        stack2_start = stack.step_no
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches0 = sum(st.layer.launch_count for st in stack.layers)
+        e0.record()
+        for s in range(steps):
+            stack.step([d_x[s, l] for l in range(L)], [outs[l] for l in range(L)], record=False)
+        e1.record(); torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        launches = sum(st.layer.launch_count for st in stack.layers) - launches0
+        load_s = stack.loader_seconds()
+        loads, bytes_loaded, stalls = stack.loads, stack.bytes_loaded, stack.stalls
+        status = [st.layer.device_status() for st in stack.layers]
+        assert all(s == (0, 0) for s in status), status
+        del stack
+        # pass 1b: the same loop with the scheduler switched off (no importance reads, no swaps):
+        # what the kernels alone allow, to separate compute from PCIe traffic
+        stack = make_stack(False, frequency=1 << 30)
+        for s in range(min(8, steps)):
+            stack.step([d_x[s, l] for l in range(L)], [outs[l] for l in range(L)], record=False)
+        torch.cuda.synchronize()
+        e0.record()
+        for s in range(steps):
+            stack.step([d_x[s, l] for l in range(L)], [outs[l] for l in range(L)], record=False)
+        e1.record(); torch.cuda.synchronize()
+        ms_noswap = e0.elapsed_time(e1)
+        del stack
+        # pass 2: same inputs, slot counts tapped after every forward -> touched slots for the roofline
+        stack = make_stack(False)
+        touched = 0
+        for s in range(min(8, steps)):
+            stack.step([d_x[s, l] for l in range(L)], [outs[l] for l in range(L)], record=False)
+        for s in range(steps):
+            n = stack.step_no
+            for li, st in enumerate(stack.layers):
+                stack._commit_due(st, n)
+                st.layer.forward(d_x[s, li], outs[li])
+                touched += int(np.count_nonzero(st.layer.tap("count")))
+            if (n + 1) % stack.frequency == 0:
+                for li, st in enumerate(stack.layers):
+                    stack._decide(li, st, n)
+            for st in stack.layers:
+                stack._issue_loads(st, n)
+            stack.step_no += 1
+        torch.cuda.synchronize()
+        del stack
+        bytes_alg = touched * expert_bytes + steps * L * (2 * B * cfg.d * cfg.nb + cfg.E * cfg.d * cfg.nb)
+        t_roof = bytes_alg / (peaks["hbm_gbs"] * 1e9)
+        results[str(B)] = {
+            "tokens_per_s": steps * B / (ms * 1e-3), "ms_per_step": ms / steps,
+            "us_per_layer": ms / steps / L * 1e3, "gpu_launches": int(launches),
+            "touched_slots_per_layer_step": touched / (steps * L),
+            "roofline_us_per_layer": t_roof / (steps * L) * 1e6, "roofline_frac": t_roof * 1e3 / ms,
+            "loads": loads, "loaded_GB": bytes_loaded / 1e9,
+            "loader_GBps": (bytes_loaded / load_s / 1e9) if load_s > 0 else None,
+            "loader_frac_of_pcie_probe": (bytes_loaded / load_s / 1e9 / pcie_gbs) if load_s > 0 else None,
+            "stalls": stalls,
+            "pcie_seconds_needed": bytes_loaded / (pcie_gbs * 1e9), "loop_seconds": ms * 1e-3,
+            "no_swap": {"tokens_per_s": steps * B / (ms_noswap * 1e-3), "us_per_layer": ms_noswap / steps / L * 1e3},
+        }
+    Bmax = str(max(args.batches))
+    return {
+        "metric": METRIC, "value": results[Bmax]["tokens_per_s"], "unit": UNIT, "n_gpus": 1, "steps": steps,
+        "warmup": 8, "ms_per_step": results[Bmax]["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "cfg4 decode loop: %d layers d_model=%d d_ff=%d E=%d top1 K=%d, %d steps, "
+                               "B in %s tokens per step; frequency 8, <=1 load/layer/step, commit lag 2, 2 spare "
+                               "slots; value = B=%s" % (L, cfg.d, cfg.f, cfg.E, cfg.K, steps, args.batches, Bmax),
+                   "expert_bank": "one bank of %d experts, copied into %d per-layer pinned buffers" % (cfg.E, L),
+                   "launch": "eager (host policy in the loop)"},
+        "gpu_launches": results[Bmax]["gpu_launches"],
+        "pcie_probe_GBps": pcie_gbs, "per_batch": results,
+    }
+
+
 # ----------------------------------------------------------------------------- the oracle arm
 def oracle_sample(cfg, steps=1, warmup=0):
     """Times the CPU oracle, as it stands, on the workload's batch (host cores)."""
@@ -379,7 +521,8 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg5"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--batches", type=int, nargs="+", default=[1, 4, 16, 64], help="cfg4: tokens per decode step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
@@ -390,6 +533,9 @@ def main():
         res = run_reference(args, cfg)
         if res is not None:
             print(json.dumps(res), flush=True)
+        return
+    if args.workload == "cfg4":
+        print(json.dumps(run_decode(args, cfg)), flush=True)
         return
     args.steps = 2000 if args.steps is None else args.steps
     args.warmup = 50 if args.warmup is None else max(3, args.warmup)

@@ -13,6 +13,7 @@
 #include "common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "ffn_fused.cuh"
 #include "permute.cuh"
 #include "router_gate.cuh"
 #include "router_tc.cuh"
@@ -31,6 +32,9 @@ struct swapmoe_layer {
   int32_t *uidx, *midx, *slot, *cta_hist, *cta_base, *count, *offset, *pad_offset;
   int32_t *perm, *inv, *inv_pad, *row_pair, *n_tiles, *e2s, *phys, *s2e, *status;
   unsigned* ticket;
+  int32_t* done;               // per-row-tile counters of the fused FFN kernel
+  int32_t n_done;
+  bool fused_ffn;              // both grouped GEMMs in one launch
   TileDesc* tiles;
   void *xp, *h, *x_stage, *out_stage;
   // host state
@@ -89,7 +93,8 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   const int n_cta = (T + tok_tile - 1) / tok_tile;
   const int n_pairs = T * c.top_k;
   const bool use_tc = tc_selected(L->gemm_path, c, T);
-  const int tile_rows = use_tc ? kTcBM : kSimtBM;
+  const int mt = use_tc ? tc_row_subtiles(c, T) : 1;
+  const int tile_rows = use_tc ? kTcBM * mt : kSimtBM;
   const int max_tiles = (n_pairs + tile_rows - 1) / tile_rows + c.K;
 
   RouterArgs ra;
@@ -103,6 +108,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   sa.cta_base = L->cta_base; sa.count = L->count; sa.offset = L->offset;
   sa.pad_offset = L->pad_offset; sa.tiles = L->tiles; sa.n_tiles = L->n_tiles; sa.imp = L->imp;
   sa.ticket = L->ticket;
+  sa.done = L->done; sa.n_done = L->n_done;
   sa.n_cta = n_cta; sa.K = c.K; sa.E = c.E; sa.tile_rows = tile_rows;
   ra.pf_base[0] = ra.pf_base[1] = nullptr;
   ra.pf_slot_bytes[0] = ra.pf_slot_bytes[1] = 16384;
@@ -165,8 +171,15 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   bool combined = false;
   if (use_tc) {
     cudaEvent_t mid = L->stage_events ? static_cast<cudaEvent_t>(L->stage_events[4]) : nullptr;
-    const int32_t rc = tc_ffn(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->row_pair, L->mgate, max_tiles,
-                              L->status, st, pdl, &L->launches, &combined, mid);
+    int32_t rc;
+    if (L->fused_ffn && mt == 1) {
+      rc = tc_ffn_fused(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->done, L->row_pair, L->mgate, max_tiles,
+                        L->status, st, pdl, &L->launches, &combined);
+      if (mid) cudaEventRecord(mid, st);      // one kernel: the GEMM-2 stage reads as zero
+    } else {
+      rc = tc_ffn(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->row_pair, L->mgate, max_tiles, mt,
+                  L->status, st, pdl, &L->launches, &combined, mid);
+    }
     if (rc != SWAPMOE_OK) return rc;
   } else {
     SimtGemmArgs g1;
@@ -256,6 +269,8 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   {
     const char* env = std::getenv("SWAPMOE_PDL");      // SWAPMOE_PDL=0 launches every kernel fully serialised
     L->use_pdl = !(env && env[0] == '0');
+    env = std::getenv("SWAPMOE_FUSED_FFN");             // SWAPMOE_FUSED_FFN=1: both grouped GEMMs in one launch
+    L->fused_ffn = env && env[0] == '1';                // off by default: measured slower than two launches
     env = std::getenv("SWAPMOE_PREFETCH");              // SWAPMOE_PREFETCH=0 disables the L2 weight prefetch
     L->prefetch = !(env && env[0] == '0');
     // The prefetch must drain while the router runs (about 15 us on 16-64 SMs): what HBM delivers
@@ -290,6 +305,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_phys = cv.take<int32_t>(kMaxSlots), o_s2e = cv.take<int32_t>(kMaxSlots);
   const size_t o_status = cv.take<int32_t>(4);
   const size_t o_ticket = cv.take<unsigned>(4);
+  const size_t o_done = cv.take<int32_t>(max_tiles);
   const size_t o_tiles = cv.take<TileDesc>(max_tiles);
   const size_t o_xp = cv.take<char>(rows_pad * c.d_model * L->elem);
   const size_t o_h = cv.take<char>(rows_pad * c.d_ff * L->elem);
@@ -310,6 +326,8 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   L->n_tiles = (int32_t*)(b + o_ntiles); L->e2s = (int32_t*)(b + o_e2s); L->phys = (int32_t*)(b + o_phys);
   L->s2e = (int32_t*)(b + o_s2e); L->status = (int32_t*)(b + o_status);
   L->ticket = (unsigned*)(b + o_ticket);
+  L->done = (int32_t*)(b + o_done);
+  L->n_done = (int32_t)max_tiles;
   L->tiles = (TileDesc*)(b + o_tiles);
   L->xp = b + o_xp; L->h = b + o_h; L->y = (float*)(b + o_y);
   L->x_stage = b + o_xs; L->out_stage = b + o_os;

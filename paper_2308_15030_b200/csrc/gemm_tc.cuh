@@ -38,6 +38,8 @@ struct TcGemmArgs {
   int32_t k_blocks;         // contraction length / 64
   int32_t b_rows_per_phys;  // rows of the flattened weight map per arena entry
   int32_t b_rows_gate;      // row offset of the second input matrix (SwiGLU), else 0
+  int32_t row_split;        // 128-row sub-tiles per tile-list entry handled as SEPARATE work items
+                            // (2 when a one-sub-tile kernel walks a list built for 256-row tiles)
   const int32_t* row_pair;  // [rows_pad] pair index of each padded row (scatter epilogue)
   const float* gate;        // [T*k] masked gate values (scatter epilogue)
   int32_t top_k;
@@ -167,26 +169,32 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, vol
   }
 }
 
-template <int BN>
+// MT = row sub-tiles of 128 rows that one CTA multiplies against the same weight tile.
+template <int BN, int MT = 1>
 struct TcSmem {
-  static constexpr int kABytes = kTcBM * kTcBK * 2;
+  static constexpr int kABytes = MT * kTcBM * kTcBK * 2;
   static constexpr int kBBytes = BN * kTcBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kStages = (kTcSmemBudget - 2048) / kStageBytes;
   static constexpr int kBytes = kStages * kStageBytes + 2048;  // + alignment slack and barriers
 };
 
-// C tile [128, BN (or BN/2 for SwiGLU)] = epi(A[row0:row0+128, :] * B[brow:brow+BN, :]^T)
-template <int BN, int EPI>
+// C tile [128*MT, BN (or BN/2 for SwiGLU)] = epi(A[row0:row0+128*MT, :] * B[brow:brow+BN, :]^T).
+// With MT = 2 a slot's weight tile is loaded once for two 128-row sub-tiles (two TMEM
+// accumulators), which halves the weight bytes the SM has to ingest for slots with more
+// than 128 rows; a tile with <= 128 valid rows skips the second half entirely.
+template <int BN, int EPI, int MT = 1>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const TcGemmArgs a) {
-  using S = TcSmem<BN>;
+  using S = TcSmem<BN, MT>;
+  constexpr int kAccBufs = (2 * MT * BN <= 512) ? 2 : 1;   // TMEM accumulator sets
+  constexpr int kHalfBytes = kTcBM * kTcBK * 2;
   constexpr int kStages = S::kStages;
   constexpr int kNB = (EPI == kTcEpiSwigluBf16) ? 2 : 1;   // weight boxes per stage
   constexpr int kBoxRows = BN / kNB;
   constexpr int kOutCols = BN / kNB;                        // output columns per tile
-  constexpr uint32_t kTmemCols = 2 * BN;                    // two accumulator buffers
+  constexpr uint32_t kTmemCols = kAccBufs * MT * BN;
   constexpr uint32_t kIdesc = make_idesc_bf16(kTcBM, BN);
 
   extern __shared__ unsigned char smem_raw[];
@@ -223,7 +231,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   pdl_wait();      // the tile list and the operands come from the preceding kernels
   pdl_trigger();
-  const int n_row_tiles = *a.n_tiles;
+  const int n_row_tiles = *a.n_tiles * a.row_split;
   const int total = n_row_tiles * a.n_col_tiles;
 
   if (warp == 0) {
@@ -233,14 +241,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t phase = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
-        const int rt = t / a.n_col_tiles, ct = t - rt * a.n_col_tiles;   // column tiles vary fastest
-        const TileDesc td = a.tiles[rt];
+        const int ct = t / n_row_tiles, rt = t - ct * n_row_tiles;   // row tiles vary fastest
+        TileDesc td = a.tiles[rt / a.row_split];
+        if (a.row_split > 1) {
+          const int off = (rt % a.row_split) * kTcBM;
+          td.row0 += off;
+          td.rows = min(td.rows - off, kTcBM);
+          if (td.rows <= 0) continue;              // this entry has no second sub-tile
+        }
         const int brow = td.phys * a.b_rows_per_phys + ct * kBoxRows;
+        const int halves = (MT == 2 && td.rows > kTcBM) ? 2 : 1;
         for (int kb = 0; kb < a.k_blocks; ++kb) {
           ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 1);
           if (!ok) break;
-          ptx::mbar_expect_tx(&full[stage], S::kStageBytes);
-          ptx::tma_load_2d(sA + stage * S::kABytes, &tmA, &full[stage], kb * kTcBK, td.row0);
+          ptx::mbar_expect_tx(&full[stage], (uint32_t)(halves * kHalfBytes + S::kBBytes));
+          for (int hf = 0; hf < halves; ++hf)
+            ptx::tma_load_2d(sA + stage * S::kABytes + hf * kHalfBytes, &tmA, &full[stage], kb * kTcBK,
+                             td.row0 + hf * kTcBM);
 #pragma unroll
           for (int j = 0; j < kNB; ++j)
             ptx::tma_load_2d(sB + stage * S::kBBytes + j * kBoxRows * kTcBK * 2, &tmB, &full[stage],
@@ -261,28 +278,37 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        int halves = 1;
+        {
+          const int rt = t % n_row_tiles;
+          const int rows = a.tiles[rt / a.row_split].rows - (rt % a.row_split) * kTcBM;
+          if (rows <= 0) continue;
+          if (MT == 2) halves = rows > kTcBM ? 2 : 1;
+        }
         ok = bounded_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, a.status, 2);
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BN);
+        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * MT * BN);
         for (int kb = 0; kb < a.k_blocks; ++kb) {
           ok = bounded_wait(&full[stage], phase, abort_flag, a.status, 3);
           if (!ok) break;
           ptx::tc_fence_after();
-          const uint64_t da = make_kmajor_sw128_desc(ptx::smem_u32(sA + stage * S::kABytes));
           const uint64_t db = make_kmajor_sw128_desc(ptx::smem_u32(sB + stage * S::kBBytes));
+          for (int hf = 0; hf < halves; ++hf) {
+            const uint64_t da = make_kmajor_sw128_desc(ptx::smem_u32(sA + stage * S::kABytes + hf * kHalfBytes));
 #pragma unroll
-          for (int k = 0; k < kTcBK / kTcUmmaK; ++k) {
-            // advancing 16 elements along K inside the swizzled row = +32 bytes = +2 in the address field
-            ptx::umma_bf16(tmem_d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), kIdesc,
-                           (kb > 0 || k > 0) ? 1u : 0u);
+            for (int k = 0; k < kTcBK / kTcUmmaK; ++k) {
+              // advancing 16 elements along K inside the swizzled row = +32 bytes = +2 in the address field
+              ptx::umma_bf16(tmem_d + (uint32_t)(hf * BN), da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), kIdesc,
+                             (kb > 0 || k > 0) ? 1u : 0u);
+            }
           }
           ptx::umma_commit(&empty[stage]);   // frees the stage once these MMAs have read it
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
         ptx::umma_commit(&acc_full[acc]);    // accumulator complete
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1u; }
       }
     }
   } else if (warp >= 4) {
@@ -293,17 +319,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
-      const int rt = t / a.n_col_tiles, ct = t - rt * a.n_col_tiles;
-      const TileDesc td = a.tiles[rt];
+      const int ct = t / n_row_tiles, rt = t - ct * n_row_tiles;
+      TileDesc td = a.tiles[rt / a.row_split];
+      if (a.row_split > 1) {
+        const int off = (rt % a.row_split) * kTcBM;
+        td.row0 += off;
+        td.rows = min(td.rows - off, kTcBM);
+        if (td.rows <= 0) continue;
+      }
       ok = bounded_wait(&acc_full[acc], acc_phase, abort_flag, a.status, 4);
       if (!ok) break;
       ptx::tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
-      const bool row_ok = r < td.rows;
-      size_t crow = (size_t)(td.row0 + r) * a.ldc + (size_t)ct * kOutCols;
+      const int halves = (MT == 2 && td.rows > kTcBM) ? 2 : 1;
+      for (int hf = 0; hf < halves; ++hf) {
+      const int rr = r + hf * kTcBM;             // row inside the (up to 256-row) tile
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)((acc * MT + hf) * BN);
+      const bool row_ok = rr < td.rows;
+      size_t crow = (size_t)(td.row0 + rr) * a.ldc + (size_t)ct * kOutCols;
       float gate = 1.f;
       if (EPI == kTcEpiScatterBf16 && row_ok) {
-        const int p = a.row_pair[td.row0 + r];
+        const int p = a.row_pair[td.row0 + rr];
         gate = a.gate[p];
         crow = (size_t)(p / a.top_k) * a.ldc + (size_t)ct * kOutCols;
       }
@@ -347,9 +382,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
       }
+      }
       ptx::tc_fence_before();
       ptx::mbar_arrive(&acc_empty[acc]);       // 128 arrivals hand the buffer back to the MMA warp
-      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1u; }
     }
   }
   ptx::tc_fence_before();
@@ -372,6 +408,7 @@ struct TcState {
   PFN_encodeTiled encode;
   CUtensorMap map_xp, map_h;          // activations: [rows_pad, d], [rows_pad, f], box 64 x 128
   CUtensorMap map_win, map_wout;      // weights flattened to 2D, box 64 x (rows per load)
+  CUtensorMap map_wout256;            // W_out with 256-row boxes (two-sub-tile kernels)
   CUtensorMap map_wr;                 // router matrix [E, d], box 64 x Epad
   int bn2;                            // column tile of the second GEMM
   bool arena_bound;
@@ -380,6 +417,14 @@ struct TcState {
 
 inline bool tc_supported(const swapmoe_config_t& c) {
   return c.dtype == SWAPMOE_BF16 && c.d_model % 128 == 0 && c.d_ff % 256 == 0;
+}
+
+// Row sub-tiles per CTA for a forward of T tokens: two when the average slot has well over
+// 128 rows (weight tiles are then shared by two sub-tiles), one for small slots (nothing to
+// share) and for very large ones (tensor-bound: keep the double-buffered accumulators).
+inline int tc_row_subtiles(const swapmoe_config_t& c, int T) {
+  const long long rows_per_slot = (long long)T * c.top_k / c.K;
+  return (rows_per_slot >= 160 && rows_per_slot < 1024 && c.d_model % 256 == 0) ? 2 : 1;
 }
 
 // Automatic choice: tensor cores whenever the shape allows it.
@@ -399,10 +444,10 @@ inline bool tc_encode_2d(PFN_encodeTiled enc, CUtensorMap* m, const void* base, 
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int EPI>
+template <int BN, int EPI, int MT = 1>
 inline bool tc_set_smem_attr() {
-  return cudaFuncSetAttribute(tc_gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              TcSmem<BN>::kBytes) == cudaSuccess;
+  return cudaFuncSetAttribute(tc_gemm_kernel<BN, EPI, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              TcSmem<BN, MT>::kBytes) == cudaSuccess;
 }
 
 inline int32_t tc_init(TcState& s, const swapmoe_config_t& c, void* xp, void* h, float* /*y*/, int rows_pad) {
@@ -425,7 +470,8 @@ inline int32_t tc_init(TcState& s, const swapmoe_config_t& c, void* xp, void* h,
   if (!tc_encode_2d(s.encode, &s.map_h, h, (uint64_t)rows_pad, (uint64_t)c.d_ff, kTcBM)) return SWAPMOE_ERR_CUDA;
   bool ok = tc_set_smem_attr<256, kTcEpiReluBf16>() && tc_set_smem_attr<256, kTcEpiSwigluBf16>() &&
             tc_set_smem_attr<256, kTcEpiF32>() && tc_set_smem_attr<128, kTcEpiF32>() &&
-            tc_set_smem_attr<256, kTcEpiScatterBf16>() && tc_set_smem_attr<128, kTcEpiScatterBf16>();
+            tc_set_smem_attr<256, kTcEpiScatterBf16>() && tc_set_smem_attr<128, kTcEpiScatterBf16>() &&
+            tc_set_smem_attr<256, kTcEpiF32, 2>() && tc_set_smem_attr<256, kTcEpiScatterBf16, 2>();
   if (!ok) return SWAPMOE_ERR_CUDA;
   s.bn2 = (c.d_model % 256 == 0 && c.d_model >= 2048) ? 256 : 128;
   s.enabled = true;
@@ -440,6 +486,9 @@ inline int32_t tc_bind_arena(TcState& s, const swapmoe_config_t& c, const void* 
   if (!tc_encode_2d(s.encode, &s.map_win, arena_in, (uint64_t)P * nin * c.d_ff, (uint64_t)c.d_model, box_in))
     return SWAPMOE_ERR_CUDA;
   if (!tc_encode_2d(s.encode, &s.map_wout, arena_out, (uint64_t)P * c.d_model, (uint64_t)c.d_ff, (uint32_t)s.bn2))
+    return SWAPMOE_ERR_CUDA;
+  if (c.d_model % 256 == 0 &&
+      !tc_encode_2d(s.encode, &s.map_wout256, arena_out, (uint64_t)P * c.d_model, (uint64_t)c.d_ff, 256))
     return SWAPMOE_ERR_CUDA;
   s.arena_bound = true;
   return SWAPMOE_OK;
@@ -463,7 +512,7 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
 // Runs both grouped GEMMs.  With top_k == 1 the second GEMM writes gate * y straight into
 // `out` (*combined = true) and no combine kernel is needed.
 inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, void* out, const TileDesc* tiles,
-                      const int32_t* n_tiles, const int32_t* row_pair, const float* mgate, int max_tiles,
+                      const int32_t* n_tiles, const int32_t* row_pair, const float* mgate, int max_tiles, int mt,
                       int32_t* status, cudaStream_t st, bool pdl, int64_t* launches, bool* combined,
                       cudaEvent_t between = nullptr) {
   if (!s.enabled || !s.arena_bound) return SWAPMOE_ERR_NOT_READY;
@@ -476,6 +525,12 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
   g1.b_rows_gate = swiglu ? c.d_ff : 0;
   g1.row_pair = nullptr; g1.gate = nullptr; g1.top_k = c.top_k;
   int grid = max_tiles * g1.n_col_tiles;
+  if (grid > s.sm_count) grid = s.sm_count;
+  // GEMM-1's k-loop is short (d_model / 64 blocks), so its epilogue must overlap the next tile's
+  // MMAs: it always runs one sub-tile per CTA with two TMEM buffers, and simply walks a 256-row
+  // tile list as two work items per entry.
+  g1.row_split = mt;
+  grid = max_tiles * mt * g1.n_col_tiles;
   if (grid > s.sm_count) grid = s.sm_count;
   cudaError_t e;
   if (swiglu)
@@ -492,15 +547,25 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
   TcGemmArgs g2;
   g2.C = scatter ? out : static_cast<void*>(y);
   g2.tiles = tiles; g2.n_tiles = n_tiles; g2.status = status; g2.ldc = c.d_model;
-  g2.n_col_tiles = c.d_model / s.bn2;
+  const int bn2 = mt == 2 ? 256 : s.bn2;
+  g2.n_col_tiles = c.d_model / bn2;
   g2.k_blocks = c.d_ff / kTcBK;
   g2.b_rows_per_phys = c.d_model;
   g2.b_rows_gate = 0;
   g2.row_pair = row_pair; g2.gate = mgate; g2.top_k = c.top_k;
+  g2.row_split = 1;
   grid = max_tiles * g2.n_col_tiles;
   if (grid > s.sm_count) grid = s.sm_count;
   const bool pdl2 = pdl && between == nullptr;
-  if (s.bn2 == 256) {
+  const CUtensorMap& map_wout = bn2 == 256 ? s.map_wout256 : s.map_wout;
+  if (mt == 2) {
+    if (scatter)
+      e = launch_kernel(tc_gemm_kernel<256, kTcEpiScatterBf16, 2>, dim3(grid), dim3(kTcThreads),
+                        TcSmem<256, 2>::kBytes, st, pdl2, s.map_h, map_wout, g2);
+    else
+      e = launch_kernel(tc_gemm_kernel<256, kTcEpiF32, 2>, dim3(grid), dim3(kTcThreads), TcSmem<256, 2>::kBytes, st,
+                        pdl2, s.map_h, map_wout, g2);
+  } else if (s.bn2 == 256) {
     if (scatter)
       e = launch_kernel(tc_gemm_kernel<256, kTcEpiScatterBf16>, dim3(grid), dim3(kTcThreads), TcSmem<256>::kBytes, st,
                         pdl2, s.map_h, s.map_wout, g2);

@@ -17,7 +17,8 @@ struct ScanArgs {
   int32_t* n_tiles;          // [1]
   float* imp;                // [E] accumulator of Eq. (1)
   unsigned* ticket;          // [1] router CTAs finished so far (returns to 0)
-  int32_t n_cta, K, E, tile_rows;
+  int32_t* done;             // [n_done] per-row-tile progress counters of the fused FFN kernel (zeroed here)
+  int32_t n_cta, K, E, tile_rows, n_done;
 };
 
 // Work of the LAST router CTA to finish (all of its threads call this).  Warp w scans
@@ -46,6 +47,7 @@ __device__ __forceinline__ void scan_reduce_block(const ScanArgs& a) {
       s_count[s] = running;
     }
   }
+  for (int i = tid; i < a.n_done; i += blockDim.x) a.done[i] = 0;
   for (int e = tid; e < a.E; e += blockDim.x) {
     float acc = 0.f;
 #pragma unroll 16

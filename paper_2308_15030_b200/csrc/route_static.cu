@@ -99,6 +99,7 @@ extern "C" int32_t swapmoe_route_static(const void* x_dev, const void* Wr_dev, c
   sa.n_tiles = reinterpret_cast<int32_t*>(s + kOffNTiles);
   sa.imp = imp_dev;
   sa.ticket = reinterpret_cast<unsigned*>(s + kOffTicket);
+  sa.done = nullptr; sa.n_done = 0;
   sa.n_cta = n_cta; sa.K = K; sa.E = E; sa.tile_rows = kSimtBMStatic;
   if (dtype == SWAPMOE_BF16)
     router_gate_kernel<bf16><<<n_cta, 256, router_smem_bytes(E), st>>>(ra);

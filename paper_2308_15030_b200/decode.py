@@ -51,7 +51,7 @@ class DecodeStack:
     """L independent layers driven step by step; records the slot tables each step used."""
 
     def __init__(self, layers: Sequence[LayerState], frequency: int = 8, loads_per_step: int = 1,
-                 lag: int = 2, compute_stream=None, side_stream=None):
+                 lag: int = 2, compute_stream=None, side_stream=None, time_loads: bool = False):
         import torch
         self.layers = list(layers)
         self.frequency, self.loads_per_step, self.lag = int(frequency), int(loads_per_step), int(lag)
@@ -63,6 +63,8 @@ class DecodeStack:
         self.stalls = 0            # commits whose copy had not finished when the flip was enqueued
         self.loads = 0
         self.bytes_loaded = 0
+        self.time_loads = time_loads
+        self.load_events = []      # (start, stop) events around every copy when time_loads is set
         for st in self.layers:
             st.layer.set_resident(st.s2e, st.arena_in, st.arena_out, st.phys, stream=self.compute)
 
@@ -81,6 +83,10 @@ class DecodeStack:
         for st in self.layers:
             self._issue_loads(st, n)
         self.step_no += 1
+
+    def loader_seconds(self) -> float:
+        """Sum of the device-side durations of all copies issued so far (needs time_loads)."""
+        return sum(a.elapsed_time(b) for a, b in self.load_events) * 1e-3
 
     def _commit_due(self, st: LayerState, n: int) -> None:
         due = [p for p in st.pending if p.commit_step <= n]
@@ -124,6 +130,11 @@ class DecodeStack:
             # the spare entry may still be read by forwards already enqueued before its slot
             # was flipped away: order the copy after everything enqueued so far
             self.side.wait_stream(self.compute)
+            if self.time_loads:
+                t0 = torch.cuda.Event(enable_timing=True)
+                ev = torch.cuda.Event(enable_timing=True)
+                t0.record(self.side)
+                self.load_events.append((t0, ev))
             st.layer.load_slot_async(phys, st.host_in[expert], st.host_out[expert], self.side, ev)
             st.pending.append(_Pending(n + self.lag, slot, expert, phys, ev))
             issued += 1

@@ -177,3 +177,34 @@ def test_cfg5_mixtral_shape_sampled():
     sub = np.sort(np.random.default_rng(5).choice(cfg.T, size=48, replace=False)).astype(np.int32)
     check_against_oracle(case, out, token_subset=sub)
     assert np.all(np.isfinite(out))
+
+
+def test_fused_ffn_kernel_option(monkeypatch):
+    """SWAPMOE_FUSED_FFN=1 runs both grouped GEMMs in one persistent launch; results must not change."""
+    from harness import Case, check_against_oracle
+    monkeypatch.setenv("SWAPMOE_FUSED_FFN", "1")
+    for k, act, renorm in ((1, I.ACT_RELU, 0), (2, I.ACT_SWIGLU, 1)):
+        cfg = _cfg(T=900 // k, d=256, f=512, E=16, K=6, k=k, act=act, renorm=renorm, zipf_s=1.1)
+        case = Case(cfg)
+        n0 = case.layer.launch_count
+        out = case.run()
+        assert case.layer.launch_count - n0 == (3 if k == 1 else 4)
+        check_against_oracle(case, out)
+
+
+def test_two_row_subtiles_per_cta():
+    """Slots with 160..1023 rows on average take the kernels that share a weight tile between two
+    128-row sub-tiles; include slots above and below 128 rows and a ragged last sub-tile."""
+    import oracle
+    from harness import Case, check_against_oracle
+    for k, act, renorm in ((1, I.ACT_RELU, 0), (2, I.ACT_SWIGLU, 1)):
+        cfg = _cfg(T=1500 // k, d=256, f=512, E=12, K=5, k=k, act=act, renorm=renorm, zipf_s=1.3)
+        probe = Case(cfg)                                   # ranks the experts by importance
+        lg = oracle.logits(probe.x, probe.Wr)
+        ui, ug = oracle.gate(lg, cfg.k, cfg.renorm)
+        order = oracle.topk_importance(oracle.importance(probe.x, ui, ug, probe.enorm), cfg.E)
+        case = Case(cfg, s2e=list(order[:3]) + list(order[-2:]))   # three popular and two rare experts
+        res = check_against_oracle(case, case.run())
+        cnt = res["oracle"]["count"]
+        # covered: entries with two full sub-tiles, and entries whose second sub-tile is absent
+        assert cnt.max() > 256 and any(0 < c % 256 <= 128 for c in cnt), cnt
