@@ -373,7 +373,9 @@ def run_decode(args, cfg):
         d_x = dev(x.reshape(-1, cfg.d)).reshape(steps, L, B, cfg.d)
         outs = torch.empty((L, B, cfg.d), dtype=torch.bfloat16, device="cuda")
 
-        def make_stack(time_loads, frequency=8):
+        xbuf = torch.empty((L, B, cfg.d), dtype=torch.bfloat16, device="cuda")
+
+        def make_stack(time_loads, frequency=8, graph=False):
             states = []
             for l in range(L):
                 P = cfg.K + spare
@@ -386,7 +388,8 @@ def run_decode(args, cfg):
                 states.append(LayerState(layer, np.arange(cfg.K, dtype=np.int32), np.arange(cfg.K, dtype=np.int32),
                                          list(range(cfg.K, P)), a_in, a_out, host_in[l], host_out[l]))
             torch.cuda.synchronize()
-            return DecodeStack(states, frequency=frequency, loads_per_step=1, lag=2, time_loads=time_loads)
+            return DecodeStack(states, frequency=frequency, loads_per_step=1, lag=2, time_loads=time_loads,
+                               graph_buffers=(xbuf, outs) if graph else None)
 
         # pass 1: timed, nothing read back except the importance every 8 steps
         stack = make_stack(True)
@@ -418,6 +421,28 @@ def run_decode(args, cfg):
             stack.step([d_x[s, l] for l in range(L)], [outs[l] for l in range(L)], record=False)
         e1.record(); torch.cuda.synchronize()
         ms_noswap = e0.elapsed_time(e1)
+        del stack
+        # pass 1c: scheduler off, the step's 12 forwards replayed as one CUDA graph
+        stack = make_stack(False, frequency=1 << 30, graph=True)
+        for s in range(min(8, steps)):
+            stack.step_graph(d_x[s])
+        torch.cuda.synchronize()
+        e0.record()
+        for s in range(steps):
+            stack.step_graph(d_x[s])
+        e1.record(); torch.cuda.synchronize()
+        ms_graph = e0.elapsed_time(e1)
+        del stack
+        # pass 1d: scheduler ON with the graph
+        stack = make_stack(False, frequency=8, graph=True)
+        for s in range(min(8, steps)):
+            stack.step_graph(d_x[s])
+        torch.cuda.synchronize()
+        e0.record()
+        for s in range(steps):
+            stack.step_graph(d_x[s])
+        e1.record(); torch.cuda.synchronize()
+        ms_graph_swap = e0.elapsed_time(e1)
         del stack
         # pass 2: same inputs, slot counts tapped after every forward -> touched slots for the roofline
         stack = make_stack(False)
@@ -451,6 +476,10 @@ def run_decode(args, cfg):
             "stalls": stalls,
             "pcie_seconds_needed": bytes_loaded / (pcie_gbs * 1e9), "loop_seconds": ms * 1e-3,
             "no_swap": {"tokens_per_s": steps * B / (ms_noswap * 1e-3), "us_per_layer": ms_noswap / steps / L * 1e3},
+            "no_swap_graph": {"tokens_per_s": steps * B / (ms_graph * 1e-3), "us_per_layer": ms_graph / steps / L * 1e3,
+                              "roofline_frac": t_roof * 1e3 / ms_graph},
+            "swap_graph": {"tokens_per_s": steps * B / (ms_graph_swap * 1e-3),
+                           "us_per_layer": ms_graph_swap / steps / L * 1e3},
         }
     Bmax = str(max(args.batches))
     return {

@@ -115,7 +115,8 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   ra.pf_total_bytes[0] = ra.pf_total_bytes[1] = 0;
   ra.pf_phys = L->phys;
   int pf_ctas = 0;
-  if (tc_router && use_tc && L->prefetch && n_pairs >= 8 * c.K) {
+  if (tc_router && use_tc && L->prefetch && n_pairs >= 8 * c.K &&
+      (long long)c.K * (L->nin + 1) * c.d_ff * c.d_model * (long long)L->elem <= (256ll << 20)) {
     // Every slot will most likely be touched: pull the resident weights towards L2 now, while the
     // router and the permutation leave HBM idle.  GEMM-1's matrices first, then as much of GEMM-2's
     // as the L2 budget allows.
@@ -177,7 +178,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
                         L->status, st, pdl, &L->launches, &combined);
       if (mid) cudaEventRecord(mid, st);      // one kernel: the GEMM-2 stage reads as zero
     } else {
-      rc = tc_ffn(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->row_pair, L->mgate, max_tiles, mt,
+      rc = tc_ffn(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->row_pair, L->mgate, max_tiles, mt, T,
                   L->status, st, pdl, &L->launches, &combined, mid);
     }
     if (rc != SWAPMOE_OK) return rc;

@@ -286,7 +286,7 @@ inline cudaError_t tc_ffn_launch_one(const TcState& s, const TcFfnArgs& a, int g
     attr_done = true;
   }
   return launch_kernel(tc_ffn_kernel<EPI1, BN2, EPI2>, dim3(grid), dim3(kTcThreads), kFfnSmemBytes, st, pdl,
-                       s.map_xp, s.map_win, s.map_h, s.map_wout, a);
+                       s.map_xp[0], s.map_win[0], s.map_h[0], s.map_wout[BN2 == 256 ? 0 : 1], a);
 }
 
 // One launch for both GEMMs.  *combined tells whether out was written (top_k == 1).
@@ -295,6 +295,7 @@ inline int32_t tc_ffn_fused(TcState& s, const swapmoe_config_t& c, void* h, floa
                             int max_tiles, int32_t* status, cudaStream_t st, bool pdl, int64_t* launches,
                             bool* combined) {
   if (!s.enabled || !s.arena_bound) return SWAPMOE_ERR_NOT_READY;
+  const int bn2 = (c.d_model % 256 == 0 && c.d_model >= 2048) ? 256 : 128;
   const bool swiglu = c.act == SWAPMOE_ACT_SWIGLU;
   const bool scatter = c.top_k == 1;
   TcFfnArgs a;
@@ -306,7 +307,7 @@ inline int32_t tc_ffn_fused(TcState& s, const swapmoe_config_t& c, void* h, floa
   a.kb1 = c.d_model / kTcBK;
   a.b_rows_per_phys1 = swiglu ? 2 * c.d_ff : c.d_ff;
   a.b_rows_gate1 = swiglu ? c.d_ff : 0;
-  a.n_col2 = c.d_model / s.bn2;
+  a.n_col2 = c.d_model / bn2;
   a.kb2 = c.d_ff / kTcBK;
   a.b_rows_per_phys2 = c.d_model;
   long long work = (long long)max_tiles * (a.n_col1 + a.n_col2);
@@ -314,10 +315,10 @@ inline int32_t tc_ffn_fused(TcState& s, const swapmoe_config_t& c, void* h, floa
   cudaError_t e;
 #define SWAPMOE_FFN_CASE(E1, B2, E2) e = tc_ffn_launch_one<E1, B2, E2>(s, a, grid, st, pdl)
   if (swiglu) {
-    if (s.bn2 == 256) { if (scatter) SWAPMOE_FFN_CASE(kTcEpiSwigluBf16, 256, kTcEpiScatterBf16); else SWAPMOE_FFN_CASE(kTcEpiSwigluBf16, 256, kTcEpiF32); }
+    if (bn2 == 256) { if (scatter) SWAPMOE_FFN_CASE(kTcEpiSwigluBf16, 256, kTcEpiScatterBf16); else SWAPMOE_FFN_CASE(kTcEpiSwigluBf16, 256, kTcEpiF32); }
     else              { if (scatter) SWAPMOE_FFN_CASE(kTcEpiSwigluBf16, 128, kTcEpiScatterBf16); else SWAPMOE_FFN_CASE(kTcEpiSwigluBf16, 128, kTcEpiF32); }
   } else {
-    if (s.bn2 == 256) { if (scatter) SWAPMOE_FFN_CASE(kTcEpiReluBf16, 256, kTcEpiScatterBf16); else SWAPMOE_FFN_CASE(kTcEpiReluBf16, 256, kTcEpiF32); }
+    if (bn2 == 256) { if (scatter) SWAPMOE_FFN_CASE(kTcEpiReluBf16, 256, kTcEpiScatterBf16); else SWAPMOE_FFN_CASE(kTcEpiReluBf16, 256, kTcEpiF32); }
     else              { if (scatter) SWAPMOE_FFN_CASE(kTcEpiReluBf16, 128, kTcEpiScatterBf16); else SWAPMOE_FFN_CASE(kTcEpiReluBf16, 128, kTcEpiF32); }
   }
 #undef SWAPMOE_FFN_CASE

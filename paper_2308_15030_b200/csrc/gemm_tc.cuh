@@ -38,6 +38,9 @@ struct TcGemmArgs {
   int32_t k_blocks;         // contraction length / 64
   int32_t b_rows_per_phys;  // rows of the flattened weight map per arena entry
   int32_t b_rows_gate;      // row offset of the second input matrix (SwiGLU), else 0
+  int32_t a_box_bytes;      // bytes one activation TMA box delivers (box rows * 128): small batches
+                            // load only the first 16/32/64 rows of the 128-row MMA tile, the rest
+                            // of the tile is stale shared memory whose output rows are never stored
   int32_t row_split;        // 128-row sub-tiles per tile-list entry handled as SEPARATE work items
                             // (2 when a one-sub-tile kernel walks a list built for 256-row tiles)
   const int32_t* row_pair;  // [rows_pad] pair index of each padded row (scatter epilogue)
@@ -254,7 +257,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int kb = 0; kb < a.k_blocks; ++kb) {
           ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 1);
           if (!ok) break;
-          ptx::mbar_expect_tx(&full[stage], (uint32_t)(halves * kHalfBytes + S::kBBytes));
+          ptx::mbar_expect_tx(&full[stage], (uint32_t)(halves * a.a_box_bytes + S::kBBytes));
           for (int hf = 0; hf < halves; ++hf)
             ptx::tma_load_2d(sA + stage * S::kABytes + hf * kHalfBytes, &tmA, &full[stage], kb * kTcBK,
                              td.row0 + hf * kTcBM);
@@ -402,15 +405,19 @@ typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_
                                     CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                     CUtensorMapFloatOOBfill);
 
+// Column-tile widths the kernels are built for.  Narrow tiles exist for small batches
+// (decode): with few row tiles, wide column tiles would leave most SMs without work.
+constexpr int kBn1Options[3] = {256, 128, 64};
+constexpr int kBn2Options[4] = {256, 128, 64, 32};
+
 struct TcState {
   bool enabled;
   int sm_count;
   PFN_encodeTiled encode;
-  CUtensorMap map_xp, map_h;          // activations: [rows_pad, d], [rows_pad, f], box 64 x 128
-  CUtensorMap map_win, map_wout;      // weights flattened to 2D, box 64 x (rows per load)
-  CUtensorMap map_wout256;            // W_out with 256-row boxes (two-sub-tile kernels)
+  CUtensorMap map_xp[4], map_h[4];    // activations [rows_pad, d] / [rows_pad, f]; box rows 128, 64, 32, 16
+  CUtensorMap map_win[3];             // W_in flattened to 2D, one map per entry of kBn1Options
+  CUtensorMap map_wout[4];            // W_out flattened to 2D, one map per entry of kBn2Options
   CUtensorMap map_wr;                 // router matrix [E, d], box 64 x Epad
-  int bn2;                            // column tile of the second GEMM
   bool arena_bound;
   bool router_ok;                     // tensor-core router usable (bf16 layer)
 };
@@ -466,14 +473,21 @@ inline int32_t tc_init(TcState& s, const swapmoe_config_t& c, void* xp, void* h,
   s.encode = reinterpret_cast<PFN_encodeTiled>(fn);
   s.router_ok = true;
   if (!tc_supported(c)) return SWAPMOE_OK;
-  if (!tc_encode_2d(s.encode, &s.map_xp, xp, (uint64_t)rows_pad, (uint64_t)c.d_model, kTcBM)) return SWAPMOE_ERR_CUDA;
-  if (!tc_encode_2d(s.encode, &s.map_h, h, (uint64_t)rows_pad, (uint64_t)c.d_ff, kTcBM)) return SWAPMOE_ERR_CUDA;
-  bool ok = tc_set_smem_attr<256, kTcEpiReluBf16>() && tc_set_smem_attr<256, kTcEpiSwigluBf16>() &&
+  for (int i = 0; i < 4; ++i) {
+    if (!tc_encode_2d(s.encode, &s.map_xp[i], xp, (uint64_t)rows_pad, (uint64_t)c.d_model, (uint32_t)(kTcBM >> i)))
+      return SWAPMOE_ERR_CUDA;
+    if (!tc_encode_2d(s.encode, &s.map_h[i], h, (uint64_t)rows_pad, (uint64_t)c.d_ff, (uint32_t)(kTcBM >> i)))
+      return SWAPMOE_ERR_CUDA;
+  }
+  bool ok = tc_set_smem_attr<256, kTcEpiReluBf16>() && tc_set_smem_attr<128, kTcEpiReluBf16>() &&
+            tc_set_smem_attr<64, kTcEpiReluBf16>() && tc_set_smem_attr<256, kTcEpiSwigluBf16>() &&
+            tc_set_smem_attr<128, kTcEpiSwigluBf16>() && tc_set_smem_attr<64, kTcEpiSwigluBf16>() &&
             tc_set_smem_attr<256, kTcEpiF32>() && tc_set_smem_attr<128, kTcEpiF32>() &&
+            tc_set_smem_attr<64, kTcEpiF32>() && tc_set_smem_attr<32, kTcEpiF32>() &&
             tc_set_smem_attr<256, kTcEpiScatterBf16>() && tc_set_smem_attr<128, kTcEpiScatterBf16>() &&
+            tc_set_smem_attr<64, kTcEpiScatterBf16>() && tc_set_smem_attr<32, kTcEpiScatterBf16>() &&
             tc_set_smem_attr<256, kTcEpiF32, 2>() && tc_set_smem_attr<256, kTcEpiScatterBf16, 2>();
   if (!ok) return SWAPMOE_ERR_CUDA;
-  s.bn2 = (c.d_model % 256 == 0 && c.d_model >= 2048) ? 256 : 128;
   s.enabled = true;
   return SWAPMOE_OK;
 }
@@ -482,14 +496,14 @@ inline int32_t tc_bind_arena(TcState& s, const swapmoe_config_t& c, const void* 
   if (!s.enabled) return SWAPMOE_OK;
   const int P = c.K + c.spare_slots;
   const int nin = c.act == SWAPMOE_ACT_SWIGLU ? 2 : 1;
-  const uint32_t box_in = nin == 2 ? 128 : 256;
-  if (!tc_encode_2d(s.encode, &s.map_win, arena_in, (uint64_t)P * nin * c.d_ff, (uint64_t)c.d_model, box_in))
-    return SWAPMOE_ERR_CUDA;
-  if (!tc_encode_2d(s.encode, &s.map_wout, arena_out, (uint64_t)P * c.d_model, (uint64_t)c.d_ff, (uint32_t)s.bn2))
-    return SWAPMOE_ERR_CUDA;
-  if (c.d_model % 256 == 0 &&
-      !tc_encode_2d(s.encode, &s.map_wout256, arena_out, (uint64_t)P * c.d_model, (uint64_t)c.d_ff, 256))
-    return SWAPMOE_ERR_CUDA;
+  for (int i = 0; i < 3; ++i)     // SwiGLU loads W1 and W3 as two boxes of half the tile width
+    if (!tc_encode_2d(s.encode, &s.map_win[i], arena_in, (uint64_t)P * nin * c.d_ff, (uint64_t)c.d_model,
+                      (uint32_t)(kBn1Options[i] / nin)))
+      return SWAPMOE_ERR_CUDA;
+  for (int i = 0; i < 4; ++i)
+    if (!tc_encode_2d(s.encode, &s.map_wout[i], arena_out, (uint64_t)P * c.d_model, (uint64_t)c.d_ff,
+                      (uint32_t)kBn2Options[i]))
+      return SWAPMOE_ERR_CUDA;
   s.arena_bound = true;
   return SWAPMOE_OK;
 }
@@ -509,76 +523,105 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Column-tile width (index into `options`) that minimises the bytes the busiest SM has to pull:
+// (tiles per SM) x (k-blocks) x (activation box + weight box).  Wide tiles amortise the
+// activation box, narrow ones give every SM work when there are few row tiles.
+inline int tc_pick_bn(const int* options, int n_options, int n, long long row_tiles, int sm_count, int a_box_bytes,
+                      int min_bn) {
+  int pick = -1;
+  long long best = 0;
+  for (int i = 0; i < n_options; ++i) {
+    if (n % options[i] || options[i] < min_bn) continue;
+    const long long tiles = row_tiles * (n / options[i]);
+    const long long per_sm = (tiles + sm_count - 1) / sm_count;
+    const long long cost = per_sm * (a_box_bytes + (long long)options[i] * kTcBK * 2);
+    if (pick < 0 || cost < best) { pick = i; best = cost; }
+  }
+  return pick;
+}
+
+typedef void (*TcGemmKernel)(const CUtensorMap, const CUtensorMap, const TcGemmArgs);
+
 // Runs both grouped GEMMs.  With top_k == 1 the second GEMM writes gate * y straight into
 // `out` (*combined = true) and no combine kernel is needed.
 inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, void* out, const TileDesc* tiles,
                       const int32_t* n_tiles, const int32_t* row_pair, const float* mgate, int max_tiles, int mt,
-                      int32_t* status, cudaStream_t st, bool pdl, int64_t* launches, bool* combined,
+                      int n_tokens, int32_t* status, cudaStream_t st, bool pdl, int64_t* launches, bool* combined,
                       cudaEvent_t between = nullptr) {
   if (!s.enabled || !s.arena_bound) return SWAPMOE_ERR_NOT_READY;
   const bool swiglu = c.act == SWAPMOE_ACT_SWIGLU;
+  const bool scatter = c.top_k == 1;
+  // row tiles expected: every touched slot (at most min(pairs, K)) has at least one, and large slots
+  // have pairs / 128 in total plus on average half a ragged tile each
+  const long long pairs = (long long)n_tokens * c.top_k;
+  const long long touched = pairs < c.K ? pairs : c.K;
+  const long long by_rows = pairs / kTcBM + touched / 2;
+  const long long row_tiles_est = touched > by_rows ? touched : by_rows;
+  // no tile holds more rows than there are pairs: small batches fetch only the rows that can be valid
+  int ia = 0;
+  while (ia < 3 && (kTcBM >> (ia + 1)) >= pairs) ++ia;
+  if (mt == 2) ia = 0;
+  const int a_box_bytes = (kTcBM >> ia) * kTcBK * 2;
+
+  // ---- GEMM-1: h = act(xp * W_in^T).  Its k-loop is short (d_model / 64 blocks), so its epilogue must
+  // overlap the next tile's MMAs: always one sub-tile per CTA with two TMEM buffers; a 256-row tile
+  // list is walked as two work items per entry.
+  const int i1 = tc_pick_bn(kBn1Options, 3, c.d_ff, row_tiles_est * mt, s.sm_count, a_box_bytes, swiglu ? 64 : 32);
+  if (i1 < 0) return SWAPMOE_ERR_UNSUPPORTED;
+  const int bn1 = kBn1Options[i1];
+  const int out1 = swiglu ? bn1 / 2 : bn1;      // output columns per tile
   TcGemmArgs g1;
   g1.C = h; g1.tiles = tiles; g1.n_tiles = n_tiles; g1.status = status; g1.ldc = c.d_ff;
-  g1.n_col_tiles = swiglu ? c.d_ff / 128 : c.d_ff / 256;
+  g1.n_col_tiles = c.d_ff / out1;
   g1.k_blocks = c.d_model / kTcBK;
   g1.b_rows_per_phys = swiglu ? 2 * c.d_ff : c.d_ff;
   g1.b_rows_gate = swiglu ? c.d_ff : 0;
   g1.row_pair = nullptr; g1.gate = nullptr; g1.top_k = c.top_k;
-  int grid = max_tiles * g1.n_col_tiles;
-  if (grid > s.sm_count) grid = s.sm_count;
-  // GEMM-1's k-loop is short (d_model / 64 blocks), so its epilogue must overlap the next tile's
-  // MMAs: it always runs one sub-tile per CTA with two TMEM buffers, and simply walks a 256-row
-  // tile list as two work items per entry.
   g1.row_split = mt;
-  grid = max_tiles * mt * g1.n_col_tiles;
-  if (grid > s.sm_count) grid = s.sm_count;
-  cudaError_t e;
-  if (swiglu)
-    e = launch_kernel(tc_gemm_kernel<256, kTcEpiSwigluBf16>, dim3(grid), dim3(kTcThreads), TcSmem<256>::kBytes, st, pdl,
-                      s.map_xp, s.map_win, g1);
-  else
-    e = launch_kernel(tc_gemm_kernel<256, kTcEpiReluBf16>, dim3(grid), dim3(kTcThreads), TcSmem<256>::kBytes, st, pdl,
-                      s.map_xp, s.map_win, g1);
-  if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
+  g1.a_box_bytes = a_box_bytes;
+  long long work = (long long)max_tiles * mt * g1.n_col_tiles;
+  int grid = work > s.sm_count ? s.sm_count : (int)work;
+  static const TcGemmKernel k1[2][3] = {
+      {tc_gemm_kernel<256, kTcEpiReluBf16>, tc_gemm_kernel<128, kTcEpiReluBf16>, tc_gemm_kernel<64, kTcEpiReluBf16>},
+      {tc_gemm_kernel<256, kTcEpiSwigluBf16>, tc_gemm_kernel<128, kTcEpiSwigluBf16>,
+       tc_gemm_kernel<64, kTcEpiSwigluBf16>}};
+  static const int smem1[3] = {TcSmem<256>::kBytes, TcSmem<128>::kBytes, TcSmem<64>::kBytes};
+  if (launch_kernel(k1[swiglu ? 1 : 0][i1], dim3(grid), dim3(kTcThreads), smem1[i1], st, pdl, s.map_xp[ia], s.map_win[i1],
+                    g1) != cudaSuccess)
+    return SWAPMOE_ERR_CUDA;
   ++*launches;
   if (between) cudaEventRecord(between, st);
 
-  const bool scatter = c.top_k == 1;
+  // ---- GEMM-2: y = h * W_out^T (or out = gate * y for top-1)
+  const int i2 = mt == 2 ? 0 : tc_pick_bn(kBn2Options, 4, c.d_model, row_tiles_est, s.sm_count, a_box_bytes, 32);
+  if (i2 < 0 || c.d_model % kBn2Options[i2]) return SWAPMOE_ERR_UNSUPPORTED;
+  const int bn2 = kBn2Options[i2];
   TcGemmArgs g2;
   g2.C = scatter ? out : static_cast<void*>(y);
   g2.tiles = tiles; g2.n_tiles = n_tiles; g2.status = status; g2.ldc = c.d_model;
-  const int bn2 = mt == 2 ? 256 : s.bn2;
   g2.n_col_tiles = c.d_model / bn2;
   g2.k_blocks = c.d_ff / kTcBK;
   g2.b_rows_per_phys = c.d_model;
   g2.b_rows_gate = 0;
   g2.row_pair = row_pair; g2.gate = mgate; g2.top_k = c.top_k;
   g2.row_split = 1;
-  grid = max_tiles * g2.n_col_tiles;
-  if (grid > s.sm_count) grid = s.sm_count;
+  g2.a_box_bytes = a_box_bytes;
+  work = (long long)max_tiles * g2.n_col_tiles;
+  grid = work > s.sm_count ? s.sm_count : (int)work;
   const bool pdl2 = pdl && between == nullptr;
-  const CUtensorMap& map_wout = bn2 == 256 ? s.map_wout256 : s.map_wout;
+  static const TcGemmKernel k2[2][4] = {
+      {tc_gemm_kernel<256, kTcEpiF32>, tc_gemm_kernel<128, kTcEpiF32>, tc_gemm_kernel<64, kTcEpiF32>,
+       tc_gemm_kernel<32, kTcEpiF32>},
+      {tc_gemm_kernel<256, kTcEpiScatterBf16>, tc_gemm_kernel<128, kTcEpiScatterBf16>,
+       tc_gemm_kernel<64, kTcEpiScatterBf16>, tc_gemm_kernel<32, kTcEpiScatterBf16>}};
+  static const int smem2[4] = {TcSmem<256>::kBytes, TcSmem<128>::kBytes, TcSmem<64>::kBytes, TcSmem<32>::kBytes};
+  cudaError_t e;
   if (mt == 2) {
-    if (scatter)
-      e = launch_kernel(tc_gemm_kernel<256, kTcEpiScatterBf16, 2>, dim3(grid), dim3(kTcThreads),
-                        TcSmem<256, 2>::kBytes, st, pdl2, s.map_h, map_wout, g2);
-    else
-      e = launch_kernel(tc_gemm_kernel<256, kTcEpiF32, 2>, dim3(grid), dim3(kTcThreads), TcSmem<256, 2>::kBytes, st,
-                        pdl2, s.map_h, map_wout, g2);
-  } else if (s.bn2 == 256) {
-    if (scatter)
-      e = launch_kernel(tc_gemm_kernel<256, kTcEpiScatterBf16>, dim3(grid), dim3(kTcThreads), TcSmem<256>::kBytes, st,
-                        pdl2, s.map_h, s.map_wout, g2);
-    else
-      e = launch_kernel(tc_gemm_kernel<256, kTcEpiF32>, dim3(grid), dim3(kTcThreads), TcSmem<256>::kBytes, st, pdl2,
-                        s.map_h, s.map_wout, g2);
+    const TcGemmKernel k = scatter ? tc_gemm_kernel<256, kTcEpiScatterBf16, 2> : tc_gemm_kernel<256, kTcEpiF32, 2>;
+    e = launch_kernel(k, dim3(grid), dim3(kTcThreads), TcSmem<256, 2>::kBytes, st, pdl2, s.map_h[0], s.map_wout[0], g2);
   } else {
-    if (scatter)
-      e = launch_kernel(tc_gemm_kernel<128, kTcEpiScatterBf16>, dim3(grid), dim3(kTcThreads), TcSmem<128>::kBytes, st,
-                        pdl2, s.map_h, s.map_wout, g2);
-    else
-      e = launch_kernel(tc_gemm_kernel<128, kTcEpiF32>, dim3(grid), dim3(kTcThreads), TcSmem<128>::kBytes, st, pdl2,
-                        s.map_h, s.map_wout, g2);
+    e = launch_kernel(k2[scatter ? 1 : 0][i2], dim3(grid), dim3(kTcThreads), smem2[i2], st, pdl2, s.map_h[ia],
+                      s.map_wout[i2], g2);
   }
   if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
   ++*launches;

@@ -51,7 +51,8 @@ class DecodeStack:
     """L independent layers driven step by step; records the slot tables each step used."""
 
     def __init__(self, layers: Sequence[LayerState], frequency: int = 8, loads_per_step: int = 1,
-                 lag: int = 2, compute_stream=None, side_stream=None, time_loads: bool = False):
+                 lag: int = 2, compute_stream=None, side_stream=None, time_loads: bool = False,
+                 graph_buffers=None):
         import torch
         self.layers = list(layers)
         self.frequency, self.loads_per_step, self.lag = int(frequency), int(loads_per_step), int(lag)
@@ -65,6 +66,11 @@ class DecodeStack:
         self.bytes_loaded = 0
         self.time_loads = time_loads
         self.load_events = []      # (start, stop) events around every copy when time_loads is set
+        # graph_buffers = (x_buf, out_buf), device tensors [L, B, d_model]: the L forwards of a step
+        # are then captured once into a CUDA graph over these fixed buffers and replayed
+        # (step_graph); slot-table flips and expert copies stay outside the graph.
+        self.graph_buffers = graph_buffers
+        self.graph = None
         for st in self.layers:
             st.layer.set_resident(st.s2e, st.arena_in, st.arena_out, st.phys, stream=self.compute)
 
@@ -77,6 +83,35 @@ class DecodeStack:
             if record:
                 self.trace.append((n, li, st.s2e.copy(), st.phys.copy()))
             st.layer.forward(xs[li], outs[li], stream=self.compute)
+        if (n + 1) % self.frequency == 0:
+            for li, st in enumerate(self.layers):
+                self._decide(li, st, n)
+        for st in self.layers:
+            self._issue_loads(st, n)
+        self.step_no += 1
+
+    def step_graph(self, x_step, record: bool = False) -> None:
+        """One step through the captured graph: x_step [L, B, d_model] is copied into the fixed
+        input buffer, due table flips are enqueued, the graph runs, the scheduler acts."""
+        import torch
+        x_buf, out_buf = self.graph_buffers
+        n = self.step_no
+        with torch.cuda.stream(self.compute):
+            if self.graph is None:
+                for li, st in enumerate(self.layers):          # eager once: lazily built state
+                    st.layer.forward(x_buf[li], out_buf[li], stream=self.compute)
+                    st.layer.read_importance(reset=True, stream=self.compute)
+                self.compute.synchronize()
+                self.graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(self.graph):        # captured on torch's own side stream
+                    for li, st in enumerate(self.layers):
+                        st.layer.forward(x_buf[li], out_buf[li], stream=None)
+            x_buf.copy_(x_step, non_blocking=True)
+            for li, st in enumerate(self.layers):
+                self._commit_due(st, n)
+                if record:
+                    self.trace.append((n, li, st.s2e.copy(), st.phys.copy()))
+            self.graph.replay()
         if (n + 1) % self.frequency == 0:
             for li, st in enumerate(self.layers):
                 self._decide(li, st, n)

@@ -140,3 +140,27 @@ def test_cfg4_shape_sampled():
             err = np.max(np.abs(outs[s, l][sub] - ref)) / max(1e-30, np.max(np.abs(ref)))
             assert err <= TOL_OUT[cfg.dtype], (B, s, l, err)
         del stack, host
+
+
+def test_decode_loop_through_cuda_graph_matches_replay():
+    """The step's forwards captured as a CUDA graph (fixed buffers), table flips outside it."""
+    import torch
+    from harness import to_host_f32, TOL_OUT
+    cfg = I.LayerConfig("decg", I.BF16, T=6, d=128, f=256, E=16, k=1, K=4, zipf_s=1.1, seed=2)
+    L, B, steps = 2, 6, 24
+    stack, host, x, d_x = _build(cfg, L, B, steps, frequency=4, lag=1, spare=2)
+    xbuf = torch.empty((L, B, cfg.d), dtype=d_x.dtype, device="cuda")
+    obuf = torch.empty_like(xbuf)
+    stack.graph_buffers = (xbuf, obuf)
+    outs = torch.empty((steps, L, B, cfg.d), dtype=d_x.dtype, device="cuda")
+    for s in range(steps):
+        stack.step_graph(d_x[s], record=True)
+        outs[s].copy_(obuf)
+    torch.cuda.synchronize()
+    outs = to_host_f32(outs.reshape(-1, cfg.d)).reshape(steps, L, B, cfg.d)
+    assert stack.loads > 0
+    for entry in stack.trace:
+        s, l, _, _ = entry
+        ref = _replay(cfg, host, x, entry)["out"]
+        err = np.max(np.abs(outs[s, l] - ref)) / max(1e-30, np.max(np.abs(ref)))
+        assert err <= TOL_OUT[cfg.dtype], (s, l, err)
