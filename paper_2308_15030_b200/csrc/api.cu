@@ -47,6 +47,7 @@ struct swapmoe_layer {
   int32_t rows_pad_max;
   int32_t sm_count;
   bool use_pdl;                // programmatic dependent launch between the kernels of a forward
+  int32_t router_tok;          // 0 = automatic token-tile size of the tensor-core router, else 32/64/128
   bool prefetch;               // pull resident weights into L2 from the router kernel
   long long l2_prefetch_bytes; // how much of them (L2 capacity minus head room)
   void* const* stage_events;   // 7 cudaEvent_t of the forward being enqueued, or nullptr
@@ -89,7 +90,8 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   const swapmoe_config_t& c = L->cfg;
   const bool pdl = L->use_pdl && L->stage_events == nullptr;
   const bool tc_router = L->tc.router_ok && ext_logits == nullptr;
-  const int tok_tile = tc_router ? kRtTok : kTokTile;
+  int tok_tile = tc_router ? router_tc_tok(T) : kTokTile;
+  if (tc_router && L->router_tok) tok_tile = L->router_tok;
   const int n_cta = (T + tok_tile - 1) / tok_tile;
   const int n_pairs = T * c.top_k;
   const bool use_tc = tc_selected(L->gemm_path, c, T);
@@ -137,12 +139,14 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   mark(L, 0, st);
   if (tc_router) {
     if (x != L->map_x_ptr || T != L->map_x_T) {   // the token map is re-encoded only when x or T changes
-      if (!tc_encode_2d(L->tc.encode, &L->map_x, x, (uint64_t)T, (uint64_t)c.d_model, kRtTok)) return SWAPMOE_ERR_CUDA;
+      if (!tc_encode_2d(L->tc.encode, &L->map_x, x, (uint64_t)T, (uint64_t)c.d_model, (uint32_t)tok_tile))
+        return SWAPMOE_ERR_CUDA;
       L->map_x_ptr = x;
       L->map_x_T = T;
     }
-    if (launch_kernel(router_tc_kernel, dim3(n_cta + pf_ctas), dim3(kRtThreads), router_tc_smem_bytes(c.E), st, pdl,
-                      L->map_x, L->tc.map_wr, ra, L->status, router_tc_stages(c.E)) != cudaSuccess)
+    if (launch_kernel(router_tc_kernel, dim3(n_cta + pf_ctas), dim3(kRtThreads), router_tc_smem_bytes(c.E, tok_tile),
+                      st, pdl, L->map_x, L->tc.map_wr, ra, L->status, router_tc_stages(c.E, tok_tile), tok_tile) !=
+        cudaSuccess)
       return SWAPMOE_ERR_CUDA;
   } else {
     if (launch_kernel(router_gate_kernel<DT>, dim3(n_cta), dim3(256), router_smem_bytes(c.E), st, pdl, ra) !=
@@ -272,6 +276,9 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
     L->use_pdl = !(env && env[0] == '0');
     env = std::getenv("SWAPMOE_FUSED_FFN");             // SWAPMOE_FUSED_FFN=1: both grouped GEMMs in one launch
     L->fused_ffn = env && env[0] == '1';                // off by default: measured slower than two launches
+    env = std::getenv("SWAPMOE_ROUTER_TOK");            // force the router's token tile (32, 64 or 128)
+    L->router_tok = env ? std::atoi(env) : 0;
+    if (L->router_tok != 32 && L->router_tok != 64 && L->router_tok != 128) L->router_tok = 0;
     env = std::getenv("SWAPMOE_PREFETCH");              // SWAPMOE_PREFETCH=0 disables the L2 weight prefetch
     L->prefetch = !(env && env[0] == '0');
     // The prefetch must drain while the router runs (about 15 us on 16-64 SMs): what HBM delivers
@@ -337,7 +344,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   ok = ok && cuda_ok(cudaMemset(L->status, 0, sizeof(int32_t) * 4));
   ok = ok && cuda_ok(cudaMemset(L->ticket, 0, sizeof(unsigned) * 4));
   ok = ok && cuda_ok(cudaFuncSetAttribute(router_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          200 * 1024));
+                                          210 * 1024));
   // Rows of the padded workspaces that no pair occupies are computed on but never
   // read back; start them at zero so they hold finite values.
   ok = ok && cuda_ok(cudaMemset(L->xp, 0, rows_pad * c.d_model * L->elem));

@@ -21,26 +21,36 @@ struct ScanArgs {
   int32_t n_cta, K, E, tile_rows, n_done;
 };
 
-// Work of the LAST router CTA to finish (all of its threads call this).  Warp w scans
-// slot w, w+nwarp, ... over the router CTAs in order; then thread s lays out slot s
-// (offsets, padded offsets, tile list); warps also reduce the per-CTA importance
-// partials in a fixed order.  Loads bypass L1: the data was written by other CTAs.
-__device__ __forceinline__ void scan_reduce_block(const ScanArgs& a) {
+// Work of the LAST router CTA to finish (all of its threads call this).  The per-CTA
+// histograms and importance partials written by the other CTAs are first staged into shared
+// memory with coalesced L1-bypassing loads (one latency for everything) when `stage` is large
+// enough, else read in place.  Then thread s walks slot s over the router CTAs in order and lays
+// out the slot (offsets, padded offsets, tile list); thread e adds expert e's partials in CTA
+// order, which fixes the summation order of Eq. (1) run to run.
+__device__ __forceinline__ void scan_reduce_block(const ScanArgs& a, void* stage, int stage_bytes) {
   __shared__ int32_t s_count[kMaxSlots];
   const int tid = threadIdx.x;
-
-  // Thread s walks slot s over the router CTAs in order (the loads do not depend on the
-  // running sum, so they pipeline); thread e likewise adds expert e's importance partials
-  // in CTA order, which fixes the summation order of Eq. (1) run to run.
+  const int n_hist = a.n_cta * a.K, n_imp = a.n_cta * a.E;
+  const int32_t* hist = a.cta_hist;
+  const float* impp = a.cta_imp;
+  if (stage != nullptr && (size_t)(n_hist + n_imp) * 4 <= (size_t)stage_bytes) {
+    int32_t* sh = static_cast<int32_t*>(stage);
+    float* si = reinterpret_cast<float*>(sh + n_hist);
+    for (int i = tid; i < n_hist; i += blockDim.x) sh[i] = __ldcg(a.cta_hist + i);
+    for (int i = tid; i < n_imp; i += blockDim.x) si[i] = __ldcg(a.cta_imp + i);
+    __syncthreads();
+    hist = sh;
+    impp = si;
+  }
   // Slots are walked by the LAST K threads and experts by the first E threads, so the two
-  // chains of dependent global loads run side by side.
+  // chains run side by side.
   {
     const int s = (int)blockDim.x - 1 - tid;
     if (s < a.K) {
       int running = 0;
 #pragma unroll 16
       for (int c = 0; c < a.n_cta; ++c) {
-        const int v = __ldcg(a.cta_hist + (size_t)c * a.K + s);
+        const int v = hist[(size_t)c * a.K + s];
         a.cta_base[(size_t)c * a.K + s] = running;
         running += v;
       }
@@ -51,7 +61,7 @@ __device__ __forceinline__ void scan_reduce_block(const ScanArgs& a) {
   for (int e = tid; e < a.E; e += blockDim.x) {
     float acc = 0.f;
 #pragma unroll 16
-    for (int c = 0; c < a.n_cta; ++c) acc += __ldcg(a.cta_imp + (size_t)c * a.E + e);
+    for (int c = 0; c < a.n_cta; ++c) acc += impp[(size_t)c * a.E + e];
     a.imp[e] += acc;
   }
   __syncthreads();
@@ -87,7 +97,7 @@ __device__ __forceinline__ void scan_reduce_block(const ScanArgs& a) {
 
 // Called by every thread of a router CTA after its partials are written: the CTA
 // that draws the last ticket runs the scan.  No CTA waits for another.
-__device__ __forceinline__ void finish_router_cta(const ScanArgs& a) {
+__device__ __forceinline__ void finish_router_cta(const ScanArgs& a, void* stage = nullptr, int stage_bytes = 0) {
   __shared__ int s_last;
   __threadfence();
   __syncthreads();
@@ -98,7 +108,7 @@ __device__ __forceinline__ void finish_router_cta(const ScanArgs& a) {
   __syncthreads();
   if (s_last) {
     __threadfence();
-    scan_reduce_block(a);
+    scan_reduce_block(a, stage, stage_bytes);
     if (threadIdx.x == 0) *a.ticket = 0u;
   }
 }

@@ -1,12 +1,15 @@
 // Router product on the tensor cores with the whole gate fused into its epilogue
 // (SwapMoE Section 2: G(x); Fig. 4: Masked Gating; Eq. 1: importance terms).
 //
-// One CTA = 128 tokens.  logits[128, E] = x_tile * Wr^T is accumulated in TMEM by
-// tcgen05.mma (bf16 -> fp32) from TMA-staged tiles; TMEM lane = token row, so in the
-// epilogue ONE THREAD OWNS ONE TOKEN: it reads its E logits, picks the unmasked and the
-// masked top-k, evaluates the softmax gates, looks up the slot and emits the token's
-// importance term.  While the tiles stream through shared memory the same four warps
-// accumulate ||x||^2 of their rows.  The last CTA to finish runs the slot scan.
+// One CTA = tok (32, 64 or 128) tokens.  logits[tok, E] = x_tile * Wr^T is accumulated in TMEM
+// by tcgen05.mma (bf16 -> fp32, M = 128: rows beyond tok are stale shared memory whose
+// accumulator lanes are never read) from TMA-staged tiles; while the tiles stream through
+// shared memory four warps accumulate ||x||^2 of their rows.  The logits then go TMEM ->
+// shared memory and the gate runs with 256 / tok threads per token: half of them for the
+// off-the-shelf gate, half for the masked gate (Fig. 4), each scanning its share of the
+// experts; per-token candidates are merged in expert order so ties keep the lowest index.
+// Small token tiles keep many SMs busy on small batches.  The last CTA to finish runs the
+// slot scan.
 #pragma once
 #include "gemm_tc.cuh"
 #include "permute.cuh"
@@ -42,20 +45,33 @@ struct TopK {
 constexpr int kRtSmemBudget = 190 * 1024;
 
 inline int router_tc_epad(int E) { return (E + 15) / 16 * 16; }
-inline int router_tc_stage_bytes(int E) { return kRtTok * kTcBK * 2 + router_tc_epad(E) * kTcBK * 2; }
-inline int router_tc_stages(int E) {
-  int s = kRtSmemBudget / router_tc_stage_bytes(E);
-  return s > 8 ? 8 : s;
+// tokens per CTA: every CTA re-reads the whole router matrix, so tiles shrink only for small
+// batches (measured on B200: 64 is best at T = 2048, 128 at T = 8192)
+inline int router_tc_tok(int T) { return T <= 1024 ? 32 : (T <= 4096 ? 64 : 128); }
+// A stage holds tok token rows and Epad router rows of one 64-column k-block.  (The MMA always
+// reads 128 token rows: those beyond tok fall into neighbouring stage memory and only feed
+// accumulator lanes that nobody reads.)
+inline int router_tc_stage_bytes(int E, int tok) { return tok * kTcBK * 2 + router_tc_epad(E) * kTcBK * 2; }
+constexpr int kRtMaxStages = 16;
+inline int router_tc_stages(int E, int tok) {
+  int s = (kRtSmemBudget - kRtTok * kTcBK * 2) / router_tc_stage_bytes(E, tok);
+  return s > kRtMaxStages ? kRtMaxStages : s;
 }
-inline size_t router_tc_smem_bytes(int E) {
-  return (size_t)router_tc_stages(E) * router_tc_stage_bytes(E) + 2048 +
+inline size_t router_tc_smem_bytes(int E, int tok) {
+  // + one full 128-row tile of slack behind the stages for the MMA's over-read, and room for the
+  // logits tile [tok][E+1] that later reuses the stage memory
+  size_t stages = (size_t)router_tc_stages(E, tok) * router_tc_stage_bytes(E, tok) + kRtTok * kTcBK * 2;
+  const size_t logit_tile = (size_t)tok * (E + 1) * 4;
+  if (stages < logit_tile) stages = logit_tile;
+  return stages + 2048 +
          (sizeof(int) * 2 + sizeof(float)) * kRtTok * kMaxTopK + sizeof(float) * kRtTok +
-         (sizeof(int) + sizeof(float)) * kMaxE + sizeof(uint32_t) * 24;
+         (sizeof(int) + sizeof(float)) * kMaxE + sizeof(uint32_t) * 24 + 1024 + 8 * (2 * kRtMaxStages + 8) +
+         (sizeof(float) + sizeof(int)) * kRtTok * 2 * 4 * kMaxTopK / 4 + sizeof(float) * kRtThreads + 1024;
 }
 
 __global__ void __launch_bounds__(kRtThreads, 1)
 router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW,
-                 const RouterArgs a, int32_t* status, int n_stages) {
+                 const RouterArgs a, int32_t* status, int n_stages, int tok) {
   if ((int)blockIdx.x >= a.scan.n_cta) {
     // ---------------------------------------------------- weight-prefetch blocks
     pdl_wait();
@@ -77,32 +93,39 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   }
   const int E = a.E, k = a.k;
   const int Epad = (E + 15) / 16 * 16;
-  const int a_bytes = kRtTok * kTcBK * 2, b_bytes = Epad * kTcBK * 2;
-  const int stage_bytes = a_bytes + b_bytes;
+  const int a_bytes = tok * kTcBK * 2, b_bytes = Epad * kTcBK * 2;   // token box, router box
+  const int a_box_bytes = a_bytes;
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  unsigned char* sA = smem;
-  unsigned char* sB = smem + n_stages * a_bytes;
-  float* slog = reinterpret_cast<float*>(smem);           // [128][E+1], reuses the stage buffers
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + n_stages * stage_bytes);
-  uint64_t* full = bars;                  // [8]
-  uint64_t* empty = bars + 8;             // [8]
-  uint64_t* acc_full = bars + 16;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
+  // layout: router tiles of all stages, then token tiles of all stages, then 16 KB of slack that
+  // the 128-row MMA read of the last token tile may run into
+  unsigned char* sB = smem;
+  unsigned char* sA = smem + n_stages * b_bytes;
+  float* slog = reinterpret_cast<float*>(smem);           // [tok][E+1], reuses the stage buffers
+  const int stage_area = max(n_stages * (a_bytes + b_bytes) + kRtTok * kTcBK * 2, tok * (E + 1) * 4);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + ((stage_area + 1023) & ~1023));
+  uint64_t* full = bars;                  // [16]
+  uint64_t* empty = bars + kRtMaxStages;  // [16]
+  uint64_t* acc_full = bars + 2 * kRtMaxStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kRtMaxStages + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  int* pe = reinterpret_cast<int*>(bars + 24);            // [128*k] unmasked expert per pair
-  int* ps = pe + kRtTok * kMaxTopK;                       // [128*k] slot per pair
+  int* pe = reinterpret_cast<int*>(bars + 2 * kRtMaxStages + 8);   // [tok*k] unmasked expert per pair
+  int* ps = pe + kRtTok * kMaxTopK;                       // [tok*k] slot per pair
   float* pt = reinterpret_cast<float*>(ps + kRtTok * kMaxTopK);
-  float* snorm = pt + kRtTok * kMaxTopK;                  // [128] ||x_t||
+  float* snorm = pt + kRtTok * kMaxTopK;                  // [tok] ||x_t||
   int* s_e2s = reinterpret_cast<int*>(snorm + kRtTok);    // [256] expert -> slot
   float* s_enorm = reinterpret_cast<float*>(s_e2s + kMaxE);   // [256] ||E_e||
   uint32_t* s_mask = reinterpret_cast<uint32_t*>(s_enorm + kMaxE);  // [2][8] valid / resident bits
   uint32_t* s_present = s_mask + 16;                       // [8] experts selected (unmasked) in this tile
+  float* cand_v = reinterpret_cast<float*>(s_present + 8); // [256 threads][kMaxTopK] per-thread top-k values
+  int* cand_e = reinterpret_cast<int*>(cand_v + kRtThreads * kMaxTopK);   // ... and experts
+  float* part_den = reinterpret_cast<float*>(cand_e + kRtThreads * kMaxTopK);   // [256] partial denominators
+  float* s_m = part_den + kRtThreads;                      // [tok][2] row maximum per gate
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int tok0 = blockIdx.x * kRtTok;
+  const int tok0 = blockIdx.x * tok;
   const int k_blocks = a.d / kTcBK;
 #ifdef SWAPMOE_PHASE_TIMING
   __shared__ unsigned long long dbg[16];
@@ -150,7 +173,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       int stage = 0; uint32_t phase = 0;
       for (int kb = 0; kb < k_blocks; ++kb) {
         if (!bounded_wait(&empty[stage], phase ^ 1u, abort_flag, status, 11)) break;
-        ptx::mbar_expect_tx(&full[stage], (uint32_t)stage_bytes);
+        ptx::mbar_expect_tx(&full[stage], (uint32_t)(a_box_bytes + b_bytes));
         ptx::tma_load_2d(sA + stage * a_bytes, &tmX, &full[stage], kb * kTcBK, tok0);
         ptx::tma_load_2d(sB + stage * b_bytes, &tmW, &full[stage], kb * kTcBK, 0);
         if (++stage == n_stages) { stage = 0; phase ^= 1u; }
@@ -183,37 +206,40 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   } else if (warp >= 4) {
     // ------------------------------------------------ ||x||^2 while the tiles stream through
     const int q = warp - 4, r = q * 32 + lane;
+    const bool warp_has_rows = q * 32 < tok;       // whole warps beyond the token tile only keep the pipeline moving
     float sumsq = 0.f;
     int stage = 0; uint32_t phase = 0;
     bool ok = true;
     for (int kb = 0; kb < k_blocks; ++kb) {
       ok = bounded_wait(&full[stage], phase, abort_flag, status, 13);
       if (!ok) break;
-      const uint4* row = reinterpret_cast<const uint4*>(sA + stage * a_bytes + r * 128);
+      if (warp_has_rows) {
+        const uint4* row = reinterpret_cast<const uint4*>(sA + stage * a_bytes + r * 128);
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        // the 16-byte chunks of a row may be visited in any order: rotate by the row
-        // index so the threads of a quarter-warp hit different banks
-        const uint4 u = row[(c + r) & 7];
-        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+        for (int c = 0; c < 8; ++c) {
+          // the 16-byte chunks of a row may be visited in any order: rotate by the row
+          // index so the threads of a quarter-warp hit different banks
+          const uint4 u = row[(c + r) & 7];
+          const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
-          sumsq = fmaf(lo, lo, sumsq);
-          sumsq = fmaf(hi, hi, sumsq);
+          for (int i = 0; i < 4; ++i) {
+            const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+            sumsq = fmaf(lo, lo, sumsq);
+            sumsq = fmaf(hi, hi, sumsq);
+          }
         }
       }
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&empty[stage]);
       if (++stage == n_stages) { stage = 0; phase ^= 1u; }
     }
-    snorm[r] = sqrtf(sumsq);
+    if (warp_has_rows) snorm[r] = sqrtf(sumsq);
     STAMP(2);
     // ------------------------------------------------ logits: TMEM lane r -> shared-memory row r
     // (all MMAs have completed once acc_full fires, so the stage buffers are free to reuse)
     if (ok) ok = bounded_wait(acc_full, 0, abort_flag, status, 14);
     STAMP(3);
-    if (ok) {
+    if (ok && warp_has_rows) {
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
       float* srow = slog + (size_t)r * (E + 1);
@@ -234,15 +260,10 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     ptx::tmem_dealloc(tmem_base, tmem_cols);
   }
   STAMP(4);
-  // ---------------------------------------------------- gate: two threads per token
-  // Thread t < 128 evaluates the off-the-shelf gate of token t, thread t + 128 its masked
-  // gate (Fig. 4): each scans the token's row of logits in shared memory once for the
-  // top-k (ties -> lowest index, kept by scanning in index order with a strict compare)
-  // and once for the softmax denominator.  No shuffles, no cross-thread dependencies.
   const bool failed = *abort_flag != 0;
   {
     // coalesced copy of the logits: a warp writes a token's row; four rows are in flight
-    const int rows = min(kRtTok, a.T - tok0);
+    const int rows = min(tok, a.T - tok0);
     for (int t0 = warp * 4; t0 < rows; t0 += (kRtThreads / 32) * 4) {
       for (int e = lane; e < E; e += 32) {
         float v[4];
@@ -255,36 +276,42 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     }
   }
   STAMP(8);
+  // ---------------------------------------------------- gate: 256 / tok threads per token
+  // Thread t serves token t % tok.  Its group g = t / tok splits into the gate it evaluates
+  // (first half of the groups: off-the-shelf gate; second half: masked gate) and the share of
+  // the expert range it scans (whole 32-expert chunks, contiguous and ascending per share).
+  const int tl = tid % tok, grp = tid / tok;
+  const int parts = (kRtThreads / tok) >> 1;                // threads per token and gate: 1, 2 or 4
+  const bool masked = grp >= parts;
+  const int part = masked ? grp - parts : grp;
+  const int token = tok0 + tl;
+  const float* row = slog + (size_t)tl * (E + 1);
+  const uint32_t* allow = s_mask + (masked ? 8 : 0);
+  const int n_chunks = (E + 31) >> 5, cpp = (n_chunks + parts - 1) / parts;
+  const int e_lo = min(E, part * cpp * 32), e_hi = min(E, (part + 1) * cpp * 32);
   {
-    const bool masked = tid >= kRtTok;
-    const int tl = tid & (kRtTok - 1);
-    const int tok = tok0 + tl;
-    const float* row = slog + (size_t)tl * (E + 1);
-    const uint32_t* allow = s_mask + (masked ? 8 : 0);
+    // The loops below run once per CTA, so they are kept rolled (short bodies that stay in the
+    // instruction cache) rather than unrolled over the whole expert range.
     TopK tk;
     tk.init();
-    // The loops below run once per CTA, so they are kept rolled (short bodies that stay
-    // in the instruction cache) rather than unrolled over the whole expert range.
     if (k == 1) {
-      // top-1: branch-free running maximum; the first allowed expert seeds it and a strict
-      // compare keeps the lowest index among equal logits
       float best = -INFINITY;
       int bi = -1;
 #pragma unroll 4
-      for (int e = 0; e < E; ++e) {
+      for (int e = e_lo; e < e_hi; ++e) {
         const float l = row[e];
         const bool take = ((allow[e >> 5] >> (e & 31)) & 1u) && (bi < 0 || l > best);
         best = take ? l : best;
         bi = take ? e : bi;
       }
-      tk.v[0] = failed ? 0.f : best;
+      tk.v[0] = best;
       tk.e[0] = bi;
     } else {
       float thr = -INFINITY;
       int filled = 0;
 #pragma unroll 1
-      for (int e = 0; e < E; ++e) {
-        const float l = failed ? 0.f : row[e];
+      for (int e = e_lo; e < e_hi; ++e) {
+        const float l = row[e];
         if (((allow[e >> 5] >> (e & 31)) & 1u) && (filled < k || l > thr)) {
           tk.push(l, e, k);
           ++filled;
@@ -292,38 +319,66 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         }
       }
     }
-    STAMP(9);
-    const float m = tk.v[0];
+#pragma unroll
+    for (int j = 0; j < kMaxTopK; ++j) { cand_v[tid * kMaxTopK + j] = tk.v[j]; cand_e[tid * kMaxTopK + j] = tk.e[j]; }
+  }
+  __syncthreads();
+  STAMP(9);
+  // merge the shares of one (token, gate) in ascending expert order: a candidate only displaces
+  // an entry it strictly beats, so equal logits keep the lowest expert index
+  TopK fin;
+  fin.init();
+  if (part == 0) {
+    for (int pp = 0; pp < parts; ++pp) {
+      const int src = ((masked ? parts : 0) + pp) * tok + tl;
+#pragma unroll
+      for (int j = 0; j < kMaxTopK; ++j)
+        if (j < k && cand_e[src * kMaxTopK + j] >= 0) fin.push(cand_v[src * kMaxTopK + j], cand_e[src * kMaxTopK + j], k);
+    }
+    s_m[tl * 2 + (masked ? 1 : 0)] = fin.v[0];
+  }
+  __syncthreads();
+  {
+    const float m = s_m[tl * 2 + (masked ? 1 : 0)];
+    float den = 0.f;
+    if (!a.renorm) {
+      // eight interleaved partial sums: short dependency chains and a tree-shaped total
+      float acc8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+      for (int e0 = e_lo; e0 < e_hi; e0 += 8) {
+        const uint32_t w = allow[e0 >> 5] >> (e0 & 31);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float t = __expf(row[e0 + i] - m);
+          acc8[i] += ((w >> i) & 1u) ? t : 0.f;
+        }
+      }
+      den = ((acc8[0] + acc8[1]) + (acc8[2] + acc8[3])) + ((acc8[4] + acc8[5]) + (acc8[6] + acc8[7]));
+    }
+    part_den[tid] = den;
+  }
+  __syncthreads();
+  STAMP(10);
+  if (part == 0) {
+    const float m = fin.v[0];
     float den = 0.f;
     if (a.renorm) {
 #pragma unroll
       for (int j = 0; j < kMaxTopK; ++j)
-        if (j < k) den += expf(tk.v[j] - m);
+        if (j < k) den += expf(fin.v[j] - m);
     } else {
-      // eight interleaved partial sums: short dependency chains and a tree-shaped total
-      float part[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
-      for (int e0 = 0; e0 < E; e0 += 8) {
-        const uint32_t w = allow[e0 >> 5] >> (e0 & 31);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float t = __expf((failed ? 0.f : row[e0 + i]) - m);
-          part[i] += ((w >> i) & 1u) ? t : 0.f;
-        }
-      }
-      den = ((part[0] + part[1]) + (part[2] + part[3])) + ((part[4] + part[5]) + (part[6] + part[7]));
+      for (int pp = 0; pp < parts; ++pp) den += part_den[((masked ? parts : 0) + pp) * tok + tl];
     }
-    STAMP(10);
     const float xn = snorm[tl];
 #pragma unroll
     for (int j = 0; j < kMaxTopK; ++j) {
       if (j < k) {
         const int pl = tl * k + j;
-        const size_t p = (size_t)tok * k + j;
-        const float g = expf(tk.v[j] - m) / den;
-        const int e = tk.e[j];
+        const size_t p = (size_t)token * k + j;
+        const float g = failed ? 0.f : expf(fin.v[j] - m) / den;
+        const int e = fin.e[j];
         if (!masked) {
-          if (tok < a.T) {
+          if (token < a.T) {
             a.uidx[p] = e; a.ugate[p] = g;
             pe[pl] = e; pt[pl] = xn * fabsf(g) * s_enorm[e];   // one term of Eq. (1)
             atomicOr(&s_present[e >> 5], 1u << (e & 31));
@@ -331,7 +386,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             pe[pl] = -1; pt[pl] = 0.f;
           }
         } else {
-          if (tok < a.T) {
+          if (token < a.T) {
             const int sl = s_e2s[e];
             a.midx[p] = e; a.mgate[p] = g; a.slot[p] = sl;
             ps[pl] = sl;
@@ -341,15 +396,15 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         }
       }
     }
-    if (!masked && tok < a.T) a.xnorm[tok] = xn;
-    STAMP(11);
+    if (!masked && token < a.T) a.xnorm[token] = xn;
   }
+  STAMP(11);
   __syncthreads();
   STAMP(5);
   // Per-CTA partial sums with a fixed association (lane-strided partials, then the
   // shuffle tree), so the result does not depend on scheduling.  Only experts that some
   // token of this tile selected are visited; the others get an exact zero.
-  const int npair = kRtTok * k;
+  const int npair = tok * k;
   for (int e = tid; e < E; e += kRtThreads) a.cta_imp[(size_t)blockIdx.x * E + e] = 0.f;
   for (int sl = tid; sl < a.K; sl += kRtThreads) a.cta_hist[(size_t)blockIdx.x * a.K + sl] = 0;
   __syncthreads();
@@ -372,13 +427,13 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     c = __reduce_add_sync(0xffffffffu, c);
     if (lane == 0 && c) a.cta_hist[(size_t)blockIdx.x * a.K + sl] = c;
   }
-  finish_router_cta(a.scan);
+  finish_router_cta(a.scan, smem, stage_area);      // the stage memory is free again: stage the scan inputs there
 #ifdef SWAPMOE_PHASE_TIMING
   __syncthreads();
   STAMP(6);
   if (tid == 128)   // phase stamps replace the first logits of this CTA's first token (instrumented build only)
     for (int i = 0; i < 12; ++i)
-      reinterpret_cast<unsigned long long*>(a.logits + (size_t)blockIdx.x * kRtTok * E)[i] = dbg[i];
+      reinterpret_cast<unsigned long long*>(a.logits + (size_t)blockIdx.x * tok * E)[i] = dbg[i];
 #endif
 }
 
