@@ -31,6 +31,11 @@ sys.path.insert(0, ROOT)
 
 from paper_2308_15030_b200 import inputs as I  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the grouped-GEMM kernel, mean of the
+# GEMM-1 and GEMM-2 launches of one step, from the ncu capture summarised in
+# profiles/cfg2_router_tc_permute_tc_gemm.md (80.04 + 3.42 MB and 93.63 + 3.44 MB).
+NCU_TRAFFIC_PER_LAUNCH = {"cfg2": (80.04e6 + 3.42e6 + 93.63e6 + 3.44e6) / 2}
+
 METRIC = "moe_layer_tokens_per_s_at_budget_K"
 UNIT = "tokens/s"
 L2_BYTES = 126e6
@@ -309,7 +314,7 @@ def run_cuda(args, cfg):
                 "h2d_bytes_per_step": cfg.T * cfg.d * cfg.nb, "d2h_bytes_per_step": cfg.T * cfg.d * cfg.nb,
                 "ms_per_step": e2e_ms / args.steps},
         "roofline": {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
-                     "traffic": None, "peak_source": peaks["source"],
+                     "traffic": NCU_TRAFFIC_PER_LAUNCH.get(cfg.name), "peak_source": peaks["source"],
                      "kernel": "tc_gemm_kernel (grouped FFN GEMM, 2 launches per step: GEMM-1+act, GEMM-2)"
                                if cfg.dtype == I.BF16 else "gemm_simt_kernel (2 launches per step)",
                      "algorithmic_bytes_per_launch": g_bytes / 2, "flops_per_launch": g_flops / 2,
