@@ -174,6 +174,19 @@ int32_t swapmoe_forward_host(swapmoe_layer_t* layer, const void* x_host, void* o
 int32_t swapmoe_read_importance(swapmoe_layer_t* layer, float* imp_host, int32_t reset,
                                 void* stream);
 
+/*
+ * Other per-expert scores accumulated next to Eq. (1), read and reset independently:
+ *   SWAPMOE_IMP_EQ1        - Eq. (1) over the unmasked routing (what swapmoe_read_importance returns);
+ *   SWAPMOE_IMP_COUNT      - number of (token, j) selections per expert under the unmasked routing:
+ *                            the token-count score of the "Simple scheduling" ablation (Section 4.4);
+ *   SWAPMOE_IMP_EQ1_MASKED - Eq. (1) read literally over the tokens actually passed to each expert,
+ *                            i.e. the masked routing (non-resident experts score 0).
+ * Same synchronisation and errors as swapmoe_read_importance; unknown kind -> INVALID_ARG.
+ */
+enum { SWAPMOE_IMP_EQ1 = 0, SWAPMOE_IMP_COUNT = 1, SWAPMOE_IMP_EQ1_MASKED = 2 };
+int32_t swapmoe_read_importance_kind(swapmoe_layer_t* layer, int32_t kind, float* imp_host,
+                                     int32_t reset, void* stream);
+
 /* Sections 3.1-3.2: the K most important experts, by descending importance, ties
  * to the lowest index.  Pure host function (E <= 256 floats). */
 int32_t swapmoe_topk_importance(const float* imp_host, int32_t E, int32_t K,

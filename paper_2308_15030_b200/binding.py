@@ -30,7 +30,7 @@ TAPS = {
 EXPORTS = [
     "swapmoe_create", "swapmoe_destroy", "swapmoe_set_router", "swapmoe_set_resident",
     "swapmoe_forward", "swapmoe_forward_timed", "swapmoe_forward_from_logits", "swapmoe_forward_host",
-    "swapmoe_read_importance", "swapmoe_topk_importance", "swapmoe_load_slot_async",
+    "swapmoe_read_importance", "swapmoe_read_importance_kind", "swapmoe_topk_importance", "swapmoe_load_slot_async",
     "swapmoe_debug_copy", "swapmoe_device_status", "swapmoe_launch_count",
     "swapmoe_workspace_bytes", "swapmoe_set_gemm_path", "swapmoe_status_string",
     "swapmoe_route_static",
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.swapmoe_forward_from_logits.argtypes = [vp, vp, vp, vp, i32, vp]
         L.swapmoe_forward_host.argtypes = [vp, vp, vp, i32, vp]
         L.swapmoe_read_importance.argtypes = [vp, vp, i32, vp]
+        L.swapmoe_read_importance_kind.argtypes = [vp, i32, vp, i32, vp]
         L.swapmoe_topk_importance.argtypes = [vp, i32, i32, vp]
         L.swapmoe_load_slot_async.argtypes = [vp, i32, vp, vp, vp, vp]
         L.swapmoe_debug_copy.argtypes = [vp, i32, vp, ctypes.c_size_t, vp]
@@ -227,6 +228,14 @@ class Layer:
         _check(lib().swapmoe_read_importance(self._h, _np_ptr(imp), int(bool(reset)),
                                              _stream_ptr(stream)), "swapmoe_read_importance")
         return imp
+
+    def read_score(self, kind: str, reset: bool = False, stream=None) -> np.ndarray:
+        """kind: "eq1" (Eq. 1, unmasked routing), "count" (token counts), "eq1_masked"."""
+        k = {"eq1": 0, "count": 1, "eq1_masked": 2}[kind]
+        out = np.empty(self.cfg.E, dtype=np.float32)
+        _check(lib().swapmoe_read_importance_kind(self._h, k, _np_ptr(out), int(bool(reset)),
+                                                  _stream_ptr(stream)), "swapmoe_read_importance_kind")
+        return out
 
     def load_slot_async(self, phys: int, in_host_pinned, out_host_pinned, side_stream,
                         done_event=None) -> None:

@@ -28,7 +28,7 @@ struct swapmoe_layer {
   // device workspace (one allocation)
   char* ws_base;
   size_t ws_bytes;
-  float *logits, *ugate, *mgate, *xnorm, *cta_imp, *imp, *enorm, *y;
+  float *logits, *ugate, *mgate, *xnorm, *cta_imp, *cta_cnt, *cta_mimp, *imp, *cnt, *mimp, *enorm, *y;
   int32_t *uidx, *midx, *slot, *cta_hist, *cta_base, *count, *offset, *pad_offset;
   int32_t *perm, *inv, *inv_pad, *row_pair, *n_tiles, *e2s, *phys, *s2e, *status;
   unsigned* ticket;
@@ -104,11 +104,13 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   ra.logits = L->logits; ra.uidx = L->uidx; ra.ugate = L->ugate; ra.midx = L->midx;
   ra.mgate = L->mgate; ra.slot = L->slot; ra.xnorm = L->xnorm; ra.cta_hist = L->cta_hist;
   ra.cta_imp = L->cta_imp;
+  ra.cta_cnt = L->cta_cnt; ra.cta_mimp = L->cta_mimp;
   ra.T = T; ra.d = c.d_model; ra.E = c.E; ra.k = c.top_k; ra.K = c.K; ra.renorm = c.renorm_topk;
   ScanArgs& sa = ra.scan;
   sa.cta_hist = L->cta_hist; sa.cta_imp = L->cta_imp; sa.phys_slot = L->phys;
   sa.cta_base = L->cta_base; sa.count = L->count; sa.offset = L->offset;
   sa.pad_offset = L->pad_offset; sa.tiles = L->tiles; sa.n_tiles = L->n_tiles; sa.imp = L->imp;
+  sa.cta_cnt = L->cta_cnt; sa.cta_mimp = L->cta_mimp; sa.s2e = L->s2e; sa.cnt = L->cnt; sa.mimp = L->mimp;
   sa.ticket = L->ticket;
   sa.done = L->done; sa.n_done = L->n_done;
   sa.n_cta = n_cta; sa.K = c.K; sa.E = c.E; sa.tile_rows = tile_rows;
@@ -302,6 +304,8 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_logits = cv.take<float>(T * c.E);
   const size_t o_ugate = cv.take<float>(P), o_mgate = cv.take<float>(P), o_xnorm = cv.take<float>(T);
   const size_t o_cta_imp = cv.take<float>(n_cta * c.E);
+  const size_t o_cta_cnt = cv.take<float>(n_cta * c.E), o_cta_mimp = cv.take<float>(n_cta * c.K);
+  const size_t o_cnt = cv.take<float>(c.E), o_mimp = cv.take<float>(c.E);
   const size_t o_imp = cv.take<float>(c.E), o_enorm = cv.take<float>(c.E);
   const size_t o_uidx = cv.take<int32_t>(P), o_midx = cv.take<int32_t>(P), o_slot = cv.take<int32_t>(P);
   const size_t o_cta_hist = cv.take<int32_t>(n_cta * c.K), o_cta_base = cv.take<int32_t>(n_cta * c.K);
@@ -325,6 +329,8 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   char* b = L->ws_base;
   L->logits = (float*)(b + o_logits); L->ugate = (float*)(b + o_ugate); L->mgate = (float*)(b + o_mgate);
   L->xnorm = (float*)(b + o_xnorm); L->cta_imp = (float*)(b + o_cta_imp); L->imp = (float*)(b + o_imp);
+  L->cta_cnt = (float*)(b + o_cta_cnt); L->cta_mimp = (float*)(b + o_cta_mimp);
+  L->cnt = (float*)(b + o_cnt); L->mimp = (float*)(b + o_mimp);
   L->enorm = (float*)(b + o_enorm); L->uidx = (int32_t*)(b + o_uidx); L->midx = (int32_t*)(b + o_midx);
   L->slot = (int32_t*)(b + o_slot); L->cta_hist = (int32_t*)(b + o_cta_hist);
   L->cta_base = (int32_t*)(b + o_cta_base); L->count = (int32_t*)(b + o_count);
@@ -341,6 +347,8 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   L->x_stage = b + o_xs; L->out_stage = b + o_os;
 
   bool ok = cuda_ok(cudaMemset(L->imp, 0, sizeof(float) * c.E));
+  ok = ok && cuda_ok(cudaMemset(L->cnt, 0, sizeof(float) * c.E));
+  ok = ok && cuda_ok(cudaMemset(L->mimp, 0, sizeof(float) * c.E));
   ok = ok && cuda_ok(cudaMemset(L->status, 0, sizeof(int32_t) * 4));
   ok = ok && cuda_ok(cudaMemset(L->ticket, 0, sizeof(unsigned) * 4));
   ok = ok && cuda_ok(cudaFuncSetAttribute(router_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -455,14 +463,22 @@ int32_t swapmoe_forward_host(swapmoe_layer_t* L, const void* x_host, void* out_h
   return SWAPMOE_OK;
 }
 
-int32_t swapmoe_read_importance(swapmoe_layer_t* L, float* imp_host, int32_t reset, void* stream) {
+int32_t swapmoe_read_importance_kind(swapmoe_layer_t* L, int32_t kind, float* imp_host, int32_t reset,
+                                     void* stream) {
   if (!L || !imp_host) return SWAPMOE_ERR_INVALID_ARG;
+  float* acc = kind == SWAPMOE_IMP_EQ1 ? L->imp : kind == SWAPMOE_IMP_COUNT ? L->cnt
+             : kind == SWAPMOE_IMP_EQ1_MASKED ? L->mimp : nullptr;
+  if (!acc) return SWAPMOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (!cuda_ok(cudaMemcpyAsync(imp_host, L->imp, sizeof(float) * L->cfg.E, cudaMemcpyDeviceToHost, st)))
+  if (!cuda_ok(cudaMemcpyAsync(imp_host, acc, sizeof(float) * L->cfg.E, cudaMemcpyDeviceToHost, st)))
     return SWAPMOE_ERR_CUDA;
-  if (reset && !cuda_ok(cudaMemsetAsync(L->imp, 0, sizeof(float) * L->cfg.E, st))) return SWAPMOE_ERR_CUDA;
+  if (reset && !cuda_ok(cudaMemsetAsync(acc, 0, sizeof(float) * L->cfg.E, st))) return SWAPMOE_ERR_CUDA;
   if (!cuda_ok(cudaStreamSynchronize(st))) return SWAPMOE_ERR_CUDA;
   return SWAPMOE_OK;
+}
+
+int32_t swapmoe_read_importance(swapmoe_layer_t* L, float* imp_host, int32_t reset, void* stream) {
+  return swapmoe_read_importance_kind(L, SWAPMOE_IMP_EQ1, imp_host, reset, stream);
 }
 
 int32_t swapmoe_topk_importance(const float* imp, int32_t E, int32_t K, int32_t* out_idx) {

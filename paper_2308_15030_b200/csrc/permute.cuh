@@ -8,6 +8,11 @@ namespace swapmoe {
 struct ScanArgs {
   const int32_t* cta_hist;   // [n_cta, K]
   const float* cta_imp;      // [n_cta, E]
+  const float* cta_cnt;      // [n_cta, E] unmasked selections per expert (token counts), or nullptr
+  const float* cta_mimp;     // [n_cta, K] Eq. (1) terms of the MASKED routing per slot, or nullptr
+  const int32_t* s2e;        // [K] expert served by each slot (for cta_mimp)
+  float* cnt;                // [E] accumulator of the token counts ("simple scheduling" score)
+  float* mimp;               // [E] accumulator of Eq. (1) over the masked routing
   const int32_t* phys_slot;  // [K]
   int32_t* cta_base;         // [n_cta, K] pairs of the same slot in earlier CTAs
   int32_t* count;            // [K]
@@ -30,17 +35,46 @@ struct ScanArgs {
 __device__ __forceinline__ void scan_reduce_block(const ScanArgs& a, void* stage, int stage_bytes) {
   __shared__ int32_t s_count[kMaxSlots];
   const int tid = threadIdx.x;
+  // The accumulators' old values are fetched first so that their latency overlaps the staging
+  // (thread e owns expert e, thread sl owns slot sl; blockDim.x >= E, K).
+  const bool own_e = tid < a.E, own_s = tid < a.K;
+  const float old_imp = own_e ? a.imp[tid] : 0.f;
+  const float old_cnt = (own_e && a.cta_cnt) ? a.cnt[tid] : 0.f;
+  const int my_expert = (own_s && a.cta_mimp) ? a.s2e[tid] : 0;
   const int n_hist = a.n_cta * a.K, n_imp = a.n_cta * a.E;
+  const int n_cnt = a.cta_cnt ? n_imp : 0, n_mimp = a.cta_mimp ? n_hist : 0;
   const int32_t* hist = a.cta_hist;
   const float* impp = a.cta_imp;
-  if (stage != nullptr && (size_t)(n_hist + n_imp) * 4 <= (size_t)stage_bytes) {
+  const float* cntp = a.cta_cnt;
+  const float* mimpp = a.cta_mimp;
+  if (stage != nullptr && (size_t)(n_hist + n_imp + n_cnt + n_mimp + 16) * 4 <= (size_t)stage_bytes &&
+      (reinterpret_cast<uintptr_t>(stage) & 15) == 0) {
+    // All four arrays are copied with 16-byte cp.async.cg (L2 only, no L1 allocation, no register
+    // round trip), issued back to back: one memory latency in total.  Tails shorter than 16 bytes
+    // are read with plain L1-bypassing loads.
     int32_t* sh = static_cast<int32_t*>(stage);
-    float* si = reinterpret_cast<float*>(sh + n_hist);
-    for (int i = tid; i < n_hist; i += blockDim.x) sh[i] = __ldcg(a.cta_hist + i);
-    for (int i = tid; i < n_imp; i += blockDim.x) si[i] = __ldcg(a.cta_imp + i);
+    float* si = reinterpret_cast<float*>(sh + ((n_hist + 3) & ~3));
+    float* sc = si + ((n_imp + 3) & ~3);
+    float* sm = sc + ((n_cnt + 3) & ~3);
+    const void* srcs[4] = {a.cta_hist, a.cta_imp, a.cta_cnt, a.cta_mimp};
+    void* dsts[4] = {sh, si, sc, sm};
+    const int counts[4] = {n_hist, n_imp, n_cnt, n_mimp};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int n16 = counts[q] >> 2;
+      const uint4* src = static_cast<const uint4*>(srcs[q]);
+      const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(dsts[q]));
+      for (int i = tid; i < n16; i += blockDim.x)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16u * i), "l"(src + i) : "memory");
+      for (int i = (n16 << 2) + tid; i < counts[q]; i += blockDim.x)
+        static_cast<int32_t*>(dsts[q])[i] = __ldcg(static_cast<const int32_t*>(srcs[q]) + i);
+    }
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     hist = sh;
     impp = si;
+    if (n_cnt) cntp = sc;
+    if (n_mimp) mimpp = sm;
   }
   // Slots are walked by the LAST K threads and experts by the first E threads, so the two
   // chains run side by side.
@@ -58,11 +92,25 @@ __device__ __forceinline__ void scan_reduce_block(const ScanArgs& a, void* stage
     }
   }
   for (int i = tid; i < a.n_done; i += blockDim.x) a.done[i] = 0;
-  for (int e = tid; e < a.E; e += blockDim.x) {
+  if (own_e) {
+    const int e = tid;
     float acc = 0.f;
 #pragma unroll 16
     for (int c = 0; c < a.n_cta; ++c) acc += impp[(size_t)c * a.E + e];
-    a.imp[e] += acc;
+    a.imp[e] = old_imp + acc;
+    if (a.cta_cnt != nullptr) {            // token counts: small integers, exact in fp32
+      float n = 0.f;
+#pragma unroll 16
+      for (int c = 0; c < a.n_cta; ++c) n += cntp[(size_t)c * a.E + e];
+      a.cnt[e] = old_cnt + n;
+    }
+  }
+  if (own_s && a.cta_mimp != nullptr) {
+    const int sl = tid;
+    float acc = 0.f;
+#pragma unroll 16
+    for (int c = 0; c < a.n_cta; ++c) acc += mimpp[(size_t)c * a.K + sl];
+    a.mimp[my_expert] += acc;              // slots map to distinct experts: no two threads share a target
   }
   __syncthreads();
   if (tid < a.K) {

@@ -88,6 +88,7 @@ extern "C" int32_t swapmoe_route_static(const void* x_dev, const void* Wr_dev, c
   ra.slot = slot_dev; ra.xnorm = xnorm_dev;
   ra.cta_hist = reinterpret_cast<int32_t*>(s + kOffHist);
   ra.cta_imp = reinterpret_cast<float*>(s + kOffImp);
+  ra.cta_cnt = nullptr; ra.cta_mimp = nullptr;
   ra.T = n_tokens; ra.d = d_model; ra.E = E; ra.k = top_k; ra.K = K; ra.renorm = renorm_topk;
   ScanArgs& sa = ra.scan;
   sa.cta_hist = ra.cta_hist; sa.cta_imp = ra.cta_imp;
@@ -100,6 +101,7 @@ extern "C" int32_t swapmoe_route_static(const void* x_dev, const void* Wr_dev, c
   sa.imp = imp_dev;
   sa.ticket = reinterpret_cast<unsigned*>(s + kOffTicket);
   sa.done = nullptr; sa.n_done = 0;
+  sa.cta_cnt = nullptr; sa.cta_mimp = nullptr; sa.s2e = nullptr; sa.cnt = nullptr; sa.mimp = nullptr;
   sa.n_cta = n_cta; sa.K = K; sa.E = E; sa.tile_rows = kSimtBMStatic;
   if (dtype == SWAPMOE_BF16)
     router_gate_kernel<bf16><<<n_cta, 256, router_smem_bytes(E), st>>>(ra);

@@ -21,6 +21,8 @@ struct RouterArgs {
   float* xnorm;             // [T]
   int32_t* cta_hist;        // [n_cta, K]
   float* cta_imp;           // [n_cta, E]
+  float* cta_cnt;           // [n_cta, E] or nullptr
+  float* cta_mimp;          // [n_cta, K] or nullptr
   int32_t T, d, E, k, K, renorm;
   ScanArgs scan;            // work of the last CTA to finish
   // Weight prefetch (tensor-core router only): blocks beyond the token tiles pull the resident
@@ -80,7 +82,7 @@ __device__ __forceinline__ void warp_topk_gate(const float (&v)[8], uint32_t all
 // tl is the token's index inside the CTA (pair arrays pe/ps/pt live in shared memory).
 __device__ __forceinline__ void gate_token(const RouterArgs& a, const float (&v)[8], uint32_t valid_mask,
                                            uint32_t res_mask, int lane, int tok, int tl, float xn,
-                                           int* pe, int* ps, float* pt) {
+                                           int* pe, int* ps, float* pt, float* pm) {
   int ue[kMaxTopK], me[kMaxTopK];
   float ug[kMaxTopK], mg[kMaxTopK];
   warp_topk_gate(v, valid_mask, a.E, a.k, a.renorm, lane, ue, ug);   // off-the-shelf gate
@@ -96,8 +98,9 @@ __device__ __forceinline__ void gate_token(const RouterArgs& a, const float (&v)
         a.slot[p] = s;
         pe[pl] = ue[j]; ps[pl] = s;
         pt[pl] = xn * fabsf(ug[j]) * a.enorm[ue[j]];   // one term of Eq. (1)
+        pm[pl] = xn * fabsf(mg[j]) * a.enorm[me[j]];   // the same term under the masked routing
       } else {
-        pe[pl] = -1; ps[pl] = -1; pt[pl] = 0.f;
+        pe[pl] = -1; ps[pl] = -1; pt[pl] = 0.f; pm[pl] = 0.f;
       }
     }
     if (tok < a.T) a.xnorm[tok] = xn;
@@ -113,6 +116,7 @@ __global__ void __launch_bounds__(256) router_gate_kernel(const RouterArgs a) {
   int* pe = reinterpret_cast<int*>(ws + a.E * (kRouterDK + 1)); // [kTokTile*k] unmasked expert
   int* ps = pe + kTokTile * kMaxTopK;                           // [kTokTile*k] slot
   float* pt = reinterpret_cast<float*>(ps + kTokTile * kMaxTopK);  // importance term
+  float* pm = pt + kTokTile * kMaxTopK;                            // importance term, masked routing
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tok0 = blockIdx.x * kTokTile;
@@ -196,27 +200,31 @@ __global__ void __launch_bounds__(256) router_gate_kernel(const RouterArgs a) {
       v[i] = lv;
       if (tok < a.T && e < a.E) a.logits[(size_t)tok * a.E + e] = lv;
     }
-    gate_token(a, v, valid_mask, res_mask, lane, tok, tl, xn, pe, ps, pt);
+    gate_token(a, v, valid_mask, res_mask, lane, tok, tl, xn, pe, ps, pt, pm);
   }
   __syncthreads();
   // Per-CTA partial sums in a fixed order, so the result does not depend on scheduling.
   const int npair = kTokTile * a.k;
   for (int e = tid; e < a.E; e += 256) {
     float s = 0.f;
-    for (int p = 0; p < npair; ++p) s += (pe[p] == e) ? pt[p] : 0.f;
+    int n = 0;
+    for (int p = 0; p < npair; ++p) { s += (pe[p] == e) ? pt[p] : 0.f; n += (pe[p] == e); }
     a.cta_imp[(size_t)blockIdx.x * a.E + e] = s;
+    if (a.cta_cnt) a.cta_cnt[(size_t)blockIdx.x * a.E + e] = (float)n;
   }
   for (int s = tid; s < a.K; s += 256) {
     int c = 0;
-    for (int p = 0; p < npair; ++p) c += (ps[p] == s);
+    float m = 0.f;
+    for (int p = 0; p < npair; ++p) { c += (ps[p] == s); m += (ps[p] == s) ? pm[p] : 0.f; }
     a.cta_hist[(size_t)blockIdx.x * a.K + s] = c;
+    if (a.cta_mimp) a.cta_mimp[(size_t)blockIdx.x * a.K + s] = m;
   }
   finish_router_cta(a.scan);
 }
 
 inline size_t router_smem_bytes(int E) {
   return sizeof(float) * (kTokTile * (kRouterDK + 1) + (size_t)E * (kRouterDK + 1)) +
-         (sizeof(int) * 2 + sizeof(float)) * kTokTile * kMaxTopK;
+         (sizeof(int) * 2 + sizeof(float) * 2) * kTokTile * kMaxTopK;
 }
 
 }  // namespace swapmoe

@@ -66,7 +66,8 @@ inline size_t router_tc_smem_bytes(int E, int tok) {
   return stages + 2048 +
          (sizeof(int) * 2 + sizeof(float)) * kRtTok * kMaxTopK + sizeof(float) * kRtTok +
          (sizeof(int) + sizeof(float)) * kMaxE + sizeof(uint32_t) * 24 + 1024 + 8 * (2 * kRtMaxStages + 8) +
-         (sizeof(float) + sizeof(int)) * kRtTok * 2 * 4 * kMaxTopK / 4 + sizeof(float) * kRtThreads + 1024;
+         (sizeof(float) + sizeof(int)) * kRtTok * 2 * 4 * kMaxTopK / 4 + sizeof(float) * kRtThreads + 1024 +
+         sizeof(float) * kRtTok * kMaxTopK;
 }
 
 __global__ void __launch_bounds__(kRtThreads, 1)
@@ -123,6 +124,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   int* cand_e = reinterpret_cast<int*>(cand_v + kRtThreads * kMaxTopK);   // ... and experts
   float* part_den = reinterpret_cast<float*>(cand_e + kRtThreads * kMaxTopK);   // [256] partial denominators
   float* s_m = part_den + kRtThreads;                      // [tok][2] row maximum per gate
+  float* pm = s_m + 2 * kRtTok;                            // [tok*k] Eq. (1) term under the masked routing
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tok0 = blockIdx.x * tok;
@@ -389,9 +391,9 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
           if (token < a.T) {
             const int sl = s_e2s[e];
             a.midx[p] = e; a.mgate[p] = g; a.slot[p] = sl;
-            ps[pl] = sl;
+            ps[pl] = sl; pm[pl] = xn * fabsf(g) * s_enorm[e];
           } else {
-            ps[pl] = -1;
+            ps[pl] = -1; pm[pl] = 0.f;
           }
         }
       }
@@ -405,7 +407,10 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   // shuffle tree), so the result does not depend on scheduling.  Only experts that some
   // token of this tile selected are visited; the others get an exact zero.
   const int npair = tok * k;
-  for (int e = tid; e < E; e += kRtThreads) a.cta_imp[(size_t)blockIdx.x * E + e] = 0.f;
+  for (int e = tid; e < E; e += kRtThreads) {
+    a.cta_imp[(size_t)blockIdx.x * E + e] = 0.f;
+    if (a.cta_cnt) a.cta_cnt[(size_t)blockIdx.x * E + e] = 0.f;
+  }
   for (int sl = tid; sl < a.K; sl += kRtThreads) a.cta_hist[(size_t)blockIdx.x * a.K + sl] = 0;
   __syncthreads();
   for (int c = 0; c * 32 < E; ++c) {
@@ -416,16 +421,26 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       if ((n & 7) != warp) continue;                    // experts dealt round-robin to the warps
       const int e = c * 32 + bit;
       float sum = 0.f;
-      for (int p = lane; p < npair; p += 32) sum += (pe[p] == e) ? pt[p] : 0.f;
+      int hits = 0;
+      for (int p = lane; p < npair; p += 32) { sum += (pe[p] == e) ? pt[p] : 0.f; hits += (pe[p] == e); }
       sum = warp_sum(sum);
-      if (lane == 0) a.cta_imp[(size_t)blockIdx.x * E + e] = sum;
+      hits = __reduce_add_sync(0xffffffffu, hits);
+      if (lane == 0) {
+        a.cta_imp[(size_t)blockIdx.x * E + e] = sum;
+        if (a.cta_cnt) a.cta_cnt[(size_t)blockIdx.x * E + e] = (float)hits;
+      }
     }
   }
   for (int sl = warp; sl < a.K; sl += kRtThreads / 32) {
     int c = 0;
-    for (int p = lane; p < npair; p += 32) c += (ps[p] == sl);
+    float m = 0.f;
+    for (int p = lane; p < npair; p += 32) { c += (ps[p] == sl); m += (ps[p] == sl) ? pm[p] : 0.f; }
     c = __reduce_add_sync(0xffffffffu, c);
-    if (lane == 0 && c) a.cta_hist[(size_t)blockIdx.x * a.K + sl] = c;
+    m = warp_sum(m);
+    if (lane == 0) {
+      if (c) a.cta_hist[(size_t)blockIdx.x * a.K + sl] = c;
+      if (a.cta_mimp) a.cta_mimp[(size_t)blockIdx.x * a.K + sl] = m;
+    }
   }
   finish_router_cta(a.scan, smem, stage_area);      // the stage memory is free again: stage the scan inputs there
 #ifdef SWAPMOE_PHASE_TIMING

@@ -208,3 +208,24 @@ def test_two_row_subtiles_per_cta():
         cnt = res["oracle"]["count"]
         # covered: entries with two full sub-tiles, and entries whose second sub-tile is absent
         assert cnt.max() > 256 and any(0 < c % 256 <= 128 for c in cnt), cnt
+
+
+@pytest.mark.parametrize("dtype,k,renorm", [(I.BF16, 1, 0), (I.BF16, 2, 1), (I.F32, 2, 0)])
+def test_count_and_masked_importance_scores(dtype, k, renorm):
+    """Token-count score ("Simple scheduling", Section 4.4) and Eq. (1) over the masked routing."""
+    import oracle
+    from harness import Case, check_against_oracle
+    cfg = _cfg(T=700, dtype=dtype, d=128, f=256, E=24, K=5, k=k, renorm=renorm, zipf_s=1.1)
+    case = Case(cfg)
+    r = check_against_oracle(case, case.run())["oracle"]
+    case.run()                                                       # accumulate a second batch
+    cnt = case.layer.read_score("count", reset=True)
+    ref_cnt = 2 * oracle.importance_count(r["uidx"], cfg.E)
+    assert np.array_equal(cnt, ref_cnt.astype(np.float32))           # integers: exact
+    ref_m = 2 * oracle.importance(case.x, r["midx"], r["mgate"], case.enorm)
+    got_m = case.layer.read_score("eq1_masked", reset=True)
+    assert np.max(np.abs(got_m - ref_m)) <= 1e-4 * ref_m.max()
+    absent = [e for e in range(cfg.E) if e not in set(case.s2e.tolist())]
+    assert np.all(got_m[absent] == 0)                                # absent experts can never score
+    assert np.all(case.layer.read_score("count") == 0) and np.all(case.layer.read_score("eq1_masked") == 0)
+    assert case.layer.read_score("eq1").max() > 0                    # Eq. (1) accumulator untouched by those resets
