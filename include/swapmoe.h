@@ -165,6 +165,18 @@ int32_t swapmoe_forward_timed(swapmoe_layer_t* layer, const void* x_dev, void* o
 int32_t swapmoe_forward_host(swapmoe_layer_t* layer, const void* x_host, void* out_host,
                              int32_t n_tokens, void* stream);
 
+/* Pipelined form of swapmoe_forward_host for streams of requests: the copy of x_host (PINNED)
+ * into the layer's staging buffer runs on a copy stream owned by the layer, the forward on
+ * `stream` behind it, the copy of the result to out_host (PINNED) on a second copy stream; the
+ * call returns at once.  x_host must stay untouched, and out_host is defined, only after
+ * swapmoe_host_wait(layer) has returned.  Calls on one layer queue up behind each other (one
+ * staging buffer each way); calls on different layers overlap their copies with each other's
+ * compute.  Same errors as swapmoe_forward_host. */
+int32_t swapmoe_forward_host_async(swapmoe_layer_t* layer, const void* x_host, void* out_host,
+                                   int32_t n_tokens, void* stream);
+/* Blocks until the most recent swapmoe_forward_host_async of this layer has delivered out_host. */
+int32_t swapmoe_host_wait(swapmoe_layer_t* layer);
+
 /*
  * Eq. (1): importance(E_i, X) = sum_{x in X_i} ||x|| * |G(x)_i| * ||E_i||, X_i =
  * tokens whose unmasked top-k contains i, accumulated over every forward since

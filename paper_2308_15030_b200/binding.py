@@ -30,6 +30,7 @@ TAPS = {
 EXPORTS = [
     "swapmoe_create", "swapmoe_destroy", "swapmoe_set_router", "swapmoe_set_resident",
     "swapmoe_forward", "swapmoe_forward_timed", "swapmoe_forward_from_logits", "swapmoe_forward_host",
+    "swapmoe_forward_host_async", "swapmoe_host_wait",
     "swapmoe_read_importance", "swapmoe_read_importance_kind", "swapmoe_topk_importance", "swapmoe_load_slot_async",
     "swapmoe_debug_copy", "swapmoe_device_status", "swapmoe_launch_count",
     "swapmoe_workspace_bytes", "swapmoe_set_gemm_path", "swapmoe_status_string",
@@ -70,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.swapmoe_forward_timed.argtypes = [vp, vp, vp, i32, vp, ctypes.POINTER(vp)]
         L.swapmoe_forward_from_logits.argtypes = [vp, vp, vp, vp, i32, vp]
         L.swapmoe_forward_host.argtypes = [vp, vp, vp, i32, vp]
+        L.swapmoe_forward_host_async.argtypes = [vp, vp, vp, i32, vp]
+        L.swapmoe_host_wait.argtypes = [vp]
         L.swapmoe_read_importance.argtypes = [vp, vp, i32, vp]
         L.swapmoe_read_importance_kind.argtypes = [vp, i32, vp, i32, vp]
         L.swapmoe_topk_importance.argtypes = [vp, i32, i32, vp]
@@ -221,6 +224,16 @@ class Layer:
         op = out_host.data_ptr() if hasattr(out_host, "data_ptr") else out_host.ctypes.data
         _check(lib().swapmoe_forward_host(self._h, xp, op, T, _stream_ptr(stream)),
                "swapmoe_forward_host")
+
+    def forward_host_async(self, x_host, out_host, n_tokens: Optional[int] = None, stream=None) -> None:
+        """Pipelined host path (pinned CPU tensors); out_host is valid after host_wait()."""
+        T = int(x_host.shape[0]) if n_tokens is None else int(n_tokens)
+        self.last_T = T
+        _check(lib().swapmoe_forward_host_async(self._h, x_host.data_ptr(), out_host.data_ptr(), T,
+                                                _stream_ptr(stream)), "swapmoe_forward_host_async")
+
+    def host_wait(self) -> None:
+        _check(lib().swapmoe_host_wait(self._h), "swapmoe_host_wait")
 
     # -- importance and swapping
     def read_importance(self, reset: bool = False, stream=None) -> np.ndarray:

@@ -47,6 +47,8 @@ struct swapmoe_layer {
   int32_t rows_pad_max;
   int32_t sm_count;
   bool use_pdl;                // programmatic dependent launch between the kernels of a forward
+  cudaStream_t s_in, s_out;    // private copy streams of the asynchronous host path
+  cudaEvent_t ev_in, ev_comp, ev_out;
   int32_t router_tok;          // 0 = automatic token-tile size of the tensor-core router, else 32/64/128
   bool prefetch;               // pull resident weights into L2 from the router kernel
   long long l2_prefetch_bytes; // how much of them (L2 capacity minus head room)
@@ -363,6 +365,11 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)router_smem_bytes(kMaxE)));
   ok = ok && tc_init(L->tc, c, L->xp, L->h, L->y, L->rows_pad_max) == SWAPMOE_OK;
+  ok = ok && cuda_ok(cudaStreamCreateWithFlags(&L->s_in, cudaStreamNonBlocking));
+  ok = ok && cuda_ok(cudaStreamCreateWithFlags(&L->s_out, cudaStreamNonBlocking));
+  ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_in, cudaEventDisableTiming));
+  ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_comp, cudaEventDisableTiming));
+  ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_out, cudaEventDisableTiming));
   if (!ok) { cudaGetLastError(); cudaFree(L->ws_base); delete L; return SWAPMOE_ERR_CUDA; }
   *out = L;
   return SWAPMOE_OK;
@@ -370,6 +377,11 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
 
 int32_t swapmoe_destroy(swapmoe_layer_t* L) {
   if (!L) return SWAPMOE_OK;
+  if (L->s_in) cudaStreamDestroy(L->s_in);
+  if (L->s_out) cudaStreamDestroy(L->s_out);
+  if (L->ev_in) cudaEventDestroy(L->ev_in);
+  if (L->ev_comp) cudaEventDestroy(L->ev_comp);
+  if (L->ev_out) cudaEventDestroy(L->ev_out);
   cudaFree(L->ws_base);
   delete L;
   return SWAPMOE_OK;
@@ -461,6 +473,38 @@ int32_t swapmoe_forward_host(swapmoe_layer_t* L, const void* x_host, void* out_h
   if (!cuda_ok(cudaMemcpyAsync(out_host, L->out_stage, bytes, cudaMemcpyDeviceToHost, st))) return SWAPMOE_ERR_CUDA;
   if (!cuda_ok(cudaStreamSynchronize(st))) return SWAPMOE_ERR_CUDA;
   return SWAPMOE_OK;
+}
+
+int32_t swapmoe_forward_host_async(swapmoe_layer_t* L, const void* x_host, void* out_host, int32_t T,
+                                   void* stream) {
+  if (!L || T < 0) return SWAPMOE_ERR_INVALID_ARG;
+  if (T == 0) return SWAPMOE_OK;
+  if (!x_host || !out_host) return SWAPMOE_ERR_INVALID_ARG;
+  if (T > L->cfg.max_tokens) return SWAPMOE_ERR_TOO_MANY_TOKENS;
+  if (!L->router_set || !L->resident_set) return SWAPMOE_ERR_NOT_READY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)T * L->cfg.d_model * L->elem;
+  // copy-in stream: the staging buffer is free once the previous forward of this layer has run
+  bool ok = cuda_ok(cudaStreamWaitEvent(L->s_in, L->ev_comp, 0));
+  ok = ok && cuda_ok(cudaMemcpyAsync(L->x_stage, x_host, bytes, cudaMemcpyHostToDevice, L->s_in));
+  ok = ok && cuda_ok(cudaEventRecord(L->ev_in, L->s_in));
+  // compute stream: needs the tokens, and the output staging buffer must have been copied out
+  ok = ok && cuda_ok(cudaStreamWaitEvent(st, L->ev_in, 0));
+  ok = ok && cuda_ok(cudaStreamWaitEvent(st, L->ev_out, 0));
+  if (!ok) return SWAPMOE_ERR_CUDA;
+  const int32_t rc = forward_checked(L, L->x_stage, nullptr, L->out_stage, T, stream);
+  if (rc != SWAPMOE_OK) return rc;
+  ok = cuda_ok(cudaEventRecord(L->ev_comp, st));
+  // copy-out stream
+  ok = ok && cuda_ok(cudaStreamWaitEvent(L->s_out, L->ev_comp, 0));
+  ok = ok && cuda_ok(cudaMemcpyAsync(out_host, L->out_stage, bytes, cudaMemcpyDeviceToHost, L->s_out));
+  ok = ok && cuda_ok(cudaEventRecord(L->ev_out, L->s_out));
+  return ok ? SWAPMOE_OK : SWAPMOE_ERR_CUDA;
+}
+
+int32_t swapmoe_host_wait(swapmoe_layer_t* L) {
+  if (!L) return SWAPMOE_ERR_INVALID_ARG;
+  return cuda_ok(cudaEventSynchronize(L->ev_out)) ? SWAPMOE_OK : SWAPMOE_ERR_CUDA;
 }
 
 int32_t swapmoe_read_importance_kind(swapmoe_layer_t* L, int32_t kind, float* imp_host, int32_t reset,

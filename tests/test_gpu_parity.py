@@ -229,3 +229,23 @@ def test_count_and_masked_importance_scores(dtype, k, renorm):
     assert np.all(got_m[absent] == 0)                                # absent experts can never score
     assert np.all(case.layer.read_score("count") == 0) and np.all(case.layer.read_score("eq1_masked") == 0)
     assert case.layer.read_score("eq1").max() > 0                    # Eq. (1) accumulator untouched by those resets
+
+
+def test_host_paths_sync_and_pipelined():
+    """swapmoe_forward_host and the pipelined swapmoe_forward_host_async give the device path's bits."""
+    import torch
+    from harness import Case, to_host_f32
+    cfg = _cfg(T=300, d=128, f=256, E=16, K=5)
+    case = Case(cfg)
+    ref = case.run().copy()
+    xh = case.d_x.cpu().pin_memory()
+    o1 = torch.empty_like(xh).pin_memory()
+    case.layer.forward_host(xh, o1)
+    assert np.array_equal(to_host_f32(o1), ref)
+    outs = [torch.empty_like(xh).pin_memory() for _ in range(3)]
+    for o in outs:                                   # three requests queued on one layer
+        case.layer.forward_host_async(xh, o)
+    case.layer.host_wait()
+    torch.cuda.synchronize()
+    for o in outs:
+        assert np.array_equal(to_host_f32(o), ref)
