@@ -14,6 +14,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "ffn_fused.cuh"
+#include "gemm_tc_small.cuh"
 #include "permute.cuh"
 #include "router_gate.cuh"
 #include "router_tc.cuh"
@@ -35,6 +36,8 @@ struct swapmoe_layer {
   int32_t* done;               // per-row-tile counters of the fused FFN kernel
   int32_t n_done;
   bool fused_ffn;              // both grouped GEMMs in one launch
+  bool small_path;             // small-batch GEMM kernels for <= 64 pairs
+  TcSmallCache small;
   TileDesc* tiles;
   void *xp, *h, *x_stage, *out_stage;
   // host state
@@ -181,7 +184,11 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   if (use_tc) {
     cudaEvent_t mid = L->stage_events ? static_cast<cudaEvent_t>(L->stage_events[4]) : nullptr;
     int32_t rc;
-    if (L->fused_ffn && mt == 1) {
+    if (L->small_path && n_pairs <= 64 && c.act == SWAPMOE_ACT_RELU) {
+      rc = tc_ffn_small(L->tc, L->small, c, L->xp, L->h, L->y, out, L->rows_pad_max, L->arena_in, L->arena_out,
+                        L->tiles, L->n_tiles, L->row_pair, L->mgate, max_tiles, T, L->status, st, pdl,
+                        &L->launches, &combined, mid);
+    } else if (L->fused_ffn && mt == 1) {
       rc = tc_ffn_fused(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->done, L->row_pair, L->mgate, max_tiles,
                         L->status, st, pdl, &L->launches, &combined);
       if (mid) cudaEventRecord(mid, st);      // one kernel: the GEMM-2 stage reads as zero
@@ -283,6 +290,8 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
     env = std::getenv("SWAPMOE_ROUTER_TOK");            // force the router's token tile (32, 64 or 128)
     L->router_tok = env ? std::atoi(env) : 0;
     if (L->router_tok != 32 && L->router_tok != 64 && L->router_tok != 128) L->router_tok = 0;
+    env = std::getenv("SWAPMOE_SMALL_PATH");            // SWAPMOE_SMALL_PATH=0: general GEMM kernels for small batches too
+    L->small_path = !(env && env[0] == '0');
     env = std::getenv("SWAPMOE_PREFETCH");              // SWAPMOE_PREFETCH=0 disables the L2 weight prefetch
     L->prefetch = !(env && env[0] == '0');
     // The prefetch must drain while the router runs (about 15 us on 16-64 SMs): what HBM delivers
@@ -365,6 +374,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)router_smem_bytes(kMaxE)));
   ok = ok && tc_init(L->tc, c, L->xp, L->h, L->y, L->rows_pad_max) == SWAPMOE_OK;
+  if (ok && L->tc.enabled) ok = tc_small_set_attrs();
   ok = ok && cuda_ok(cudaStreamCreateWithFlags(&L->s_in, cudaStreamNonBlocking));
   ok = ok && cuda_ok(cudaStreamCreateWithFlags(&L->s_out, cudaStreamNonBlocking));
   ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_in, cudaEventDisableTiming));
@@ -426,6 +436,7 @@ int32_t swapmoe_set_resident(swapmoe_layer_t* L, const int32_t* s2e, const int32
     t.phys[s] = p;
   }
   if (arena_in != L->arena_in || arena_out != L->arena_out) {
+    L->small.valid = false;
     const int32_t rc = tc_bind_arena(L->tc, c, arena_in, arena_out);
     if (rc != SWAPMOE_OK) return rc;
   }
