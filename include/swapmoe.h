@@ -229,6 +229,13 @@ int32_t swapmoe_debug_copy(swapmoe_layer_t* layer, int32_t which, void* host, si
  * the wait.  The word is cleared. */
 int32_t swapmoe_device_status(swapmoe_layer_t* layer, int32_t* detail, void* stream);
 
+/* Failure-detection self-test.  Launches one small kernel in which a single thread waits on an
+ * mbarrier that nothing will ever complete, through the same bounded wait the tensor-core
+ * kernels use but with a limit of limit_ms (1..1000) milliseconds.  The wait must give up: the
+ * kernel then returns normally and the layer's status word reads SWAPMOE_ERR_DEVICE_TIMEOUT
+ * with detail 99 at the next swapmoe_device_status; the CUDA context stays usable. */
+int32_t swapmoe_selftest_bounded_wait(swapmoe_layer_t* layer, int32_t limit_ms, void* stream);
+
 /* Number of kernels of this library launched by the layer so far (host counter). */
 int64_t swapmoe_launch_count(const swapmoe_layer_t* layer);
 

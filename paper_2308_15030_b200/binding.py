@@ -34,7 +34,7 @@ EXPORTS = [
     "swapmoe_read_importance", "swapmoe_read_importance_kind", "swapmoe_topk_importance", "swapmoe_load_slot_async",
     "swapmoe_debug_copy", "swapmoe_device_status", "swapmoe_launch_count",
     "swapmoe_workspace_bytes", "swapmoe_set_gemm_path", "swapmoe_status_string",
-    "swapmoe_route_static",
+    "swapmoe_route_static", "swapmoe_selftest_bounded_wait",
 ]
 
 
@@ -85,6 +85,7 @@ def lib() -> ctypes.CDLL:
         L.swapmoe_workspace_bytes.restype = i64
         L.swapmoe_set_gemm_path.argtypes = [vp, i32]
         L.swapmoe_route_static.argtypes = [vp] * 4 + [i32] * 7 + [vp] * 11
+        L.swapmoe_selftest_bounded_wait.argtypes = [vp, i32, vp]
         L.swapmoe_status_string.argtypes = [i32]
         L.swapmoe_status_string.restype = ctypes.c_char_p
         for n in EXPORTS:
@@ -274,6 +275,10 @@ class Layer:
         detail = ctypes.c_int32(0)
         st = lib().swapmoe_device_status(self._h, ctypes.byref(detail), _stream_ptr(stream))
         return int(st), int(detail.value)
+
+    def selftest_bounded_wait(self, limit_ms: int = 20, stream=None) -> None:
+        _check(lib().swapmoe_selftest_bounded_wait(self._h, int(limit_ms), _stream_ptr(stream)),
+               "swapmoe_selftest_bounded_wait")
 
     @property
     def launch_count(self) -> int:

@@ -610,6 +610,14 @@ int32_t swapmoe_device_status(swapmoe_layer_t* L, int32_t* detail, void* stream)
   return w[0] != 0 ? SWAPMOE_ERR_DEVICE_TIMEOUT : SWAPMOE_OK;
 }
 
+int32_t swapmoe_selftest_bounded_wait(swapmoe_layer_t* L, int32_t limit_ms, void* stream) {
+  if (!L || limit_ms < 1 || limit_ms > 1000) return SWAPMOE_ERR_INVALID_ARG;
+  bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+      L->status, 99, (unsigned long long)limit_ms * 1000000ull);
+  L->launches++;
+  return check_launch();
+}
+
 int64_t swapmoe_launch_count(const swapmoe_layer_t* L) { return L ? L->launches : 0; }
 int64_t swapmoe_workspace_bytes(const swapmoe_layer_t* L) { return L ? (int64_t)L->ws_bytes : 0; }
 

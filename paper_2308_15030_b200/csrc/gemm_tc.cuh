@@ -156,20 +156,35 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N) {
 // Bounded wait: polls the barrier, and every 256 polls checks a 2-second deadline.
 // Returns false (after recording `code`) when the wait gave up or another role aborted.
 __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                             int32_t* status, int code) {
+                                             int32_t* status, int code, uint64_t limit_ns = 2000000000ull) {
   if (ptx::mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = ptx::globaltimer_ns();
   for (uint32_t spin = 1;; ++spin) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     if ((spin & 255u) == 0) {
       if (*abort_flag) return false;
-      if (ptx::globaltimer_ns() - t0 > 2000000000ull) {
+      if (ptx::globaltimer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         if (atomicCAS(status, 0, 1) == 0) status[1] = code;
         return false;
       }
     }
   }
+}
+
+// Self-test of the bounded wait: one thread waits on an mbarrier that nobody will ever complete,
+// with a short limit; the wait must give up, record `code` and let the kernel return normally.
+__global__ void bounded_wait_selftest_kernel(int32_t* status, int code, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) bounded_wait(&bar, 0u, &abort_flag, status, code, limit_ns);
+  __syncthreads();
 }
 
 // MT = row sub-tiles of 128 rows that one CTA multiplies against the same weight tile.

@@ -249,3 +249,21 @@ def test_host_paths_sync_and_pipelined():
     torch.cuda.synchronize()
     for o in outs:
         assert np.array_equal(to_host_f32(o), ref)
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """A device wait that nothing completes runs into its limit, the kernel returns, the status word
+    names the wait, and the layer keeps working afterwards (no hang, no fault)."""
+    import time
+    import torch
+    from harness import Case, check_against_oracle
+    cfg = _cfg(T=64)
+    case = Case(cfg)
+    assert case.layer.device_status() == (0, 0)
+    t0 = time.perf_counter()
+    case.layer.selftest_bounded_wait(limit_ms=20)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 1.0
+    assert case.layer.device_status() == (-6, 99)          # SWAPMOE_ERR_DEVICE_TIMEOUT, wait code
+    assert case.layer.device_status() == (0, 0)            # cleared by the read
+    check_against_oracle(case, case.run())                 # the context is still usable
