@@ -461,6 +461,23 @@ def run_decode(args, cfg):
         e1.record(); torch.cuda.synchronize()
         ms_graph_swap = e0.elapsed_time(e1)
         del stack
+        # pass 1e (optional): Section 3.4.1's search - run the loop at several update frequencies,
+        # from rare to frequent updates, and report where swapping starts to cost latency
+        sweep = {}
+        if args.sweep_frequency and B == max(args.batches):
+            for freq in args.sweep_frequency:
+                stack = make_stack(False, frequency=freq, graph=True)
+                for s in range(min(8, steps)):
+                    stack.step_graph(d_x[s])
+                torch.cuda.synchronize()
+                l0, st0 = stack.loads, stack.stalls
+                e0.record()
+                for s in range(steps):
+                    stack.step_graph(d_x[s])
+                e1.record(); torch.cuda.synchronize()
+                sweep[str(freq)] = {"us_per_layer": e0.elapsed_time(e1) / steps / L * 1e3,
+                                    "loads": stack.loads - l0, "stalls": stack.stalls - st0}
+                del stack
         # pass 2: same inputs, slot counts tapped after every forward -> touched slots for the roofline
         stack = make_stack(False)
         touched = 0
@@ -492,6 +509,7 @@ def run_decode(args, cfg):
             "loader_frac_of_pcie_probe": (bytes_loaded / load_s / 1e9 / pcie_gbs) if load_s > 0 else None,
             "stalls": stalls,
             "pcie_seconds_needed": bytes_loaded / (pcie_gbs * 1e9), "loop_seconds": ms * 1e-3,
+            "frequency_sweep": sweep,
             "no_swap": {"tokens_per_s": steps * B / (ms_noswap * 1e-3), "us_per_layer": ms_noswap / steps / L * 1e3},
             "no_swap_graph": {"tokens_per_s": steps * B / (ms_graph * 1e-3), "us_per_layer": ms_graph / steps / L * 1e3,
                               "roofline_frac": t_roof * 1e3 / ms_graph},
@@ -569,6 +587,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--batches", type=int, nargs="+", default=[1, 4, 16, 64], help="cfg4: tokens per decode step")
+    ap.add_argument("--sweep-frequency", type=int, nargs="*", default=None,
+                    help="cfg4: also run the loop (largest batch) at these update frequencies (steps between updates)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
