@@ -129,13 +129,6 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tok0 = blockIdx.x * tok;
   const int k_blocks = a.d / kTcBK;
-#ifdef SWAPMOE_PHASE_TIMING
-  __shared__ unsigned long long dbg[16];
-#define STAMP(i) do { if (tid == 128) dbg[i] = ptx::globaltimer_ns(); } while (0)
-#else
-#define STAMP(i) do { } while (0)
-#endif
-  STAMP(0);
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < Epad) tmem_cols <<= 1;
 
@@ -168,7 +161,6 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  STAMP(1);
 
   if (warp == 0) {
     if (lane == 0) {
@@ -236,11 +228,9 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       if (++stage == n_stages) { stage = 0; phase ^= 1u; }
     }
     if (warp_has_rows) snorm[r] = sqrtf(sumsq);
-    STAMP(2);
     // ------------------------------------------------ logits: TMEM lane r -> shared-memory row r
     // (all MMAs have completed once acc_full fires, so the stage buffers are free to reuse)
     if (ok) ok = bounded_wait(acc_full, 0, abort_flag, status, 14);
-    STAMP(3);
     if (ok && warp_has_rows) {
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -261,7 +251,6 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, tmem_cols);
   }
-  STAMP(4);
   const bool failed = *abort_flag != 0;
   {
     // coalesced copy of the logits: a warp writes a token's row; four rows are in flight
@@ -277,7 +266,6 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       }
     }
   }
-  STAMP(8);
   // ---------------------------------------------------- gate: 256 / tok threads per token
   // Thread t serves token t % tok.  Its group g = t / tok splits into the gate it evaluates
   // (first half of the groups: off-the-shelf gate; second half: masked gate) and the share of
@@ -325,7 +313,6 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     for (int j = 0; j < kMaxTopK; ++j) { cand_v[tid * kMaxTopK + j] = tk.v[j]; cand_e[tid * kMaxTopK + j] = tk.e[j]; }
   }
   __syncthreads();
-  STAMP(9);
   // merge the shares of one (token, gate) in ascending expert order: a candidate only displaces
   // an entry it strictly beats, so equal logits keep the lowest expert index
   TopK fin;
@@ -360,7 +347,6 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     part_den[tid] = den;
   }
   __syncthreads();
-  STAMP(10);
   if (part == 0) {
     const float m = fin.v[0];
     float den = 0.f;
@@ -400,9 +386,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     }
     if (!masked && token < a.T) a.xnorm[token] = xn;
   }
-  STAMP(11);
   __syncthreads();
-  STAMP(5);
   // Per-CTA partial sums with a fixed association (lane-strided partials, then the
   // shuffle tree), so the result does not depend on scheduling.  Only experts that some
   // token of this tile selected are visited; the others get an exact zero.
@@ -443,13 +427,6 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     }
   }
   finish_router_cta(a.scan, smem, stage_area);      // the stage memory is free again: stage the scan inputs there
-#ifdef SWAPMOE_PHASE_TIMING
-  __syncthreads();
-  STAMP(6);
-  if (tid == 128)   // phase stamps replace the first logits of this CTA's first token (instrumented build only)
-    for (int i = 0; i < 12; ++i)
-      reinterpret_cast<unsigned long long*>(a.logits + (size_t)blockIdx.x * tok * E)[i] = dbg[i];
-#endif
 }
 
 }  // namespace swapmoe
