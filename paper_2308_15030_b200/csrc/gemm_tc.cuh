@@ -13,6 +13,8 @@
 #pragma once
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "../../include/swapmoe.h"
 #include "common.cuh"
 
@@ -41,6 +43,7 @@ struct TcGemmArgs {
   int32_t a_box_bytes;      // bytes one activation TMA box delivers (box rows * 128): small batches
                             // load only the first 16/32/64 rows of the 128-row MMA tile, the rest
                             // of the tile is stale shared memory whose output rows are never stored
+  int32_t row_group;        // row tiles per scheduling group (see decode_tile)
   int32_t row_split;        // 128-row sub-tiles per tile-list entry handled as SEPARATE work items
                             // (2 when a one-sub-tile kernel walks a list built for 256-row tiles)
   const int32_t* row_pair;  // [rows_pad] pair index of each padded row (scatter epilogue)
@@ -187,6 +190,21 @@ __global__ void bounded_wait_selftest_kernel(int32_t* status, int code, unsigned
   __syncthreads();
 }
 
+// Work item t -> (row tile, column tile).  Row tiles vary fastest inside a group of `group` row
+// tiles, column tiles next, groups last: the row tiles of a slot (which share weights) run side
+// by side, and for large problems the activations of one group stay in L2 while its column
+// tiles are walked (group >= n_row_tiles: one group).
+__device__ __forceinline__ void decode_tile(int t, int n_row_tiles, int n_col_tiles, int group, int* rt, int* ct) {
+  group = min(group, n_row_tiles);
+  const int per_group = group * n_col_tiles;
+  const int g = t / per_group;
+  const int r0 = g * group;
+  const int rows_here = min(group, n_row_tiles - r0);
+  const int u = t - g * per_group;
+  *ct = u / rows_here;
+  *rt = r0 + (u - *ct * rows_here);
+}
+
 // MT = row sub-tiles of 128 rows that one CTA multiplies against the same weight tile.
 template <int BN, int MT = 1>
 struct TcSmem {
@@ -259,7 +277,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t phase = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
-        const int ct = t / n_row_tiles, rt = t - ct * n_row_tiles;   // row tiles vary fastest
+        int rt, ct;
+        decode_tile(t, n_row_tiles, a.n_col_tiles, a.row_group, &rt, &ct);
         TileDesc td = a.tiles[rt / a.row_split];
         if (a.row_split > 1) {
           const int off = (rt % a.row_split) * kTcBM;
@@ -298,7 +317,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
         int halves = 1;
         {
-          const int rt = t % n_row_tiles;
+          int rt, ct_unused;
+          decode_tile(t, n_row_tiles, a.n_col_tiles, a.row_group, &rt, &ct_unused);
           const int rows = a.tiles[rt / a.row_split].rows - (rt % a.row_split) * kTcBM;
           if (rows <= 0) continue;
           if (MT == 2) halves = rows > kTcBM ? 2 : 1;
@@ -337,7 +357,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint32_t acc_phase = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
-      const int ct = t / n_row_tiles, rt = t - ct * n_row_tiles;
+      int rt, ct;
+      decode_tile(t, n_row_tiles, a.n_col_tiles, a.row_group, &rt, &ct);
       TileDesc td = a.tiles[rt / a.row_split];
       if (a.row_split > 1) {
         const int off = (rt % a.row_split) * kTcBM;
@@ -578,6 +599,14 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
   if (mt == 2) ia = 0;
   const int a_box_bytes = (kTcBM >> ia) * kTcBK * 2;
 
+  // Large activation matrices (tens of MB) are walked in groups of 32 row tiles so that a group's
+  // rows stay in L2 across its column tiles; small ones are a single group.
+  int row_group = 1 << 30;
+  {
+    const char* env = std::getenv("SWAPMOE_ROW_GROUP");
+    if (env) row_group = std::atoi(env) > 0 ? std::atoi(env) : row_group;
+    else if (pairs * (long long)c.d_model * 2 > (48ll << 20)) row_group = 32;
+  }
   // ---- GEMM-1: h = act(xp * W_in^T).  Its k-loop is short (d_model / 64 blocks), so its epilogue must
   // overlap the next tile's MMAs: always one sub-tile per CTA with two TMEM buffers; a 256-row tile
   // list is walked as two work items per entry.
@@ -593,6 +622,7 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
   g1.b_rows_gate = swiglu ? c.d_ff : 0;
   g1.row_pair = nullptr; g1.gate = nullptr; g1.top_k = c.top_k;
   g1.row_split = mt;
+  g1.row_group = row_group;
   g1.a_box_bytes = a_box_bytes;
   long long work = (long long)max_tiles * mt * g1.n_col_tiles;
   int grid = work > s.sm_count ? s.sm_count : (int)work;
@@ -620,6 +650,7 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
   g2.b_rows_gate = 0;
   g2.row_pair = row_pair; g2.gate = mgate; g2.top_k = c.top_k;
   g2.row_split = 1;
+  g2.row_group = row_group;
   g2.a_box_bytes = a_box_bytes;
   work = (long long)max_tiles * g2.n_col_tiles;
   grid = work > s.sm_count ? s.sm_count : (int)work;
