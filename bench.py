@@ -62,7 +62,7 @@ def workload_string(cfg):
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
@@ -70,6 +70,11 @@ class ClockSampler:
         self.index = index
         self.proc = None
         self.lines = []
+        self.t_begin = None      # wall-clock window of the timed regions (samples outside are dropped)
+
+    def mark_begin(self):
+        import datetime
+        self.t_begin = datetime.datetime.now()
 
     def start(self):
         try:
@@ -94,13 +99,19 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
+        import datetime
+        t_end = datetime.datetime.now()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             f = [s.strip() for s in ln.split(",")]
-            if len(f) < 7:
+            if len(f) < 8:
                 continue
             try:
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f")
+                if self.t_begin is not None and not (self.t_begin <= ts <= t_end):
+                    continue
+                f = f[1:]
                 sm.append(float(f[0])); mx.append(float(f[1]))
             except ValueError:
                 continue
@@ -198,6 +209,9 @@ def run_cuda(args, cfg):
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()          # started early: nvidia-smi needs a moment before its first sample
     # ---- timed region 1: device-resident inputs
     with torch.cuda.stream(stream):
         for i in range(args.warmup):
@@ -212,15 +226,13 @@ def run_cuda(args, cfg):
         # loop replays it.  forward() neither synchronises nor allocates, so it captures as is.
         torch.cuda.synchronize()
         graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=stream):
+        with torch.cuda.graph(graph, stream=stream, capture_error_mode="thread_local"):
             for j in range(copies):
                 step(j, st=None)
         for _ in range(3):
             graph.replay()
     barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
+    sampler.mark_begin()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     with torch.cuda.stream(stream):
@@ -246,7 +258,6 @@ def run_cuda(args, cfg):
             j = i % copies
             layers[j].forward_timed(d_x[j], d_out[j], evs[i], stream=stream)
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
     stage_ms = np.array([[evs[i][s].elapsed_time(evs[i][s + 1]) for s in range(nst)]
                          for i in range(args.steps)])
     stage_avg = stage_ms.mean(axis=0)
@@ -276,6 +287,7 @@ def run_cuda(args, cfg):
         layers[i % copies].forward_host(xh, ohs[i % copies], stream=stream)
     e2e_sync_ms = (time.perf_counter() - t1) / 20 * 1e3
 
+    clocks = sampler.stop() if rank == 0 else None     # sampled over all three timed regions (all under load)
     st = [L.device_status() for L in layers]
     if any(s[0] != 0 for s in st):
         raise SystemExit("device status error: %r" % (st,))

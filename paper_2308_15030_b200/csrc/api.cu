@@ -39,6 +39,8 @@ struct swapmoe_layer {
   bool small_path;             // small-batch GEMM kernels for <= 64 pairs
   TcSmallCache small;
   TileDesc* tiles;
+  TileDesc* tiles_b;           // 128-row work list kept beside a 256-row one (see forward_impl)
+  int32_t* n_tiles_b;
   void *xp, *h, *x_stage, *out_stage;
   // host state
   const void *Wr, *arena_in, *arena_out;
@@ -119,6 +121,9 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   sa.ticket = L->ticket;
   sa.done = L->done; sa.n_done = L->n_done;
   sa.n_cta = n_cta; sa.K = c.K; sa.E = c.E; sa.tile_rows = tile_rows;
+  // GEMM-2 with two row sub-tiles per CTA walks 256-row tiles; GEMM-1 then gets its own compact
+  // list of 128-row tiles (walking the 256-row list as pairs would leave holes in its schedule).
+  sa.tiles_b = mt == 2 ? L->tiles_b : nullptr; sa.n_tiles_b = L->n_tiles_b; sa.tile_rows_b = kTcBM;
   ra.pf_base[0] = ra.pf_base[1] = nullptr;
   ra.pf_slot_bytes[0] = ra.pf_slot_bytes[1] = 16384;
   ra.pf_total_bytes[0] = ra.pf_total_bytes[1] = 0;
@@ -193,7 +198,8 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
                         L->status, st, pdl, &L->launches, &combined);
       if (mid) cudaEventRecord(mid, st);      // one kernel: the GEMM-2 stage reads as zero
     } else {
-      rc = tc_ffn(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->row_pair, L->mgate, max_tiles, mt, T,
+      rc = tc_ffn(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->tiles_b, L->n_tiles_b, L->row_pair, L->mgate,
+                  max_tiles, mt, T,
                   L->status, st, pdl, &L->launches, &combined, mid);
     }
     if (rc != SWAPMOE_OK) return rc;
@@ -330,6 +336,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_ticket = cv.take<unsigned>(4);
   const size_t o_done = cv.take<int32_t>(max_tiles);
   const size_t o_tiles = cv.take<TileDesc>(max_tiles);
+  const size_t o_tiles_b = cv.take<TileDesc>(max_tiles), o_ntiles_b = cv.take<int32_t>(4);
   const size_t o_xp = cv.take<char>(rows_pad * c.d_model * L->elem);
   const size_t o_h = cv.take<char>(rows_pad * c.d_ff * L->elem);
   const size_t o_y = cv.take<float>(rows_pad * c.d_model);
@@ -354,6 +361,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   L->done = (int32_t*)(b + o_done);
   L->n_done = (int32_t)max_tiles;
   L->tiles = (TileDesc*)(b + o_tiles);
+  L->tiles_b = (TileDesc*)(b + o_tiles_b); L->n_tiles_b = (int32_t*)(b + o_ntiles_b);
   L->xp = b + o_xp; L->h = b + o_h; L->y = (float*)(b + o_y);
   L->x_stage = b + o_xs; L->out_stage = b + o_os;
 

@@ -581,7 +581,8 @@ typedef void (*TcGemmKernel)(const CUtensorMap, const CUtensorMap, const TcGemmA
 // Runs both grouped GEMMs.  With top_k == 1 the second GEMM writes gate * y straight into
 // `out` (*combined = true) and no combine kernel is needed.
 inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, void* out, const TileDesc* tiles,
-                      const int32_t* n_tiles, const int32_t* row_pair, const float* mgate, int max_tiles, int mt,
+                      const int32_t* n_tiles, const TileDesc* tiles128, const int32_t* n_tiles128,
+                      const int32_t* row_pair, const float* mgate, int max_tiles, int mt,
                       int n_tokens, int32_t* status, cudaStream_t st, bool pdl, int64_t* launches, bool* combined,
                       cudaEvent_t between = nullptr) {
   if (!s.enabled || !s.arena_bound) return SWAPMOE_ERR_NOT_READY;
@@ -608,20 +609,21 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
     else if (pairs * (long long)c.d_model * 2 > (48ll << 20)) row_group = 32;
   }
   // ---- GEMM-1: h = act(xp * W_in^T).  Its k-loop is short (d_model / 64 blocks), so its epilogue must
-  // overlap the next tile's MMAs: always one sub-tile per CTA with two TMEM buffers; a 256-row tile
-  // list is walked as two work items per entry.
+  // overlap the next tile's MMAs: always one sub-tile per CTA with two TMEM buffers.
   const int i1 = tc_pick_bn(kBn1Options, 3, c.d_ff, row_tiles_est * mt, s.sm_count, a_box_bytes, swiglu ? 64 : 32);
   if (i1 < 0) return SWAPMOE_ERR_UNSUPPORTED;
   const int bn1 = kBn1Options[i1];
   const int out1 = swiglu ? bn1 / 2 : bn1;      // output columns per tile
   TcGemmArgs g1;
-  g1.C = h; g1.tiles = tiles; g1.n_tiles = n_tiles; g1.status = status; g1.ldc = c.d_ff;
+  g1.C = h; g1.status = status; g1.ldc = c.d_ff;
+  g1.tiles = mt == 2 ? tiles128 : tiles;          // always a list of 128-row tiles
+  g1.n_tiles = mt == 2 ? n_tiles128 : n_tiles;
   g1.n_col_tiles = c.d_ff / out1;
   g1.k_blocks = c.d_model / kTcBK;
   g1.b_rows_per_phys = swiglu ? 2 * c.d_ff : c.d_ff;
   g1.b_rows_gate = swiglu ? c.d_ff : 0;
   g1.row_pair = nullptr; g1.gate = nullptr; g1.top_k = c.top_k;
-  g1.row_split = mt;
+  g1.row_split = 1;
   g1.row_group = row_group;
   g1.a_box_bytes = a_box_bytes;
   long long work = (long long)max_tiles * mt * g1.n_col_tiles;

@@ -23,7 +23,9 @@ struct ScanArgs {
   float* imp;                // [E] accumulator of Eq. (1)
   unsigned* ticket;          // [1] router CTAs finished so far (returns to 0)
   int32_t* done;             // [n_done] per-row-tile progress counters of the fused FFN kernel (zeroed here)
-  int32_t n_cta, K, E, tile_rows, n_done;
+  TileDesc* tiles_b;         // optional second work list with tile_rows_b rows per tile (or nullptr)
+  int32_t* n_tiles_b;
+  int32_t n_cta, K, E, tile_rows, tile_rows_b, n_done;
 };
 
 // Work of the LAST router CTA to finish (all of its threads call this).  The per-CTA
@@ -139,6 +141,20 @@ __device__ __forceinline__ void scan_reduce_block(const ScanArgs& a, void* stage
       a.offset[a.K] = off + c;
       a.pad_offset[a.K] = pad + (c + kSegAlign - 1) / kSegAlign * kSegAlign;
       *a.n_tiles = t0 + nt;
+    }
+    if (a.tiles_b != nullptr) {            // same segments cut into tiles of another height
+      int tb = 0;
+      for (int s = 0; s < tid; ++s) tb += (s_count[s] + a.tile_rows_b - 1) / a.tile_rows_b;
+      const int ntb = (c + a.tile_rows_b - 1) / a.tile_rows_b;
+      for (int i = 0; i < ntb; ++i) {
+        TileDesc td;
+        td.phys = ph;
+        td.row0 = pad + i * a.tile_rows_b;
+        td.rows = min(a.tile_rows_b, c - i * a.tile_rows_b);
+        td.slot = tid;
+        a.tiles_b[tb + i] = td;
+      }
+      if (tid == a.K - 1) *a.n_tiles_b = tb + ntb;
     }
   }
 }

@@ -101,6 +101,7 @@ extern "C" int32_t swapmoe_route_static(const void* x_dev, const void* Wr_dev, c
   sa.imp = imp_dev;
   sa.ticket = reinterpret_cast<unsigned*>(s + kOffTicket);
   sa.done = nullptr; sa.n_done = 0;
+  sa.tiles_b = nullptr; sa.n_tiles_b = nullptr; sa.tile_rows_b = 0;
   sa.cta_cnt = nullptr; sa.cta_mimp = nullptr; sa.s2e = nullptr; sa.cnt = nullptr; sa.mimp = nullptr;
   sa.n_cta = n_cta; sa.K = K; sa.E = E; sa.tile_rows = kSimtBMStatic;
   if (dtype == SWAPMOE_BF16)

@@ -103,7 +103,7 @@ class DecodeStack:
                     st.layer.read_importance(reset=True, stream=self.compute)
                 self.compute.synchronize()
                 self.graph = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(self.graph):        # captured on torch's own side stream
+                with torch.cuda.graph(self.graph, capture_error_mode="thread_local"):   # torch's own side stream
                     for li, st in enumerate(self.layers):
                         st.layer.forward(x_buf[li], out_buf[li], stream=None)
             x_buf.copy_(x_step, non_blocking=True)
