@@ -267,3 +267,33 @@ def test_bounded_wait_gives_up_and_reports():
     assert case.layer.device_status() == (-6, 99)          # SWAPMOE_ERR_DEVICE_TIMEOUT, wait code
     assert case.layer.device_status() == (0, 0)            # cleared by the read
     check_against_oracle(case, case.run())                 # the context is still usable
+
+
+def test_cfg2_in_the_benchmark_launch_configuration():
+    """Full-size cfg2 the way bench.py times it: several layer replicas with their own weight copies,
+    their forwards captured into one CUDA graph (programmatic dependent launch, L2 weight prefetch)
+    and replayed; every replica's output of the last replay is compared with the oracle."""
+    import torch
+    from harness import Case, check_against_oracle, to_host_f32
+    cfg = I.CONFIGS["cfg2"]
+    cases = [Case(cfg) for _ in range(2)]
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for c in cases:                                   # eager warm-up on the capture stream
+            c.layer.forward(c.d_x, c.d_out, stream=stream)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream, capture_error_mode="thread_local"):
+            for c in cases:
+                c.layer.forward(c.d_x, c.d_out, stream=None)
+        for c in cases:
+            c.d_out.fill_(float("nan"))
+            c.layer.read_importance(reset=True, stream=stream)
+        for _ in range(3):
+            graph.replay()
+    torch.cuda.synchronize()
+    for c in cases:
+        out = to_host_f32(c.d_out[: c.T])
+        # three replays accumulated three batches of importance: start the oracle from two of them
+        r0 = c.oracle(c.layer.tap("logits"))
+        check_against_oracle(c, out, imp_before=2 * r0["imp"])
