@@ -44,8 +44,6 @@ struct TcGemmArgs {
                             // load only the first 16/32/64 rows of the 128-row MMA tile, the rest
                             // of the tile is stale shared memory whose output rows are never stored
   int32_t row_group;        // row tiles per scheduling group (see decode_tile)
-  int32_t row_split;        // 128-row sub-tiles per tile-list entry handled as SEPARATE work items
-                            // (2 when a one-sub-tile kernel walks a list built for 256-row tiles)
   const int32_t* row_pair;  // [rows_pad] pair index of each padded row (scatter epilogue)
   const float* gate;        // [T*k] masked gate values (scatter epilogue)
   int32_t top_k;
@@ -267,7 +265,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   pdl_wait();      // the tile list and the operands come from the preceding kernels
   pdl_trigger();
-  const int n_row_tiles = *a.n_tiles * a.row_split;
+  const int n_row_tiles = *a.n_tiles;
   const int total = n_row_tiles * a.n_col_tiles;
 
   if (warp == 0) {
@@ -279,13 +277,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
         int rt, ct;
         decode_tile(t, n_row_tiles, a.n_col_tiles, a.row_group, &rt, &ct);
-        TileDesc td = a.tiles[rt / a.row_split];
-        if (a.row_split > 1) {
-          const int off = (rt % a.row_split) * kTcBM;
-          td.row0 += off;
-          td.rows = min(td.rows - off, kTcBM);
-          if (td.rows <= 0) continue;              // this entry has no second sub-tile
-        }
+        const TileDesc td = a.tiles[rt];
         const int brow = td.phys * a.b_rows_per_phys + ct * kBoxRows;
         const int halves = (MT == 2 && td.rows > kTcBM) ? 2 : 1;
         for (int kb = 0; kb < a.k_blocks; ++kb) {
@@ -319,9 +311,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         {
           int rt, ct_unused;
           decode_tile(t, n_row_tiles, a.n_col_tiles, a.row_group, &rt, &ct_unused);
-          const int rows = a.tiles[rt / a.row_split].rows - (rt % a.row_split) * kTcBM;
-          if (rows <= 0) continue;
-          if (MT == 2) halves = rows > kTcBM ? 2 : 1;
+          if (MT == 2) halves = a.tiles[rt].rows > kTcBM ? 2 : 1;
         }
         ok = bounded_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, a.status, 2);
         if (!ok) break;
@@ -359,13 +349,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
       int rt, ct;
       decode_tile(t, n_row_tiles, a.n_col_tiles, a.row_group, &rt, &ct);
-      TileDesc td = a.tiles[rt / a.row_split];
-      if (a.row_split > 1) {
-        const int off = (rt % a.row_split) * kTcBM;
-        td.row0 += off;
-        td.rows = min(td.rows - off, kTcBM);
-        if (td.rows <= 0) continue;
-      }
+      const TileDesc td = a.tiles[rt];
       ok = bounded_wait(&acc_full[acc], acc_phase, abort_flag, a.status, 4);
       if (!ok) break;
       ptx::tc_fence_after();
@@ -623,7 +607,6 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
   g1.b_rows_per_phys = swiglu ? 2 * c.d_ff : c.d_ff;
   g1.b_rows_gate = swiglu ? c.d_ff : 0;
   g1.row_pair = nullptr; g1.gate = nullptr; g1.top_k = c.top_k;
-  g1.row_split = 1;
   g1.row_group = row_group;
   g1.a_box_bytes = a_box_bytes;
   long long work = (long long)max_tiles * mt * g1.n_col_tiles;
@@ -651,7 +634,6 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
   g2.b_rows_per_phys = c.d_model;
   g2.b_rows_gate = 0;
   g2.row_pair = row_pair; g2.gate = mgate; g2.top_k = c.top_k;
-  g2.row_split = 1;
   g2.row_group = row_group;
   g2.a_box_bytes = a_box_bytes;
   work = (long long)max_tiles * g2.n_col_tiles;
