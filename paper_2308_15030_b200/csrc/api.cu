@@ -50,6 +50,7 @@ struct swapmoe_layer {
   int64_t launches;
   int32_t gemm_path;
   int32_t rows_pad_max;
+  int32_t y_copies;            // copies of y in the workspace (slices of a split contraction)
   int32_t sm_count;
   bool use_pdl;                // programmatic dependent launch between the kernels of a forward
   cudaStream_t s_in, s_out;    // private copy streams of the asynchronous host path
@@ -57,6 +58,10 @@ struct swapmoe_layer {
   int32_t router_tok;          // 0 = automatic token-tile size of the tensor-core router, else 32/64/128
   bool prefetch;               // pull resident weights into L2 from the router kernel
   long long l2_prefetch_bytes; // how much of them (L2 capacity minus head room)
+  int32_t side_prefetch;       // >0: prefetch from a kernel on a private stream instead (experiment switch)
+  long long side_mb0, side_mb1;// bytes of the first wave (with the router) and of the second (with GEMM-1)
+  cudaStream_t s_pf;
+  cudaEvent_t ev_pf_fork, ev_pf_mid, ev_pf_join;
   void* const* stage_events;   // 7 cudaEvent_t of the forward being enqueued, or nullptr
   CUtensorMap map_x;           // TMA view of the last token matrix [T, d]
   const void* map_x_ptr;
@@ -83,6 +88,29 @@ inline bool cuda_ok(cudaError_t e) { return e == cudaSuccess; }
 struct EnormTable { float v[kMaxE]; };
 __global__ void set_enorm_kernel(const EnormTable t, int E, float* enorm) {
   for (int i = threadIdx.x; i < E; i += blockDim.x) enorm[i] = t.v[i];
+}
+
+// Pulls bytes [begin, end) of the resident weights, counted over logical slots in order with
+// GEMM-1's matrices before GEMM-2's, towards L2.
+struct PrefetchArgs {
+  const char* base[2];
+  long long slot_bytes[2];
+  long long total[2];
+  const int32_t* phys;
+  long long begin, end;
+};
+__global__ void __launch_bounds__(256) prefetch_l2_kernel(const PrefetchArgs a) {
+  constexpr long long kChunk = 16384;
+  const long long n_thr = (long long)gridDim.x * blockDim.x;
+  for (long long c = a.begin / kChunk + (long long)blockIdx.x * blockDim.x + threadIdx.x; c * kChunk < a.end; c += n_thr) {
+    long long off = c * kChunk;
+    int m = 0;
+    if (off >= a.total[0]) { off -= a.total[0]; m = 1; }
+    if (off >= a.total[m]) break;
+    const long long sl = off / a.slot_bytes[m], o = off - sl * a.slot_bytes[m];
+    const char* src = a.base[m] + (long long)a.phys[sl] * a.slot_bytes[m] + o;
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"((unsigned)kChunk) : "memory");
+  }
 }
 
 inline void mark(swapmoe_layer* L, int i, cudaStream_t st) {
@@ -148,6 +176,21 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     if (pf_ctas < 0) pf_ctas = 0;
     if (pf_ctas > 64) pf_ctas = 64;
   }
+  bool side = false;
+  PrefetchArgs pfa;
+  if (pf_ctas > 0 && L->side_prefetch && L->stage_events == nullptr) {
+    side = true;
+    pfa.base[0] = ra.pf_base[0]; pfa.base[1] = ra.pf_base[1];
+    pfa.slot_bytes[0] = ra.pf_slot_bytes[0]; pfa.slot_bytes[1] = ra.pf_slot_bytes[1];
+    pfa.total[0] = pfa.slot_bytes[0] * c.K; pfa.total[1] = pfa.slot_bytes[1] * c.K;
+    pfa.phys = L->phys;
+    pfa.begin = 0; pfa.end = L->side_mb0;
+    ra.pf_total_bytes[0] = ra.pf_total_bytes[1] = 0;
+    pf_ctas = 0;
+    if (!cuda_ok(cudaEventRecord(L->ev_pf_fork, st)) || !cuda_ok(cudaStreamWaitEvent(L->s_pf, L->ev_pf_fork, 0)))
+      return SWAPMOE_ERR_CUDA;
+    prefetch_l2_kernel<<<L->side_prefetch, 256, 0, L->s_pf>>>(pfa);
+  }
   mark(L, 0, st);
   if (tc_router) {
     if (x != L->map_x_ptr || T != L->map_x_T) {   // the token map is re-encoded only when x or T changes
@@ -161,7 +204,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
         cudaSuccess)
       return SWAPMOE_ERR_CUDA;
   } else {
-    if (launch_kernel(router_gate_kernel<DT>, dim3(n_cta), dim3(256), router_smem_bytes(c.E), st, pdl, ra) !=
+    if (launch_kernel(router_gate_fn<DT>(c.E), dim3(n_cta), dim3(256), router_smem_bytes(c.E), st, pdl, ra) !=
         cudaSuccess)
       return SWAPMOE_ERR_CUDA;
   }
@@ -183,9 +226,17 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
       cudaSuccess)
     return SWAPMOE_ERR_CUDA;
   L->launches++;
+  if (side && L->side_mb1 > 0) {
+    // second wave: starts when the permutation has finished, i.e. alongside GEMM-1
+    pfa.begin = L->side_mb0; pfa.end = L->side_mb0 + L->side_mb1;
+    if (!cuda_ok(cudaEventRecord(L->ev_pf_mid, st)) || !cuda_ok(cudaStreamWaitEvent(L->s_pf, L->ev_pf_mid, 0)))
+      return SWAPMOE_ERR_CUDA;
+    prefetch_l2_kernel<<<L->side_prefetch, 256, 0, L->s_pf>>>(pfa);
+  }
 
   mark(L, 3, st);
   bool combined = false;
+  int y_split = 1;
   if (use_tc) {
     cudaEvent_t mid = L->stage_events ? static_cast<cudaEvent_t>(L->stage_events[4]) : nullptr;
     int32_t rc;
@@ -208,13 +259,13 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     g1.A = L->xp; g1.W = L->arena_in; g1.C = L->h; g1.tiles = L->tiles; g1.n_tiles = L->n_tiles;
     g1.slot_stride = (long long)L->nin * c.d_ff * c.d_model;
     g1.gate_offset = (long long)c.d_ff * c.d_model;
-    g1.N = c.d_ff; g1.Kdim = c.d_model;
+    g1.N = c.d_ff; g1.Kdim = c.d_model; g1.split_stride = 0;
     const dim3 grid1(c.d_ff / kSimtBN, max_tiles);
     cudaError_t e;
     if (c.act == SWAPMOE_ACT_SWIGLU)
-      e = launch_kernel(gemm_simt_kernel<DT, DT, DT, kEpiSwiglu>, grid1, dim3(256), 0, st, pdl, g1);
+      e = launch_kernel(gemm_simt_kernel<DT, DT, DT, kEpiSwiglu>, grid1, dim3(kSimtThreads), 0, st, pdl, g1);
     else
-      e = launch_kernel(gemm_simt_kernel<DT, DT, DT, kEpiRelu>, grid1, dim3(256), 0, st, pdl, g1);
+      e = launch_kernel(gemm_simt_kernel<DT, DT, DT, kEpiRelu>, grid1, dim3(kSimtThreads), 0, st, pdl, g1);
     if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
     L->launches++;
     mark(L, 4, st);
@@ -223,8 +274,14 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     g2.slot_stride = (long long)c.d_ff * c.d_model;
     g2.gate_offset = 0;
     g2.N = c.d_model; g2.Kdim = c.d_ff;
-    const dim3 grid2(c.d_model / kSimtBN, max_tiles);
-    if (launch_kernel(gemm_simt_kernel<DT, DT, float, kEpiNone>, grid2, dim3(256), 0, st, pdl, g2) != cudaSuccess)
+    // Few output tiles and a long contraction: slice the contraction so that every SM has work.
+    // The slices land in separate copies of y and the combine kernel adds them in order.
+    const long long tiles_est = ((long long)n_pairs / kSimtBM + (n_pairs < c.K ? n_pairs : c.K) / 2 + 1) *
+                                (c.d_model / kSimtBN);
+    y_split = simt_pick_split(tiles_est, L->sm_count, c.d_ff, L->y_copies);
+    g2.split_stride = (long long)L->rows_pad_max * c.d_model;
+    const dim3 grid2(c.d_model / kSimtBN, max_tiles, y_split);
+    if (launch_kernel(gemm_simt_kernel<DT, DT, float, kEpiNone>, grid2, dim3(kSimtThreads), 0, st, pdl, g2) != cudaSuccess)
       return SWAPMOE_ERR_CUDA;
     L->launches++;
   }
@@ -232,6 +289,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   CombineArgs ca;
   ca.y = L->y; ca.inv_pad = L->inv_pad; ca.mgate = L->mgate; ca.out = out;
   ca.T = T; ca.d = c.d_model; ca.k = c.top_k;
+  ca.n_split = y_split; ca.split_stride = (long long)L->rows_pad_max * c.d_model;
   const long long work = (long long)T * (c.d_model / 8);
   mark(L, 5, st);
   if (!combined) {
@@ -241,6 +299,8 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     L->launches++;
   }
   mark(L, 6, st);
+  if (side && (!cuda_ok(cudaEventRecord(L->ev_pf_join, L->s_pf)) || !cuda_ok(cudaStreamWaitEvent(st, L->ev_pf_join, 0))))
+    return SWAPMOE_ERR_CUDA;
   return check_launch();
 }
 
@@ -307,6 +367,12 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
     L->l2_prefetch_bytes = l2 > (80ll << 20) ? (56ll << 20) : 0;
     env = std::getenv("SWAPMOE_PREFETCH_MB");
     if (env) L->l2_prefetch_bytes = std::atoll(env) << 20;
+    env = std::getenv("SWAPMOE_SIDE_PREFETCH");         // CTAs of the side-stream prefetch kernel, 0 = off
+    L->side_prefetch = env ? std::atoi(env) : 0;
+    env = std::getenv("SWAPMOE_SIDE_MB0");
+    L->side_mb0 = (env ? std::atoll(env) : 56) << 20;
+    env = std::getenv("SWAPMOE_SIDE_MB1");
+    L->side_mb1 = (env ? std::atoll(env) : 0) << 20;
   }
   L->nin = c.act == SWAPMOE_ACT_SWIGLU ? 2 : 1;
   L->elem = c.dtype == SWAPMOE_BF16 ? 2 : 4;
@@ -339,7 +405,9 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_tiles_b = cv.take<TileDesc>(max_tiles), o_ntiles_b = cv.take<int32_t>(4);
   const size_t o_xp = cv.take<char>(rows_pad * c.d_model * L->elem);
   const size_t o_h = cv.take<char>(rows_pad * c.d_ff * L->elem);
-  const size_t o_y = cv.take<float>(rows_pad * c.d_model);
+  // up to four copies of y for a sliced contraction in the CUDA-core GEMM-2, when they stay small
+  L->y_copies = (rows_pad * c.d_model * sizeof(float) * 4 <= (size_t)(64u << 20)) ? 4 : 1;
+  const size_t o_y = cv.take<float>(rows_pad * c.d_model * L->y_copies);
   const size_t o_xs = cv.take<char>(T * c.d_model * L->elem);
   const size_t o_os = cv.take<char>(T * c.d_model * L->elem);
   L->ws_bytes = cv.off;
@@ -375,12 +443,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   // Rows of the padded workspaces that no pair occupies are computed on but never
   // read back; start them at zero so they hold finite values.
   ok = ok && cuda_ok(cudaMemset(L->xp, 0, rows_pad * c.d_model * L->elem));
-  ok = ok && cuda_ok(cudaFuncSetAttribute(router_gate_kernel<float>,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)router_smem_bytes(kMaxE)));
-  ok = ok && cuda_ok(cudaFuncSetAttribute(router_gate_kernel<bf16>,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)router_smem_bytes(kMaxE)));
+  ok = ok && cuda_ok(router_gate_set_smem_limit<float>()) && cuda_ok(router_gate_set_smem_limit<bf16>());
   ok = ok && tc_init(L->tc, c, L->xp, L->h, L->y, L->rows_pad_max) == SWAPMOE_OK;
   if (ok && L->tc.enabled) ok = tc_small_set_attrs();
   ok = ok && cuda_ok(cudaStreamCreateWithFlags(&L->s_in, cudaStreamNonBlocking));
@@ -388,6 +451,10 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_in, cudaEventDisableTiming));
   ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_comp, cudaEventDisableTiming));
   ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_out, cudaEventDisableTiming));
+  ok = ok && cuda_ok(cudaStreamCreateWithFlags(&L->s_pf, cudaStreamNonBlocking));
+  ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_pf_fork, cudaEventDisableTiming));
+  ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_pf_mid, cudaEventDisableTiming));
+  ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_pf_join, cudaEventDisableTiming));
   if (!ok) { cudaGetLastError(); cudaFree(L->ws_base); delete L; return SWAPMOE_ERR_CUDA; }
   *out = L;
   return SWAPMOE_OK;
@@ -400,6 +467,10 @@ int32_t swapmoe_destroy(swapmoe_layer_t* L) {
   if (L->ev_in) cudaEventDestroy(L->ev_in);
   if (L->ev_comp) cudaEventDestroy(L->ev_comp);
   if (L->ev_out) cudaEventDestroy(L->ev_out);
+  if (L->s_pf) cudaStreamDestroy(L->s_pf);
+  if (L->ev_pf_fork) cudaEventDestroy(L->ev_pf_fork);
+  if (L->ev_pf_mid) cudaEventDestroy(L->ev_pf_mid);
+  if (L->ev_pf_join) cudaEventDestroy(L->ev_pf_join);
   cudaFree(L->ws_base);
   delete L;
   return SWAPMOE_OK;

@@ -2,99 +2,196 @@
 // layer's contraction (a tensor-core fp32 path would need split-TF32 to hold the
 // 1e-4 output tolerance) and the small-shape path of the bf16 layer.
 // SwapMoE Section 2: E_i(x) = W_out * act(W_in * x), evaluated per slot segment.
+//
+// One CTA (256 threads) = 64 rows x 64 columns of one slot segment.  The two halves of the CTA
+// (128 threads each) split every contraction chunk between them and add their accumulators at
+// the end, which doubles the warps that hide latency without shrinking the per-thread micro-tile
+// of 8 x 4 (rows 8 ty .. 8 ty + 7, columns tx + 16 j).  Shared memory keeps both operands
+// row-major with the contraction index contiguous, as they sit in global memory, so a chunk is
+// staged with 16-byte stores and read back 16 bytes (four contraction indices) at a time:
+// twelve reads feed 128 FFMAs, and the row pitch of 20 words spreads them over the banks.  The
+// contraction runs in chunks of 16 through two shared-memory buffers and two register sets: the
+// global loads of chunk c + 2 are issued before the arithmetic of chunk c, and chunk c + 1 (in
+// registers since the previous round) moves to the other buffer afterwards; one barrier per
+// chunk.  gridDim.z > 1 splits the contraction: slice z writes its partial sums to
+// C + z * split_stride and the consumer adds the slices in order (a fixed order, so results
+// repeat run to run).
 #pragma once
 #include "common.cuh"
 
 namespace swapmoe {
 
-constexpr int kSimtBM = 64, kSimtBN = 64, kSimtBK = 16;
+constexpr int kSimtBM = 64, kSimtBN = 64, kSimtBK = 16, kSimtThreads = 256;
 
 struct SimtGemmArgs {
   const void* A;          // [rows_pad, Kdim] activations (TA)
   const void* W;          // arena: entry stride `slot_stride` elements; matrix [N, Kdim] (TW)
-  void* C;                // [rows_pad, N] (TC)
+  void* C;                // [rows_pad, N] (TC); slice z of a split contraction at C + z * split_stride
   const TileDesc* tiles;
   const int32_t* n_tiles;
   long long slot_stride;  // elements between arena entries
   long long gate_offset;  // elements from W1 to W3 inside an entry (SwiGLU only)
+  long long split_stride; // elements between the partial outputs of a split contraction
   int32_t N, Kdim;
 };
 
 enum { kEpiNone = 0, kEpiRelu = 1, kEpiSwiglu = 2 };
 
-// C[tile rows, 64 cols] = epi(A[tile rows, :] * W[phys][n0:n0+64, :]^T); grid = (N/64, max tiles).
+__device__ __forceinline__ void store1(float* p, float v) { *p = v; }
+__device__ __forceinline__ void store1(bf16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+// C[tile rows, 64 cols] = epi(A[tile rows, :] * W[phys][n0:n0+64, :]^T);
+// grid = (N/64, max tiles, contraction slices).
 template <typename TA, typename TW, typename TC, int EPI>
-__global__ void __launch_bounds__(256) gemm_simt_kernel(const SimtGemmArgs a) {
+__global__ void __launch_bounds__(kSimtThreads, EPI == kEpiSwiglu ? 1 : 2) gemm_simt_kernel(const SimtGemmArgs a) {
   pdl_wait();
   pdl_trigger();
   if ((int)blockIdx.y >= *a.n_tiles) return;
   const TileDesc td = a.tiles[blockIdx.y];
-  constexpr int LD = kSimtBM + 4;
-  __shared__ __align__(16) float As[kSimtBK][LD];
-  __shared__ __align__(16) float Bs[kSimtBK][LD];
-  __shared__ __align__(16) float Gs[EPI == kEpiSwiglu ? kSimtBK : 1][LD];
+  constexpr int LD = kSimtBK + 4;
+  constexpr bool kGate = EPI == kEpiSwiglu;
+  constexpr int kOperands = kGate ? 3 : 2;
+  // [buffer][operand A / W / gate][row][LD]; reused at the end for the accumulator exchange
+  __shared__ __align__(16) float smem[2 * kOperands * kSimtBM * LD];
+  static_assert(2 * kOperands * kSimtBM * LD >= kSimtBM * kSimtBN, "accumulator exchange must fit");
+  auto tile = [&](int buf, int op) { return smem + (size_t)(buf * kOperands + op) * kSimtBM * LD; };
 
   const int tid = threadIdx.x;
   const int n0 = blockIdx.x * kSimtBN;
-  const TA* A = static_cast<const TA*>(a.A) + (size_t)td.row0 * a.Kdim;
-  const TW* W = static_cast<const TW*>(a.W) + (size_t)td.phys * a.slot_stride + (size_t)n0 * a.Kdim;
+  const int k_len = a.Kdim / (int)gridDim.z, k_begin = (int)blockIdx.z * k_len;
+  const TA* A = static_cast<const TA*>(a.A) + (size_t)td.row0 * a.Kdim + k_begin;
+  const TW* W = static_cast<const TW*>(a.W) + (size_t)td.phys * a.slot_stride + (size_t)n0 * a.Kdim + k_begin;
   const TW* G = W + a.gate_offset;
 
-  const int lr = tid >> 2, lc = (tid & 3) * 4;   // staged element: row lr, k-columns lc..lc+3
-  const int ty = tid >> 4, tx = tid & 15;        // micro-tile: rows 4ty.., cols 4tx..
+  const int lr = tid >> 2, lc = (tid & 3) * 4;   // staging: row lr, contraction columns lc..lc+3
+  const int half = tid >> 7;                     // which half of every chunk this thread multiplies
+  const int ty = (tid & 127) >> 4, tx = tid & 15;
 
-  float acc[4][4], acg[4][4];
+  float acc[8][4], acg[kGate ? 8 : 1][4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < 8; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) { acc[i][j] = 0.f; acg[i][j] = 0.f; }
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll
+  for (int i = 0; i < (kGate ? 8 : 1); ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acg[i][j] = 0.f;
 
-  for (int k0 = 0; k0 < a.Kdim; k0 += kSimtBK) {
-    float av[4], bv[4], gv[4];
-    load4(A + (size_t)lr * a.Kdim + k0 + lc, av);
-    load4(W + (size_t)lr * a.Kdim + k0 + lc, bv);
-    if (EPI == kEpiSwiglu) load4(G + (size_t)lr * a.Kdim + k0 + lc, gv);
-    __syncthreads();
+  float av[2][4], bv[2][4], gv[kGate ? 2 : 1][4];   // two register sets
+  auto load_chunk = [&](int k0, int set) {
+    load4(A + (size_t)lr * a.Kdim + k0 + lc, av[set]);
+    load4(W + (size_t)lr * a.Kdim + k0 + lc, bv[set]);
+    if (kGate) load4(G + (size_t)lr * a.Kdim + k0 + lc, gv[kGate ? set : 0]);
+  };
+  auto store_chunk = [&](int buf, int set) {
+    store4(tile(buf, 0) + lr * LD + lc, av[set]);
+    store4(tile(buf, 1) + lr * LD + lc, bv[set]);
+    if (kGate) store4(tile(buf, kGate ? 2 : 0) + lr * LD + lc, gv[kGate ? set : 0]);
+  };
+  auto compute_chunk = [&](int buf) {
+    const float* As = tile(buf, 0);
+    const float* Bs = tile(buf, 1);
+    const float* Gs = tile(buf, kGate ? 2 : 0);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      As[lc + q][lr] = av[q];
-      Bs[lc + q][lr] = bv[q];
-      if (EPI == kEpiSwiglu) Gs[lc + q][lr] = gv[q];
-    }
-    __syncthreads();
+    for (int s4 = 0; s4 < kSimtBK / 2; s4 += 4) {
+      const int k4 = half * (kSimtBK / 2) + s4;
+      float ar[8][4], br[4][4];
 #pragma unroll
-    for (int kk = 0; kk < kSimtBK; ++kk) {
-      const float4 a4 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
-      const float4 b4 = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
-      const float ar[4] = {a4.x, a4.y, a4.z, a4.w};
-      const float br[4] = {b4.x, b4.y, b4.z, b4.w};
+      for (int i = 0; i < 8; ++i) load4(As + (ty * 8 + i) * LD + k4, ar[i]);
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int j = 0; j < 4; ++j) load4(Bs + (tx + 16 * j) * LD + k4, br[j]);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(ar[i], br[j], acc[i][j]);
-      if (EPI == kEpiSwiglu) {
-        const float4 g4 = *reinterpret_cast<const float4*>(&Gs[kk][tx * 4]);
-        const float gr[4] = {g4.x, g4.y, g4.z, g4.w};
+      for (int q = 0; q < 4; ++q)        // contraction indices in ascending order
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
+        for (int i = 0; i < 8; ++i)
 #pragma unroll
-          for (int j = 0; j < 4; ++j) acg[i][j] = fmaf(ar[i], gr[j], acg[i][j]);
+          for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(ar[i][q], br[j][q], acc[i][j]);
+      if (kGate) {
+        float gr[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) load4(Gs + (tx + 16 * j) * LD + k4, gr[j]);
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+#pragma unroll
+          for (int i = 0; i < (kGate ? 8 : 1); ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acg[i][j] = fmaf(ar[i][q], gr[j][q], acg[i][j]);
       }
     }
+  };
+  // The chunk loop is unrolled by two so that the register sets are addressed statically.
+  const int n_chunks = k_len / kSimtBK;
+  load_chunk(0, 0);
+  store_chunk(0, 0);
+  if (n_chunks > 1) load_chunk(kSimtBK, 1);
+  __syncthreads();
+  for (int c = 0; c < n_chunks; c += 2) {
+    // even chunk c: computes buffer 0; chunk c + 1 waits in set 1; chunk c + 2 is fetched into set 0
+    if (c + 2 < n_chunks) load_chunk((c + 2) * kSimtBK, 0);
+    compute_chunk(0);
+    if (c + 1 < n_chunks) store_chunk(1, 1);
+    __syncthreads();
+    if (c + 1 >= n_chunks) break;
+    // odd chunk c + 1: computes buffer 1; chunk c + 2 waits in set 0; chunk c + 3 is fetched into set 1
+    if (c + 3 < n_chunks) load_chunk((c + 3) * kSimtBK, 1);
+    compute_chunk(1);
+    if (c + 2 < n_chunks) store_chunk(0, 0);
+    __syncthreads();
   }
-  TC* C = static_cast<TC*>(a.C) + (size_t)td.row0 * a.N + n0;
+  // The upper half hands its accumulators to the lower half through shared memory (every thread
+  // has passed the loop's last barrier, so the operand buffers are free).
+  float* xch = smem;   // [64][64]
+  if (half == 1) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float o[4];
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) xch[(ty * 8 + i) * kSimtBN + tx + 16 * j] = acc[i][j];
+  }
+  __syncthreads();
+  if (half == 0) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] += xch[(ty * 8 + i) * kSimtBN + tx + 16 * j];
+  }
+  if (kGate) {
+    __syncthreads();
+    if (half == 1) {
+#pragma unroll
+      for (int i = 0; i < (kGate ? 8 : 1); ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) xch[(ty * 8 + i) * kSimtBN + tx + 16 * j] = acg[i][j];
+    }
+    __syncthreads();
+    if (half == 0) {
+#pragma unroll
+      for (int i = 0; i < (kGate ? 8 : 1); ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acg[i][j] += xch[(ty * 8 + i) * kSimtBN + tx + 16 * j];
+    }
+  }
+  if (half != 0) return;
+  TC* C = static_cast<TC*>(a.C) + (size_t)blockIdx.z * a.split_stride + (size_t)td.row0 * a.N + n0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       float v = acc[i][j];
       if (EPI == kEpiRelu) v = fmaxf(v, 0.f);
-      if (EPI == kEpiSwiglu) v = v / (1.f + expf(-v)) * acg[i][j];
-      o[j] = v;
+      if (kGate) v = v / (1.f + expf(-v)) * acg[kGate ? i : 0][j];
+      store1(C + (size_t)(ty * 8 + i) * a.N + tx + 16 * j, v);
     }
-    store4(C + (size_t)(ty * 4 + i) * a.N + tx * 4, o);
   }
+}
+
+// Number of contraction slices for a GEMM with `tiles` output tiles of the 64 x 64 shape: enough
+// to give every SM about two CTAs, at most `max_split`, and only slicings that leave whole chunks.
+inline int simt_pick_split(long long tiles, int sm_count, int Kdim, int max_split) {
+  int split = 1;
+  while (split * 2 <= max_split && tiles * split < 2ll * sm_count && Kdim % (split * 2 * kSimtBK) == 0 &&
+         Kdim / (split * 2) >= 4 * kSimtBK)
+    split *= 2;
+  return split;
 }
 
 }  // namespace swapmoe

@@ -259,7 +259,8 @@ struct CombineArgs {
   const int32_t* inv_pad;    // [T*k]
   const float* mgate;        // [T*k]
   void* out;                 // [T, d]
-  int32_t T, d, k;
+  long long split_stride;    // elements between the copies of y
+  int32_t T, d, k, n_split;  // n_split copies of y hold partial sums that are added here, in order
 };
 
 // out[t, c] = sum_j mgate[t,j] * y[inv_pad[t,j], c]; each thread owns 8 columns.
@@ -275,8 +276,14 @@ __global__ void __launch_bounds__(256) combine_kernel(const CombineArgs a) {
   for (int j = 0; j < a.k; ++j) {
     const float g = a.mgate[(size_t)t * a.k + j];
     const float* yr = a.y + (size_t)a.inv_pad[(size_t)t * a.k + j] * a.d + c;
-    const float4 y0 = reinterpret_cast<const float4*>(yr)[0];
-    const float4 y1 = reinterpret_cast<const float4*>(yr)[1];
+    float4 y0 = reinterpret_cast<const float4*>(yr)[0];
+    float4 y1 = reinterpret_cast<const float4*>(yr)[1];
+    for (int z = 1; z < a.n_split; ++z) {
+      const float4 p0 = reinterpret_cast<const float4*>(yr + (size_t)z * a.split_stride)[0];
+      const float4 p1 = reinterpret_cast<const float4*>(yr + (size_t)z * a.split_stride)[1];
+      y0.x += p0.x; y0.y += p0.y; y0.z += p0.z; y0.w += p0.w;
+      y1.x += p1.x; y1.y += p1.y; y1.z += p1.z; y1.w += p1.w;
+    }
     acc[0] = fmaf(g, y0.x, acc[0]); acc[1] = fmaf(g, y0.y, acc[1]);
     acc[2] = fmaf(g, y0.z, acc[2]); acc[3] = fmaf(g, y0.w, acc[3]);
     acc[4] = fmaf(g, y1.x, acc[4]); acc[5] = fmaf(g, y1.y, acc[5]);

@@ -48,6 +48,11 @@ int32_t scratch_for_current_device(unsigned char** out) {
   if (!g_scratch_dev[dev]) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_route_scratch) != cudaSuccess || !p) { cudaGetLastError(); return SWAPMOE_ERR_CUDA; }
+    // large expert counts need more dynamic shared memory than the default limit
+    if (router_gate_set_smem_limit<float>() != cudaSuccess || router_gate_set_smem_limit<bf16>() != cudaSuccess) {
+      cudaGetLastError();
+      return SWAPMOE_ERR_CUDA;
+    }
     g_scratch_dev[dev] = static_cast<unsigned char*>(p);
   }
   *out = g_scratch_dev[dev];
@@ -105,8 +110,8 @@ extern "C" int32_t swapmoe_route_static(const void* x_dev, const void* Wr_dev, c
   sa.cta_cnt = nullptr; sa.cta_mimp = nullptr; sa.s2e = nullptr; sa.cnt = nullptr; sa.mimp = nullptr;
   sa.n_cta = n_cta; sa.K = K; sa.E = E; sa.tile_rows = kSimtBMStatic;
   if (dtype == SWAPMOE_BF16)
-    router_gate_kernel<bf16><<<n_cta, 256, router_smem_bytes(E), st>>>(ra);
+    router_gate_fn<bf16>(E)<<<n_cta, 256, router_smem_bytes(E), st>>>(ra);
   else
-    router_gate_kernel<float><<<n_cta, 256, router_smem_bytes(E), st>>>(ra);
+    router_gate_fn<float>(E)<<<n_cta, 256, router_smem_bytes(E), st>>>(ra);
   return cudaGetLastError() == cudaSuccess ? SWAPMOE_OK : SWAPMOE_ERR_CUDA;
 }

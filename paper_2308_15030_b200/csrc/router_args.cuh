@@ -1,0 +1,35 @@
+// Arguments of the router kernels (SwapMoE Section 2, Fig. 4, Eq. 1).
+#pragma once
+#include "common.cuh"
+#include "permute.cuh"
+
+namespace swapmoe {
+
+struct RouterArgs {
+  const void* x;            // [T, d] layer dtype
+  const void* Wr;           // [E, d] layer dtype
+  const float* ext_logits;  // [T, E] or nullptr
+  const int32_t* e2s;       // [E] expert -> slot, -1 = not resident
+  const float* enorm;       // [E]
+  float* logits;            // [T, E]
+  int32_t* uidx;            // [T, k]
+  float* ugate;             // [T, k]
+  int32_t* midx;            // [T, k]
+  float* mgate;             // [T, k]
+  int32_t* slot;            // [T, k]
+  float* xnorm;             // [T]
+  int32_t* cta_hist;        // [n_cta, K]
+  float* cta_imp;           // [n_cta, E]
+  float* cta_cnt;           // [n_cta, E] or nullptr
+  float* cta_mimp;          // [n_cta, K] or nullptr
+  int32_t T, d, E, k, K, renorm;
+  ScanArgs scan;            // work of the last CTA to finish
+  // Weight prefetch (tensor-core router only): blocks beyond the token tiles pull the resident
+  // experts' matrices into L2 while the router runs, when HBM is otherwise idle.
+  const char* pf_base[2];       // arena_in, arena_out
+  long long pf_slot_bytes[2];   // bytes of one arena entry
+  long long pf_total_bytes[2];  // bytes to prefetch, counted over logical slots 0..K-1 in order
+  const int32_t* pf_phys;       // [K] arena entry of each logical slot
+};
+
+}  // namespace swapmoe

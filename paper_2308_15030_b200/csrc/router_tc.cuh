@@ -14,34 +14,13 @@
 #include "gemm_tc.cuh"
 #include "permute.cuh"
 #include "router_gate.cuh"
+#include "gate_epilogue.cuh"
 
 namespace swapmoe {
 
 constexpr int kRtTok = 128;      // tokens per CTA
 constexpr int kRtThreads = 256;
 
-// Running top-k list, descending by value; a candidate is inserted below every entry
-// that is >= it, so equal values stay in arrival (= expert index) order.
-struct TopK {
-  float v[kMaxTopK];
-  int e[kMaxTopK];
-  __device__ __forceinline__ void init() {
-#pragma unroll
-    for (int j = 0; j < kMaxTopK; ++j) { v[j] = -INFINITY; e[j] = -1; }
-  }
-  __device__ __forceinline__ void push(float cv, int ce, int k) {
-    bool shifting = false;
-#pragma unroll
-    for (int j = 0; j < kMaxTopK; ++j) {
-      if (j < k && (shifting || e[j] < 0 || cv > v[j])) {
-        const float tv = v[j]; const int te = e[j];
-        v[j] = cv; e[j] = ce;
-        cv = tv; ce = te;
-        shifting = true;
-      }
-    }
-  }
-};
 constexpr int kRtSmemBudget = 190 * 1024;
 
 inline int router_tc_epad(int E) { return (E + 15) / 16 * 16; }
@@ -63,11 +42,7 @@ inline size_t router_tc_smem_bytes(int E, int tok) {
   size_t stages = (size_t)router_tc_stages(E, tok) * router_tc_stage_bytes(E, tok) + kRtTok * kTcBK * 2;
   const size_t logit_tile = (size_t)tok * (E + 1) * 4;
   if (stages < logit_tile) stages = logit_tile;
-  return stages + 2048 +
-         (sizeof(int) * 2 + sizeof(float)) * kRtTok * kMaxTopK + sizeof(float) * kRtTok +
-         (sizeof(int) + sizeof(float)) * kMaxE + sizeof(uint32_t) * 24 + 1024 + 8 * (2 * kRtMaxStages + 8) +
-         (sizeof(float) + sizeof(int)) * kRtTok * 2 * 4 * kMaxTopK / 4 + sizeof(float) * kRtThreads + 1024 +
-         sizeof(float) * kRtTok * kMaxTopK;
+  return stages + 2048 + 1024 + 8 * (2 * kRtMaxStages + 8) + 16 + gate_smem_bytes();
 }
 
 __global__ void __launch_bounds__(kRtThreads, 1)
@@ -92,7 +67,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     }
     return;
   }
-  const int E = a.E, k = a.k;
+  const int E = a.E;
   const int Epad = (E + 15) / 16 * 16;
   const int a_bytes = tok * kTcBK * 2, b_bytes = Epad * kTcBK * 2;   // token box, router box
   const int a_box_bytes = a_bytes;
@@ -112,19 +87,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   uint64_t* acc_full = bars + 2 * kRtMaxStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kRtMaxStages + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  int* pe = reinterpret_cast<int*>(bars + 2 * kRtMaxStages + 8);   // [tok*k] unmasked expert per pair
-  int* ps = pe + kRtTok * kMaxTopK;                       // [tok*k] slot per pair
-  float* pt = reinterpret_cast<float*>(ps + kRtTok * kMaxTopK);
-  float* snorm = pt + kRtTok * kMaxTopK;                  // [tok] ||x_t||
-  int* s_e2s = reinterpret_cast<int*>(snorm + kRtTok);    // [256] expert -> slot
-  float* s_enorm = reinterpret_cast<float*>(s_e2s + kMaxE);   // [256] ||E_e||
-  uint32_t* s_mask = reinterpret_cast<uint32_t*>(s_enorm + kMaxE);  // [2][8] valid / resident bits
-  uint32_t* s_present = s_mask + 16;                       // [8] experts selected (unmasked) in this tile
-  float* cand_v = reinterpret_cast<float*>(s_present + 8); // [256 threads][kMaxTopK] per-thread top-k values
-  int* cand_e = reinterpret_cast<int*>(cand_v + kRtThreads * kMaxTopK);   // ... and experts
-  float* part_den = reinterpret_cast<float*>(cand_e + kRtThreads * kMaxTopK);   // [256] partial denominators
-  float* s_m = part_den + kRtThreads;                      // [tok][2] row maximum per gate
-  float* pm = s_m + 2 * kRtTok;                            // [tok*k] Eq. (1) term under the masked routing
+  const GateSmem g = gate_smem_carve(bars + 2 * kRtMaxStages + 8);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tok0 = blockIdx.x * tok;
@@ -146,17 +109,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   }
   pdl_wait();      // everything above touched only shared memory, TMEM and kernel parameters
   pdl_trigger();
-  for (int e = tid; e < kMaxE; e += kRtThreads) {
-    s_e2s[e] = e < E ? a.e2s[e] : -1;
-    s_enorm[e] = e < E ? a.enorm[e] : 0.f;
-  }
-  {
-    // warp w builds word w of the valid-expert mask and of the resident-expert mask
-    const int e = warp * 32 + lane;
-    const int sl = e < E ? a.e2s[e] : -1;
-    const uint32_t wv = __ballot_sync(0xffffffffu, e < E), wr = __ballot_sync(0xffffffffu, sl >= 0);
-    if (lane == 0) { s_mask[warp] = wv; s_mask[8 + warp] = wr; s_present[warp] = 0u; }
-  }
+  gate_load_tables(a, g);
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
@@ -227,7 +180,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       if (lane == 0) ptx::mbar_arrive(&empty[stage]);
       if (++stage == n_stages) { stage = 0; phase ^= 1u; }
     }
-    if (warp_has_rows) snorm[r] = sqrtf(sumsq);
+    if (warp_has_rows) g.snorm[r] = sqrtf(sumsq);
     // ------------------------------------------------ logits: TMEM lane r -> shared-memory row r
     // (all MMAs have completed once acc_full fires, so the stage buffers are free to reuse)
     if (ok) ok = bounded_wait(acc_full, 0, abort_flag, status, 14);
@@ -252,181 +205,8 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     ptx::tmem_dealloc(tmem_base, tmem_cols);
   }
   const bool failed = *abort_flag != 0;
-  {
-    // coalesced copy of the logits: a warp writes a token's row; four rows are in flight
-    const int rows = min(tok, a.T - tok0);
-    for (int t0 = warp * 4; t0 < rows; t0 += (kRtThreads / 32) * 4) {
-      for (int e = lane; e < E; e += 32) {
-        float v[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) v[q] = slog[(size_t)(t0 + q) * (E + 1) + e];
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-          if (t0 + q < rows) a.logits[(size_t)(tok0 + t0 + q) * E + e] = failed ? 0.f : v[q];
-      }
-    }
-  }
-  // ---------------------------------------------------- gate: 256 / tok threads per token
-  // Thread t serves token t % tok.  Its group g = t / tok splits into the gate it evaluates
-  // (first half of the groups: off-the-shelf gate; second half: masked gate) and the share of
-  // the expert range it scans (whole 32-expert chunks, contiguous and ascending per share).
-  const int tl = tid % tok, grp = tid / tok;
-  const int parts = (kRtThreads / tok) >> 1;                // threads per token and gate: 1, 2 or 4
-  const bool masked = grp >= parts;
-  const int part = masked ? grp - parts : grp;
-  const int token = tok0 + tl;
-  const float* row = slog + (size_t)tl * (E + 1);
-  const uint32_t* allow = s_mask + (masked ? 8 : 0);
-  const int n_chunks = (E + 31) >> 5, cpp = (n_chunks + parts - 1) / parts;
-  const int e_lo = min(E, part * cpp * 32), e_hi = min(E, (part + 1) * cpp * 32);
-  {
-    // The loops below run once per CTA, so they are kept rolled (short bodies that stay in the
-    // instruction cache) rather than unrolled over the whole expert range.
-    TopK tk;
-    tk.init();
-    if (k == 1) {
-      float best = -INFINITY;
-      int bi = -1;
-#pragma unroll 4
-      for (int e = e_lo; e < e_hi; ++e) {
-        const float l = row[e];
-        const bool take = ((allow[e >> 5] >> (e & 31)) & 1u) && (bi < 0 || l > best);
-        best = take ? l : best;
-        bi = take ? e : bi;
-      }
-      tk.v[0] = best;
-      tk.e[0] = bi;
-    } else {
-      float thr = -INFINITY;
-      int filled = 0;
-#pragma unroll 1
-      for (int e = e_lo; e < e_hi; ++e) {
-        const float l = row[e];
-        if (((allow[e >> 5] >> (e & 31)) & 1u) && (filled < k || l > thr)) {
-          tk.push(l, e, k);
-          ++filled;
-          thr = (k == 2) ? tk.v[1] : (k == 3) ? tk.v[2] : tk.v[3];
-        }
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < kMaxTopK; ++j) { cand_v[tid * kMaxTopK + j] = tk.v[j]; cand_e[tid * kMaxTopK + j] = tk.e[j]; }
-  }
-  __syncthreads();
-  // merge the shares of one (token, gate) in ascending expert order: a candidate only displaces
-  // an entry it strictly beats, so equal logits keep the lowest expert index
-  TopK fin;
-  fin.init();
-  if (part == 0) {
-    for (int pp = 0; pp < parts; ++pp) {
-      const int src = ((masked ? parts : 0) + pp) * tok + tl;
-#pragma unroll
-      for (int j = 0; j < kMaxTopK; ++j)
-        if (j < k && cand_e[src * kMaxTopK + j] >= 0) fin.push(cand_v[src * kMaxTopK + j], cand_e[src * kMaxTopK + j], k);
-    }
-    s_m[tl * 2 + (masked ? 1 : 0)] = fin.v[0];
-  }
-  __syncthreads();
-  {
-    const float m = s_m[tl * 2 + (masked ? 1 : 0)];
-    float den = 0.f;
-    if (!a.renorm) {
-      // eight interleaved partial sums: short dependency chains and a tree-shaped total
-      float acc8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
-      for (int e0 = e_lo; e0 < e_hi; e0 += 8) {
-        const uint32_t w = allow[e0 >> 5] >> (e0 & 31);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float t = __expf(row[e0 + i] - m);
-          acc8[i] += ((w >> i) & 1u) ? t : 0.f;
-        }
-      }
-      den = ((acc8[0] + acc8[1]) + (acc8[2] + acc8[3])) + ((acc8[4] + acc8[5]) + (acc8[6] + acc8[7]));
-    }
-    part_den[tid] = den;
-  }
-  __syncthreads();
-  if (part == 0) {
-    const float m = fin.v[0];
-    float den = 0.f;
-    if (a.renorm) {
-#pragma unroll
-      for (int j = 0; j < kMaxTopK; ++j)
-        if (j < k) den += expf(fin.v[j] - m);
-    } else {
-      for (int pp = 0; pp < parts; ++pp) den += part_den[((masked ? parts : 0) + pp) * tok + tl];
-    }
-    const float xn = snorm[tl];
-#pragma unroll
-    for (int j = 0; j < kMaxTopK; ++j) {
-      if (j < k) {
-        const int pl = tl * k + j;
-        const size_t p = (size_t)token * k + j;
-        const float g = failed ? 0.f : expf(fin.v[j] - m) / den;
-        const int e = fin.e[j];
-        if (!masked) {
-          if (token < a.T) {
-            a.uidx[p] = e; a.ugate[p] = g;
-            pe[pl] = e; pt[pl] = xn * fabsf(g) * s_enorm[e];   // one term of Eq. (1)
-            atomicOr(&s_present[e >> 5], 1u << (e & 31));
-          } else {
-            pe[pl] = -1; pt[pl] = 0.f;
-          }
-        } else {
-          if (token < a.T) {
-            const int sl = s_e2s[e];
-            a.midx[p] = e; a.mgate[p] = g; a.slot[p] = sl;
-            ps[pl] = sl; pm[pl] = xn * fabsf(g) * s_enorm[e];
-          } else {
-            ps[pl] = -1; pm[pl] = 0.f;
-          }
-        }
-      }
-    }
-    if (!masked && token < a.T) a.xnorm[token] = xn;
-  }
-  __syncthreads();
-  // Per-CTA partial sums with a fixed association (lane-strided partials, then the
-  // shuffle tree), so the result does not depend on scheduling.  Only experts that some
-  // token of this tile selected are visited; the others get an exact zero.
-  const int npair = tok * k;
-  for (int e = tid; e < E; e += kRtThreads) {
-    a.cta_imp[(size_t)blockIdx.x * E + e] = 0.f;
-    if (a.cta_cnt) a.cta_cnt[(size_t)blockIdx.x * E + e] = 0.f;
-  }
-  for (int sl = tid; sl < a.K; sl += kRtThreads) a.cta_hist[(size_t)blockIdx.x * a.K + sl] = 0;
-  __syncthreads();
-  for (int c = 0; c * 32 < E; ++c) {
-    uint32_t present = s_present[c];
-    for (int n = 0; present; ++n) {
-      const int bit = __ffs(present) - 1;
-      present &= present - 1;
-      if ((n & 7) != warp) continue;                    // experts dealt round-robin to the warps
-      const int e = c * 32 + bit;
-      float sum = 0.f;
-      int hits = 0;
-      for (int p = lane; p < npair; p += 32) { sum += (pe[p] == e) ? pt[p] : 0.f; hits += (pe[p] == e); }
-      sum = warp_sum(sum);
-      hits = __reduce_add_sync(0xffffffffu, hits);
-      if (lane == 0) {
-        a.cta_imp[(size_t)blockIdx.x * E + e] = sum;
-        if (a.cta_cnt) a.cta_cnt[(size_t)blockIdx.x * E + e] = (float)hits;
-      }
-    }
-  }
-  for (int sl = warp; sl < a.K; sl += kRtThreads / 32) {
-    int c = 0;
-    float m = 0.f;
-    for (int p = lane; p < npair; p += 32) { c += (ps[p] == sl); m += (ps[p] == sl) ? pm[p] : 0.f; }
-    c = __reduce_add_sync(0xffffffffu, c);
-    m = warp_sum(m);
-    if (lane == 0) {
-      if (c) a.cta_hist[(size_t)blockIdx.x * a.K + sl] = c;
-      if (a.cta_mimp) a.cta_mimp[(size_t)blockIdx.x * a.K + sl] = m;
-    }
-  }
-  finish_router_cta(a.scan, smem, stage_area);      // the stage memory is free again: stage the scan inputs there
+  // the stage memory is free again: the last CTA stages the scan inputs there
+  gate_epilogue(a, g, slog, tok, tok0, failed, smem, stage_area);
 }
 
 }  // namespace swapmoe
