@@ -11,6 +11,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "decode_fused.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "ffn_fused.cuh"
@@ -50,6 +51,11 @@ struct swapmoe_layer {
   int64_t launches;
   int32_t gemm_path;
   int32_t rows_pad_max;
+  bool decode_path;            // one-launch forward for a handful of tokens (bf16)
+  int32_t decode_max_tokens;   // ... used up to this many tokens (the kernel takes up to 8)
+  float* dec_ws;               // its partial-row workspace
+  unsigned* dec_tickets;
+  CUtensorMap dec_map_wo;      // W_out viewed for the decode kernel's column-slice loads
   int32_t y_copies;            // copies of y in the workspace (slices of a split contraction)
   int32_t sm_count;
   bool use_pdl;                // programmatic dependent launch between the kernels of a forward
@@ -58,10 +64,6 @@ struct swapmoe_layer {
   int32_t router_tok;          // 0 = automatic token-tile size of the tensor-core router, else 32/64/128
   bool prefetch;               // pull resident weights into L2 from the router kernel
   long long l2_prefetch_bytes; // how much of them (L2 capacity minus head room)
-  int32_t side_prefetch;       // >0: prefetch from a kernel on a private stream instead (experiment switch)
-  long long side_mb0, side_mb1;// bytes of the first wave (with the router) and of the second (with GEMM-1)
-  cudaStream_t s_pf;
-  cudaEvent_t ev_pf_fork, ev_pf_mid, ev_pf_join;
   void* const* stage_events;   // 7 cudaEvent_t of the forward being enqueued, or nullptr
   CUtensorMap map_x;           // TMA view of the last token matrix [T, d]
   const void* map_x_ptr;
@@ -90,29 +92,6 @@ __global__ void set_enorm_kernel(const EnormTable t, int E, float* enorm) {
   for (int i = threadIdx.x; i < E; i += blockDim.x) enorm[i] = t.v[i];
 }
 
-// Pulls bytes [begin, end) of the resident weights, counted over logical slots in order with
-// GEMM-1's matrices before GEMM-2's, towards L2.
-struct PrefetchArgs {
-  const char* base[2];
-  long long slot_bytes[2];
-  long long total[2];
-  const int32_t* phys;
-  long long begin, end;
-};
-__global__ void __launch_bounds__(256) prefetch_l2_kernel(const PrefetchArgs a) {
-  constexpr long long kChunk = 16384;
-  const long long n_thr = (long long)gridDim.x * blockDim.x;
-  for (long long c = a.begin / kChunk + (long long)blockIdx.x * blockDim.x + threadIdx.x; c * kChunk < a.end; c += n_thr) {
-    long long off = c * kChunk;
-    int m = 0;
-    if (off >= a.total[0]) { off -= a.total[0]; m = 1; }
-    if (off >= a.total[m]) break;
-    const long long sl = off / a.slot_bytes[m], o = off - sl * a.slot_bytes[m];
-    const char* src = a.base[m] + (long long)a.phys[sl] * a.slot_bytes[m] + o;
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"((unsigned)kChunk) : "memory");
-  }
-}
-
 inline void mark(swapmoe_layer* L, int i, cudaStream_t st) {
   if (L->stage_events) cudaEventRecord(static_cast<cudaEvent_t>(L->stage_events[i]), st);
 }
@@ -124,6 +103,29 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
                      cudaStream_t st) {
   const swapmoe_config_t& c = L->cfg;
   const bool pdl = L->use_pdl && L->stage_events == nullptr;
+  if (L->decode_path && T <= L->decode_max_tokens && c.dtype == SWAPMOE_BF16) {
+    // a handful of tokens: routing, both expert products and the combine in one launch
+    DecodeArgs da;
+    da.x = static_cast<const bf16*>(x); da.Wr = static_cast<const bf16*>(L->Wr); da.ext_logits = ext_logits;
+    da.e2s = L->e2s; da.s2e = L->s2e; da.phys = L->phys; da.enorm = L->enorm;
+    da.arena_in = static_cast<const bf16*>(L->arena_in); da.arena_out = static_cast<const bf16*>(L->arena_out);
+    da.in_stride = (long long)L->nin * c.d_ff * c.d_model; da.out_stride = (long long)c.d_ff * c.d_model;
+    da.logits = L->logits; da.uidx = L->uidx; da.ugate = L->ugate; da.midx = L->midx; da.mgate = L->mgate;
+    da.slot = L->slot; da.xnorm = L->xnorm; da.count = L->count; da.offset = L->offset; da.perm = L->perm;
+    da.inv = L->inv; da.imp = L->imp; da.cnt = L->cnt; da.mimp = L->mimp;
+    const size_t n_jb = c.d_ff / kDecJB;
+    da.ypart = L->dec_ws; da.gpart = L->dec_ws + n_jb * (size_t)(kDecMaxTokens * c.top_k) * c.d_model;
+    da.tickets = L->dec_tickets; da.out = static_cast<bf16*>(out); da.status = L->status;
+    da.T = T; da.d = c.d_model; da.f = c.d_ff; da.E = c.E; da.k = c.top_k; da.K = c.K; da.renorm = c.renorm_topk;
+    da.swiglu = c.act == SWAPMOE_ACT_SWIGLU;
+    mark(L, 0, st);
+    if (launch_kernel(decode_fused_kernel, dim3(L->sm_count), dim3(kDecThreads), decode_smem_bytes(c.d_model), st, pdl,
+                      L->dec_map_wo, da) != cudaSuccess)
+      return SWAPMOE_ERR_CUDA;
+    L->launches++;
+    for (int i = 1; i <= 6; ++i) mark(L, i, st);
+    return check_launch();
+  }
   const bool tc_router = L->tc.router_ok && ext_logits == nullptr;
   int tok_tile = tc_router ? router_tc_tok(T) : kTokTile;
   if (tc_router && L->router_tok) tok_tile = L->router_tok;
@@ -176,21 +178,6 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     if (pf_ctas < 0) pf_ctas = 0;
     if (pf_ctas > 64) pf_ctas = 64;
   }
-  bool side = false;
-  PrefetchArgs pfa;
-  if (pf_ctas > 0 && L->side_prefetch && L->stage_events == nullptr) {
-    side = true;
-    pfa.base[0] = ra.pf_base[0]; pfa.base[1] = ra.pf_base[1];
-    pfa.slot_bytes[0] = ra.pf_slot_bytes[0]; pfa.slot_bytes[1] = ra.pf_slot_bytes[1];
-    pfa.total[0] = pfa.slot_bytes[0] * c.K; pfa.total[1] = pfa.slot_bytes[1] * c.K;
-    pfa.phys = L->phys;
-    pfa.begin = 0; pfa.end = L->side_mb0;
-    ra.pf_total_bytes[0] = ra.pf_total_bytes[1] = 0;
-    pf_ctas = 0;
-    if (!cuda_ok(cudaEventRecord(L->ev_pf_fork, st)) || !cuda_ok(cudaStreamWaitEvent(L->s_pf, L->ev_pf_fork, 0)))
-      return SWAPMOE_ERR_CUDA;
-    prefetch_l2_kernel<<<L->side_prefetch, 256, 0, L->s_pf>>>(pfa);
-  }
   mark(L, 0, st);
   if (tc_router) {
     if (x != L->map_x_ptr || T != L->map_x_T) {   // the token map is re-encoded only when x or T changes
@@ -226,14 +213,6 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
       cudaSuccess)
     return SWAPMOE_ERR_CUDA;
   L->launches++;
-  if (side && L->side_mb1 > 0) {
-    // second wave: starts when the permutation has finished, i.e. alongside GEMM-1
-    pfa.begin = L->side_mb0; pfa.end = L->side_mb0 + L->side_mb1;
-    if (!cuda_ok(cudaEventRecord(L->ev_pf_mid, st)) || !cuda_ok(cudaStreamWaitEvent(L->s_pf, L->ev_pf_mid, 0)))
-      return SWAPMOE_ERR_CUDA;
-    prefetch_l2_kernel<<<L->side_prefetch, 256, 0, L->s_pf>>>(pfa);
-  }
-
   mark(L, 3, st);
   bool combined = false;
   int y_split = 1;
@@ -299,8 +278,6 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     L->launches++;
   }
   mark(L, 6, st);
-  if (side && (!cuda_ok(cudaEventRecord(L->ev_pf_join, L->s_pf)) || !cuda_ok(cudaStreamWaitEvent(st, L->ev_pf_join, 0))))
-    return SWAPMOE_ERR_CUDA;
   return check_launch();
 }
 
@@ -367,12 +344,6 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
     L->l2_prefetch_bytes = l2 > (80ll << 20) ? (56ll << 20) : 0;
     env = std::getenv("SWAPMOE_PREFETCH_MB");
     if (env) L->l2_prefetch_bytes = std::atoll(env) << 20;
-    env = std::getenv("SWAPMOE_SIDE_PREFETCH");         // CTAs of the side-stream prefetch kernel, 0 = off
-    L->side_prefetch = env ? std::atoi(env) : 0;
-    env = std::getenv("SWAPMOE_SIDE_MB0");
-    L->side_mb0 = (env ? std::atoll(env) : 56) << 20;
-    env = std::getenv("SWAPMOE_SIDE_MB1");
-    L->side_mb1 = (env ? std::atoll(env) : 0) << 20;
   }
   L->nin = c.act == SWAPMOE_ACT_SWIGLU ? 2 : 1;
   L->elem = c.dtype == SWAPMOE_BF16 ? 2 : 4;
@@ -410,6 +381,19 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_y = cv.take<float>(rows_pad * c.d_model * L->y_copies);
   const size_t o_xs = cv.take<char>(T * c.d_model * L->elem);
   const size_t o_os = cv.take<char>(T * c.d_model * L->elem);
+  {
+    // Measured on B200 (d_model 1024, d_ff 4096): the one-launch path costs 20 us + 9.5 us per extra
+    // touched slot, the general kernels 42-46 us up to four tokens: it wins up to three tokens.
+    L->decode_max_tokens = 3;
+    const char* envt = std::getenv("SWAPMOE_DECODE_MAX_T");  // 1..8: use the one-launch path up to this many tokens
+    if (envt && std::atoi(envt) >= 1 && std::atoi(envt) <= kDecMaxTokens) L->decode_max_tokens = std::atoi(envt);
+    const char* env = std::getenv("SWAPMOE_DECODE_PATH");   // SWAPMOE_DECODE_PATH=0: general kernels for tiny batches too
+    L->decode_path = c.dtype == SWAPMOE_BF16 && !(env && env[0] == '0') &&
+                     decode_smem_bytes(c.d_model) <= (size_t)(226 << 10) &&
+                     decode_ws_floats(c.d_model, c.d_ff, c.top_k) * sizeof(float) <= ((size_t)64 << 20);
+  }
+  const size_t o_dec_ws = cv.take<float>(L->decode_path ? decode_ws_floats(c.d_model, c.d_ff, c.top_k) : 1);
+  const size_t o_dec_tk = cv.take<unsigned>(L->decode_path ? decode_ticket_count(c.d_ff, c.K) : 1);
   L->ws_bytes = cv.off;
   if (!cuda_ok(cudaMalloc(&L->ws_base, L->ws_bytes))) { cudaGetLastError(); delete L; return SWAPMOE_ERR_CUDA; }
   char* b = L->ws_base;
@@ -432,12 +416,17 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   L->tiles_b = (TileDesc*)(b + o_tiles_b); L->n_tiles_b = (int32_t*)(b + o_ntiles_b);
   L->xp = b + o_xp; L->h = b + o_h; L->y = (float*)(b + o_y);
   L->x_stage = b + o_xs; L->out_stage = b + o_os;
+  L->dec_ws = (float*)(b + o_dec_ws); L->dec_tickets = (unsigned*)(b + o_dec_tk);
 
   bool ok = cuda_ok(cudaMemset(L->imp, 0, sizeof(float) * c.E));
   ok = ok && cuda_ok(cudaMemset(L->cnt, 0, sizeof(float) * c.E));
   ok = ok && cuda_ok(cudaMemset(L->mimp, 0, sizeof(float) * c.E));
   ok = ok && cuda_ok(cudaMemset(L->status, 0, sizeof(int32_t) * 4));
   ok = ok && cuda_ok(cudaMemset(L->ticket, 0, sizeof(unsigned) * 4));
+  if (L->decode_path) {
+    ok = ok && cuda_ok(cudaMemset(L->dec_tickets, 0, sizeof(unsigned) * decode_ticket_count(c.d_ff, c.K)));
+    ok = ok && cuda_ok(decode_fused_set_smem_limit((int)decode_smem_bytes(c.d_model)));
+  }
   ok = ok && cuda_ok(cudaFuncSetAttribute(router_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           210 * 1024));
   // Rows of the padded workspaces that no pair occupies are computed on but never
@@ -445,16 +434,13 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   ok = ok && cuda_ok(cudaMemset(L->xp, 0, rows_pad * c.d_model * L->elem));
   ok = ok && cuda_ok(router_gate_set_smem_limit<float>()) && cuda_ok(router_gate_set_smem_limit<bf16>());
   ok = ok && tc_init(L->tc, c, L->xp, L->h, L->y, L->rows_pad_max) == SWAPMOE_OK;
+  if (L->tc.encode == nullptr) L->decode_path = false;     // its W_out loads need a tensor map
   if (ok && L->tc.enabled) ok = tc_small_set_attrs();
   ok = ok && cuda_ok(cudaStreamCreateWithFlags(&L->s_in, cudaStreamNonBlocking));
   ok = ok && cuda_ok(cudaStreamCreateWithFlags(&L->s_out, cudaStreamNonBlocking));
   ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_in, cudaEventDisableTiming));
   ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_comp, cudaEventDisableTiming));
   ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_out, cudaEventDisableTiming));
-  ok = ok && cuda_ok(cudaStreamCreateWithFlags(&L->s_pf, cudaStreamNonBlocking));
-  ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_pf_fork, cudaEventDisableTiming));
-  ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_pf_mid, cudaEventDisableTiming));
-  ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_pf_join, cudaEventDisableTiming));
   if (!ok) { cudaGetLastError(); cudaFree(L->ws_base); delete L; return SWAPMOE_ERR_CUDA; }
   *out = L;
   return SWAPMOE_OK;
@@ -467,10 +453,6 @@ int32_t swapmoe_destroy(swapmoe_layer_t* L) {
   if (L->ev_in) cudaEventDestroy(L->ev_in);
   if (L->ev_comp) cudaEventDestroy(L->ev_comp);
   if (L->ev_out) cudaEventDestroy(L->ev_out);
-  if (L->s_pf) cudaStreamDestroy(L->s_pf);
-  if (L->ev_pf_fork) cudaEventDestroy(L->ev_pf_fork);
-  if (L->ev_pf_mid) cudaEventDestroy(L->ev_pf_mid);
-  if (L->ev_pf_join) cudaEventDestroy(L->ev_pf_join);
   cudaFree(L->ws_base);
   delete L;
   return SWAPMOE_OK;
@@ -518,6 +500,11 @@ int32_t swapmoe_set_resident(swapmoe_layer_t* L, const int32_t* s2e, const int32
     L->small.valid = false;
     const int32_t rc = tc_bind_arena(L->tc, c, arena_in, arena_out);
     if (rc != SWAPMOE_OK) return rc;
+    // column slices of W_out for the one-launch decode kernel: 32 columns x 256 rows, 64-byte swizzle
+    if (L->decode_path &&
+        !tc_encode_2d_box(L->tc.encode, &L->dec_map_wo, arena_out, (uint64_t)P * c.d_model, (uint64_t)c.d_ff,
+                          (uint32_t)kDecJB, (uint32_t)kDecOutRows, CU_TENSOR_MAP_SWIZZLE_64B))
+      return SWAPMOE_ERR_CUDA;
   }
   set_tables_kernel<<<1, 256, 0, static_cast<cudaStream_t>(stream)>>>(t, c.E, c.K, L->e2s, L->phys, L->s2e);
   L->launches++;

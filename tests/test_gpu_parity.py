@@ -297,3 +297,77 @@ def test_cfg2_in_the_benchmark_launch_configuration():
         # three replays accumulated three batches of importance: start the oracle from two of them
         r0 = c.oracle(c.layer.tap("logits"))
         check_against_oracle(c, out, imp_before=2 * r0["imp"])
+
+
+DECODE = [
+    _cfg(T=1, d=256, f=512, E=64, K=16, zipf_s=1.1),
+    _cfg(T=2, d=1024, f=4096, E=64, K=16, zipf_s=1.1),
+    _cfg(T=3, d=192, f=320, E=40, K=7, k=2, renorm=0),
+    _cfg(T=5, d=128, f=256, E=8, K=4, k=2, renorm=1, act=I.ACT_SWIGLU),
+    _cfg(T=8, d=256, f=1088, E=256, K=33, k=4, renorm=1, zipf_s=1.1),     # 34 blocks of hidden units: ragged last group
+    _cfg(T=8, d=128, f=128, E=1, K=1, k=1),                               # every token in one slot
+]
+
+
+@pytest.mark.parametrize("cfg", DECODE, ids=lambda c: "T%d_d%d_f%d_E%d_k%d_K%d_%s" % (
+    c.T, c.d, c.f, c.E, c.k, c.K, "swiglu" if c.act else "relu"))
+def test_one_launch_decode_path(cfg, monkeypatch):
+    """The single-launch path (bf16, up to 8 tokens; by default used up to 3) must match the
+    oracle like the general kernels, twice in a row (its tickets reset themselves), and be
+    repeatable bit for bit."""
+    from harness import Case, check_against_oracle
+    monkeypatch.setenv("SWAPMOE_DECODE_MAX_T", "8")
+    case = Case(cfg, spare=2, phys=np.arange(cfg.K, dtype=np.int32)[::-1] + 2)
+    n0 = case.layer.launch_count
+    out = case.run()
+    assert case.layer.launch_count - n0 == 1
+    r = check_against_oracle(case, out)
+    out2 = case.run()
+    assert np.array_equal(out, out2)
+    check_against_oracle(case, out2, imp_before=r["oracle"]["imp"])
+
+
+def test_decode_path_matches_general_kernels(monkeypatch):
+    """Same inputs through the single-launch path and through the general kernels."""
+    from harness import Case
+    cfg = _cfg(T=6, d=256, f=512, E=64, K=16, k=2, renorm=1, zipf_s=1.1)
+    monkeypatch.setenv("SWAPMOE_DECODE_MAX_T", "8")
+    a = Case(cfg)
+    n0 = a.layer.launch_count
+    out_a = a.run()
+    assert a.layer.launch_count - n0 == 1
+    monkeypatch.setenv("SWAPMOE_DECODE_PATH", "0")
+    b = Case(cfg)
+    n0 = b.layer.launch_count
+    out_b = b.run()
+    assert b.layer.launch_count - n0 > 1
+    for name in ("uidx", "midx", "slot", "count", "offset", "perm", "inv"):
+        assert np.array_equal(a.layer.tap(name), b.layer.tap(name)), name
+    scale = np.max(np.abs(out_b))
+    assert np.max(np.abs(out_a - out_b)) <= 2e-2 * scale
+    for kind in ("eq1", "count", "eq1_masked"):
+        ia, ib = a.layer.read_score(kind), b.layer.read_score(kind)
+        assert np.max(np.abs(ia - ib)) <= 1e-4 * max(1e-30, np.max(np.abs(ib))), kind
+
+
+def test_decode_path_external_logits_with_ties(monkeypatch):
+    from harness import Case, check_against_oracle
+    monkeypatch.setenv("SWAPMOE_DECODE_MAX_T", "8")
+    cfg = _cfg(T=4, d=128, f=256, E=16, K=6, k=2)
+    case = Case(cfg)
+    lg = np.zeros((cfg.T, cfg.E), np.float32)
+    lg[:, 3] = lg[:, 9] = 1.0          # ties: the lower index must win
+    lg[2, :] = 0.5                     # a full tie
+    out = case.run(ext_logits=lg)
+    check_against_oracle(case, out, check_logits=False)
+
+
+def test_decode_path_default_threshold():
+    """Without overrides the single-launch path serves up to three tokens, the general kernels the rest."""
+    from harness import Case, check_against_oracle
+    for T, one in ((3, True), (4, False)):
+        case = Case(_cfg(T=T, d=256, f=512, E=64, K=16, zipf_s=1.1))
+        n0 = case.layer.launch_count
+        out = case.run()
+        assert (case.layer.launch_count - n0 == 1) == one
+        check_against_oracle(case, out)
