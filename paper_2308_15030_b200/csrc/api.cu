@@ -428,7 +428,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
     ok = ok && cuda_ok(decode_fused_set_smem_limit((int)decode_smem_bytes(c.d_model)));
   }
   ok = ok && cuda_ok(cudaFuncSetAttribute(router_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          210 * 1024));
+                                          226 * 1024));
   // Rows of the padded workspaces that no pair occupies are computed on but never
   // read back; start them at zero so they hold finite values.
   ok = ok && cuda_ok(cudaMemset(L->xp, 0, rows_pad * c.d_model * L->elem));
