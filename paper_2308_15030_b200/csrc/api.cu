@@ -52,7 +52,7 @@ struct swapmoe_layer {
   int32_t gemm_path;
   int32_t rows_pad_max;
   bool decode_path;            // one-launch forward for a handful of tokens (bf16)
-  int32_t decode_max_tokens;   // ... used up to this many tokens (the kernel takes up to 8)
+  int32_t decode_max_pairs;    // ... used up to this many (token, expert) pairs (the kernel takes 8 tokens)
   float* dec_ws;               // its partial-row workspace
   unsigned* dec_tickets;
   CUtensorMap dec_map_wo;      // W_out viewed for the decode kernel's column-slice loads
@@ -103,7 +103,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
                      cudaStream_t st) {
   const swapmoe_config_t& c = L->cfg;
   const bool pdl = L->use_pdl && L->stage_events == nullptr;
-  if (L->decode_path && T <= L->decode_max_tokens && c.dtype == SWAPMOE_BF16) {
+  if (L->decode_path && T <= kDecMaxTokens && T * c.top_k <= L->decode_max_pairs && c.dtype == SWAPMOE_BF16) {
     // a handful of tokens: routing, both expert products and the combine in one launch
     DecodeArgs da;
     da.x = static_cast<const bf16*>(x); da.Wr = static_cast<const bf16*>(L->Wr); da.ext_logits = ext_logits;
@@ -382,11 +382,11 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_xs = cv.take<char>(T * c.d_model * L->elem);
   const size_t o_os = cv.take<char>(T * c.d_model * L->elem);
   {
-    // Measured on B200 (d_model 1024, d_ff 4096): the one-launch path costs 20 us + 9.5 us per extra
-    // touched slot, the general kernels 42-46 us up to four tokens: it wins up to three tokens.
-    L->decode_max_tokens = 3;
-    const char* envt = std::getenv("SWAPMOE_DECODE_MAX_T");  // 1..8: use the one-launch path up to this many tokens
-    if (envt && std::atoi(envt) >= 1 && std::atoi(envt) <= kDecMaxTokens) L->decode_max_tokens = std::atoi(envt);
+    // Measured on B200 (d_model 1024, d_ff 4096, top-1): the one-launch path costs about 21 us + 5.5 us
+    // per extra touched slot, the general kernels 42-54 us up to eight tokens: it wins up to six pairs.
+    L->decode_max_pairs = 6;
+    const char* envt = std::getenv("SWAPMOE_DECODE_MAX_PAIRS");  // 1..32: use the one-launch path up to this many pairs
+    if (envt && std::atoi(envt) >= 1 && std::atoi(envt) <= kDecMaxPairs) L->decode_max_pairs = std::atoi(envt);
     const char* env = std::getenv("SWAPMOE_DECODE_PATH");   // SWAPMOE_DECODE_PATH=0: general kernels for tiny batches too
     L->decode_path = c.dtype == SWAPMOE_BF16 && !(env && env[0] == '0') &&
                      decode_smem_bytes(c.d_model) <= (size_t)(226 << 10) &&

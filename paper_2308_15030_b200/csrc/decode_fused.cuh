@@ -389,11 +389,16 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
   const int out_rows = kDecOutRows * kDecOutBoxes;   // 1024
   const int n_out = (d + out_rows - 1) / out_rows;
   const int wpi = n_in * n_mats + n_out;             // waves per item
-  const int my_items = n_items > (int)blockIdx.x ? (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  // A CTA takes a contiguous range of items: consecutive items are consecutive blocks of hidden
+  // units of one slot, so their partial output rows can be added in registers (a "run") and only
+  // one set of partial rows, one fence and one ticket are spent per run instead of per item.
+  const int ipc = (n_items + (int)gridDim.x - 1) / (int)gridDim.x;      // items per CTA
+  const int item0 = (int)blockIdx.x * ipc;
+  const int my_items = max(0, min(ipc, n_items - item0));
   const int total = my_items * wpi;
   auto issue_item_wave = [&](int v) {                // all of warp 0
     const int it = v / wpi, wi = v - it * wpi;
-    const int item = blockIdx.x + it * gridDim.x;
+    const int item = item0 + it;
     const int ti = item / n_jb, jb = item - ti * n_jb;
     const int ph = R->phys[R->touched[ti]];
     const int w = n_rw + v;
@@ -461,12 +466,20 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
     }
   }
 
+  float yacc[kDecOutBoxes][4];      // a run's partial output rows: tile warp + 16 i, mma accumulator layout
+  int run_jb = -1;                  // first hidden block of the current run, -1 = none open
 #pragma unroll 1
   for (int v = 0; v < total; ++v) {
     const int it = v / wpi, wi = v - it * wpi;
-    const int item = blockIdx.x + it * gridDim.x;
+    const int item = item0 + it;
     const int ti = item / n_jb, jb = item - ti * n_jb;
     const int s = R->touched[ti], n_s = R->tcount[ti], q0 = R->toffset[ti];
+    const int grp = jb / kDecGroup;
+    // runs need the whole output in one wave and all the slot's pairs in one mma
+    const bool runs = n_out == 1 && n_s <= 8;
+    // the run ends with this item unless the CTA's next item is in the same slot and group
+    const bool run_ends = !runs || it + 1 >= my_items || (item + 1) / n_jb != ti ||
+                          (item + 1 - ti * n_jb) / kDecGroup != grp;
     const int w = n_rw + v;
     if (!dec_wait_wave(bars, w, R, a.status, 22)) { alive = false; break; }
     const unsigned char* st = ring + (w & 1) * kDecHalfBytes;
@@ -499,41 +512,61 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
         const int nn = min(8, n_s - nb);
         const unsigned char* hrow = reinterpret_cast<const unsigned char*>(hsb) + (nb + min(g, nn - 1)) * (kDecHPitch * 2) + t * 4;
         const uint32_t b00 = lds32(hrow), b01 = lds32(hrow + 16), b10 = lds32(hrow + 32), b11 = lds32(hrow + 48);
-#pragma unroll 1
-        for (int tile = warp; tile * 16 < out_rows; tile += kDecWarps) {
-          const int r0 = tile * 16 + g, r1 = r0 + 8;      // rows of the wave
+        if (!runs || run_jb < 0) {              // a new run (without runs: every item, batch and wave)
+          run_jb = jb;
+#pragma unroll
+          for (int i = 0; i < kDecOutBoxes; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) yacc[i][j] = 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < kDecOutBoxes; ++i) {
+          const int r0 = (warp + kDecWarps * i) * 16 + g, r1 = r0 + 8;      // rows of the wave
           // 16-byte chunk j of row r sits at chunk j ^ ((r >> 1) & 3)
           const unsigned char* p0 = st + r0 * 64 + t * 4;
           const unsigned char* p1 = st + r1 * 64 + t * 4;
           const int x0 = (r0 >> 1) & 3, x1 = (r1 >> 1) & 3;
-          float acc[4] = {0.f, 0.f, 0.f, 0.f};
-          mma_bf16_16x8x16(acc, lds32(p0 + ((0 ^ x0) << 4)), lds32(p1 + ((0 ^ x1) << 4)), lds32(p0 + ((1 ^ x0) << 4)),
+          mma_bf16_16x8x16(yacc[i], lds32(p0 + ((0 ^ x0) << 4)), lds32(p1 + ((0 ^ x1) << 4)), lds32(p0 + ((1 ^ x0) << 4)),
                            lds32(p1 + ((1 ^ x1) << 4)), b00, b01);
-          mma_bf16_16x8x16(acc, lds32(p0 + ((2 ^ x0) << 4)), lds32(p1 + ((2 ^ x1) << 4)), lds32(p0 + ((3 ^ x0) << 4)),
+          mma_bf16_16x8x16(yacc[i], lds32(p0 + ((2 ^ x0) << 4)), lds32(p1 + ((2 ^ x1) << 4)), lds32(p0 + ((3 ^ x0) << 4)),
                            lds32(p1 + ((3 ^ x1) << 4)), b10, b11);
-          const int c0 = ow * out_rows + r0, c1 = c0 + 8;
+        }
+        if (run_ends) {
+          // partial rows of the run go out under the run's first hidden block
+          float* yp = a.ypart + ((size_t)run_jb * P + q0 + nb) * d + ow * out_rows + g;
           const int n0 = 2 * t, n1 = 2 * t + 1;
-          if (c0 < d) {
-            if (n0 < nn) a.ypart[((size_t)jb * P + q0 + nb + n0) * d + c0] = acc[0];
-            if (n1 < nn) a.ypart[((size_t)jb * P + q0 + nb + n1) * d + c0] = acc[1];
-          }
-          if (c1 < d) {
-            if (n0 < nn) a.ypart[((size_t)jb * P + q0 + nb + n0) * d + c1] = acc[2];
-            if (n1 < nn) a.ypart[((size_t)jb * P + q0 + nb + n1) * d + c1] = acc[3];
+#pragma unroll
+          for (int i = 0; i < kDecOutBoxes; ++i) {
+            const int c0 = (warp + kDecWarps * i) * 16;          // + g (in yp), + 8 for the second half
+            if (ow * out_rows + c0 + g < d) {
+              if (n0 < nn) yp[(size_t)n0 * d + c0] = yacc[i][0];
+              if (n1 < nn) yp[(size_t)n1 * d + c0] = yacc[i][1];
+            }
+            if (ow * out_rows + c0 + g + 8 < d) {
+              if (n0 < nn) yp[(size_t)n0 * d + c0 + 8] = yacc[i][2];
+              if (n1 < nn) yp[(size_t)n1 * d + c0 + 8] = yacc[i][3];
+            }
           }
         }
       }
     }
-    if (wi == wpi - 1) __threadfence();           // the item's partial rows, before its ticket
+    const bool flush = wi == wpi - 1 && run_ends;
+    if (flush) __threadfence();                   // the run's partial rows, before its ticket
     __syncthreads();                              // the buffer is free; the activations are complete / free
     if (warp == 0 && v + 2 < total) {
       ptx::fence_proxy_async();
       issue_item_wave(v + 2);
     }
-    if (wi != wpi - 1) continue;
-    // ---- first-step sum: whoever finishes the group's last item adds its partial rows
-    const int grp = jb / kDecGroup, g_first = grp * kDecGroup, g_size = min(kDecGroup, n_jb - g_first);
-    if (tid == 0) R->last = atomicAdd(&a.tickets[s * n_groups + grp], 1u) == (unsigned)(g_size - 1);
+    if (!flush) continue;
+    run_jb = -1;
+    // ---- first-step sum: whoever delivers the group's last set of partial rows adds them all.
+    // The group's sets: one per item, or with runs one per CTA whose item range meets the group
+    // (CTA c holds items c*ipc ..; its set is filed under the first of them inside the group).
+    const int g_first = grp * kDecGroup, g_size = min(kDecGroup, n_jb - g_first);
+    const int gs = ti * n_jb + g_first;           // the group's first item, numbered over all items
+    const int c_lo = gs / ipc, c_hi = (gs + g_size - 1) / ipc;
+    const int n_sets = runs ? c_hi - c_lo + 1 : g_size;
+    if (tid == 0) R->last = atomicAdd(&a.tickets[s * n_groups + grp], 1u) == (unsigned)(n_sets - 1);
     __syncthreads();
     if (R->last) {
       __threadfence();
@@ -553,7 +586,8 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
 #pragma unroll
           for (int j = 0; j < 4; ++j) {           // all loads first: one round trip
             const int jj = sub * 4 + j;
-            pv[j] = jj < g_size ? __ldcg(reinterpret_cast<const float4*>(a.ypart + ((size_t)(g_first + jj) * P + q0 + n) * d) + c4)
+            const int jbf = runs ? max(gs, (c_lo + jj) * ipc) - ti * n_jb : g_first + jj;   // where set jj was filed
+            pv[j] = jj < n_sets ? __ldcg(reinterpret_cast<const float4*>(a.ypart + ((size_t)jbf * P + q0 + n) * d) + c4)
                                 : make_float4(0.f, 0.f, 0.f, 0.f);
           }
 #pragma unroll

@@ -312,11 +312,11 @@ DECODE = [
 @pytest.mark.parametrize("cfg", DECODE, ids=lambda c: "T%d_d%d_f%d_E%d_k%d_K%d_%s" % (
     c.T, c.d, c.f, c.E, c.k, c.K, "swiglu" if c.act else "relu"))
 def test_one_launch_decode_path(cfg, monkeypatch):
-    """The single-launch path (bf16, up to 8 tokens; by default used up to 3) must match the
+    """The single-launch path (bf16, up to 8 tokens; by default used up to 6 pairs) must match the
     oracle like the general kernels, twice in a row (its tickets reset themselves), and be
     repeatable bit for bit."""
     from harness import Case, check_against_oracle
-    monkeypatch.setenv("SWAPMOE_DECODE_MAX_T", "8")
+    monkeypatch.setenv("SWAPMOE_DECODE_MAX_PAIRS", "32")
     case = Case(cfg, spare=2, phys=np.arange(cfg.K, dtype=np.int32)[::-1] + 2)
     n0 = case.layer.launch_count
     out = case.run()
@@ -331,7 +331,7 @@ def test_decode_path_matches_general_kernels(monkeypatch):
     """Same inputs through the single-launch path and through the general kernels."""
     from harness import Case
     cfg = _cfg(T=6, d=256, f=512, E=64, K=16, k=2, renorm=1, zipf_s=1.1)
-    monkeypatch.setenv("SWAPMOE_DECODE_MAX_T", "8")
+    monkeypatch.setenv("SWAPMOE_DECODE_MAX_PAIRS", "32")
     a = Case(cfg)
     n0 = a.layer.launch_count
     out_a = a.run()
@@ -352,7 +352,7 @@ def test_decode_path_matches_general_kernels(monkeypatch):
 
 def test_decode_path_external_logits_with_ties(monkeypatch):
     from harness import Case, check_against_oracle
-    monkeypatch.setenv("SWAPMOE_DECODE_MAX_T", "8")
+    monkeypatch.setenv("SWAPMOE_DECODE_MAX_PAIRS", "32")
     cfg = _cfg(T=4, d=128, f=256, E=16, K=6, k=2)
     case = Case(cfg)
     lg = np.zeros((cfg.T, cfg.E), np.float32)
@@ -363,9 +363,10 @@ def test_decode_path_external_logits_with_ties(monkeypatch):
 
 
 def test_decode_path_default_threshold():
-    """Without overrides the single-launch path serves up to three tokens, the general kernels the rest."""
+    """Without overrides the single-launch path serves up to six (token, expert) pairs, the general
+    kernels the rest."""
     from harness import Case, check_against_oracle
-    for T, one in ((3, True), (4, False)):
+    for T, one in ((6, True), (7, False)):
         case = Case(_cfg(T=T, d=256, f=512, E=64, K=16, zipf_s=1.1))
         n0 = case.layer.launch_count
         out = case.run()
