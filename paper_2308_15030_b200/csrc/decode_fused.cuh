@@ -551,7 +551,6 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
       }
     }
     const bool flush = wi == wpi - 1 && run_ends;
-    if (flush) __threadfence();                   // the run's partial rows, before its ticket
     __syncthreads();                              // the buffer is free; the activations are complete / free
     if (warp == 0 && v + 2 < total) {
       ptx::fence_proxy_async();
@@ -566,10 +565,17 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
     const int gs = ti * n_jb + g_first;           // the group's first item, numbered over all items
     const int c_lo = gs / ipc, c_hi = (gs + g_size - 1) / ipc;
     const int n_sets = runs ? c_hi - c_lo + 1 : g_size;
-    if (tid == 0) R->last = atomicAdd(&a.tickets[s * n_groups + grp], 1u) == (unsigned)(n_sets - 1);
+    // One thread publishes for the whole CTA: the block barrier above ordered everybody's stores
+    // before its fence (fences are cumulative), and its second fence orders the ticket before the
+    // reads of the other CTAs' rows (L2 loads below).
+    if (tid == 0) {
+      __threadfence();
+      const bool last = atomicAdd(&a.tickets[s * n_groups + grp], 1u) == (unsigned)(n_sets - 1);
+      __threadfence();
+      R->last = last;
+    }
     __syncthreads();
     if (R->last) {
-      __threadfence();
       const int d4 = d / 4;
       // thread (sub, col): sub = tid / 128 adds partial rows 4 sub .. 4 sub + 3 of 128 float4 columns;
       // the four sub-sums meet in shared memory (the per-warp product area is free here) and are
@@ -605,15 +611,17 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
         }
         __syncthreads();
       }
-      if (tid == 0) a.tickets[s * n_groups + grp] = 0u;
-      __threadfence();
       __syncthreads();
-      if (tid == 0)
-        R->last = atomicAdd(&a.tickets[K * n_groups], 1u) == (unsigned)(R->n_touched * n_groups - 1);
+      if (tid == 0) {
+        a.tickets[s * n_groups + grp] = 0u;
+        __threadfence();
+        const bool last = atomicAdd(&a.tickets[K * n_groups], 1u) == (unsigned)(R->n_touched * n_groups - 1);
+        __threadfence();
+        R->last = last;
+      }
       __syncthreads();
       if (R->last) {
         // ---- second step: all groups are in; gate-weighted sum into out (Section 2's combine)
-        __threadfence();
 #pragma unroll 1
         for (int i = tid; i < T * d4; i += kDecThreads) {
           const int t = i / d4, c4 = i - t * d4;
