@@ -198,10 +198,14 @@ constexpr int kPermThreads = 512;
 // pairs in earlier warps of this CTA + earlier lanes of this warp (match + popc),
 // which is exactly a stable counting sort.  gridDim.y CTAs share one token tile: each
 // recomputes the (cheap) positions and copies every gridDim.y-th row of the tile.
+// The kernel is a chain of memory round trips, so the independent ones are started together:
+// the token rows (inputs of the layer, so even before the wait on the predecessor) go to
+// registers while the slots, the CTA's base counts and the offsets are fetched.
 template <typename T>
 __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const PermuteArgs a) {
   __shared__ int32_t wcount[kPermThreads / 32][kMaxSlots];
   __shared__ int32_t dst_row[kPermThreads];
+  __shared__ int32_t s_base[kMaxSlots], s_off[kMaxSlots], s_pad[kMaxSlots];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int npair = a.tok_tile * a.k;          // <= 512
   const int nwarp_p = (npair + 31) >> 5;
@@ -209,24 +213,46 @@ __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const Perm
   const int n_total = a.T * a.k;
 
   for (int i = tid; i < (kPermThreads / 32) * kMaxSlots; i += kPermThreads) (&wcount[0][0])[i] = 0;
+  // this CTA's rows: local pair pl = ri * gridDim.y + blockIdx.y; the first kPre 16-byte pieces per
+  // thread are fetched now
+  constexpr int kPre = 4;
+  const int vec_per_row = a.d * (int)sizeof(T) / 16;
+  const uint4* src = static_cast<const uint4*>(a.x);
+  const int my_rows = (npair - (int)blockIdx.y + (int)gridDim.y - 1) / (int)gridDim.y;
+  uint4 pre[kPre];
+#pragma unroll
+  for (int u = 0; u < kPre; ++u) {
+    const int i = tid + u * kPermThreads;
+    pre[u] = make_uint4(0u, 0u, 0u, 0u);
+    if (i < my_rows * vec_per_row) {
+      const int ri = i / vec_per_row, v = i - ri * vec_per_row;
+      const int pg = p0 + ri * (int)gridDim.y + (int)blockIdx.y;
+      if (pg < n_total) pre[u] = src[(size_t)(pg / a.k) * vec_per_row + v];
+    }
+  }
   pdl_wait();
   pdl_trigger();
-  __syncthreads();
   int s = -1, rank = 0;
   const int p = p0 + tid;
+  if (tid < npair && p < n_total) s = a.slot[p];
+  if (tid < a.K) {
+    s_base[tid] = a.cta_base[(size_t)blockIdx.x * a.K + tid];
+    s_off[tid] = a.offset[tid];
+    s_pad[tid] = a.pad_offset[tid];
+  }
+  __syncthreads();
   if (warp < nwarp_p) {
-    if (tid < npair && p < n_total) s = a.slot[p];
     const uint32_t same = __match_any_sync(0xffffffffu, s);
     rank = __popc(same & ((1u << lane) - 1u));
     if (s >= 0 && rank == 0) wcount[warp][s] = __popc(same);
   }
   __syncthreads();
   if (s >= 0) {
-    int before = a.cta_base[(size_t)blockIdx.x * a.K + s];
+    int before = s_base[s];
     for (int w = 0; w < warp; ++w) before += wcount[w][s];
     const int within = before + rank;
-    const int pos = a.offset[s] + within;
-    const int row = a.pad_offset[s] + within;
+    const int pos = s_off[s] + within;
+    const int row = s_pad[s] + within;
     if (blockIdx.y == 0) {
       a.perm[pos] = p;
       a.inv[p] = pos;
@@ -239,11 +265,17 @@ __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const Perm
   }
   __syncthreads();
   // Gather: copy each pair's token row into its slot segment, 16 bytes per access.
-  const int vec_per_row = a.d * (int)sizeof(T) / 16;
-  const uint4* src = static_cast<const uint4*>(a.x);
   uint4* dst = static_cast<uint4*>(a.xp);
-  const int my_rows = (npair - (int)blockIdx.y + (int)gridDim.y - 1) / (int)gridDim.y;
-  for (int i = tid; i < my_rows * vec_per_row; i += kPermThreads) {
+#pragma unroll
+  for (int u = 0; u < kPre; ++u) {
+    const int i = tid + u * kPermThreads;
+    if (i < my_rows * vec_per_row) {
+      const int ri = i / vec_per_row, v = i - ri * vec_per_row;
+      const int row = dst_row[ri * gridDim.y + blockIdx.y];
+      if (row >= 0) dst[(size_t)row * vec_per_row + v] = pre[u];
+    }
+  }
+  for (int i = tid + kPre * kPermThreads; i < my_rows * vec_per_row; i += kPermThreads) {
     const int ri = i / vec_per_row, v = i - ri * vec_per_row;
     const int pl = ri * gridDim.y + blockIdx.y;
     const int row = dst_row[pl];
