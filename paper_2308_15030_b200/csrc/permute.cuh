@@ -115,46 +115,78 @@ __device__ __forceinline__ void scan_reduce_block(const ScanArgs& a, void* stage
     a.mimp[my_expert] += acc;              // slots map to distinct experts: no two threads share a target
   }
   __syncthreads();
-  if (tid < a.K) {
-    int off = 0, pad = 0, t0 = 0;
-    for (int s = 0; s < tid; ++s) {
-      const int c = s_count[s];
-      off += c;
-      pad += (c + kSegAlign - 1) / kSegAlign * kSegAlign;
-      t0 += (c + a.tile_rows - 1) / a.tile_rows;
+  // Slot layout by the first warp: lane l owns slots l and l + 32 (K <= 64); offsets, padded
+  // offsets and first-tile indices are exclusive prefix sums over the slots, taken with warp scans
+  // (tile heights are powers of two: shifts, no divisions — this code runs once, every dependent
+  // instruction counts).
+  if (tid < 32) {
+    const int lane = tid;
+    const int sh_a = 31 - __clz(a.tile_rows);
+    const int sh_b = a.tiles_b != nullptr ? 31 - __clz(a.tile_rows_b) : 0;
+    int c[2], off[2], pad[2], ta[2], tb[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int s = lane + 32 * h;
+      c[h] = s < a.K ? s_count[s] : 0;
+      off[h] = c[h];
+      pad[h] = (c[h] + kSegAlign - 1) & ~(kSegAlign - 1);
+      ta[h] = (c[h] + a.tile_rows - 1) >> sh_a;
+      tb[h] = a.tiles_b != nullptr ? (c[h] + a.tile_rows_b - 1) >> sh_b : 0;
     }
-    const int c = s_count[tid];
-    a.count[tid] = c;
-    a.offset[tid] = off;
-    a.pad_offset[tid] = pad;
-    const int nt = (c + a.tile_rows - 1) / a.tile_rows;
-    const int ph = a.phys_slot[tid];
-    for (int i = 0; i < nt; ++i) {
-      TileDesc td;
-      td.phys = ph;
-      td.row0 = pad + i * a.tile_rows;
-      td.rows = min(a.tile_rows, c - i * a.tile_rows);
-      td.slot = tid;
-      a.tiles[t0 + i] = td;
-    }
-    if (tid == a.K - 1) {
-      a.offset[a.K] = off + c;
-      a.pad_offset[a.K] = pad + (c + kSegAlign - 1) / kSegAlign * kSegAlign;
-      *a.n_tiles = t0 + nt;
-    }
-    if (a.tiles_b != nullptr) {            // same segments cut into tiles of another height
-      int tb = 0;
-      for (int s = 0; s < tid; ++s) tb += (s_count[s] + a.tile_rows_b - 1) / a.tile_rows_b;
-      const int ntb = (c + a.tile_rows_b - 1) / a.tile_rows_b;
-      for (int i = 0; i < ntb; ++i) {
-        TileDesc td;
-        td.phys = ph;
-        td.row0 = pad + i * a.tile_rows_b;
-        td.rows = min(a.tile_rows_b, c - i * a.tile_rows_b);
-        td.slot = tid;
-        a.tiles_b[tb + i] = td;
+    // inclusive scans of the four quantities over 64 slots
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int u0 = __shfl_up_sync(0xffffffffu, off[h], o), u1 = __shfl_up_sync(0xffffffffu, pad[h], o);
+        const int u2 = __shfl_up_sync(0xffffffffu, ta[h], o), u3 = __shfl_up_sync(0xffffffffu, tb[h], o);
+        if (lane >= o) { off[h] += u0; pad[h] += u1; ta[h] += u2; tb[h] += u3; }
       }
-      if (tid == a.K - 1) *a.n_tiles_b = tb + ntb;
+    }
+    {
+      const int t0 = __shfl_sync(0xffffffffu, off[0], 31), t1 = __shfl_sync(0xffffffffu, pad[0], 31);
+      const int t2 = __shfl_sync(0xffffffffu, ta[0], 31), t3 = __shfl_sync(0xffffffffu, tb[0], 31);
+      off[1] += t0; pad[1] += t1; ta[1] += t2; tb[1] += t3;
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int s = lane + 32 * h;
+      if (s < a.K) {
+        const int cnt = c[h];
+        const int padded = (cnt + kSegAlign - 1) & ~(kSegAlign - 1);
+        const int nt = (cnt + a.tile_rows - 1) >> sh_a;
+        const int o_excl = off[h] - cnt, p_excl = pad[h] - padded, t_excl = ta[h] - nt;
+        a.count[s] = cnt;
+        a.offset[s] = o_excl;
+        a.pad_offset[s] = p_excl;
+        const int ph = a.phys_slot[s];
+        for (int i = 0; i < nt; ++i) {
+          TileDesc td;
+          td.phys = ph;
+          td.row0 = p_excl + i * a.tile_rows;
+          td.rows = min(a.tile_rows, cnt - i * a.tile_rows);
+          td.slot = s;
+          a.tiles[t_excl + i] = td;
+        }
+        if (s == a.K - 1) {
+          a.offset[a.K] = off[h];
+          a.pad_offset[a.K] = pad[h];
+          *a.n_tiles = ta[h];
+        }
+        if (a.tiles_b != nullptr) {            // same segments cut into tiles of another height
+          const int ntb = (cnt + a.tile_rows_b - 1) >> sh_b;
+          const int tb_excl = tb[h] - ntb;
+          for (int i = 0; i < ntb; ++i) {
+            TileDesc td;
+            td.phys = ph;
+            td.row0 = p_excl + i * a.tile_rows_b;
+            td.rows = min(a.tile_rows_b, cnt - i * a.tile_rows_b);
+            td.slot = s;
+            a.tiles_b[tb_excl + i] = td;
+          }
+          if (s == a.K - 1) *a.n_tiles_b = tb[h];
+        }
+      }
     }
   }
 }
