@@ -133,6 +133,7 @@ struct DecRoute {
   float ug[kDecMaxPairs], mg[kDecMaxPairs];
   int q[kDecMaxPairs];          // position of pair p in slot-sorted order
   int pair_at[kDecMaxPairs];    // inverse: pair at sorted position
+  int tok_at[kDecMaxPairs];     // token of the pair at sorted position
   int touched[kDecMaxPairs];    // slots with pairs, ascending
   int tcount[kDecMaxPairs];     // ... their pair counts
   int toffset[kDecMaxPairs];    // ... and the position of their first pair in sorted order
@@ -279,10 +280,23 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
   pdl_wait();
   pdl_trigger();
   // ------------------------------------------------------------------ routing, in every CTA
+  // (integer divisions are kept out of this kernel's once-run paths: each costs dozens of
+  // dependent instructions)
+  // token t is copied by warps t and t + 8 (T <= 8, 16 warps), four independent loads per lane and round
+  {
+    const int t = warp & (kDecMaxTokens - 1);
+    if (t < T) {
 #pragma unroll 1
-  for (int i = tid; i < T * chunks; i += kDecThreads) {
-    const int t = i / chunks, c = i - t * chunks;
-    *reinterpret_cast<uint4*>(xs + t * pitch + c * 16) = reinterpret_cast<const uint4*>(a.x)[i];
+      for (int c0 = (warp >> 3) * 32 + lane; c0 < chunks; c0 += 256) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (c0 + 64 * u < chunks) v[u] = reinterpret_cast<const uint4*>(a.x)[t * chunks + c0 + 64 * u];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (c0 + 64 * u < chunks) *reinterpret_cast<uint4*>(xs + t * pitch + (c0 + 64 * u) * 16) = v[u];
+      }
+    }
   }
   if (tid < kMaxE) R->e2s[tid] = tid < E ? a.e2s[tid] : -1;
   if (tid < K) R->phys[tid] = a.phys[tid];
@@ -369,6 +383,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
       const int q = less + rank;
       R->q[lane] = q;
       R->pair_at[q] = lane;
+      R->tok_at[q] = lane / k;
       if (rank == 0) {
         R->touched[leaders_less] = my;
         R->tcount[leaders_less] = __popc(peers);
@@ -396,14 +411,17 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
   const int item0 = (int)blockIdx.x * ipc;
   const int my_items = max(0, min(ipc, n_items - item0));
   const int total = my_items * wpi;
-  auto issue_item_wave = [&](int v) {                // all of warp 0
-    const int it = v / wpi, wi = v - it * wpi;
-    const int item = item0 + it;
-    const int ti = item / n_jb, jb = item - ti * n_jb;
+  // issue cursor of warp 0 (waves are requested strictly in order): wave, its index inside the
+  // item, the item's slot index and hidden block
+  int iv = 0, iwi = 0, iti = n_items > 0 ? item0 / n_jb : 0, ijb = n_items > 0 ? item0 - iti * n_jb : 0;
+  auto issue_item_wave = [&]() {                     // all of warp 0; requests wave iv and advances
+    const int wi = iwi, ti = iti, jb = ijb;
     const int ph = R->phys[R->touched[ti]];
-    const int w = n_rw + v;
+    const int w = n_rw + iv;
+    ++iv;
+    if (++iwi == wpi) { iwi = 0; if (++ijb == n_jb) { ijb = 0; ++iti; } }
     if (wi < n_in * n_mats) {
-      const int mat = wi / n_in, rp = wi - mat * n_in;
+      const int mat = wi >= n_in ? 1 : 0, rp = wi - mat * n_in;
       issue_rows(w, a.arena_in + (size_t)ph * a.in_stride + (size_t)mat * f * d + (size_t)(jb * kDecJB + rp * RW) * d, RW);
     } else {
       const int ow = wi - n_in * n_mats;
@@ -418,8 +436,8 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
   };
   if (warp == 0) {
     ptx::fence_proxy_async();
-    if (total > 0) issue_item_wave(0);
-    if (total > 1) issue_item_wave(1);
+    if (total > 0) issue_item_wave();
+    if (total > 1) issue_item_wave();
   }
 
   if (blockIdx.x == gridDim.x - 1 && alive) {
@@ -468,28 +486,31 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
 
   float yacc[kDecOutBoxes][4];      // a run's partial output rows: tile warp + 16 i, mma accumulator layout
   int run_jb = -1;                  // first hidden block of the current run, -1 = none open
+  // consumer cursor: item index, wave inside the item, slot index, hidden block
+  int it = 0, wi = 0, ti = n_items > 0 ? item0 / n_jb : 0, jb = n_items > 0 ? item0 - ti * n_jb : 0;
 #pragma unroll 1
-  for (int v = 0; v < total; ++v) {
-    const int it = v / wpi, wi = v - it * wpi;
-    const int item = item0 + it;
-    const int ti = item / n_jb, jb = item - ti * n_jb;
+  for (int v = 0; v < total; ++v, ++wi) {
+    if (wi == wpi) {                            // next item
+      wi = 0;
+      ++it;
+      if (++jb == n_jb) { jb = 0; ++ti; }
+    }
     const int s = R->touched[ti], n_s = R->tcount[ti], q0 = R->toffset[ti];
     const int grp = jb / kDecGroup;
     // runs need the whole output in one wave and all the slot's pairs in one mma
     const bool runs = n_out == 1 && n_s <= 8;
     // the run ends with this item unless the CTA's next item is in the same slot and group
-    const bool run_ends = !runs || it + 1 >= my_items || (item + 1) / n_jb != ti ||
-                          (item + 1 - ti * n_jb) / kDecGroup != grp;
+    const bool run_ends = !runs || it + 1 >= my_items || jb + 1 == n_jb || (jb + 1) / kDecGroup != grp;
     const int w = n_rw + v;
     if (!dec_wait_wave(bars, w, R, a.status, 22)) { alive = false; break; }
     const unsigned char* st = ring + (w & 1) * kDecHalfBytes;
     if (wi < n_in * n_mats) {
       // ---- RW of the item's 32 hidden units: raw products W1 x (and W3 x), eight pairs at a time
-      const int mat = wi / n_in, rp = wi - mat * n_in;
+      const int mat = wi >= n_in ? 1 : 0, rp = wi - mat * n_in;
 #pragma unroll 1
       for (int nb = 0; nb < n_s; nb += 8) {
         const int nn = min(8, n_s - nb);
-        if (tid < 8) R->tok[tid] = R->pair_at[q0 + nb + min(tid, nn - 1)] / k;
+        if (tid < 8) R->tok[tid] = R->tok_at[q0 + nb + min(tid, nn - 1)];
         __syncthreads();
         dec_wave_dots(st, RW, d, xs, R, nn, red, (mat == 0 ? hraw : hraw3) + nb * kDecJB + rp * RW, kDecJB);
       }
@@ -554,7 +575,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
     __syncthreads();                              // the buffer is free; the activations are complete / free
     if (warp == 0 && v + 2 < total) {
       ptx::fence_proxy_async();
-      issue_item_wave(v + 2);
+      issue_item_wave();
     }
     if (!flush) continue;
     run_jb = -1;
