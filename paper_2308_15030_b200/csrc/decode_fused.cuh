@@ -598,39 +598,38 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
     __syncthreads();
     if (R->last) {
       const int d4 = d / 4;
-      // thread (sub, col): sub = tid / 128 adds partial rows 4 sub .. 4 sub + 3 of 128 float4 columns;
-      // the four sub-sums meet in shared memory (the per-warp product area is free here) and are
-      // added in order
-      const int sub = tid >> 7, col = tid & 127;
-      float4* xch = reinterpret_cast<float4*>(red);       // [4][128] float4 = 8 KB
+      // thread (sub, col): sub = tid / 256 adds sets 8 sub .. 8 sub + 7 of 256 float4 columns (all eight
+      // loads in flight together: one round trip per pair row at d_model 1024); the two sub-sums meet
+      // in shared memory (the per-warp product area is free here) and are added in order
+      const int sub = tid >> 8, col = tid & 255;
+      float4* xch = reinterpret_cast<float4*>(red);       // [2][256] float4 = 8 KB
 #pragma unroll 1
-      for (int i0 = 0; i0 < n_s * d4; i0 += 128) {
-        const int i = i0 + col;
-        const int n = i / d4, c4 = i - n * d4;
-        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (i < n_s * d4) {
-          float4 pv[4];
+      for (int n = 0; n < n_s; ++n) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < d4; c0 += 256) {
+          const int c4 = c0 + col;
+          float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (c4 < d4) {
+            float4 pv[8];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {           // all loads first: one round trip
-            const int jj = sub * 4 + j;
-            const int jbf = runs ? max(gs, (c_lo + jj) * ipc) - ti * n_jb : g_first + jj;   // where set jj was filed
-            pv[j] = jj < n_sets ? __ldcg(reinterpret_cast<const float4*>(a.ypart + ((size_t)jbf * P + q0 + n) * d) + c4)
-                                : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int j = 0; j < 8; ++j) {
+              const int jj = sub * 8 + j;
+              const int jbf = runs ? max(gs, (c_lo + jj) * ipc) - ti * n_jb : g_first + jj;   // where set jj was filed
+              pv[j] = jj < n_sets ? __ldcg(reinterpret_cast<const float4*>(a.ypart + ((size_t)jbf * P + q0 + n) * d) + c4)
+                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { sum.x += pv[j].x; sum.y += pv[j].y; sum.z += pv[j].z; sum.w += pv[j].w; }
           }
-#pragma unroll
-          for (int j = 0; j < 4; ++j) { sum.x += pv[j].x; sum.y += pv[j].y; sum.z += pv[j].z; sum.w += pv[j].w; }
-        }
-        xch[sub * 128 + col] = sum;
-        __syncthreads();
-        if (sub == 0 && i < n_s * d4) {
-#pragma unroll
-          for (int q = 1; q < 4; ++q) {
-            const float4 o = xch[q * 128 + col];
+          xch[sub * 256 + col] = sum;
+          __syncthreads();
+          if (sub == 0 && c4 < d4) {
+            const float4 o = xch[256 + col];
             sum.x += o.x; sum.y += o.y; sum.z += o.z; sum.w += o.w;
+            reinterpret_cast<float4*>(a.gpart + ((size_t)grp * P + q0 + n) * d)[c4] = sum;
           }
-          reinterpret_cast<float4*>(a.gpart + ((size_t)grp * P + q0 + n) * d)[c4] = sum;
+          __syncthreads();
         }
-        __syncthreads();
       }
       __syncthreads();
       if (tid == 0) {
@@ -644,8 +643,9 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
       if (R->last) {
         // ---- second step: all groups are in; gate-weighted sum into out (Section 2's combine)
 #pragma unroll 1
-        for (int i = tid; i < T * d4; i += kDecThreads) {
-          const int t = i / d4, c4 = i - t * d4;
+        for (int t = 0; t < T; ++t) {
+#pragma unroll 1
+          for (int c4 = tid; c4 < d4; c4 += kDecThreads) {
           float o[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
           for (int j = 0; j < k; ++j) {
@@ -661,6 +661,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
             o[2] = fmaf(gt, sum.z, o[2]); o[3] = fmaf(gt, sum.w, o[3]);
           }
           store4(a.out + (size_t)t * d + c4 * 4, o);
+          }
         }
         if (tid == 0) a.tickets[K * n_groups] = 0u;
       }
