@@ -119,14 +119,17 @@ __device__ __forceinline__ void gate_epilogue(const RouterArgs& a, const GateSme
       }
     }
   }
-  const int tl = tid % tok, grp = tid / tok;
-  const int parts = (kGateThreads / tok) >> 1;              // threads per token and gate: 1, 2 or 4
+  // tok is a power of two (32, 64, 128): shifts, not integer divisions, which cost dozens of
+  // dependent instructions each in code that runs once
+  const int tok_shift = 31 - __clz(tok);
+  const int tl = tid & (tok - 1), grp = tid >> tok_shift;
+  const int parts = (kGateThreads >> tok_shift) >> 1;       // threads per token and gate: 1, 2 or 4
   const bool masked = grp >= parts;
   const int part = masked ? grp - parts : grp;
   const int token = tok0 + tl;
   const float* row = slog + (size_t)tl * (E + 1);
   const uint32_t* allow = g.s_mask + (masked ? 8 : 0);
-  const int n_chunks = (E + 31) >> 5, cpp = (n_chunks + parts - 1) / parts;
+  const int n_chunks = (E + 31) >> 5, cpp = (n_chunks + parts - 1) >> (parts == 4 ? 2 : parts - 1);
   const int e_lo = min(E, part * cpp * 32), e_hi = min(E, (part + 1) * cpp * 32);
   {
     // The loops below run once per CTA, so they are kept rolled (short bodies that stay in the
