@@ -357,21 +357,33 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int rt, ct;
       decode_tile(t, n_row_tiles, a.n_col_tiles, a.row_group, &rt, &ct);
       const TileDesc td = a.tiles[rt];
+      const int halves = (MT == 2 && td.rows > kTcBM) ? 2 : 1;
+      // where this thread's rows go (and, for the scatter epilogue, their gate values): two dependent
+      // global loads, fetched while the tile's MMAs are still running
+      size_t crow_h[MT];
+      float gate_h[MT];
+#pragma unroll
+      for (int hf = 0; hf < MT; ++hf) {
+        const int rr = r + hf * kTcBM;
+        crow_h[hf] = (size_t)(td.row0 + rr) * a.ldc + (size_t)ct * kOutCols;
+        gate_h[hf] = 1.f;
+        if (EPI == kTcEpiScatterBf16 && hf < halves && rr < td.rows) {
+          const int p = a.row_pair[td.row0 + rr];
+          gate_h[hf] = a.gate[p];
+          crow_h[hf] = (size_t)(p / a.top_k) * a.ldc + (size_t)ct * kOutCols;
+        }
+      }
       ok = bounded_wait(&acc_full[acc], acc_phase, abort_flag, a.status, 4);
       if (!ok) break;
       ptx::tc_fence_after();
-      const int halves = (MT == 2 && td.rows > kTcBM) ? 2 : 1;
-      for (int hf = 0; hf < halves; ++hf) {
+#pragma unroll
+      for (int hf = 0; hf < MT; ++hf) {
+      if (hf < halves) {
       const int rr = r + hf * kTcBM;             // row inside the (up to 256-row) tile
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)((acc * MT + hf) * BN);
       const bool row_ok = rr < td.rows;
-      size_t crow = (size_t)(td.row0 + rr) * a.ldc + (size_t)ct * kOutCols;
-      float gate = 1.f;
-      if (EPI == kTcEpiScatterBf16 && row_ok) {
-        const int p = a.row_pair[td.row0 + rr];
-        gate = a.gate[p];
-        crow = (size_t)(p / a.top_k) * a.ldc + (size_t)ct * kOutCols;
-      }
+      const size_t crow = crow_h[hf];
+      const float gate = gate_h[hf];
 #pragma unroll 1
       for (int c0 = 0; c0 < kOutCols; c0 += 32) {
         uint32_t v[32];
@@ -411,6 +423,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           }
         }
+      }
       }
       }
       ptx::tc_fence_before();

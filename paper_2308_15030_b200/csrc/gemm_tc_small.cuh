@@ -151,10 +151,8 @@ tc_gemm_small_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
       const int ct = t / n_row_tiles, rt = t - ct * n_row_tiles;
       const TileDesc td = a.tiles[rt];
-      ok = bounded_wait(&acc_full[acc], acc_phase, abort_flag, a.status, 34);
-      if (!ok) break;
-      ptx::tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+      // the row's destination and gate value (two dependent global loads) are fetched while the
+      // tile's MMAs are still running
       const bool row_ok = r < td.rows;
       size_t crow = (size_t)(td.row0 + r) * a.ldc + (size_t)ct * BN;
       float gate = 1.f;
@@ -163,6 +161,10 @@ tc_gemm_small_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         gate = a.gate[p];
         crow = (size_t)(p / a.top_k) * a.ldc + (size_t)ct * BN;
       }
+      ok = bounded_wait(&acc_full[acc], acc_phase, abort_flag, a.status, 34);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         uint32_t v[32];
