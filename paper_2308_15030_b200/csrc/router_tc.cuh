@@ -25,8 +25,9 @@ constexpr int kRtSmemBudget = 190 * 1024;
 
 inline int router_tc_epad(int E) { return (E + 15) / 16 * 16; }
 // tokens per CTA: every CTA re-reads the whole router matrix, so tiles shrink only for small
-// batches (measured on B200: 64 is best at T = 2048, 128 at T = 8192)
-inline int router_tc_tok(int T) { return T <= 1024 ? 32 : (T <= 4096 ? 64 : 128); }
+// batches (measured on B200: 32 and 64 tie at T = 2048, 64 beats 128 at T = 8192 by 5 us once
+// the slot scan of the last CTA is cheap; 128-token tiles keep the grid within one wave beyond)
+inline int router_tc_tok(int T) { return T <= 1024 ? 32 : (T <= 8192 ? 64 : 128); }
 // A stage holds tok token rows and Epad router rows of one 64-column k-block.  (The MMA always
 // reads 128 token rows: those beyond tok fall into neighbouring stage memory and only feed
 // accumulator lanes that nobody reads.)
