@@ -545,6 +545,11 @@ def run_decode(args, cfg):
                    "expert_bank": "one bank of %d experts, copied into %d per-layer pinned buffers" % (cfg.E, L),
                    "launch": "eager (host policy in the loop)"},
         "gpu_launches": results[Bmax]["gpu_launches"],
+        # the layer kernels with the scheduler off (graph replay), against the HBM time of the touched slots' weights
+        "roofline": {"bound": "hbm", "unit": "GB/s", "peak": peaks["hbm_gbs"], "peak_source": peaks["source"],
+                     "achieved": peaks["hbm_gbs"] * results[Bmax]["no_swap_graph"]["roofline_frac"],
+                     "frac": results[Bmax]["no_swap_graph"]["roofline_frac"], "traffic": None,
+                     "kernel": "whole layer forward (router .. combine), B = %s, scheduler off" % Bmax},
         "pcie_probe_GBps": pcie_gbs, "per_batch": results,
     }
 
