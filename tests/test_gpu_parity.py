@@ -20,6 +20,7 @@ SMALL = [
     _cfg(T=1000, d=64, f=64, E=256, K=33, k=4, renorm=1, zipf_s=1.1),
     _cfg(T=513, d=256, f=512, E=64, K=64, k=1, zipf_s=1.1),          # K = E: unrestricted layer
     _cfg(T=64, d=128, f=128, E=1, K=1, k=1),                          # dense MLP
+    _cfg(T=12000, dtype=I.F32, d=128, f=128, E=8, K=4),               # fp32 with enough tiles that GEMM-2 is not sliced
 ]
 
 
