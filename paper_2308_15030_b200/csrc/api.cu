@@ -56,6 +56,7 @@ struct swapmoe_layer {
   float* dec_ws;               // its partial-row workspace
   unsigned* dec_tickets;
   CUtensorMap dec_map_wo;      // W_out viewed for the decode kernel's column-slice loads
+  bool fp32_ffma;              // CUDA-core FFMA grouped GEMM instead of the split-TF32 tensor-core one
   int32_t y_copies;            // copies of y in the workspace (slices of a split contraction)
   int32_t sm_count;
   bool use_pdl;                // programmatic dependent launch between the kernels of a forward
@@ -241,10 +242,17 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     g1.N = c.d_ff; g1.Kdim = c.d_model; g1.split_stride = 0;
     const dim3 grid1(c.d_ff / kSimtBN, max_tiles);
     cudaError_t e;
-    if (c.act == SWAPMOE_ACT_SWIGLU)
-      e = launch_kernel(gemm_simt_kernel<DT, DT, DT, kEpiSwiglu>, grid1, dim3(kSimtThreads), 0, st, pdl, g1);
-    else
-      e = launch_kernel(gemm_simt_kernel<DT, DT, DT, kEpiRelu>, grid1, dim3(kSimtThreads), 0, st, pdl, g1);
+    if (L->fp32_ffma) {
+      if (c.act == SWAPMOE_ACT_SWIGLU)
+        e = launch_kernel(gemm_simt_kernel<DT, DT, DT, kEpiSwiglu>, grid1, dim3(kSimtThreads), 0, st, pdl, g1);
+      else
+        e = launch_kernel(gemm_simt_kernel<DT, DT, DT, kEpiRelu>, grid1, dim3(kSimtThreads), 0, st, pdl, g1);
+    } else {
+      if (c.act == SWAPMOE_ACT_SWIGLU)
+        e = launch_kernel(gemm_tf32x3_kernel<DT, DT, DT, kEpiSwiglu>, grid1, dim3(kSimtThreads), 0, st, pdl, g1);
+      else
+        e = launch_kernel(gemm_tf32x3_kernel<DT, DT, DT, kEpiRelu>, grid1, dim3(kSimtThreads), 0, st, pdl, g1);
+    }
     if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
     L->launches++;
     mark(L, 4, st);
@@ -260,7 +268,9 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     y_split = simt_pick_split(tiles_est, L->sm_count, c.d_ff, L->y_copies);
     g2.split_stride = (long long)L->rows_pad_max * c.d_model;
     const dim3 grid2(c.d_model / kSimtBN, max_tiles, y_split);
-    if (launch_kernel(gemm_simt_kernel<DT, DT, float, kEpiNone>, grid2, dim3(kSimtThreads), 0, st, pdl, g2) != cudaSuccess)
+    if ((L->fp32_ffma ? launch_kernel(gemm_simt_kernel<DT, DT, float, kEpiNone>, grid2, dim3(kSimtThreads), 0, st, pdl, g2)
+                      : launch_kernel(gemm_tf32x3_kernel<DT, DT, float, kEpiNone>, grid2, dim3(kSimtThreads), 0, st, pdl,
+                                      g2)) != cudaSuccess)
       return SWAPMOE_ERR_CUDA;
     L->launches++;
   }
@@ -335,6 +345,8 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
     if (L->router_tok != 32 && L->router_tok != 64 && L->router_tok != 128) L->router_tok = 0;
     env = std::getenv("SWAPMOE_SMALL_PATH");            // SWAPMOE_SMALL_PATH=0: general GEMM kernels for small batches too
     L->small_path = !(env && env[0] == '0');
+    env = std::getenv("SWAPMOE_FP32_FFMA");             // SWAPMOE_FP32_FFMA=1: FFMA form of the non-tcgen05 grouped GEMM
+    L->fp32_ffma = env && env[0] == '1';
     env = std::getenv("SWAPMOE_PREFETCH");              // SWAPMOE_PREFETCH=0 disables the L2 weight prefetch
     L->prefetch = !(env && env[0] == '0');
     // The prefetch must drain while the router runs (about 15 us on 16-64 SMs): what HBM delivers
