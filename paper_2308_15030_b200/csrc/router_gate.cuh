@@ -67,32 +67,33 @@ __global__ void __launch_bounds__(kGateThreads) router_gate_kernel(const RouterA
     for (int t = 0; t < 4; ++t)
 #pragma unroll
       for (int i = 0; i < EI; ++i) acc[t][i] = 0.f;
-    float xv[4] = {0.f, 0.f, 0.f, 0.f};
-    float wv[EI][4];
-    auto load_chunk = [&](int c0) {
-      if (ltok < a.T) load4(x + (size_t)ltok * a.d + c0 + lcol, xv);
+    // two register sets: the global loads of chunk c + 2 are issued while chunk c is multiplied, so a
+    // load has two chunk periods to land (one period is shorter than the memory latency)
+    float xv[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    float wv[2][EI][4];
+    auto load_chunk = [&](int c0, int set) {
+      if (ltok < a.T) load4(x + (size_t)ltok * a.d + c0 + lcol, xv[set]);
 #pragma unroll
       for (int i = 0; i < EI; ++i) {
         const int v = tid + kGateThreads * i;
-        if (v < n_wv) load4(Wr + (size_t)(v >> 3) * a.d + c0 + (v & 7) * 4, wv[i]);
+        if (v < n_wv) load4(Wr + (size_t)(v >> 3) * a.d + c0 + (v & 7) * 4, wv[set][i]);
       }
     };
-    load_chunk(0);
-    for (int c0 = 0; c0 < a.d; c0 += kRouterDK) {
+    auto stage_and_multiply = [&](int set, int next_c0) {
       __syncthreads();                       // the previous chunk's multiply-adds are done
-      sumsq += xv[0] * xv[0] + xv[1] * xv[1] + xv[2] * xv[2] + xv[3] * xv[3];
+      sumsq += xv[set][0] * xv[set][0] + xv[set][1] * xv[set][1] + xv[set][2] * xv[set][2] + xv[set][3] * xv[set][3];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) xs[lrow * (kRouterDK + 1) + lcol + q] = xv[q];
+      for (int q = 0; q < 4; ++q) xs[lrow * (kRouterDK + 1) + lcol + q] = xv[set][q];
 #pragma unroll
       for (int i = 0; i < EI; ++i) {
         const int v = tid + kGateThreads * i;
         if (v < n_wv) {
 #pragma unroll
-          for (int q = 0; q < 4; ++q) ws[(v >> 3) * (kRouterDK + 1) + (v & 7) * 4 + q] = wv[i][q];
+          for (int q = 0; q < 4; ++q) ws[(v >> 3) * (kRouterDK + 1) + (v & 7) * 4 + q] = wv[set][i][q];
         }
       }
       __syncthreads();
-      if (c0 + kRouterDK < a.d) load_chunk(c0 + kRouterDK);
+      if (next_c0 < a.d) load_chunk(next_c0, set);
 #pragma unroll 8
       for (int kk = 0; kk < kRouterDK; ++kk) {
         float xr[4];
@@ -106,6 +107,12 @@ __global__ void __launch_bounds__(kGateThreads) router_gate_kernel(const RouterA
           for (int t = 0; t < 4; ++t) acc[t][i] = fmaf(xr[t], w, acc[t][i]);
         }
       }
+    };
+    load_chunk(0, 0);
+    if (kRouterDK < a.d) load_chunk(kRouterDK, 1);
+    for (int c0 = 0; c0 < a.d; c0 += 2 * kRouterDK) {
+      stage_and_multiply(0, c0 + 2 * kRouterDK);
+      if (c0 + kRouterDK < a.d) stage_and_multiply(1, c0 + 3 * kRouterDK);
     }
 #pragma unroll
     for (int t = 0; t < 4; ++t)
