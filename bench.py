@@ -312,8 +312,15 @@ def run_cuda(args, cfg):
     tc_peak = peaks["bf16_tflops_sustained"] if tc_kind == "sustained" else peaks["bf16_tflops"]
     t_hbm = g_bytes / (peaks["hbm_gbs"] * 1e9)
     t_tc = g_flops / (tc_peak * 1e12) if cfg.dtype == I.BF16 else 0.0
-    if cfg.dtype != I.BF16:
+    ffma = os.environ.get("SWAPMOE_FP32_FFMA") == "1"
+    # fp32 layers: the grouped GEMM runs on the tensor cores as three TF32 products per fp32 product;
+    # its peak is the measured bf16 figure x the nominal TF32 : bf16 ratio (1.1 : 2.25 PFLOP/s) / 3.
+    # (With SWAPMOE_FP32_FFMA=1 it is an FFMA kernel: 148 SMs x 128 lanes x 2 x 1.965 GHz = 74.4 TFLOP/s.)
+    tf32x3_peak = peaks["bf16_tflops"] * (1.1 / 2.25) / 3.0
+    if cfg.dtype != I.BF16 and ffma:
         bound, peak, ach, unit = "alu", 74.4, g_flops / 2 / (g_ms * 1e-3) / 1e12, "TFLOP/s"
+    elif cfg.dtype != I.BF16:
+        bound, peak, ach, unit = "tensor", tf32x3_peak, g_flops / 2 / (g_ms * 1e-3) / 1e12, "TFLOP/s"
     elif t_hbm >= t_tc:
         bound, peak, ach, unit = "hbm", peaks["hbm_gbs"], g_bytes / 2 / (g_ms * 1e-3) / 1e9, "GB/s"
     else:
@@ -322,7 +329,7 @@ def run_cuda(args, cfg):
     layer_flops = 2.0 * cfg.T * cfg.d * cfg.E + g_flops
     t_roof = max(layer_bytes / (peaks["hbm_gbs"] * 1e9),
                  layer_flops / (tc_peak * 1e12) if cfg.dtype == I.BF16
-                 else layer_flops / 74.4e12)
+                 else layer_flops / ((74.4 if ffma else tf32x3_peak) * 1e12))
     res = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
@@ -344,11 +351,14 @@ def run_cuda(args, cfg):
         "roofline": {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
                      "traffic": NCU_TRAFFIC_PER_LAUNCH.get(cfg.name), "peak_source": peaks["source"],
                      "kernel": "tc_gemm_kernel (grouped FFN GEMM, 2 launches per step: GEMM-1+act, GEMM-2)"
-                               if cfg.dtype == I.BF16 else "gemm_simt_kernel (2 launches per step)",
+                               if cfg.dtype == I.BF16 else ("gemm_simt_kernel (FFMA, 2 launches per step)" if ffma else
+                                                            "gemm_tf32x3_kernel (split-TF32 mma, 2 launches per step)"),
                      "algorithmic_bytes_per_launch": g_bytes / 2, "flops_per_launch": g_flops / 2,
                      "avg_launch_ms": g_ms,
                      "tensor_tflops": g_flops / 2 / (g_ms * 1e-3) / 1e12,
-                     "tensor_peak_kind": tc_kind if bound == "tensor" else None,
+                     "tensor_peak_kind": (tc_kind if cfg.dtype == I.BF16 else "bf16 burst x 1.1/2.25 / 3 (TF32 x3)")
+                                         if bound == "tensor" else None,
+                     "frac_of_fp32_ffma_peak": (ach / 74.4) if cfg.dtype != I.BF16 else None,
                      "frac_of_burst_tensor_peak": (ach / peaks["bf16_tflops"]) if bound == "tensor" else None},
         "layer_roofline": {"t_roof_us": t_roof * 1e6, "frac": t_roof * 1e3 / ms_step,
                            "algorithmic_bytes": layer_bytes, "flops": layer_flops},
