@@ -4,33 +4,38 @@
 #pragma once
 #include "common.cuh"
 #include "gate_epilogue.cuh"
+#include "gemm_simt.cuh"
 #include "permute.cuh"
 #include "router_args.cuh"
 
 namespace swapmoe {
 
 constexpr int kRouterDK = 32;  // contraction chunk staged in shared memory
+constexpr int kRouterLD = kRouterDK + 4;   // row pitch of the staged chunks (words): conflict-free mma fragment loads
 
 inline size_t router_stage_floats(int E) {
-  // token chunk [kTokTile][DK+1], router chunk [E][DK+1], logits [kTokTile][E+1] + 8 of slack
-  return (size_t)kTokTile * (kRouterDK + 1) + (size_t)E * (kRouterDK + 1) + (size_t)kTokTile * (E + 1) + 8;
+  // token chunk [kTokTile][LD], router chunk [E rounded up to 8][LD], logits [kTokTile][E+1] + 8 of slack
+  return (size_t)kTokTile * kRouterLD + (size_t)((E + 7) / 8 * 8) * kRouterLD + (size_t)kTokTile * (E + 1) + 8;
 }
 inline size_t router_smem_bytes(int E) {
   return ((router_stage_floats(E) * sizeof(float) + 15) & ~(size_t)15) + gate_smem_bytes();
 }
 
-// One CTA = kTokTile tokens.  In the product warp w owns tokens 4w..4w+3 and lane l owns
-// experts l + 32 i, i < EI (EI, the number of 32-expert groups, is a template parameter so that
-// a layer with few experts carries no dead multiply-adds); the next chunk's global loads are
-// issued before the current chunk's multiply-adds so their latency hides behind the arithmetic.
+// One CTA = kTokTile tokens.  The product runs as split-TF32 mma (three TF32 products per fp32
+// product, see gemm_tf32x3_kernel): warp w owns the 16 tokens of half w & 1 and the 8-expert
+// tiles (w >> 1), (w >> 1) + 4, ... (at most EI of them; EI, the number of 32-expert groups, is a
+// template parameter that sizes the accumulators).  The global loads of chunk c + 2 are issued
+// while chunk c is multiplied.
 template <typename T, int EI>
 __global__ void __launch_bounds__(kGateThreads) router_gate_kernel(const RouterArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int E = a.E;
-  float* xs = reinterpret_cast<float*>(smem_raw);              // [kTokTile][DK+1]
-  float* ws = xs + kTokTile * (kRouterDK + 1);                 // [E][DK+1]
-  float* slog = ws + E * (kRouterDK + 1);                      // [kTokTile][E+1]
-  const int stage_bytes = (int)(((size_t)(kTokTile * (kRouterDK + 1) + E * (kRouterDK + 1) +
+  const int E8 = (E + 7) & ~7;
+  float* xs = reinterpret_cast<float*>(smem_raw);              // [kTokTile][LD]
+  float* ws = xs + kTokTile * kRouterLD;                       // [E8][LD] (rows beyond E are never written: their
+                                                               //  products land in columns nobody reads)
+  float* slog = ws + E8 * kRouterLD;                           // [kTokTile][E+1]
+  const int stage_bytes = (int)(((size_t)(kTokTile * kRouterLD + E8 * kRouterLD +
                                           kTokTile * (E + 1) + 8) * sizeof(float) + 15) & ~(size_t)15);
   const GateSmem g = gate_smem_carve(smem_raw + stage_bytes);
 
@@ -62,11 +67,13 @@ __global__ void __launch_bounds__(kGateThreads) router_gate_kernel(const RouterA
       slog[r * (E + 1) + e] = (tok0 + r < a.T) ? a.ext_logits[(size_t)(tok0 + r) * E + e] : 0.f;
     }
   } else {
-    float acc[4][EI];
+    const int g = lane >> 2, t4 = lane & 3;
+    const int m0 = (warp & 1) * 16, ng = warp >> 1, NT = E8 >> 3;
+    float acc[EI][4];
 #pragma unroll
-    for (int t = 0; t < 4; ++t)
+    for (int j = 0; j < EI; ++j)
 #pragma unroll
-      for (int i = 0; i < EI; ++i) acc[t][i] = 0.f;
+      for (int q = 0; q < 4; ++q) acc[j][q] = 0.f;
     // two register sets: the global loads of chunk c + 2 are issued while chunk c is multiplied, so a
     // load has two chunk periods to land (one period is shorter than the memory latency)
     float xv[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -80,31 +87,36 @@ __global__ void __launch_bounds__(kGateThreads) router_gate_kernel(const RouterA
       }
     };
     auto stage_and_multiply = [&](int set, int next_c0) {
-      __syncthreads();                       // the previous chunk's multiply-adds are done
+      __syncthreads();                       // the previous chunk's products are done
       sumsq += xv[set][0] * xv[set][0] + xv[set][1] * xv[set][1] + xv[set][2] * xv[set][2] + xv[set][3] * xv[set][3];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) xs[lrow * (kRouterDK + 1) + lcol + q] = xv[set][q];
+      store4(xs + lrow * kRouterLD + lcol, xv[set]);
 #pragma unroll
       for (int i = 0; i < EI; ++i) {
         const int v = tid + kGateThreads * i;
-        if (v < n_wv) {
-#pragma unroll
-          for (int q = 0; q < 4; ++q) ws[(v >> 3) * (kRouterDK + 1) + (v & 7) * 4 + q] = wv[set][i][q];
-        }
+        if (v < n_wv) store4(ws + (v >> 3) * kRouterLD + (v & 7) * 4, wv[set][i]);
       }
       __syncthreads();
       if (next_c0 < a.d) load_chunk(next_c0, set);
-#pragma unroll 8
-      for (int kk = 0; kk < kRouterDK; ++kk) {
-        float xr[4];
+      const float* As = xs + (m0 + g) * kRouterLD + t4;
 #pragma unroll
-        for (int t = 0; t < 4; ++t) xr[t] = xs[(warp * 4 + t) * (kRouterDK + 1) + kk];
+      for (int k0 = 0; k0 < kRouterDK; k0 += 8) {
+        uint32_t ah[4], al[4];
+        split_tf32(As[k0], ah[0], al[0]);
+        split_tf32(As[8 * kRouterLD + k0], ah[1], al[1]);
+        split_tf32(As[k0 + 4], ah[2], al[2]);
+        split_tf32(As[8 * kRouterLD + k0 + 4], ah[3], al[3]);
 #pragma unroll
-        for (int i = 0; i < EI; ++i) {
-          const int e = lane + 32 * i;
-          const float w = (e < E) ? ws[e * (kRouterDK + 1) + kk] : 0.f;
-#pragma unroll
-          for (int t = 0; t < 4; ++t) acc[t][i] = fmaf(xr[t], w, acc[t][i]);
+        for (int j = 0; j < EI; ++j) {
+          const int nt = ng + 4 * j;
+          if (nt < NT) {
+            const float* Bs = ws + (nt * 8 + g) * kRouterLD + t4 + k0;
+            uint32_t bh[2], bl[2];
+            split_tf32(Bs[0], bh[0], bl[0]);
+            split_tf32(Bs[4], bh[1], bl[1]);
+            mma_tf32_16x8x8(acc[j], al, bh);
+            mma_tf32_16x8x8(acc[j], ah, bl);
+            mma_tf32_16x8x8(acc[j], ah, bh);
+          }
         }
       }
     };
@@ -114,13 +126,18 @@ __global__ void __launch_bounds__(kGateThreads) router_gate_kernel(const RouterA
       stage_and_multiply(0, c0 + 2 * kRouterDK);
       if (c0 + kRouterDK < a.d) stage_and_multiply(1, c0 + 3 * kRouterDK);
     }
+    // accumulator layout: [0], [1] -> token m0 + g, experts 8 nt + 2 t4, + 1; [2], [3] -> token m0 + g + 8
 #pragma unroll
-    for (int t = 0; t < 4; ++t)
+    for (int j = 0; j < EI; ++j) {
+      const int nt = ng + 4 * j;
+      if (nt < NT) {
 #pragma unroll
-      for (int i = 0; i < EI; ++i) {
-        const int e = lane + 32 * i;
-        if (e < E) slog[(warp * 4 + t) * (E + 1) + e] = acc[t][i];
+        for (int q = 0; q < 4; ++q) {
+          const int e = nt * 8 + 2 * t4 + (q & 1);
+          if (e < E) slog[(m0 + g + (q >> 1) * 8) * (E + 1) + e] = acc[j][q];
+        }
       }
+    }
   }
   // ||x||^2 of a row: 8 consecutive lanes hold its partial sums
   sumsq += __shfl_xor_sync(0xffffffffu, sumsq, 1);
