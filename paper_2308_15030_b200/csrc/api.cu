@@ -5,6 +5,7 @@
 
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -19,6 +20,7 @@
 #include "permute.cuh"
 #include "router_gate.cuh"
 #include "router_tc.cuh"
+#include "router_small.cuh"
 
 using namespace swapmoe;
 
@@ -51,6 +53,7 @@ struct swapmoe_layer {
   int64_t launches;
   int32_t gemm_path;
   int32_t rows_pad_max;
+  bool small_router;           // eight-token mma router CTAs for batches of up to 64 tokens (bf16)
   bool decode_path;            // one-launch forward for a handful of tokens (bf16)
   int32_t decode_max_pairs;    // ... used up to this many (token, expert) pairs (the kernel takes 8 tokens)
   float* dec_ws;               // its partial-row workspace
@@ -128,8 +131,11 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     return check_launch();
   }
   const bool tc_router = L->tc.router_ok && ext_logits == nullptr;
+  // up to 64 tokens: eight-token CTAs of the mma router (the tcgen05 router's fixed cost dominates there)
+  const bool small_router = tc_router && L->small_router && T <= kRsMaxTokens;
   int tok_tile = tc_router ? router_tc_tok(T) : kTokTile;
   if (tc_router && L->router_tok) tok_tile = L->router_tok;
+  if (small_router) tok_tile = kRsTok;
   const int n_cta = (T + tok_tile - 1) / tok_tile;
   const int n_pairs = T * c.top_k;
   const bool use_tc = tc_selected(L->gemm_path, c, T);
@@ -180,7 +186,11 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     if (pf_ctas > 64) pf_ctas = 64;
   }
   mark(L, 0, st);
-  if (tc_router) {
+  if (small_router) {
+    if (launch_kernel(router_small_kernel, dim3(n_cta), dim3(kDecThreads), router_small_smem_bytes(c.d_model), st, pdl,
+                      ra, L->status) != cudaSuccess)
+      return SWAPMOE_ERR_CUDA;
+  } else if (tc_router) {
     if (x != L->map_x_ptr || T != L->map_x_T) {   // the token map is re-encoded only when x or T changes
       if (!tc_encode_2d(L->tc.encode, &L->map_x, x, (uint64_t)T, (uint64_t)c.d_model, (uint32_t)tok_tile))
         return SWAPMOE_ERR_CUDA;
@@ -361,7 +371,12 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   L->elem = c.dtype == SWAPMOE_BF16 ? 2 : 4;
 
   const size_t T = (size_t)c.max_tokens, P = T * c.top_k;
-  const size_t n_cta = (T + kTokTile - 1) / kTokTile;
+  // router CTAs: 32-token tiles at least; batches of up to 64 tokens may use eight-token tiles
+  size_t n_cta = (T + kTokTile - 1) / kTokTile;
+  {
+    const size_t small = std::min<size_t>((T + kRsTok - 1) / kRsTok, kRsMaxTokens / kRsTok);
+    if (small > n_cta) n_cta = small;
+  }
   const size_t rows_pad = align_up(P + (size_t)c.K * kSegAlign, kSegAlign);
   const size_t max_tiles = (P + kSimtBM - 1) / kSimtBM + c.K;
   L->rows_pad_max = (int32_t)rows_pad;
@@ -447,6 +462,14 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   ok = ok && cuda_ok(router_gate_set_smem_limit<float>()) && cuda_ok(router_gate_set_smem_limit<bf16>());
   ok = ok && tc_init(L->tc, c, L->xp, L->h, L->y, L->rows_pad_max) == SWAPMOE_OK;
   if (L->tc.encode == nullptr) L->decode_path = false;     // its W_out loads need a tensor map
+  {
+    const char* env = std::getenv("SWAPMOE_SMALL_ROUTER");   // SWAPMOE_SMALL_ROUTER=0: tcgen05 router for small batches too
+    L->small_router = c.dtype == SWAPMOE_BF16 && !(env && env[0] == '0') &&
+                      router_small_smem_bytes(c.d_model) <= (size_t)(226 << 10);
+    if (L->small_router)
+      ok = ok && cuda_ok(cudaFuncSetAttribute(router_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)router_small_smem_bytes(c.d_model)));
+  }
   if (ok && L->tc.enabled) ok = tc_small_set_attrs();
   ok = ok && cuda_ok(cudaStreamCreateWithFlags(&L->s_in, cudaStreamNonBlocking));
   ok = ok && cuda_ok(cudaStreamCreateWithFlags(&L->s_out, cudaStreamNonBlocking));
