@@ -54,6 +54,7 @@ struct swapmoe_layer {
   int32_t gemm_path;
   int32_t rows_pad_max;
   bool small_router;           // eight-token mma router CTAs for batches of up to 64 tokens (bf16)
+  int32_t small_router_max_t;  // ... and sixteen-token CTAs up to this many tokens (0: never)
   bool decode_path;            // one-launch forward for a handful of tokens (bf16)
   int32_t decode_max_pairs;    // ... used up to this many (token, expert) pairs (the kernel takes 8 tokens)
   float* dec_ws;               // its partial-row workspace
@@ -132,10 +133,12 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   }
   const bool tc_router = L->tc.router_ok && ext_logits == nullptr;
   // up to 64 tokens: eight-token CTAs of the mma router (the tcgen05 router's fixed cost dominates there)
-  const bool small_router = tc_router && L->small_router && T <= kRsMaxTokens;
+  // (and sixteen-token CTAs while they still fit one wave of CTAs)
+  const int rs_nt = !(tc_router && L->small_router) ? 0 : (T <= kRsMaxTokens ? 1 : (T <= L->small_router_max_t ? 2 : 0));
+  const bool small_router = rs_nt > 0;
   int tok_tile = tc_router ? router_tc_tok(T) : kTokTile;
   if (tc_router && L->router_tok) tok_tile = L->router_tok;
-  if (small_router) tok_tile = kRsTok;
+  if (small_router) tok_tile = kRsTok * rs_nt;
   const int n_cta = (T + tok_tile - 1) / tok_tile;
   const int n_pairs = T * c.top_k;
   const bool use_tc = tc_selected(L->gemm_path, c, T);
@@ -187,8 +190,10 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   }
   mark(L, 0, st);
   if (small_router) {
-    if (launch_kernel(router_small_kernel, dim3(n_cta), dim3(kDecThreads), router_small_smem_bytes(c.d_model), st, pdl,
-                      ra, L->status) != cudaSuccess)
+    if ((rs_nt == 1 ? launch_kernel(router_small_kernel<1>, dim3(n_cta + pf_ctas), dim3(kDecThreads),
+                                    router_small_smem_bytes(c.d_model, 1), st, pdl, ra, L->status)
+                    : launch_kernel(router_small_kernel<2>, dim3(n_cta + pf_ctas), dim3(kDecThreads),
+                                    router_small_smem_bytes(c.d_model, 2), st, pdl, ra, L->status)) != cudaSuccess)
       return SWAPMOE_ERR_CUDA;
   } else if (tc_router) {
     if (x != L->map_x_ptr || T != L->map_x_T) {   // the token map is re-encoded only when x or T changes
@@ -376,6 +381,8 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   {
     const size_t small = std::min<size_t>((T + kRsTok - 1) / kRsTok, kRsMaxTokens / kRsTok);
     if (small > n_cta) n_cta = small;
+    const size_t mid = std::min<size_t>((T + 2 * kRsTok - 1) / (2 * kRsTok), 256);   // sixteen-token CTAs
+    if (mid > n_cta) n_cta = mid;
   }
   const size_t rows_pad = align_up(P + (size_t)c.K * kSegAlign, kSegAlign);
   const size_t max_tiles = (P + kSimtBM - 1) / kSimtBM + c.K;
@@ -465,10 +472,19 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   {
     const char* env = std::getenv("SWAPMOE_SMALL_ROUTER");   // SWAPMOE_SMALL_ROUTER=0: tcgen05 router for small batches too
     L->small_router = c.dtype == SWAPMOE_BF16 && !(env && env[0] == '0') &&
-                      router_small_smem_bytes(c.d_model) <= (size_t)(226 << 10);
+                      router_small_smem_bytes(c.d_model, 1) <= (size_t)(226 << 10);
     if (L->small_router)
-      ok = ok && cuda_ok(cudaFuncSetAttribute(router_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)router_small_smem_bytes(c.d_model)));
+      ok = ok && cuda_ok(cudaFuncSetAttribute(router_small_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)router_small_smem_bytes(c.d_model, 1)));
+    // sixteen-token CTAs: while the grid stays within one wave of CTAs and the shared memory fits
+    L->small_router_max_t = 0;
+    if (L->small_router && router_small_smem_bytes(c.d_model, 2) <= (size_t)(226 << 10)) {
+      L->small_router_max_t = 2 * kRsTok * L->sm_count;
+      const char* envm = std::getenv("SWAPMOE_SMALL_ROUTER_MAX_T");
+      if (envm) L->small_router_max_t = std::min(std::atoi(envm), 2 * kRsTok * 256);
+      ok = ok && cuda_ok(cudaFuncSetAttribute(router_small_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)router_small_smem_bytes(c.d_model, 2)));
+    }
   }
   if (ok && L->tc.enabled) ok = tc_small_set_attrs();
   ok = ok && cuda_ok(cudaStreamCreateWithFlags(&L->s_in, cudaStreamNonBlocking));

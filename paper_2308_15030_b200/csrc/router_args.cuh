@@ -32,4 +32,25 @@ struct RouterArgs {
   const int32_t* pf_phys;       // [K] arena entry of each logical slot
 };
 
+// Role of the blocks beyond the router's token tiles: pull the resident experts' matrices towards
+// L2 (GEMM-1's first, in slot order) while the router leaves HBM idle.
+__device__ __forceinline__ void router_prefetch_role(const RouterArgs& a, int n_router_ctas) {
+  constexpr long long kChunk = 16384;
+  // chunks are dealt round-robin over the prefetch blocks: an SM sustains only about 200 GB/s of
+  // prefetch requests, so the budget must be spread over enough of them to drain while the router runs
+  const long long n_blk = (long long)gridDim.x - n_router_ctas;
+  const long long n_pf = n_blk * blockDim.x;
+  const long long me = (long long)threadIdx.x * n_blk + (blockIdx.x - n_router_ctas);
+#pragma unroll 1
+  for (int m = 0; m < 2; ++m) {
+    const long long per_slot = a.pf_slot_bytes[m] / kChunk;
+    const long long n_chunks = a.pf_total_bytes[m] / kChunk;
+    for (long long c = me; c < n_chunks; c += n_pf) {
+      const long long s = c / per_slot, o = c - s * per_slot;
+      const char* src = a.pf_base[m] + (long long)a.pf_phys[s] * a.pf_slot_bytes[m] + o * kChunk;
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"((unsigned)kChunk) : "memory");
+    }
+  }
+}
+
 }  // namespace swapmoe

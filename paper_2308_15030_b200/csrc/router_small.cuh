@@ -2,7 +2,7 @@
 // SwapMoE Section 2 (G(x)), Fig. 4 (Masked Gating), Eq. 1 (importance terms).
 //
 // The tcgen05 router spends 20 us of fixed cost (TMEM hand-offs, a gate written for 32-128 token
-// tiles) on a handful of tokens.  Here a CTA takes EIGHT tokens and routes them the way the
+// tiles) on a handful of tokens.  Here a CTA takes eight or sixteen tokens and routes them the way the
 // one-launch decode kernel does: the router matrix arrives in two TMA wave buffers (requested
 // before the wait on the predecessor), the product is warp-level mma with the eight tokens as the
 // eight mma columns and the contraction split over 16 warps, and a warp computes a token's gate.
@@ -16,46 +16,114 @@
 
 namespace swapmoe {
 
-constexpr int kRsTok = kDecMaxTokens;     // tokens per CTA
-constexpr int kRsMaxTokens = 64;          // batches up to this size take this router
+constexpr int kRsTok = kDecMaxTokens;     // tokens per mma column tile
+constexpr int kRsMaxNT = 2;               // column tiles (of eight tokens) per CTA: 1 or 2
+constexpr int kRsMaxPairs = kRsTok * kRsMaxNT * kMaxTopK;
+constexpr int kRsMaxTokens = 64;          // batches up to this size use eight-token CTAs
+
+// Routing state of one CTA's tokens (shared memory).
+struct RsRoute {
+  int ue[kRsMaxPairs], sl[kRsMaxPairs];   // off-the-shelf expert and slot per pair p = t*k + j
+  float pt[kRsMaxPairs], pm[kRsMaxPairs]; // Eq. (1) term per pair: off-the-shelf routing, masked routing
+  float xn[kRsTok * kRsMaxNT];
+};
 
 struct RsSmem {
   int xs, slog, red, route, bars, pairs, total;
 };
-__host__ __device__ inline RsSmem router_small_layout(int d) {
+__host__ __device__ inline RsSmem router_small_layout(int d, int nt) {
   RsSmem m;
   int o = 2 * kDecHalfBytes;
-  m.xs = o;    o += kRsTok * (d * 2 + kDecRowPad);
-  m.slog = o;  o += kRsTok * (kMaxE + 1) * 4;
+  m.xs = o;    o += kRsTok * nt * (d * 2 + kDecRowPad);
+  m.slog = o;  o += kRsTok * nt * (kMaxE + 1) * 4;
   o = (o + 15) & ~15;
-  m.red = o;   o += kDecWarps * 32 * 8 * 4;
+  m.red = o;   o += kDecWarps * 32 * 8 * 4 * nt;
   m.route = o; o += (int)sizeof(DecRoute);
   o = (o + 15) & ~15;
   m.bars = o;  o += 16;
-  m.pairs = o; o += kDecMaxPairs * 2 * 4;   // Eq. (1) terms per pair: unmasked, masked
+  m.pairs = o; o += (int)sizeof(RsRoute);
   m.total = o;
   return m;
 }
-inline size_t router_small_smem_bytes(int d) { return (size_t)router_small_layout(d).total + 1024; }
+inline size_t router_small_smem_bytes(int d, int nt) { return (size_t)router_small_layout(d, nt).total + 1024; }
 
+// dst[(8 j + n) * dst_stride + r] = <row r of the wave buffer, token 8 j + n> for r < rows <= 32, j < NT,
+// 8 j + n < n_tok: dec_wave_dots for NT column tiles at once (the weight fragments are loaded once).
+template <int NT>
+__device__ __forceinline__ void rs_wave_dots(const unsigned char* st, int rows, int d, const unsigned char* xs,
+                                             int n_tok, float* red, float* dst, int dst_stride) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int pitch = d * 2 + kDecRowPad;
+  float acc[2][NT][4];
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int j = 0; j < NT; ++j)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) acc[i][j][q] = 0.f;
+  const unsigned char* arow = st + g * pitch + t * 4;
+#pragma unroll 2
+  for (int ks = warp; ks < d / 16; ks += kDecWarps) {
+    const int kb = ks * 32;
+    uint32_t b0[NT], b1[NT];
+#pragma unroll
+    for (int j = 0; j < NT; ++j) {
+      const unsigned char* xrow = xs + min(8 * j + g, n_tok - 1) * pitch + t * 4 + kb;
+      b0[j] = lds32(xrow);
+      b1[j] = lds32(xrow + 16);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const unsigned char* ap = arow + i * 16 * pitch + kb;
+      const uint32_t a0 = lds32(ap), a1 = lds32(ap + 8 * pitch), a2 = lds32(ap + 16), a3 = lds32(ap + 8 * pitch + 16);
+#pragma unroll
+      for (int j = 0; j < NT; ++j) mma_bf16_16x8x16(acc[i][j], a0, a1, a2, a3, b0[j], b1[j]);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int j = 0; j < NT; ++j) {
+      float* rp = red + ((warp * NT + j) * 32 + i * 16 + g) * 8 + 2 * t;
+      *reinterpret_cast<float2*>(rp) = make_float2(acc[i][j][0], acc[i][j][1]);
+      *reinterpret_cast<float2*>(rp + 8 * 8) = make_float2(acc[i][j][2], acc[i][j][3]);
+    }
+  __syncthreads();
+  if (tid < 32 * 8 * NT) {
+    const int j = tid >> 8, r = (tid >> 3) & 31, n = tid & 7;
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) s += red[((w * NT + j) * 32 + r) * 8 + n];
+    if (r < rows && 8 * j + n < n_tok) dst[(8 * j + n) * dst_stride + r] = s;
+  }
+  __syncthreads();
+}
+
+template <int NT>
 __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const RouterArgs a, int32_t* status) {
+  constexpr int TOK = kRsTok * NT;                          // tokens per CTA
+  if ((int)blockIdx.x >= a.scan.n_cta) {                    // blocks beyond the token tiles prefetch weights
+    pdl_wait();
+    pdl_trigger();
+    router_prefetch_role(a, a.scan.n_cta);
+    return;
+  }
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
   const int d = a.d, E = a.E, k = a.k, K = a.K;
   const int chunks = d / 8, pitch = d * 2 + kDecRowPad;
-  const RsSmem lay = router_small_layout(d);
+  const RsSmem lay = router_small_layout(d, NT);
   unsigned char* ring = smem;
   unsigned char* xs = smem + lay.xs;
   float* slog = reinterpret_cast<float*>(smem + lay.slog);
   float* red = reinterpret_cast<float*>(smem + lay.red);
   DecRoute* R = reinterpret_cast<DecRoute*>(smem + lay.route);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + lay.bars);
-  float* pt = reinterpret_cast<float*>(smem + lay.pairs);   // [pairs] Eq. (1) term, off-the-shelf routing
-  float* pm = pt + kDecMaxPairs;                            // [pairs] ... masked routing
+  RsRoute* Q = reinterpret_cast<RsRoute*>(smem + lay.pairs);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int tok0 = blockIdx.x * kRsTok;
-  const int T = min(kRsTok, a.T - tok0);                    // tokens of this CTA
+  const int tok0 = blockIdx.x * TOK;
+  const int T = min(TOK, a.T - tok0);                       // tokens of this CTA
   const int P = T * k;
   const bf16* x = static_cast<const bf16*>(a.x) + (size_t)tok0 * d;
   const bf16* Wr = static_cast<const bf16*>(a.Wr);
@@ -84,22 +152,23 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
   pdl_wait();
   pdl_trigger();
   {
-    const int t = warp & (kRsTok - 1);                      // token t is copied by warps t and t + 8
+    // token t is copied by the kDecWarps / TOK warps t, t + TOK, ...; four independent loads per lane and round
+    constexpr int kWpt = kDecWarps / TOK;                   // warps per token: 2 or 1
+    const int t = warp & (TOK - 1);
     if (t < T) {
 #pragma unroll 1
-      for (int c0 = (warp >> 3) * 32 + lane; c0 < chunks; c0 += 256) {
+      for (int c0 = (warp / TOK) * 32 + lane; c0 < chunks; c0 += 128 * kWpt) {
         uint4 v[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u)
-          if (c0 + 64 * u < chunks) v[u] = reinterpret_cast<const uint4*>(x)[t * chunks + c0 + 64 * u];
+          if (c0 + 32 * kWpt * u < chunks) v[u] = reinterpret_cast<const uint4*>(x)[t * chunks + c0 + 32 * kWpt * u];
 #pragma unroll
         for (int u = 0; u < 4; ++u)
-          if (c0 + 64 * u < chunks) *reinterpret_cast<uint4*>(xs + t * pitch + (c0 + 64 * u) * 16) = v[u];
+          if (c0 + 32 * kWpt * u < chunks) *reinterpret_cast<uint4*>(xs + t * pitch + (c0 + 32 * kWpt * u) * 16) = v[u];
       }
     }
   }
   if (tid < kMaxE) R->e2s[tid] = tid < E ? a.e2s[tid] : -1;
-  if (tid < kRsTok) R->tok[tid] = min(tid, T - 1);
   __syncthreads();
   if (warp < T) {
     float ss = 0.f;
@@ -115,22 +184,24 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
       }
     }
     ss = warp_sum(ss);
-    if (lane == 0) R->xn[warp] = sqrtf(ss);
+    if (lane == 0) Q->xn[warp] = sqrtf(ss);
   }
   bool alive = true;
 #pragma unroll 1
   for (int w = 0; w < n_rw; ++w) {
     if (!dec_wait_wave(bars, w, R, status, 23)) { alive = false; break; }
-    dec_wave_dots(ring + (w & 1) * kDecHalfBytes, min(RW, E - w * RW), d, xs, R, T, red, slog + w * RW, kMaxE + 1);
+    rs_wave_dots<NT>(ring + (w & 1) * kDecHalfBytes, min(RW, E - w * RW), d, xs, T, red, slog + w * RW, kMaxE + 1);
     if (warp == 0 && w + 2 < n_rw) {
       ptx::fence_proxy_async();
       issue_router_wave(w + 2);
     }
   }
   __syncthreads();
-  if (warp < 2 * kRsTok && (warp & (kRsTok - 1)) < T) {
-    // gate of token (warp & 7): warps 0-7 the off-the-shelf gate, 8-15 the masked one
-    const int t = warp & (kRsTok - 1), pass = warp / kRsTok;
+  // gates: task = (token, pass); pass 0 the off-the-shelf gate, pass 1 the masked one; 2 TOK tasks over 16 warps
+#pragma unroll 1
+  for (int task = warp; task < 2 * TOK; task += kDecWarps) {
+    const int t = task & (TOK - 1), pass = task / TOK;
+    if (t >= T) continue;
     float v[8];
     uint32_t allow = 0u;
 #pragma unroll
@@ -143,7 +214,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
     float sg[kMaxTopK];
     dec_topk_gate(v, allow, k, a.renorm, lane, se, sg);
     if (lane == 0) {
-      const float xn = R->xn[t];
+      const float xn = Q->xn[t];
 #pragma unroll
       for (int j = 0; j < kMaxTopK; ++j) {
         if (j < k) {
@@ -151,14 +222,14 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
           const size_t gp = (size_t)(tok0 + t) * k + j;
           const float gv = alive ? sg[j] : 0.f;
           if (pass == 0) {
-            R->ue[p] = se[j];
+            Q->ue[p] = se[j];
             a.uidx[gp] = se[j]; a.ugate[gp] = gv;
-            pt[p] = xn * fabsf(gv) * a.enorm[se[j]];
+            Q->pt[p] = xn * fabsf(gv) * a.enorm[se[j]];
           } else {
             const int sl = R->e2s[se[j]];
-            R->sl[p] = sl;
+            Q->sl[p] = sl;
             a.midx[gp] = se[j]; a.mgate[gp] = gv; a.slot[gp] = sl;
-            pm[p] = xn * fabsf(gv) * a.enorm[se[j]];
+            Q->pm[p] = xn * fabsf(gv) * a.enorm[se[j]];
           }
         }
       }
@@ -177,7 +248,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
     int n = 0;
 #pragma unroll 1
     for (int p = 0; p < P; ++p)
-      if (R->ue[p] == tid) { s += pt[p]; ++n; }
+      if (Q->ue[p] == tid) { s += Q->pt[p]; ++n; }
     a.cta_imp[(size_t)blockIdx.x * E + tid] = s;
     if (a.cta_cnt) a.cta_cnt[(size_t)blockIdx.x * E + tid] = (float)n;
   }
@@ -187,7 +258,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
     float m = 0.f;
 #pragma unroll 1
     for (int p = 0; p < P; ++p)
-      if (R->sl[p] == sl) { ++c; m += pm[p]; }
+      if (Q->sl[p] == sl) { ++c; m += Q->pm[p]; }
     a.cta_hist[(size_t)blockIdx.x * K + sl] = c;
     if (a.cta_mimp) a.cta_mimp[(size_t)blockIdx.x * K + sl] = m;
   }
