@@ -16,6 +16,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "ffn_fused.cuh"
+#include "gemm_tc_pair.cuh"
 #include "gemm_tc_small.cuh"
 #include "permute.cuh"
 #include "router_gate.cuh"
@@ -53,6 +54,8 @@ struct swapmoe_layer {
   int64_t launches;
   int32_t gemm_path;
   int32_t rows_pad_max;
+  int pair_min_rows;           // ... used when the slots hold at least this many rows on average (SWAPMOE_PAIR_MIN_ROWS)
+  int gemm_pairs;              // CTA pairs available to the cta_group::2 grouped GEMM (0: not used; SWAPMOE_PAIR_GEMM=0)
   bool small_router;           // eight-token mma router CTAs for batches of up to 64 tokens (bf16)
   int32_t small_router_max_t;  // ... and sixteen-token CTAs up to this many tokens (0: never)
   bool decode_path;            // one-launch forward for a handful of tokens (bf16)
@@ -142,7 +145,8 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   const int n_cta = (T + tok_tile - 1) / tok_tile;
   const int n_pairs = T * c.top_k;
   const bool use_tc = tc_selected(L->gemm_path, c, T);
-  const int mt = use_tc ? tc_row_subtiles(c, T) : 1;
+  const bool use_pairs = use_tc && tc_use_pairs(c, T, L->gemm_pairs, L->pair_min_rows);
+  const int mt = use_tc ? tc_row_subtiles(c, T, use_pairs) : 1;
   const int tile_rows = use_tc ? kTcBM * mt : kSimtBM;
   const int max_tiles = (n_pairs + tile_rows - 1) / tile_rows + c.K;
 
@@ -243,6 +247,9 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
       rc = tc_ffn_fused(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->done, L->row_pair, L->mgate, max_tiles,
                         L->status, st, pdl, &L->launches, &combined);
       if (mid) cudaEventRecord(mid, st);      // one kernel: the GEMM-2 stage reads as zero
+    } else if (mt == 2 && use_pairs) {
+      rc = tc_ffn_pair(L->tc, L->gemm_pairs, c, L->h, L->y, out, L->tiles, L->n_tiles, L->row_pair, L->mgate, max_tiles,
+                       T, L->status, st, pdl, &L->launches, &combined, mid);
     } else {
       rc = tc_ffn(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->tiles_b, L->n_tiles_b, L->row_pair, L->mgate,
                   max_tiles, mt, T,
@@ -469,6 +476,13 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   ok = ok && cuda_ok(router_gate_set_smem_limit<float>()) && cuda_ok(router_gate_set_smem_limit<bf16>());
   ok = ok && tc_init(L->tc, c, L->xp, L->h, L->y, L->rows_pad_max) == SWAPMOE_OK;
   if (L->tc.encode == nullptr) L->decode_path = false;     // its W_out loads need a tensor map
+  {
+    const char* env = std::getenv("SWAPMOE_PAIR_GEMM");      // SWAPMOE_PAIR_GEMM=0: one CTA per tile for every shape
+    L->gemm_pairs = (ok && L->tc.enabled && !(env && env[0] == '0')) ? tc_pair_init(L->sm_count) : 0;
+    env = std::getenv("SWAPMOE_PAIR_MIN_ROWS");
+    L->pair_min_rows = env ? std::max(160, std::atoi(env)) : 1024;
+    if (std::getenv("SWAPMOE_DEBUG")) std::fprintf(stderr, "swapmoe: gemm_pairs=%d\n", L->gemm_pairs);
+  }
   {
     const char* env = std::getenv("SWAPMOE_SMALL_ROUTER");   // SWAPMOE_SMALL_ROUTER=0: tcgen05 router for small batches too
     L->small_router = c.dtype == SWAPMOE_BF16 && !(env && env[0] == '0') &&

@@ -210,6 +210,101 @@ __device__ __forceinline__ void decode_tile(int t, int n_row_tiles, int n_col_ti
   *rt = r0 + (u - *ct * rows_here);
 }
 
+// ----------------------------------------------------------------------------- epilogue stores
+// An epilogue thread owns one accumulator row (a TMEM lane), so storing from its own registers
+// makes every store instruction of a warp touch 32 different rows, 16 bytes each: 32 memory
+// transactions per instruction, which saturate the load/store path that the TMA writes and the
+// tensor core's operand reads also go through (measured on the 8192-token configuration: the
+// mainloop slows down 3.5x while such an epilogue runs).  Instead each warp transposes 128 bytes
+// per row through a private 4 KB staging buffer: the owner writes its row as eight 16-byte pieces,
+// piece j at offset row * 128 + ((j ^ (row & 7)) * 16) (no bank conflicts), then lane l stores piece
+// l & 7 of rows 4 i + (l >> 3), i = 0..7: a store instruction covers four rows of 128 contiguous
+// bytes.
+constexpr int kTcEpiWarpStage = 32 * 128;                 // bytes per epilogue warp
+constexpr int kTcEpiStageBytes = 4 * kTcEpiWarpStage;     // four epilogue warps
+
+// Destination of the rows this lane stores: dst[i] = start of the tile's columns in the output row of
+// local row 4 i + (lane >> 3), plus this lane's 16 bytes; nullptr when that row is not stored.
+// `drow_own` = output row (of the matrix C) of the row this lane owns, or -1.
+__device__ __forceinline__ void epi_row_pointers(unsigned char* (&dst)[8], int drow_own, int lane, void* C, size_t ldc,
+                                                 size_t col0, int elem_bytes) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int drow = __shfl_sync(0xffffffffu, drow_own, 4 * i + (lane >> 3));
+    dst[i] = drow < 0 ? nullptr
+                      : static_cast<unsigned char*>(C) + ((size_t)drow * ldc + col0) * elem_bytes + (lane & 7) * 16;
+  }
+}
+// Stores 128 bytes of each of the warp's 32 rows: `pc` = the owned row's eight pieces, `byte_off` = offset of
+// this 128-byte chunk from the start of the tile's columns.
+__device__ __forceinline__ void epi_store_chunk(unsigned char* stg, const uint4 (&pc)[8], int lane,
+                                                unsigned char* const (&dst)[8], int byte_off) {
+  __syncwarp();                                            // the previous chunk has been read out
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    *reinterpret_cast<uint4*>(stg + lane * 128 + ((j ^ (lane & 7)) << 4)) = pc[j];
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = 4 * i + (lane >> 3);
+    const uint4 v = *reinterpret_cast<const uint4*>(stg + row * 128 + (((lane & 7) ^ (row & 7)) << 4));
+    if (dst[i] != nullptr) *reinterpret_cast<uint4*>(dst[i] + byte_off) = v;
+  }
+}
+
+// The accumulator columns [c0, c0 + 32) of this thread's TMEM lane -> activation -> four 16-byte pieces
+// (bf16 outputs) or eight (fp32 output).  `gate_cols` = distance to the gate columns (SwiGLU).
+template <int EPI>
+__device__ __forceinline__ void epi_load_pieces(uint32_t taddr, int c0, int gate_cols, float gate, uint4* pc) {
+  uint32_t v[32];
+  ptx::tmem_ld32(taddr + (uint32_t)c0, v);
+  if (EPI == kTcEpiSwigluBf16) {
+    uint32_t g[32];
+    ptx::tmem_ld32(taddr + (uint32_t)(c0 + gate_cols), g);
+    ptx::tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const float x1 = __uint_as_float(v[i]);
+      v[i] = __float_as_uint(x1 / (1.f + __expf(-x1)) * __uint_as_float(g[i]));
+    }
+  } else {
+    ptx::tmem_ld_wait();
+  }
+  if (EPI == kTcEpiF32) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) pc[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float f[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        f[j] = __uint_as_float(v[8 * i + j]);
+        if (EPI == kTcEpiReluBf16) f[j] = fmaxf(f[j], 0.f);
+        if (EPI == kTcEpiScatterBf16) f[j] *= gate;
+      }
+      pc[i] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]),
+                         pack_bf16x2(f[6], f[7]));
+    }
+  }
+}
+
+// One accumulator (kOutCols output columns of this thread's row) -> global memory, 128 bytes per row and chunk.
+template <int EPI, int kOutCols>
+__device__ __forceinline__ void epi_store_tile(uint32_t taddr, unsigned char* stg, int lane, float gate,
+                                               unsigned char* const (&dst)[8]) {
+  constexpr int kElem = (EPI == kTcEpiF32) ? 4 : 2;
+  constexpr int kChunkCols = 128 / kElem;                  // 32 fp32 or 64 bf16 columns
+  static_assert(kOutCols % kChunkCols == 0, "whole 128-byte chunks");
+#pragma unroll 1
+  for (int c0 = 0; c0 < kOutCols; c0 += kChunkCols) {
+    uint4 pc[8];
+    epi_load_pieces<EPI>(taddr, c0, kOutCols, gate, pc);
+    if (EPI != kTcEpiF32) epi_load_pieces<EPI>(taddr, c0 + 32, kOutCols, gate, pc + 4);
+    epi_store_chunk(stg, pc, lane, dst, c0 * kElem);
+  }
+}
+
 // MT = row sub-tiles of 128 rows that one CTA multiplies against the same weight tile.
 template <int BN, int MT = 1>
 struct TcSmem {
@@ -217,7 +312,8 @@ struct TcSmem {
   static constexpr int kBBytes = BN * kTcBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kStages = (kTcSmemBudget - 2048) / kStageBytes;
-  static constexpr int kBytes = kStages * kStageBytes + 2048;  // + alignment slack and barriers
+  // + alignment slack and barriers (1 KB each) + the epilogue warps' staging buffers
+  static constexpr int kBytes = kStages * kStageBytes + 2048 + kTcEpiStageBytes;
 };
 
 // C tile [128*MT, BN (or BN/2 for SwiGLU)] = epi(A[row0:row0+128*MT, :] * B[brow:brow+BN, :]^T).
@@ -250,6 +346,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   uint64_t* acc_empty = acc_full + 2;       // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  unsigned char* epi_stage = smem + kStages * S::kStageBytes + 1024;   // [4 warps][32 rows][128 bytes]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -360,17 +457,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int halves = (MT == 2 && td.rows > kTcBM) ? 2 : 1;
       // where this thread's rows go (and, for the scatter epilogue, their gate values): two dependent
       // global loads, fetched while the tile's MMAs are still running
-      size_t crow_h[MT];
+      int drow_h[MT];                            // output row of C, -1: not stored
       float gate_h[MT];
 #pragma unroll
       for (int hf = 0; hf < MT; ++hf) {
-        const int rr = r + hf * kTcBM;
-        crow_h[hf] = (size_t)(td.row0 + rr) * a.ldc + (size_t)ct * kOutCols;
+        const int rr = r + hf * kTcBM;           // row inside the (up to 256-row) tile
+        const bool valid = hf < halves && rr < td.rows;
+        drow_h[hf] = valid ? td.row0 + rr : -1;
         gate_h[hf] = 1.f;
-        if (EPI == kTcEpiScatterBf16 && hf < halves && rr < td.rows) {
+        if (EPI == kTcEpiScatterBf16 && valid) {
           const int p = a.row_pair[td.row0 + rr];
           gate_h[hf] = a.gate[p];
-          crow_h[hf] = (size_t)(p / a.top_k) * a.ldc + (size_t)ct * kOutCols;
+          drow_h[hf] = p / a.top_k;
         }
       }
       ok = bounded_wait(&acc_full[acc], acc_phase, abort_flag, a.status, 4);
@@ -378,53 +476,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       ptx::tc_fence_after();
 #pragma unroll
       for (int hf = 0; hf < MT; ++hf) {
-      if (hf < halves) {
-      const int rr = r + hf * kTcBM;             // row inside the (up to 256-row) tile
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)((acc * MT + hf) * BN);
-      const bool row_ok = rr < td.rows;
-      const size_t crow = crow_h[hf];
-      const float gate = gate_h[hf];
-#pragma unroll 1
-      for (int c0 = 0; c0 < kOutCols; c0 += 32) {
-        uint32_t v[32];
-        ptx::tmem_ld32(taddr + (uint32_t)c0, v);
-        if (EPI == kTcEpiSwigluBf16) {
-          uint32_t g[32];
-          ptx::tmem_ld32(taddr + (uint32_t)(c0 + kOutCols), g);
-          ptx::tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float x1 = __uint_as_float(v[i]);
-            v[i] = __float_as_uint(x1 / (1.f + __expf(-x1)) * __uint_as_float(g[i]));
-          }
-        } else {
-          ptx::tmem_ld_wait();
-        }
-        if (row_ok) {
-          if (EPI == kTcEpiF32) {
-            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(a.C) + crow + c0);
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-              dst[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                   __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+        if (hf < halves) {
+          const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)((acc * MT + hf) * BN);
+          constexpr int kElem = (EPI == kTcEpiF32) ? 4 : 2;
+          if constexpr ((kOutCols * kElem) % 128 == 0) {
+            unsigned char* dst[8];
+            epi_row_pointers(dst, drow_h[hf], lane, a.C, (size_t)a.ldc, (size_t)ct * kOutCols, kElem);
+            epi_store_tile<EPI, kOutCols>(taddr, epi_stage + q * kTcEpiWarpStage, lane, gate_h[hf], dst);
           } else {
-            uint4* dst = reinterpret_cast<uint4*>(static_cast<bf16*>(a.C) + crow + c0);
+            // 64 bytes per row (the narrowest bf16 tiles): every thread stores its own row
+            uint4 pc[4];
+            epi_load_pieces<EPI>(taddr, 0, kOutCols, gate_h[hf], pc);
+            if (drow_h[hf] >= 0) {
+              uint4* dst = reinterpret_cast<uint4*>(static_cast<bf16*>(a.C) + (size_t)drow_h[hf] * a.ldc +
+                                                    (size_t)ct * kOutCols);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              float f[8];
-#pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                f[j] = __uint_as_float(v[8 * i + j]);
-                if (EPI == kTcEpiReluBf16) f[j] = fmaxf(f[j], 0.f);
-                if (EPI == kTcEpiScatterBf16) f[j] *= gate;
-              }
-              dst[i] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]),
-                                  pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+              for (int i = 0; i < 4; ++i) dst[i] = pc[i];
             }
           }
         }
-      }
-      }
       }
       ptx::tc_fence_before();
       ptx::mbar_arrive(&acc_empty[acc]);       // 128 arrivals hand the buffer back to the MMA warp
@@ -469,9 +539,16 @@ inline bool tc_supported(const swapmoe_config_t& c) {
 // Row sub-tiles per CTA for a forward of T tokens: two when the average slot has well over
 // 128 rows (weight tiles are then shared by two sub-tiles), one for small slots (nothing to
 // share) and for very large ones (tensor-bound: keep the double-buffered accumulators).
-inline int tc_row_subtiles(const swapmoe_config_t& c, int T) {
+inline int tc_row_subtiles(const swapmoe_config_t& c, int T, bool cta_pairs = false) {
   const long long rows_per_slot = (long long)T * c.top_k / c.K;
+  // CTA pairs (tc_gemm_pair_kernel) keep two accumulator sets, so they take the very large slots
+  if (cta_pairs && rows_per_slot >= 1024 && c.d_model % 256 == 0) return 2;
   return (rows_per_slot >= 160 && rows_per_slot < 1024 && c.d_model % 256 == 0) ? 2 : 1;
+}
+// Whether a forward with 256-row tiles runs on CTA pairs: slots of at least `min_rows` rows on average (a
+// 256-row tile with <= 128 valid rows leaves one SM of the pair idle, so ragged small slots stay with one CTA per tile).
+inline bool tc_use_pairs(const swapmoe_config_t& c, int T, int n_pairs, int min_rows) {
+  return n_pairs > 0 && (long long)T * c.top_k / c.K >= min_rows && c.d_model % 256 == 0 && c.d_ff % 256 == 0;
 }
 
 // Automatic choice: tensor cores whenever the shape allows it.
