@@ -367,7 +367,32 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  pdl_wait();      // the tile list and the operands come from the preceding kernels
+  // The tile list was written by the router, which finished before the kernel in front of this one was
+  // allowed to start (every kernel of the chain triggers its dependents only after its own wait), and the
+  // weights are constants of the layer.  So the producer requests the weight boxes of its first stages
+  // BEFORE the dependent-launch wait; only the activations (written by the kernel in front) have to wait.
+  const bool is_producer = warp == 0 && lane == 0;
+  int pre = 0;                                   // stages whose weight boxes are already requested
+  if (is_producer) {
+    const int n_rt = __ldcg(a.n_tiles);
+    if ((int)blockIdx.x < n_rt * a.n_col_tiles) {
+      int rt, ct;
+      decode_tile((int)blockIdx.x, n_rt, a.n_col_tiles, a.row_group, &rt, &ct);
+      const int4 raw = __ldcg(reinterpret_cast<const int4*>(a.tiles + rt));
+      const TileDesc td = *reinterpret_cast<const TileDesc*>(&raw);
+      const int brow = td.phys * a.b_rows_per_phys + ct * kBoxRows;
+      const int halves = (MT == 2 && td.rows > kTcBM) ? 2 : 1;
+      pre = a.k_blocks < kStages ? a.k_blocks : kStages;
+      for (int kb = 0; kb < pre; ++kb) {
+        ptx::mbar_expect_tx(&full[kb], (uint32_t)(halves * a.a_box_bytes + S::kBBytes));
+#pragma unroll
+        for (int j = 0; j < kNB; ++j)
+          ptx::tma_load_2d(sB + kb * S::kBBytes + j * kBoxRows * kTcBK * 2, &tmB, &full[kb], kb * kTcBK,
+                           brow + j * a.b_rows_gate);
+      }
+    }
+  }
+  pdl_wait();      // the activations come from the preceding kernel
   pdl_trigger();
   const int n_row_tiles = *a.n_tiles;
   const int total = n_row_tiles * a.n_col_tiles;
@@ -385,16 +410,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int brow = td.phys * a.b_rows_per_phys + ct * kBoxRows;
         const int halves = (MT == 2 && td.rows > kTcBM) ? 2 : 1;
         for (int kb = 0; kb < a.k_blocks; ++kb) {
-          ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 1);
-          if (!ok) break;
-          ptx::mbar_expect_tx(&full[stage], (uint32_t)(halves * a.a_box_bytes + S::kBBytes));
+          const bool early = t == (int)blockIdx.x && kb < pre;   // armed and weights requested above
+          if (!early) {
+            ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 1);
+            if (!ok) break;
+            ptx::mbar_expect_tx(&full[stage], (uint32_t)(halves * a.a_box_bytes + S::kBBytes));
+          }
           for (int hf = 0; hf < halves; ++hf)
             ptx::tma_load_2d(sA + stage * S::kABytes + hf * kHalfBytes, &tmA, &full[stage], kb * kTcBK,
                              td.row0 + hf * kTcBM);
+          if (!early) {
 #pragma unroll
-          for (int j = 0; j < kNB; ++j)
-            ptx::tma_load_2d(sB + stage * S::kBBytes + j * kBoxRows * kTcBK * 2, &tmB, &full[stage],
-                             kb * kTcBK, brow + j * a.b_rows_gate);
+            for (int j = 0; j < kNB; ++j)
+              ptx::tma_load_2d(sB + stage * S::kBBytes + j * kBoxRows * kTcBK * 2, &tmB, &full[stage],
+                               kb * kTcBK, brow + j * a.b_rows_gate);
+          }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }

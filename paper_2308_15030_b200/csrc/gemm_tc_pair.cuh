@@ -137,7 +137,28 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  pdl_wait();      // the tile list and the operands come from the preceding kernels
+  // As in tc_gemm_kernel: the tile list and the weights do not depend on the kernel in front, so each
+  // producer requests the weight boxes of its first stages before the dependent-launch wait.
+  int pre = 0;
+  if (warp == 0 && lane == 0) {
+    const int n_rt = __ldcg(a.n_tiles);
+    if (pair < n_rt * a.n_col_tiles) {
+      int rt, ct;
+      decode_tile(pair, n_rt, a.n_col_tiles, a.row_group, &rt, &ct);
+      const int4 raw = __ldcg(reinterpret_cast<const int4*>(a.tiles + rt));
+      const TileDesc td = *reinterpret_cast<const TileDesc*>(&raw);
+      const int brow = td.phys * a.b_rows_per_phys +
+                       (EPI == kTcEpiSwigluBf16 ? ct * kPairHalfRows + (int)rank * a.b_rows_gate
+                                                : ct * kPairBN + (int)rank * kPairHalfRows);
+      pre = a.k_blocks < kStages ? a.k_blocks : kStages;
+      for (int kb = 0; kb < pre; ++kb) {
+        if (rank == 0)
+          ptx::mbar_expect_tx(&full[kb], (uint32_t)((td.rows > kTcBM ? 2 : 1) * kPairABytes + 2 * kPairBBytes));
+        ptx::tma_load_2d_pair(sB + kb * kPairBBytes, &tmB, ptx::map_to_cta(ptx::smem_u32(&full[kb]), 0u), kb * kTcBK, brow);
+      }
+    }
+  }
+  pdl_wait();      // the activations come from the preceding kernel
   pdl_trigger();
   const int n_row_tiles = *a.n_tiles;
   const int total = n_row_tiles * a.n_col_tiles;
@@ -160,14 +181,17 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                                                   : ct * kPairBN + (int)rank * kPairHalfRows);
         const bool load_a = rank == 0 || two_halves;
         for (int kb = 0; kb < a.k_blocks; ++kb) {
-          ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 11);
-          if (!ok) break;
+          const bool early = t == pair && kb < pre;          // armed and weights requested above
+          if (!early) {
+            ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 11);
+            if (!ok) break;
+          }
           const uint32_t full_addr = ptx::map_to_cta(ptx::smem_u32(&full[stage]), 0u);
-          if (rank == 0)
+          if (rank == 0 && !early)
             ptx::mbar_expect_tx(&full[stage], (uint32_t)((two_halves ? 2 : 1) * kPairABytes + 2 * kPairBBytes));
           if (load_a)
             ptx::tma_load_2d_pair(sA + stage * kPairABytes, &tmA, full_addr, kb * kTcBK, td.row0 + (int)rank * kTcBM);
-          ptx::tma_load_2d_pair(sB + stage * kPairBBytes, &tmB, full_addr, kb * kTcBK, brow);
+          if (!early) ptx::tma_load_2d_pair(sB + stage * kPairBBytes, &tmB, full_addr, kb * kTcBK, brow);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }

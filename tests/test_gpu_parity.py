@@ -211,6 +211,37 @@ def test_two_row_subtiles_per_cta():
         assert cnt.max() > 256 and any(0 < c % 256 <= 128 for c in cnt), cnt
 
 
+@pytest.mark.parametrize("min_rows", [None, "160"])
+def test_cta_pair_grouped_gemm(monkeypatch, min_rows):
+    """Slots of 1024+ rows on average run the grouped GEMMs on CTA pairs (one 256-row tile per two SMs,
+    cta_group::2): all four epilogues, tiles whose second half is full, ragged and absent.  With
+    SWAPMOE_PAIR_MIN_ROWS=160 the same kernels take the mid-size case of the test above; with
+    SWAPMOE_PAIR_GEMM=0 the one-CTA kernels must give the same routing and an output within tolerance."""
+    import oracle
+    from harness import Case, check_against_oracle
+    if min_rows:
+        monkeypatch.setenv("SWAPMOE_PAIR_MIN_ROWS", min_rows)
+    T = 1500 if min_rows else 5200
+    K = 5 if min_rows else 4
+    for k, act, renorm in ((1, I.ACT_RELU, 0), (2, I.ACT_SWIGLU, 1)):
+        cfg = _cfg(T=T // k, d=256, f=512, E=12, K=K, k=k, act=act, renorm=renorm, zipf_s=1.3)
+        probe = Case(cfg)
+        lg = oracle.logits(probe.x, probe.Wr)
+        ui, ug = oracle.gate(lg, cfg.k, cfg.renorm)
+        order = oracle.topk_importance(oracle.importance(probe.x, ui, ug, probe.enorm), cfg.E)
+        case = Case(cfg, s2e=list(order[:K - 2]) + list(order[-2:]))   # popular experts and two rare ones
+        out = case.run()
+        res = check_against_oracle(case, out)
+        cnt = res["oracle"]["count"]
+        assert cnt.max() > 256 and any(0 < c % 256 <= 128 for c in cnt) and any(c % 256 > 128 for c in cnt), cnt
+        monkeypatch.setenv("SWAPMOE_PAIR_GEMM", "0")
+        single = Case(cfg, s2e=list(case.s2e))
+        out1 = single.run()
+        monkeypatch.delenv("SWAPMOE_PAIR_GEMM")
+        a, b = out.astype(np.float64), out1.astype(np.float64)
+        assert np.max(np.abs(a - b)) <= 2e-2 * np.max(np.abs(b))
+
+
 @pytest.mark.parametrize("dtype,k,renorm", [(I.BF16, 1, 0), (I.BF16, 2, 1), (I.F32, 2, 0)])
 def test_count_and_masked_importance_scores(dtype, k, renorm):
     """Token-count score ("Simple scheduling", Section 4.4) and Eq. (1) over the masked routing."""
