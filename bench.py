@@ -319,6 +319,8 @@ def run_cuda(args, cfg):
     tf32x3_peak = peaks["bf16_tflops"] * (1.1 / 2.25) / 3.0
     if cfg.dtype != I.BF16 and ffma:
         bound, peak, ach, unit = "alu", 74.4, g_flops / 2 / (g_ms * 1e-3) / 1e12, "TFLOP/s"
+    elif cfg.dtype != I.BF16 and t_hbm >= g_flops / (tf32x3_peak * 1e12):
+        bound, peak, ach, unit = "hbm", peaks["hbm_gbs"], g_bytes / 2 / (g_ms * 1e-3) / 1e9, "GB/s"
     elif cfg.dtype != I.BF16:
         bound, peak, ach, unit = "tensor", tf32x3_peak, g_flops / 2 / (g_ms * 1e-3) / 1e12, "TFLOP/s"
     elif t_hbm >= t_tc:
@@ -352,13 +354,15 @@ def run_cuda(args, cfg):
                      "traffic": NCU_TRAFFIC_PER_LAUNCH.get(cfg.name), "peak_source": peaks["source"],
                      "kernel": "tc_gemm_kernel (grouped FFN GEMM, 2 launches per step: GEMM-1+act, GEMM-2)"
                                if cfg.dtype == I.BF16 else ("gemm_simt_kernel (FFMA, 2 launches per step)" if ffma else
-                                                            "gemm_tf32x3_kernel (split-TF32 mma, 2 launches per step)"),
+                                                            ("gemm_tf32x3_kernel (split-TF32 warp-level mma, 2 launches per step)"
+                                                             if os.environ.get("SWAPMOE_FP32_TC") == "0" else
+                                                             "tc_gemm_f32_kernel (split-TF32 on tcgen05, 2 launches per step)")),
                      "algorithmic_bytes_per_launch": g_bytes / 2, "flops_per_launch": g_flops / 2,
                      "avg_launch_ms": g_ms,
                      "tensor_tflops": g_flops / 2 / (g_ms * 1e-3) / 1e12,
                      "tensor_peak_kind": (tc_kind if cfg.dtype == I.BF16 else "bf16 burst x 1.1/2.25 / 3 (TF32 x3)")
                                          if bound == "tensor" else None,
-                     "frac_of_fp32_ffma_peak": (ach / 74.4) if cfg.dtype != I.BF16 else None,
+                     "frac_of_fp32_ffma_peak": (g_flops / 2 / (g_ms * 1e-3) / 1e12 / 74.4) if cfg.dtype != I.BF16 else None,
                      "frac_of_burst_tensor_peak": (ach / peaks["bf16_tflops"]) if bound == "tensor" else None},
         "layer_roofline": {"t_roof_us": t_roof * 1e6, "frac": t_roof * 1e3 / ms_step,
                            "algorithmic_bytes": layer_bytes, "flops": layer_flops},

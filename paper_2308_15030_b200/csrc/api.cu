@@ -16,6 +16,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "ffn_fused.cuh"
+#include "gemm_tc_f32.cuh"
 #include "gemm_tc_pair.cuh"
 #include "gemm_tc_small.cuh"
 #include "permute.cuh"
@@ -77,6 +78,8 @@ struct swapmoe_layer {
   const void* map_x_ptr;
   int32_t map_x_T;
   TcState tc;
+  TcF32State tc32;             // tcgen05 split-TF32 grouped GEMM of fp32 layers (SWAPMOE_FP32_TC=0: warp-level mma)
+  PFN_encodeTiled encode32;
 };
 
 namespace {
@@ -147,7 +150,8 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   const bool use_tc = tc_selected(L->gemm_path, c, T);
   const bool use_pairs = use_tc && tc_use_pairs(c, T, L->gemm_pairs, L->pair_min_rows);
   const int mt = use_tc ? tc_row_subtiles(c, T, use_pairs) : 1;
-  const int tile_rows = use_tc ? kTcBM * mt : kSimtBM;
+  const bool use_tc32 = !use_tc && L->tc32.enabled && L->tc32.arena_bound;
+  const int tile_rows = use_tc ? kTcBM * mt : (use_tc32 ? kTcBM : kSimtBM);
   const int max_tiles = (n_pairs + tile_rows - 1) / tile_rows + c.K;
 
   RouterArgs ra;
@@ -255,6 +259,11 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
                   max_tiles, mt, T,
                   L->status, st, pdl, &L->launches, &combined, mid);
     }
+    if (rc != SWAPMOE_OK) return rc;
+  } else if (use_tc32) {
+    cudaEvent_t mid = L->stage_events ? static_cast<cudaEvent_t>(L->stage_events[4]) : nullptr;
+    const int32_t rc = tc_ffn_f32(L->tc32, c, L->h, L->y, (long long)L->rows_pad_max * c.d_model, L->y_copies, L->tiles,
+                                  L->n_tiles, max_tiles, T, L->status, st, pdl, &L->launches, &y_split, mid);
     if (rc != SWAPMOE_OK) return rc;
   } else {
     SimtGemmArgs g1;
@@ -475,6 +484,15 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   ok = ok && cuda_ok(cudaMemset(L->xp, 0, rows_pad * c.d_model * L->elem));
   ok = ok && cuda_ok(router_gate_set_smem_limit<float>()) && cuda_ok(router_gate_set_smem_limit<bf16>());
   ok = ok && tc_init(L->tc, c, L->xp, L->h, L->y, L->rows_pad_max) == SWAPMOE_OK;
+  L->tc32.enabled = L->tc32.arena_bound = false;
+  L->encode32 = nullptr;
+  {
+    const char* env = std::getenv("SWAPMOE_FP32_TC");        // SWAPMOE_FP32_TC=0: warp-level mma (or FFMA) for fp32 layers
+    if (ok && c.dtype == SWAPMOE_F32 && !L->fp32_ffma && !(env && env[0] == '0')) {
+      L->encode32 = tc_get_encoder();
+      ok = tc_f32_init(L->tc32, L->encode32, c, L->xp, L->h, L->rows_pad_max, L->sm_count) == SWAPMOE_OK;
+    }
+  }
   if (L->tc.encode == nullptr) L->decode_path = false;     // its W_out loads need a tensor map
   {
     const char* env = std::getenv("SWAPMOE_PAIR_GEMM");      // SWAPMOE_PAIR_GEMM=0: one CTA per tile for every shape
@@ -563,7 +581,9 @@ int32_t swapmoe_set_resident(swapmoe_layer_t* L, const int32_t* s2e, const int32
   }
   if (arena_in != L->arena_in || arena_out != L->arena_out) {
     L->small.valid = false;
-    const int32_t rc = tc_bind_arena(L->tc, c, arena_in, arena_out);
+    int32_t rc = tc_bind_arena(L->tc, c, arena_in, arena_out);
+    if (rc != SWAPMOE_OK) return rc;
+    rc = tc_f32_bind_arena(L->tc32, L->encode32, c, arena_in, arena_out);
     if (rc != SWAPMOE_OK) return rc;
     // column slices of W_out for the one-launch decode kernel: 32 columns x 256 rows, 64-byte swizzle
     if (L->decode_path &&

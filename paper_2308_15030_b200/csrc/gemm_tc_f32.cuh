@@ -1,0 +1,392 @@
+// Grouped expert GEMM for fp32 layers on the tcgen05 tensor cores (SwapMoE Section 2: the experts'
+// FFN restricted to the resident slots), with fp32-grade accuracy from three TF32 products.
+//
+// `kind::tf32` keeps 10 mantissa bits of each operand, which cannot hold the 1e-4 output tolerance
+// over 768-3072-term dot products.  Every operand is therefore split as x = hi + lo with
+// hi = x with its low 13 mantissa bits cleared (exactly a TF32 number) and lo = x - hi (exact in
+// fp32, at most 13 significant bits, so TF32 holds it to 2^-11 relative): the product is
+// lo_a*hi_b + hi_a*lo_b + hi_a*hi_b, accumulated in fp32 in TMEM; the dropped lo*lo term and the
+// rounding of lo are below 2^-20 relative.
+//
+// TMA brings the fp32 operands (k-blocks of 32 columns = 128-byte swizzled rows) into a ring of
+// raw stages.  The split is ELEMENTWISE, so it preserves the swizzled layout: four converter warps
+// rewrite a stage in place with its hi parts and write the lo parts at the same offsets of a "lo"
+// slot (two slots), fence towards the async proxy and arrive on `conv_done`; one thread then
+// issues the 12 MMAs of the k-block (4 steps of K = 8, three products each) and commits to the
+// barriers that free the raw stage and the lo slot.  Roles (384 threads): warp 0 TMA producer,
+// warp 1 MMA issuer, warp 2 TMEM allocation, warps 4-7 epilogue (two accumulator sets, so it
+// overlaps the next item's MMAs), warps 8-11 converters.  A work item is (row tile, column tile,
+// contraction slice): GEMM-2 has few output tiles and a long contraction, so its slices go to
+// separate copies of y that the combine kernel adds in order (deterministic).
+#pragma once
+#include "gemm_tc.cuh"
+
+namespace swapmoe {
+
+constexpr int kF32BK = 32;                          // fp32 elements per k-block = one 128-byte swizzled row
+constexpr int kF32UmmaK = 8;
+constexpr int kF32BN = 128;                         // accumulator columns per tile
+constexpr int kF32Threads = 384;
+constexpr int kF32ABytes = kTcBM * kF32BK * 4;      // 16 KB
+constexpr int kF32BBytes = kF32BN * kF32BK * 4;     // 16 KB
+constexpr int kF32StageBytes = kF32ABytes + kF32BBytes;
+constexpr int kF32Stages = 4;                       // raw stages (TMA targets; hold the hi parts after conversion)
+constexpr int kF32LoSlots = 2;
+constexpr int kF32SmemBytes = (kF32Stages + kF32LoSlots) * kF32StageBytes + 2048 + kTcEpiStageBytes;
+
+// Epilogues of the fp32 path (values continue the bf16 kernels' enum)
+enum { kTcEpiReluF32 = 4, kTcEpiSwigluF32 = 5 };
+
+struct TcF32Args {
+  void* C;                  // [n_split][rows_pad, ldc] fp32
+  const TileDesc* tiles;    // 128-row tiles
+  const int32_t* n_tiles;
+  int32_t* status;
+  long long split_stride;   // elements between the copies of C
+  int32_t ldc, n_col_tiles, k_blocks, n_split;   // k_blocks per slice
+  int32_t b_rows_per_phys, b_rows_gate;
+};
+
+namespace ptx {
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n" ::"r"(tmem_d),
+      "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+}  // namespace ptx
+
+// Instruction descriptor: tf32 x tf32 -> fp32, both operands K-major, M x N tile.
+__host__ __device__ constexpr uint32_t make_idesc_tf32(int M, int N) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// accumulator columns [c0, c0 + 32) of this thread's TMEM lane -> activation -> eight 16-byte pieces of fp32
+template <int EPI>
+__device__ __forceinline__ void epi_load_pieces_f32(uint32_t taddr, int c0, int gate_cols, uint4* pc) {
+  uint32_t v[32];
+  ptx::tmem_ld32(taddr + (uint32_t)c0, v);
+  if (EPI == kTcEpiSwigluF32) {
+    uint32_t g[32];
+    ptx::tmem_ld32(taddr + (uint32_t)(c0 + gate_cols), g);
+    ptx::tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const float x1 = __uint_as_float(v[i]);
+      v[i] = __float_as_uint(x1 / (1.f + expf(-x1)) * __uint_as_float(g[i]));
+    }
+  } else {
+    ptx::tmem_ld_wait();
+    if (EPI == kTcEpiReluF32) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(fmaxf(__uint_as_float(v[i]), 0.f));
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) pc[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(kF32Threads, 1)
+tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcF32Args a) {
+  constexpr int kNB = (EPI == kTcEpiSwigluF32) ? 2 : 1;     // weight boxes per stage
+  constexpr int kBoxRows = kF32BN / kNB;
+  constexpr int kOutCols = kF32BN / kNB;
+  constexpr uint32_t kTmemCols = 2 * kF32BN;
+  constexpr uint32_t kIdesc = make_idesc_tf32(kTcBM, kF32BN);
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  unsigned char* raw = smem;                                         // [stages][A 16 KB | B 16 KB]
+  unsigned char* lo = smem + kF32Stages * kF32StageBytes;            // [slots][A 16 KB | B 16 KB]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(lo + kF32LoSlots * kF32StageBytes);
+  uint64_t* full = bars;                          // [stages]   TMA -> converters
+  uint64_t* empty = full + kF32Stages;            // [stages]   MMA -> producer
+  uint64_t* conv_done = empty + kF32Stages;       // [slots]    converters -> MMA (128 arrivals)
+  uint64_t* lo_empty = conv_done + kF32LoSlots;   // [slots]    MMA -> converters
+  uint64_t* acc_full = lo_empty + kF32LoSlots;    // [2]
+  uint64_t* acc_empty = acc_full + 2;             // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  unsigned char* epi_stage = reinterpret_cast<unsigned char*>(bars) + 1024;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kF32Stages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
+    for (int s = 0; s < kF32LoSlots; ++s) { ptx::mbar_init(&conv_done[s], 128); ptx::mbar_init(&lo_empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 128); }
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::prefetch_tmap(&tmA);
+    ptx::prefetch_tmap(&tmB);
+  }
+  if (warp == 2) {
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  pdl_wait();
+  pdl_trigger();
+  const int n_row_tiles = *a.n_tiles;
+  const int per_slice = n_row_tiles * a.n_col_tiles;
+  const int total = per_slice * a.n_split;        // item = slice * per_slice + (col tile * n_row_tiles + row tile)
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ------------------------------------------------------------------ TMA producer
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        const int z = t / per_slice, u = t - z * per_slice;
+        const int ct = u / n_row_tiles, rt = u - ct * n_row_tiles;
+        const TileDesc td = a.tiles[rt];
+        const int brow = td.phys * a.b_rows_per_phys + ct * kBoxRows;
+        const int kb0 = z * a.k_blocks;
+        for (int kb = 0; kb < a.k_blocks; ++kb) {
+          ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 31);
+          if (!ok) break;
+          unsigned char* sA = raw + stage * kF32StageBytes;
+          ptx::mbar_expect_tx(&full[stage], (uint32_t)kF32StageBytes);
+          ptx::tma_load_2d(sA, &tmA, &full[stage], (kb0 + kb) * kF32BK, td.row0);
+#pragma unroll
+          for (int j = 0; j < kNB; ++j)
+            ptx::tma_load_2d(sA + kF32ABytes + j * kBoxRows * kF32BK * 4, &tmB, &full[stage], (kb0 + kb) * kF32BK,
+                             brow + j * a.b_rows_gate);
+          if (++stage == kF32Stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // Give copies that are still in flight time to land before shared memory is released.
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ptx::globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ------------------------------------------------------------------ MMA issuer
+      int stage = 0, slot = 0, acc = 0;
+      uint32_t slot_phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        ok = bounded_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, a.status, 32);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * kF32BN);
+        for (int kb = 0; kb < a.k_blocks; ++kb) {
+          ok = bounded_wait(&conv_done[slot], slot_phase, abort_flag, a.status, 33);
+          if (!ok) break;
+          ptx::tc_fence_after();
+          const uint32_t hi_a = ptx::smem_u32(raw + stage * kF32StageBytes), hi_b = hi_a + kF32ABytes;
+          const uint32_t lo_a = ptx::smem_u32(lo + slot * kF32StageBytes), lo_b = lo_a + kF32ABytes;
+          const uint64_t dha = make_kmajor_sw128_desc(hi_a), dhb = make_kmajor_sw128_desc(hi_b);
+          const uint64_t dla = make_kmajor_sw128_desc(lo_a), dlb = make_kmajor_sw128_desc(lo_b);
+#pragma unroll
+          for (int k = 0; k < kF32BK / kF32UmmaK; ++k) {
+            // 8 fp32 along K inside the swizzled row = +32 bytes = +2 in the address field; small terms first
+            ptx::umma_tf32(tmem_d, dla + (uint64_t)(2 * k), dhb + (uint64_t)(2 * k), kIdesc, (kb > 0 || k > 0) ? 1u : 0u);
+            ptx::umma_tf32(tmem_d, dha + (uint64_t)(2 * k), dlb + (uint64_t)(2 * k), kIdesc, 1u);
+            ptx::umma_tf32(tmem_d, dha + (uint64_t)(2 * k), dhb + (uint64_t)(2 * k), kIdesc, 1u);
+          }
+          ptx::umma_commit(&empty[stage]);       // the raw stage may be refilled
+          ptx::umma_commit(&lo_empty[slot]);     // the lo slot may be rewritten
+          if (++stage == kF32Stages) stage = 0;
+          if (++slot == kF32LoSlots) { slot = 0; slot_phase ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::umma_commit(&acc_full[acc]);
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else if (warp >= 8) {
+    // ---------------------------------------------------------------------- converters: hi in place, lo beside
+    const int ctid = threadIdx.x - 8 * 32;       // 0..127
+    int stage = 0, slot = 0;
+    uint32_t phase = 0, slot_phase = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+      for (int kb = 0; kb < a.k_blocks; ++kb) {
+        ok = bounded_wait(&full[stage], phase, abort_flag, a.status, 34);
+        if (ok) ok = bounded_wait(&lo_empty[slot], slot_phase ^ 1u, abort_flag, a.status, 35);
+        if (!ok) break;
+        uint4* src = reinterpret_cast<uint4*>(raw + stage * kF32StageBytes);
+        uint4* dst = reinterpret_cast<uint4*>(lo + slot * kF32StageBytes);
+#pragma unroll 4
+        for (int i = ctid; i < kF32StageBytes / 16; i += 128) {
+          const uint4 x = src[i];
+          uint4 h, l;
+          h.x = x.x & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(x.x) - __uint_as_float(h.x));
+          h.y = x.y & 0xffffe000u; l.y = __float_as_uint(__uint_as_float(x.y) - __uint_as_float(h.y));
+          h.z = x.z & 0xffffe000u; l.z = __float_as_uint(__uint_as_float(x.z) - __uint_as_float(h.z));
+          h.w = x.w & 0xffffe000u; l.w = __float_as_uint(__uint_as_float(x.w) - __uint_as_float(h.w));
+          src[i] = h;
+          dst[i] = l;
+        }
+        ptx::fence_proxy_async();                // these writes are read by the tensor core (async proxy)
+        ptx::mbar_arrive(&conv_done[slot]);
+        if (++stage == kF32Stages) { stage = 0; phase ^= 1u; }
+        if (++slot == kF32LoSlots) { slot = 0; slot_phase ^= 1u; }
+      }
+    }
+  } else if (warp >= 4) {
+    // ---------------------------------------------------------------------- epilogue
+    const int q = warp - 4;
+    const int r = q * 32 + lane;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+      const int z = t / per_slice, u = t - z * per_slice;
+      const int ct = u / n_row_tiles, rt = u - ct * n_row_tiles;
+      const TileDesc td = a.tiles[rt];
+      const int drow = r < td.rows ? td.row0 + r : -1;
+      unsigned char* dst[8];
+      epi_row_pointers(dst, drow, lane, static_cast<float*>(a.C) + (size_t)z * a.split_stride, (size_t)a.ldc,
+                       (size_t)ct * kOutCols, 4);
+      ok = bounded_wait(&acc_full[acc], acc_phase, abort_flag, a.status, 36);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kF32BN);
+#pragma unroll 1
+      for (int c0 = 0; c0 < kOutCols; c0 += 32) {
+        uint4 pc[8];
+        epi_load_pieces_f32<EPI>(taddr, c0, kOutCols, pc);
+        epi_store_chunk(epi_stage + q * kTcEpiWarpStage, pc, lane, dst, c0 * 4);
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&acc_empty[acc]);
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ----------------------------------------------------------------------------- host side
+struct TcF32State {
+  bool enabled, arena_bound;
+  int sm_count;
+  CUtensorMap map_xp, map_h;          // activations, box 32 x 128
+  CUtensorMap map_win, map_wout;      // weights flattened to 2D; box 32 x 128 (64 for SwiGLU's W1 / W3)
+};
+
+// The driver's tensor-map encoder (nullptr when it cannot be had).
+inline PFN_encodeTiled tc_get_encoder() {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  return reinterpret_cast<PFN_encodeTiled>(fn);
+}
+
+inline bool tc_f32_supported(const swapmoe_config_t& c) {
+  return c.dtype == SWAPMOE_F32 && c.d_model % kF32BN == 0 && c.d_ff % kF32BN == 0;
+}
+
+inline bool tc_encode_2d_f32(PFN_encodeTiled enc, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                             uint32_t box_rows) {
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 4};
+  const cuuint32_t box[2] = {(cuuint32_t)kF32BK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline int32_t tc_f32_init(TcF32State& s, PFN_encodeTiled enc, const swapmoe_config_t& c, void* xp, void* h,
+                           int rows_pad, int sm_count) {
+  s.enabled = false;
+  s.arena_bound = false;
+  s.sm_count = sm_count;
+  if (!enc || !tc_f32_supported(c)) return SWAPMOE_OK;
+  if (!tc_encode_2d_f32(enc, &s.map_xp, xp, (uint64_t)rows_pad, (uint64_t)c.d_model, kTcBM) ||
+      !tc_encode_2d_f32(enc, &s.map_h, h, (uint64_t)rows_pad, (uint64_t)c.d_ff, kTcBM))
+    return SWAPMOE_ERR_CUDA;
+  if (cudaFuncSetAttribute(tc_gemm_f32_kernel<kTcEpiReluF32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kF32SmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(tc_gemm_f32_kernel<kTcEpiSwigluF32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kF32SmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(tc_gemm_f32_kernel<kTcEpiF32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kF32SmemBytes) != cudaSuccess)
+    return SWAPMOE_ERR_CUDA;
+  s.enabled = true;
+  return SWAPMOE_OK;
+}
+
+inline int32_t tc_f32_bind_arena(TcF32State& s, PFN_encodeTiled enc, const swapmoe_config_t& c, const void* arena_in,
+                                 const void* arena_out) {
+  if (!s.enabled) return SWAPMOE_OK;
+  const int P = c.K + c.spare_slots;
+  const int nin = c.act == SWAPMOE_ACT_SWIGLU ? 2 : 1;
+  if (!tc_encode_2d_f32(enc, &s.map_win, arena_in, (uint64_t)P * nin * c.d_ff, (uint64_t)c.d_model,
+                        (uint32_t)(kF32BN / nin)) ||
+      !tc_encode_2d_f32(enc, &s.map_wout, arena_out, (uint64_t)P * c.d_model, (uint64_t)c.d_ff, (uint32_t)kF32BN))
+    return SWAPMOE_ERR_CUDA;
+  s.arena_bound = true;
+  return SWAPMOE_OK;
+}
+
+// Both grouped GEMMs of an fp32 layer.  GEMM-2 writes `*y_split` partial copies of y (the combine kernel adds them).
+inline int32_t tc_ffn_f32(TcF32State& s, const swapmoe_config_t& c, void* h, float* y, long long y_copy_stride,
+                          int y_copies, const TileDesc* tiles, const int32_t* n_tiles, int max_tiles, int n_tokens,
+                          int32_t* status, cudaStream_t st, bool pdl, int64_t* launches, int* y_split,
+                          cudaEvent_t between = nullptr) {
+  if (!s.enabled || !s.arena_bound) return SWAPMOE_ERR_NOT_READY;
+  const bool swiglu = c.act == SWAPMOE_ACT_SWIGLU;
+  const int out1 = swiglu ? kF32BN / 2 : kF32BN;
+  TcF32Args g1;
+  g1.C = h; g1.tiles = tiles; g1.n_tiles = n_tiles; g1.status = status; g1.split_stride = 0;
+  g1.ldc = c.d_ff; g1.n_col_tiles = c.d_ff / out1; g1.k_blocks = c.d_model / kF32BK; g1.n_split = 1;
+  g1.b_rows_per_phys = swiglu ? 2 * c.d_ff : c.d_ff;
+  g1.b_rows_gate = swiglu ? c.d_ff : 0;
+  long long work = (long long)max_tiles * g1.n_col_tiles;
+  int grid = work > s.sm_count ? s.sm_count : (int)work;
+  cudaError_t e = swiglu ? launch_kernel(tc_gemm_f32_kernel<kTcEpiSwigluF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes,
+                                         st, pdl, s.map_xp, s.map_win, g1)
+                         : launch_kernel(tc_gemm_f32_kernel<kTcEpiReluF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes,
+                                         st, pdl, s.map_xp, s.map_win, g1);
+  if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
+  ++*launches;
+  if (between) cudaEventRecord(between, st);
+
+  // GEMM-2: few output tiles, long contraction: slice it until every SM has an item
+  const long long pairs = (long long)n_tokens * c.top_k;
+  const long long touched = pairs < c.K ? pairs : c.K;
+  const long long by_rows = pairs / kTcBM + touched / 2;
+  const long long row_tiles_est = touched > by_rows ? touched : by_rows;
+  const int n_col2 = c.d_model / kF32BN;
+  int split = 1;
+  while (split * 2 <= y_copies && row_tiles_est * n_col2 * split < s.sm_count &&
+         (c.d_ff / kF32BK) % (split * 2) == 0 && c.d_ff / kF32BK / (split * 2) >= 8)
+    split *= 2;
+  TcF32Args g2;
+  g2.C = y; g2.tiles = tiles; g2.n_tiles = n_tiles; g2.status = status; g2.split_stride = y_copy_stride;
+  g2.ldc = c.d_model; g2.n_col_tiles = n_col2; g2.k_blocks = c.d_ff / kF32BK / split; g2.n_split = split;
+  g2.b_rows_per_phys = c.d_model; g2.b_rows_gate = 0;
+  work = (long long)max_tiles * n_col2 * split;
+  grid = work > s.sm_count ? s.sm_count : (int)work;
+  e = launch_kernel(tc_gemm_f32_kernel<kTcEpiF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes, st,
+                    pdl && between == nullptr, s.map_h, s.map_wout, g2);
+  if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
+  ++*launches;
+  *y_split = split;
+  return SWAPMOE_OK;
+}
+
+}  // namespace swapmoe

@@ -136,6 +136,25 @@ def test_error_codes():
 
 
 # ------------------------------------------------------------------ the named configurations
+@pytest.mark.parametrize("path", ["tcgen05", "mma", "ffma"])
+def test_fp32_gemm_paths(monkeypatch, path):
+    """fp32 layers: split-TF32 on tcgen05 (default), the warp-level mma form (SWAPMOE_FP32_TC=0) and the
+    FFMA form (SWAPMOE_FP32_FFMA=1) all hold the fp32 tolerance; ReLU top-1 with a sliced GEMM-2 and
+    SwiGLU top-2, slots above and below one 128-row tile."""
+    from harness import Case, check_against_oracle
+    if path == "mma":
+        monkeypatch.setenv("SWAPMOE_FP32_TC", "0")
+    if path == "ffma":
+        monkeypatch.setenv("SWAPMOE_FP32_FFMA", "1")
+    for cfg in (_cfg(T=700, dtype=I.F32, d=256, f=512, E=8, K=3, zipf_s=1.2),
+                _cfg(T=300, dtype=I.F32, d=128, f=384, E=16, K=5, k=2, act=I.ACT_SWIGLU, renorm=1)):
+        case = Case(cfg)
+        n0 = case.layer.launch_count
+        res = check_against_oracle(case, case.run())
+        assert case.layer.launch_count - n0 == 5
+        assert res["out_rel_err"] <= 1e-4
+
+
 def test_cfg1_switch_fp32():
     from harness import Case, check_against_oracle
     case = Case(I.CONFIGS["cfg1"], s2e=[5, 0, 7, 2])       # fixed scrambled table
