@@ -9,11 +9,14 @@
 // rounding of lo are below 2^-20 relative.
 //
 // TMA brings the fp32 operands (k-blocks of 32 columns = 128-byte swizzled rows) into a ring of
-// raw stages.  The split is ELEMENTWISE, so it preserves the swizzled layout: four converter warps
-// rewrite a stage in place with its hi parts and write the lo parts at the same offsets of a "lo"
-// slot (two slots), fence towards the async proxy and arrive on `conv_done`; one thread then
-// issues the 12 MMAs of the k-block (4 steps of K = 8, three products each) and commits to the
-// barriers that free the raw stage and the lo slot.  Roles (384 threads): warp 0 TMA producer,
+// raw stages.  Four converter warps split a stage: the weight half elementwise (which preserves the
+// swizzled layout: hi parts in place, lo parts at the same offsets of one of two "lo" slots); the
+// activation half goes to TENSOR MEMORY: converter thread r owns row r, reads its 32 values and
+// writes hi and lo into 32 + 32 columns of TMEM lane r (`tcgen05.st`), so the MMAs take their A
+// operand from TMEM and read only B from shared memory (with both operands in shared memory a k-block
+// moved 224 KB through it and the kernel was bound by shared-memory bandwidth).  The converters
+// fence and arrive on `conv_done`; one thread then issues the 12 MMAs of the k-block (4 steps of
+// K = 8, three products each) and commits to the barriers that free the raw stage and the slot.  Roles (384 threads): warp 0 TMA producer,
 // warp 1 MMA issuer, warp 2 TMEM allocation, warps 4-7 epilogue (two accumulator sets, so it
 // overlaps the next item's MMAs), warps 8-11 converters.  A work item is (row tile, column tile,
 // contraction slice): GEMM-2 has few output tiles and a long contraction, so its slices go to
@@ -30,9 +33,11 @@ constexpr int kF32Threads = 384;
 constexpr int kF32ABytes = kTcBM * kF32BK * 4;      // 16 KB
 constexpr int kF32BBytes = kF32BN * kF32BK * 4;     // 16 KB
 constexpr int kF32StageBytes = kF32ABytes + kF32BBytes;
-constexpr int kF32Stages = 4;                       // raw stages (TMA targets; hold the hi parts after conversion)
-constexpr int kF32LoSlots = 2;
-constexpr int kF32SmemBytes = (kF32Stages + kF32LoSlots) * kF32StageBytes + 2048 + kTcEpiStageBytes;
+constexpr int kF32Stages = 5;                       // raw stages (TMA targets; the B half holds the hi parts after conversion)
+constexpr int kF32LoSlots = 2;                      // lo parts of B in shared memory; hi and lo of A in tensor memory
+constexpr int kF32SmemBytes = kF32Stages * kF32StageBytes + kF32LoSlots * kF32BBytes + 2048 + kTcEpiStageBytes;
+constexpr int kF32TmemAcc = 2 * kF32BN;             // columns of the two accumulator sets
+constexpr int kF32TmemCols = 512;                   // + 2 slots x (hi 32 + lo 32) columns of A, rounded up to a power of two
 
 // Epilogues of the fp32 path (values continue the bf16 kernels' enum)
 enum { kTcEpiReluF32 = 4, kTcEpiSwigluF32 = 5 };
@@ -56,6 +61,28 @@ __device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t desc_a, uint
       "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// A operand from tensor memory (lanes = rows, 32-bit columns = contraction index), B from shared memory.
+__device__ __forceinline__ void umma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n}\n" ::"r"(tmem_d),
+      "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 32 consecutive 32-bit columns of this thread's TMEM lane <- registers
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+      "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+      "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 }  // namespace ptx
 
 // Instruction descriptor: tf32 x tf32 -> fp32, both operands K-major, M x N tile.
@@ -94,15 +121,15 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   constexpr int kNB = (EPI == kTcEpiSwigluF32) ? 2 : 1;     // weight boxes per stage
   constexpr int kBoxRows = kF32BN / kNB;
   constexpr int kOutCols = kF32BN / kNB;
-  constexpr uint32_t kTmemCols = 2 * kF32BN;
+  constexpr uint32_t kTmemCols = kF32TmemCols;
   constexpr uint32_t kIdesc = make_idesc_tf32(kTcBM, kF32BN);
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   unsigned char* raw = smem;                                         // [stages][A 16 KB | B 16 KB]
-  unsigned char* lo = smem + kF32Stages * kF32StageBytes;            // [slots][A 16 KB | B 16 KB]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(lo + kF32LoSlots * kF32StageBytes);
+  unsigned char* lo = smem + kF32Stages * kF32StageBytes;            // [slots][B 16 KB]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(lo + kF32LoSlots * kF32BBytes);
   uint64_t* full = bars;                          // [stages]   TMA -> converters
   uint64_t* empty = full + kF32Stages;            // [stages]   MMA -> producer
   uint64_t* conv_done = empty + kF32Stages;       // [slots]    converters -> MMA (128 arrivals)
@@ -185,16 +212,15 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           ok = bounded_wait(&conv_done[slot], slot_phase, abort_flag, a.status, 33);
           if (!ok) break;
           ptx::tc_fence_after();
-          const uint32_t hi_a = ptx::smem_u32(raw + stage * kF32StageBytes), hi_b = hi_a + kF32ABytes;
-          const uint32_t lo_a = ptx::smem_u32(lo + slot * kF32StageBytes), lo_b = lo_a + kF32ABytes;
-          const uint64_t dha = make_kmajor_sw128_desc(hi_a), dhb = make_kmajor_sw128_desc(hi_b);
-          const uint64_t dla = make_kmajor_sw128_desc(lo_a), dlb = make_kmajor_sw128_desc(lo_b);
+          const uint64_t dhb = make_kmajor_sw128_desc(ptx::smem_u32(raw + stage * kF32StageBytes + kF32ABytes));
+          const uint64_t dlb = make_kmajor_sw128_desc(ptx::smem_u32(lo + slot * kF32BBytes));
+          const uint32_t a_hi = tmem_base + (uint32_t)(kF32TmemAcc + slot * 2 * kF32BK), a_lo = a_hi + kF32BK;
 #pragma unroll
           for (int k = 0; k < kF32BK / kF32UmmaK; ++k) {
-            // 8 fp32 along K inside the swizzled row = +32 bytes = +2 in the address field; small terms first
-            ptx::umma_tf32(tmem_d, dla + (uint64_t)(2 * k), dhb + (uint64_t)(2 * k), kIdesc, (kb > 0 || k > 0) ? 1u : 0u);
-            ptx::umma_tf32(tmem_d, dha + (uint64_t)(2 * k), dlb + (uint64_t)(2 * k), kIdesc, 1u);
-            ptx::umma_tf32(tmem_d, dha + (uint64_t)(2 * k), dhb + (uint64_t)(2 * k), kIdesc, 1u);
+            // 8 fp32 along K: +32 bytes = +2 in the address field of B, +8 columns of A; small terms first
+            ptx::umma_tf32_ts(tmem_d, a_lo + 8 * k, dhb + (uint64_t)(2 * k), kIdesc, (kb > 0 || k > 0) ? 1u : 0u);
+            ptx::umma_tf32_ts(tmem_d, a_hi + 8 * k, dlb + (uint64_t)(2 * k), kIdesc, 1u);
+            ptx::umma_tf32_ts(tmem_d, a_hi + 8 * k, dhb + (uint64_t)(2 * k), kIdesc, 1u);
           }
           ptx::umma_commit(&empty[stage]);       // the raw stage may be refilled
           ptx::umma_commit(&lo_empty[slot]);     // the lo slot may be rewritten
@@ -217,10 +243,30 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         ok = bounded_wait(&full[stage], phase, abort_flag, a.status, 34);
         if (ok) ok = bounded_wait(&lo_empty[slot], slot_phase ^ 1u, abort_flag, a.status, 35);
         if (!ok) break;
-        uint4* src = reinterpret_cast<uint4*>(raw + stage * kF32StageBytes);
-        uint4* dst = reinterpret_cast<uint4*>(lo + slot * kF32StageBytes);
+        ptx::tc_fence_after();
+        {
+          // A: thread = row (= TMEM lane); its 32 values sit in eight 16-byte pieces, piece j at (j ^ (row & 7))
+          const unsigned char* arow = raw + stage * kF32StageBytes + ctid * 128;
+          uint32_t h[32], l[32];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint4 x = *reinterpret_cast<const uint4*>(arow + ((j ^ (ctid & 7)) << 4));
+            const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              h[4 * j + e] = xs[e] & 0xffffe000u;
+              l[4 * j + e] = __float_as_uint(__uint_as_float(xs[e]) - __uint_as_float(h[4 * j + e]));
+            }
+          }
+          const uint32_t ta = tmem_base + ((uint32_t)((ctid >> 5) * 32) << 16) + (uint32_t)(kF32TmemAcc + slot * 2 * kF32BK);
+          ptx::tmem_st32(ta, h);
+          ptx::tmem_st32(ta + kF32BK, l);
+        }
+        // B: elementwise at identical offsets (keeps the swizzled layout): hi in place, lo into the slot
+        uint4* src = reinterpret_cast<uint4*>(raw + stage * kF32StageBytes + kF32ABytes);
+        uint4* dst = reinterpret_cast<uint4*>(lo + slot * kF32BBytes);
 #pragma unroll 4
-        for (int i = ctid; i < kF32StageBytes / 16; i += 128) {
+        for (int i = ctid; i < kF32BBytes / 16; i += 128) {
           const uint4 x = src[i];
           uint4 h, l;
           h.x = x.x & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(x.x) - __uint_as_float(h.x));
@@ -230,6 +276,8 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           src[i] = h;
           dst[i] = l;
         }
+        ptx::tmem_st_wait();
+        ptx::tc_fence_before();
         ptx::fence_proxy_async();                // these writes are read by the tensor core (async proxy)
         ptx::mbar_arrive(&conv_done[slot]);
         if (++stage == kF32Stages) { stage = 0; phase ^= 1u; }
