@@ -33,8 +33,8 @@ from paper_2308_15030_b200 import inputs as I  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the grouped-GEMM kernel, mean of the
 # GEMM-1 and GEMM-2 launches of one step, from the ncu capture summarised in
-# profiles/cfg2_router_tc_permute_tc_gemm.md (80.04 + 3.42 MB and 93.63 + 3.44 MB).
-NCU_TRAFFIC_PER_LAUNCH = {"cfg2": (80.04e6 + 3.42e6 + 93.63e6 + 3.44e6) / 2}
+# profiles/cfg2_router_permute_tc_gemm.md (80.07 + 5.99 MB and 93.63 + 3.65 MB).
+NCU_TRAFFIC_PER_LAUNCH = {"cfg2": (80.07e6 + 5.99e6 + 93.63e6 + 3.65e6) / 2}
 
 METRIC = "moe_layer_tokens_per_s_at_budget_K"
 UNIT = "tokens/s"
