@@ -251,9 +251,12 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
       rc = tc_ffn_fused(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->done, L->row_pair, L->mgate, max_tiles,
                         L->status, st, pdl, &L->launches, &combined);
       if (mid) cudaEventRecord(mid, st);      // one kernel: the GEMM-2 stage reads as zero
-    } else if (mt == 2 && use_pairs) {
+    } else if (mt == 2 && L->gemm_pairs > 0 && c.d_ff % 256 == 0) {
+      // 256-row tiles: GEMM-1 always on CTA pairs (its one-CTA form pulls 48 KB per k-block); GEMM-2 on pairs for
+      // very large slots, else on one CTA with two row sub-tiles (same bytes per flop, and a tile whose second
+      // half is empty costs half; cfg3: 128.6 -> 126.8 us)
       rc = tc_ffn_pair(L->tc, L->gemm_pairs, c, L->h, L->y, out, L->tiles, L->n_tiles, L->row_pair, L->mgate, max_tiles,
-                       T, L->status, st, pdl, &L->launches, &combined, mid);
+                       T, L->status, st, pdl, &L->launches, &combined, mid, use_pairs);
     } else {
       rc = tc_ffn(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->tiles_b, L->n_tiles_b, L->row_pair, L->mgate,
                   max_tiles, mt, T,

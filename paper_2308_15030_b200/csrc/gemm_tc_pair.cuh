@@ -308,7 +308,7 @@ inline int tc_pair_init(int sm_count) {
 inline int32_t tc_ffn_pair(TcState& s, int n_pairs, const swapmoe_config_t& c, void* h, float* y, void* out,
                            const TileDesc* tiles, const int32_t* n_tiles, const int32_t* row_pair, const float* mgate,
                            int max_tiles, int n_tokens, int32_t* status, cudaStream_t st, bool pdl, int64_t* launches,
-                           bool* combined, cudaEvent_t between = nullptr) {
+                           bool* combined, cudaEvent_t between = nullptr, bool gemm2_pairs = true) {
   if (!s.enabled || !s.arena_bound || n_pairs < 1) return SWAPMOE_ERR_NOT_READY;
   const bool swiglu = c.act == SWAPMOE_ACT_SWIGLU;
   const bool scatter = c.top_k == 1;
@@ -356,6 +356,19 @@ inline int32_t tc_ffn_pair(TcState& s, int n_pairs, const swapmoe_config_t& c, v
   work = (long long)max_tiles * g2.n_col_tiles;
   grid = 2 * (work > n_pairs ? n_pairs : (int)work);
   const bool pdl2 = pdl && between == nullptr;
+  if (!gemm2_pairs) {
+    // one CTA per 256-row tile with two row sub-tiles: the same operand bytes per flop as a pair, and a tile whose
+    // second half is empty costs half
+    g2.a_box_bytes = kTcBM * kTcBK * 2;
+    grid = work > s.sm_count ? s.sm_count : (int)work;
+    const TcGemmKernel k = scatter ? tc_gemm_kernel<256, kTcEpiScatterBf16, 2> : tc_gemm_kernel<256, kTcEpiF32, 2>;
+    if (launch_kernel(k, dim3(grid), dim3(kTcThreads), TcSmem<256, 2>::kBytes, st, pdl2, s.map_h[0], s.map_wout[0], g2) !=
+        cudaSuccess)
+      return SWAPMOE_ERR_CUDA;
+    ++*launches;
+    *combined = scatter;
+    return SWAPMOE_OK;
+  }
   e = scatter ? launch_kernel(tc_gemm_pair_kernel<kTcEpiScatterBf16>, dim3(grid), dim3(kTcThreads), kPairSmemBytes, st, pdl2,
                               s.map_h[0], s.map_wout[1], g2)
               : launch_kernel(tc_gemm_pair_kernel<kTcEpiF32>, dim3(grid), dim3(kTcThreads), kPairSmemBytes, st, pdl2,

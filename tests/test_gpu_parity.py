@@ -213,8 +213,9 @@ def test_fused_ffn_kernel_option(monkeypatch):
 
 
 def test_two_row_subtiles_per_cta():
-    """Slots with 160..1023 rows on average take the kernels that share a weight tile between two
-    128-row sub-tiles; include slots above and below 128 rows and a ragged last sub-tile."""
+    """Slots with 160..1023 rows on average run on 256-row tiles: GEMM-1 on CTA pairs, GEMM-2 on one CTA that
+    shares a weight tile between two 128-row sub-tiles; include slots above and below 128 rows and a ragged
+    last sub-tile."""
     import oracle
     from harness import Case, check_against_oracle
     for k, act, renorm in ((1, I.ACT_RELU, 0), (2, I.ACT_SWIGLU, 1)):
