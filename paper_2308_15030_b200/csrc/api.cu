@@ -73,6 +73,7 @@ struct swapmoe_layer {
   int32_t router_tok;          // 0 = automatic token-tile size of the tensor-core router, else 32/64/128
   bool prefetch;               // pull resident weights into L2 from the router kernel
   long long l2_prefetch_bytes; // how much of them (L2 capacity minus head room)
+  int prefetch_min_pairs;      // ... when the batch has at least this many HALF pairs per slot (SWAPMOE_PREFETCH_MIN_PAIRS)
   void* const* stage_events;   // 7 cudaEvent_t of the forward being enqueued, or nullptr
   CUtensorMap map_x;           // TMA view of the last token matrix [T, d]
   const void* map_x_ptr;
@@ -177,10 +178,10 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   ra.pf_total_bytes[0] = ra.pf_total_bytes[1] = 0;
   ra.pf_phys = L->phys;
   int pf_ctas = 0;
-  if (tc_router && use_tc && L->prefetch && n_pairs >= 8 * c.K &&
-      (long long)c.K * (L->nin + 1) * c.d_ff * c.d_model * (long long)L->elem <= (256ll << 20)) {
-    // Every slot will most likely be touched: pull the resident weights towards L2 now, while the
-    // router and the permutation leave HBM idle.  GEMM-1's matrices first, then as much of GEMM-2's
+  if (tc_router && use_tc && L->prefetch && 2 * n_pairs >= L->prefetch_min_pairs * c.K &&
+      (long long)c.K * (L->nin + 1) * c.d_ff * c.d_model * (long long)L->elem <= (320ll << 20)) {
+    // Most slots will be touched (at least half a pair per slot): pull the resident weights towards L2 now,
+    // while the router and the permutation leave HBM idle (a slot that stays untouched costs idle bandwidth only).  GEMM-1's matrices first, then as much of GEMM-2's
     // as the L2 budget allows.
     const long long in_slot = (long long)L->nin * c.d_ff * c.d_model * L->elem;
     const long long out_slot = (long long)c.d_ff * c.d_model * L->elem;
@@ -390,6 +391,8 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
     L->l2_prefetch_bytes = l2 > (80ll << 20) ? (56ll << 20) : 0;
     env = std::getenv("SWAPMOE_PREFETCH_MB");
     if (env) L->l2_prefetch_bytes = std::atoll(env) << 20;
+    env = std::getenv("SWAPMOE_PREFETCH_MIN_PAIRS");
+    L->prefetch_min_pairs = env ? std::max(1, std::atoi(env)) : 1;
   }
   L->nin = c.act == SWAPMOE_ACT_SWIGLU ? 2 : 1;
   L->elem = c.dtype == SWAPMOE_BF16 ? 2 : 4;
