@@ -23,6 +23,7 @@
 #include "router_gate.cuh"
 #include "router_tc.cuh"
 #include "router_small.cuh"
+#include "router_small_f32.cuh"
 
 using namespace swapmoe;
 
@@ -57,6 +58,7 @@ struct swapmoe_layer {
   int32_t rows_pad_max;
   int pair_min_rows;           // ... used when the slots hold at least this many rows on average (SWAPMOE_PAIR_MIN_ROWS)
   int gemm_pairs;              // CTA pairs available to the cta_group::2 grouped GEMM (0: not used; SWAPMOE_PAIR_GEMM=0)
+  bool small_router_f32;       // fp32 layers: eight-token CTAs of the split-TF32 mma router (SWAPMOE_SMALL_ROUTER=0: never)
   bool small_router;           // eight-token mma router CTAs for batches of up to 64 tokens (bf16)
   int32_t small_router_max_t;  // ... and sixteen-token CTAs up to this many tokens (0: never)
   bool decode_path;            // one-launch forward for a handful of tokens (bf16)
@@ -146,6 +148,9 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   int tok_tile = tc_router ? router_tc_tok(T) : kTokTile;
   if (tc_router && L->router_tok) tok_tile = L->router_tok;
   if (small_router) tok_tile = kRsTok * rs_nt;
+  // fp32 layers: eight-token CTAs of the split-TF32 mma router while they fit one wave of CTAs
+  const bool small_f32 = L->small_router_f32 && ext_logits == nullptr && T <= kRsTok * std::min(L->sm_count, 256);
+  if (small_f32) tok_tile = kRsTok;
   const int n_cta = (T + tok_tile - 1) / tok_tile;
   const int n_pairs = T * c.top_k;
   const bool use_tc = tc_selected(L->gemm_path, c, T);
@@ -214,6 +219,10 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     if (launch_kernel(router_tc_kernel, dim3(n_cta + pf_ctas), dim3(kRtThreads), router_tc_smem_bytes(c.E, tok_tile),
                       st, pdl, L->map_x, L->tc.map_wr, ra, L->status, router_tc_stages(c.E, tok_tile), tok_tile) !=
         cudaSuccess)
+      return SWAPMOE_ERR_CUDA;
+  } else if (small_f32) {
+    if (launch_kernel(router_small_f32_kernel, dim3(n_cta), dim3(kDecThreads), router_small_f32_smem_bytes(c.d_model), st,
+                      pdl, ra, L->status) != cudaSuccess)
       return SWAPMOE_ERR_CUDA;
   } else {
     if (launch_kernel(router_gate_fn<DT>(c.E), dim3(n_cta), dim3(256), router_smem_bytes(c.E), st, pdl, ra) !=
@@ -405,6 +414,8 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
     if (small > n_cta) n_cta = small;
     const size_t mid = std::min<size_t>((T + 2 * kRsTok - 1) / (2 * kRsTok), 256);   // sixteen-token CTAs
     if (mid > n_cta) n_cta = mid;
+    const size_t f32small = std::min<size_t>((T + kRsTok - 1) / kRsTok, 256);         // fp32: eight-token CTAs, one wave
+    if (c.dtype == SWAPMOE_F32 && f32small > n_cta) n_cta = f32small;
   }
   const size_t rows_pad = align_up(P + (size_t)c.K * kSegAlign, kSegAlign);
   const size_t max_tiles = (P + kSimtBM - 1) / kSimtBM + c.K;
@@ -514,6 +525,11 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
     if (L->small_router)
       ok = ok && cuda_ok(cudaFuncSetAttribute(router_small_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)router_small_smem_bytes(c.d_model, 1)));
+    L->small_router_f32 = c.dtype == SWAPMOE_F32 && !(env && env[0] == '0') &&
+                          router_small_f32_smem_bytes(c.d_model) <= (size_t)(226 << 10);
+    if (L->small_router_f32)
+      ok = ok && cuda_ok(cudaFuncSetAttribute(router_small_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)router_small_f32_smem_bytes(c.d_model)));
     // sixteen-token CTAs: while the grid stays within one wave of CTAs and the shared memory fits
     L->small_router_max_t = 0;
     if (L->small_router && router_small_smem_bytes(c.d_model, 2) <= (size_t)(226 << 10)) {
