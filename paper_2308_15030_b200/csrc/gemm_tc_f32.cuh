@@ -16,9 +16,9 @@
 // operand from TMEM and read only B from shared memory (with both operands in shared memory a k-block
 // moved 224 KB through it and the kernel was bound by shared-memory bandwidth).  The converters
 // fence and arrive on `conv_done`; one thread then issues the 12 MMAs of the k-block (4 steps of
-// K = 8, three products each) and commits to the barriers that free the raw stage and the slot.  Roles (384 threads): warp 0 TMA producer,
+// K = 8, three products each) and commits to the barriers that free the raw stage and the slot.  Roles (512 threads): warp 0 TMA producer,
 // warp 1 MMA issuer, warp 2 TMEM allocation, warps 4-7 epilogue (two accumulator sets, so it
-// overlaps the next item's MMAs), warps 8-11 converters.  A work item is (row tile, column tile,
+// overlaps the next item's MMAs), warps 8-11 and 12-15 two converter groups (one per lo slot).  A work item is (row tile, column tile,
 // contraction slice): GEMM-2 has few output tiles and a long contraction, so its slices go to
 // separate copies of y that the combine kernel adds in order (deterministic).
 #pragma once
@@ -29,7 +29,7 @@ namespace swapmoe {
 constexpr int kF32BK = 32;                          // fp32 elements per k-block = one 128-byte swizzled row
 constexpr int kF32UmmaK = 8;
 constexpr int kF32BN = 128;                         // accumulator columns per tile
-constexpr int kF32Threads = 384;
+constexpr int kF32Threads = 512;
 constexpr int kF32ABytes = kTcBM * kF32BK * 4;      // 16 KB
 constexpr int kF32BBytes = kF32BN * kF32BK * 4;     // 16 KB
 constexpr int kF32StageBytes = kF32ABytes + kF32BBytes;
@@ -234,12 +234,20 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     }
   } else if (warp >= 8) {
     // ---------------------------------------------------------------------- converters: hi in place, lo beside
-    const int ctid = threadIdx.x - 8 * 32;       // 0..127
+    // two groups of four warps: group g converts the k-blocks that use lo slot g (every other one), so two
+    // conversions are in flight; both groups walk all k-blocks to keep stage and phase counters in step
+    const int grp = (warp - 8) >> 2;
+    const int ctid = (threadIdx.x - 8 * 32) & 127;   // 0..127 inside the group = row = TMEM lane
     int stage = 0, slot = 0;
     uint32_t phase = 0, slot_phase = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
       for (int kb = 0; kb < a.k_blocks; ++kb) {
+        if (slot != grp) {
+          if (++stage == kF32Stages) { stage = 0; phase ^= 1u; }
+          if (++slot == kF32LoSlots) { slot = 0; slot_phase ^= 1u; }
+          continue;
+        }
         ok = bounded_wait(&full[stage], phase, abort_flag, a.status, 34);
         if (ok) ok = bounded_wait(&lo_empty[slot], slot_phase ^ 1u, abort_flag, a.status, 35);
         if (!ok) break;
