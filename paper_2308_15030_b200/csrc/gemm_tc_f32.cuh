@@ -160,6 +160,29 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // As in tc_gemm_kernel: the tile list (written by the router, two or more kernels back) and the weights do not
+  // depend on the kernel in front, so the producer requests the weight boxes of its first stages before the
+  // dependent-launch wait; only the activations have to wait.
+  int pre = 0;
+  if (warp == 0 && lane == 0) {
+    const int n_rt = __ldcg(a.n_tiles);
+    const int per = n_rt * a.n_col_tiles;
+    if ((int)blockIdx.x < per * a.n_split) {
+      const int z = (int)blockIdx.x / per, u = (int)blockIdx.x - z * per;
+      const int ct = u / n_rt, rt = u - ct * n_rt;
+      const int4 rawd = __ldcg(reinterpret_cast<const int4*>(a.tiles + rt));
+      const TileDesc td = *reinterpret_cast<const TileDesc*>(&rawd);
+      const int brow = td.phys * a.b_rows_per_phys + ct * kBoxRows;
+      pre = a.k_blocks < kF32Stages ? a.k_blocks : kF32Stages;
+      for (int kb = 0; kb < pre; ++kb) {
+        ptx::mbar_expect_tx(&full[kb], (uint32_t)kF32StageBytes);
+#pragma unroll
+        for (int j = 0; j < kNB; ++j)
+          ptx::tma_load_2d(raw + kb * kF32StageBytes + kF32ABytes + j * kBoxRows * kF32BK * 4, &tmB, &full[kb],
+                           (z * a.k_blocks + kb) * kF32BK, brow + j * a.b_rows_gate);
+      }
+    }
+  }
   pdl_wait();
   pdl_trigger();
   const int n_row_tiles = *a.n_tiles;
@@ -179,15 +202,20 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         const int brow = td.phys * a.b_rows_per_phys + ct * kBoxRows;
         const int kb0 = z * a.k_blocks;
         for (int kb = 0; kb < a.k_blocks; ++kb) {
-          ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 31);
-          if (!ok) break;
+          const bool early = t == (int)blockIdx.x && kb < pre;   // armed and weights requested above
           unsigned char* sA = raw + stage * kF32StageBytes;
-          ptx::mbar_expect_tx(&full[stage], (uint32_t)kF32StageBytes);
+          if (!early) {
+            ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 31);
+            if (!ok) break;
+            ptx::mbar_expect_tx(&full[stage], (uint32_t)kF32StageBytes);
+          }
           ptx::tma_load_2d(sA, &tmA, &full[stage], (kb0 + kb) * kF32BK, td.row0);
+          if (!early) {
 #pragma unroll
-          for (int j = 0; j < kNB; ++j)
-            ptx::tma_load_2d(sA + kF32ABytes + j * kBoxRows * kF32BK * 4, &tmB, &full[stage], (kb0 + kb) * kF32BK,
-                             brow + j * a.b_rows_gate);
+            for (int j = 0; j < kNB; ++j)
+              ptx::tma_load_2d(sA + kF32ABytes + j * kBoxRows * kF32BK * 4, &tmB, &full[stage], (kb0 + kb) * kF32BK,
+                               brow + j * a.b_rows_gate);
+          }
           if (++stage == kF32Stages) { stage = 0; phase ^= 1u; }
         }
       }
