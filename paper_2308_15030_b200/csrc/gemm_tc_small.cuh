@@ -80,11 +80,28 @@ tc_gemm_small_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  const int n_chunks = a.k_blocks / kps;
+  // As in tc_gemm_kernel: the tile list and the weights do not depend on the kernel in front, so the producer
+  // requests the weight boxes of its first stages before the dependent-launch wait.
+  int pre = 0;
+  if (warp == 0 && lane == 0) {
+    const int n_rt = __ldcg(a.n_tiles);
+    if ((int)blockIdx.x < n_rt * a.n_col_tiles) {
+      const int ct = (int)blockIdx.x / n_rt, rt = (int)blockIdx.x - ct * n_rt;
+      const int4 rawd = __ldcg(reinterpret_cast<const int4*>(a.tiles + rt));
+      const TileDesc td = *reinterpret_cast<const TileDesc*>(&rawd);
+      const int brow = td.phys * a.b_rows_per_phys + ct * BN;
+      pre = n_chunks < n_stages ? n_chunks : n_stages;
+      for (int c = 0; c < pre; ++c) {
+        ptx::mbar_expect_tx(&full[c], (uint32_t)(stage_a + stage_b));
+        tma_load_3d(sB + c * stage_b, &tmB, &full[c], 0, brow, c * kps);
+      }
+    }
+  }
   pdl_wait();
   pdl_trigger();
   const int n_row_tiles = *a.n_tiles;
   const int total = n_row_tiles * a.n_col_tiles;
-  const int n_chunks = a.k_blocks / kps;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -97,11 +114,14 @@ tc_gemm_small_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const TileDesc td = a.tiles[rt];
         const int brow = td.phys * a.b_rows_per_phys + ct * BN;
         for (int c = 0; c < n_chunks; ++c) {
-          ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 31);
-          if (!ok) break;
-          ptx::mbar_expect_tx(&full[stage], (uint32_t)(stage_a + stage_b));
+          const bool early = t == (int)blockIdx.x && c < pre;    // armed and weights requested above
+          if (!early) {
+            ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 31);
+            if (!ok) break;
+            ptx::mbar_expect_tx(&full[stage], (uint32_t)(stage_a + stage_b));
+          }
           tma_load_3d(sA + stage * stage_a, &tmA, &full[stage], 0, td.row0, c * kps);
-          tma_load_3d(sB + stage * stage_b, &tmB, &full[stage], 0, brow, c * kps);
+          if (!early) tma_load_3d(sB + stage * stage_b, &tmB, &full[stage], 0, brow, c * kps);
           if (++stage == n_stages) { stage = 0; phase ^= 1u; }
         }
       }
