@@ -21,6 +21,8 @@ SMALL = [
     _cfg(T=513, d=256, f=512, E=64, K=64, k=1, zipf_s=1.1),          # K = E: unrestricted layer
     _cfg(T=64, d=128, f=128, E=1, K=1, k=1),                          # dense MLP
     _cfg(T=12000, dtype=I.F32, d=128, f=128, E=8, K=4),               # fp32 with enough tiles that GEMM-2 is not sliced
+    _cfg(T=500, dtype=I.F32, d=64, f=64, E=256, K=33, k=4, renorm=1, zipf_s=1.1),   # fp32 small-batch router, 8 waves of Wr
+    _cfg(T=203, dtype=I.F32, d=384, f=256, E=40, K=7, k=2, renorm=0),               # ragged E, last CTA with 3 tokens
 ]
 
 
