@@ -154,7 +154,10 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_f32_kernel(const 
       }
     }
   }
-  if (tid < kMaxE) R->e2s[tid] = tid < E ? a.e2s[tid] : -1;
+  if (tid < kMaxE) {
+    R->e2s[tid] = tid < E ? a.e2s[tid] : -1;
+    Q->enorm[tid] = tid < E ? a.enorm[tid] : 0.f;
+  }
   __syncthreads();
   if (warp < T) {
     float ss = 0.f;
@@ -176,23 +179,24 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_f32_kernel(const 
       issue_router_wave(w + 2);
     }
   }
+  if (!alive)
+    for (int i = tid; i < TOK * (kMaxE + 1); i += kDecThreads) slog[i] = 0.f;
   __syncthreads();
   // gates: task = (token, pass); pass 0 the off-the-shelf gate, pass 1 the masked one; 2 TOK tasks over 16 warps
 #pragma unroll 1
   for (int task = warp; task < 2 * TOK; task += kDecWarps) {
     const int t = task & (TOK - 1), pass = task / TOK;
     if (t >= T) continue;
-    float v[8];
+    const int ei = (E + 31) >> 5;
     uint32_t allow = 0u;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
+#pragma unroll 1
+    for (int i = 0; i < ei; ++i) {
       const int e = lane + 32 * i;
-      v[i] = (e < E && alive) ? slog[t * (kMaxE + 1) + e] : (e < E ? 0.f : -INFINITY);
       if (e < E && (pass == 0 || R->e2s[e] >= 0)) allow |= 1u << i;
     }
     int se[kMaxTopK];
     float sg[kMaxTopK];
-    dec_topk_gate(v, allow, k, a.renorm, lane, se, sg);
+    dec_topk_gate(slog + t * (kMaxE + 1), allow, ei, k, a.renorm, lane, se, sg);
     if (lane == 0) {
       const float xn = Q->xn[t];
 #pragma unroll
@@ -204,12 +208,12 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_f32_kernel(const 
           if (pass == 0) {
             Q->ue[p] = se[j];
             a.uidx[gp] = se[j]; a.ugate[gp] = gv;
-            Q->pt[p] = xn * fabsf(gv) * a.enorm[se[j]];
+            Q->pt[p] = xn * fabsf(gv) * Q->enorm[se[j]];
           } else {
             const int sl = R->e2s[se[j]];
             Q->sl[p] = sl;
             a.midx[gp] = se[j]; a.mgate[gp] = gv; a.slot[gp] = sl;
-            Q->pm[p] = xn * fabsf(gv) * a.enorm[se[j]];
+            Q->pm[p] = xn * fabsf(gv) * Q->enorm[se[j]];
           }
         }
       }
