@@ -233,6 +233,33 @@ def test_two_row_subtiles_per_cta():
         assert cnt.max() > 256 and any(0 < c % 256 <= 128 for c in cnt), cnt
 
 
+@pytest.mark.parametrize("dtype", [I.BF16, I.F32])
+def test_back_to_back_forwards_with_changing_batches(dtype):
+    """Forwards of different batches queued back to back on one stream (no synchronisation in between, so the
+    kernels overlap through programmatic dependent launch and the grouped GEMMs read the tile list and request
+    their first weight boxes before their dependent-launch wait): every output must equal, bit for bit, what the
+    same batch gives when it runs alone."""
+    import torch
+    from harness import Case, to_host_f32
+    sizes = (1500, 400, 1100, 8, 1500, 64)
+    base = _cfg(T=1500, dtype=dtype, d=256, f=512, E=16, K=5, zipf_s=1.2)
+    s2e = [3, 7, 0, 12, 9]
+    shared = Case(base, s2e=s2e)
+    alone, outs = [], []
+    for T in sizes:
+        c = Case(_cfg(T=T, dtype=dtype, d=256, f=512, E=16, K=5, zipf_s=1.2), s2e=s2e)
+        alone.append((c, c.run()))
+        outs.append(torch.full((T, base.d), float("nan"), dtype=c.d_x.dtype, device="cuda"))
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for (c, _), o in zip(alone, outs):
+            shared.layer.forward(c.d_x, o, n_tokens=c.T)
+    torch.cuda.synchronize()
+    assert shared.layer.device_status() == (0, 0)
+    for (c, ref), o in zip(alone, outs):
+        assert np.array_equal(to_host_f32(o), ref), c.T
+
+
 @pytest.mark.parametrize("min_rows", [None, "160"])
 def test_cta_pair_grouped_gemm(monkeypatch, min_rows):
     """Slots of 1024+ rows on average run the grouped GEMMs on CTA pairs (one 256-row tile per two SMs,
