@@ -134,6 +134,74 @@ __device__ __forceinline__ void dec_topk_gate(const float* row, uint32_t allow, 
     if (j < k) sel_g[j] = expf(sel_v[j] - m) / den;
 }
 
+// The off-the-shelf gate (allow[0]) and the masked gate (allow[1]) of one token in one pass: the two selections
+// are independent instruction streams that the scheduler interleaves, so a warp that owns both gates of a token
+// needs little more time than for one (a gate is a chain of dependent shuffles and exponentials, not work).
+__device__ __forceinline__ void dec_topk_gate2(const float* row, const uint32_t (&allow)[2], int ei, int k, int renorm,
+                                               int lane, int (&sel_e)[2][kMaxTopK], float (&sel_g)[2][kMaxTopK]) {
+  float sel_v[2][kMaxTopK];
+  uint32_t avail[2] = {allow[0], allow[1]};
+#pragma unroll
+  for (int j = 0; j < kMaxTopK; ++j) {
+#pragma unroll
+    for (int p = 0; p < 2; ++p) { sel_e[p][j] = 0; sel_g[p][j] = 0.f; sel_v[p][j] = 0.f; }
+    if (j < k) {
+      float bv[2] = {-INFINITY, -INFINITY};
+      int be[2] = {0x7fffffff, 0x7fffffff};
+#pragma unroll 1
+      for (int i = 0; i < ei; ++i) {
+        const float x = row[lane + 32 * i];
+#pragma unroll
+        for (int p = 0; p < 2; ++p)
+          if (((avail[p] >> i) & 1u) && (be[p] == 0x7fffffff || x > bv[p])) { bv[p] = x; be[p] = lane + 32 * i; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        float ov[2];
+        int oe[2];
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+          ov[p] = __shfl_xor_sync(0xffffffffu, bv[p], o);
+          oe[p] = __shfl_xor_sync(0xffffffffu, be[p], o);
+        }
+#pragma unroll
+        for (int p = 0; p < 2; ++p)
+          if (oe[p] != 0x7fffffff && (be[p] == 0x7fffffff || ov[p] > bv[p] || (ov[p] == bv[p] && oe[p] < be[p]))) {
+            bv[p] = ov[p]; be[p] = oe[p];
+          }
+      }
+#pragma unroll
+      for (int p = 0; p < 2; ++p) {
+        sel_e[p][j] = be[p]; sel_v[p][j] = bv[p];
+        if ((be[p] & 31) == lane) avail[p] &= ~(1u << (be[p] >> 5));
+      }
+    }
+  }
+  const float m[2] = {sel_v[0][0], sel_v[1][0]};
+  float den[2] = {0.f, 0.f};
+  if (renorm) {
+#pragma unroll
+    for (int j = 0; j < kMaxTopK; ++j)
+      if (j < k) { den[0] += expf(sel_v[0][j] - m[0]); den[1] += expf(sel_v[1][j] - m[1]); }
+  } else {
+#pragma unroll 1
+    for (int i = 0; i < ei; ++i) {
+      const float x = row[lane + 32 * i];
+#pragma unroll
+      for (int p = 0; p < 2; ++p)
+        if ((allow[p] >> i) & 1u) den[p] += expf(x - m[p]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      den[0] += __shfl_xor_sync(0xffffffffu, den[0], o);
+      den[1] += __shfl_xor_sync(0xffffffffu, den[1], o);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < kMaxTopK; ++j)
+    if (j < k) { sel_g[0][j] = expf(sel_v[0][j] - m[0]) / den[0]; sel_g[1][j] = expf(sel_v[1][j] - m[1]) / den[1]; }
+}
+
 // Routing state of the launch, identical in every CTA (shared memory).
 struct DecRoute {
   int ue[kDecMaxPairs], me[kDecMaxPairs], sl[kDecMaxPairs];   // per pair p = t*k + j

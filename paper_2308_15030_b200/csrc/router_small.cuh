@@ -203,6 +203,44 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
   if (!alive)
     for (int i = tid; i < TOK * (kMaxE + 1); i += kDecThreads) slog[i] = 0.f;
   __syncthreads();
+  if constexpr (NT == 2) {
+    // sixteen tokens, sixteen warps: a warp computes both gates of its token in one interleaved pass
+    const int t = warp;
+    if (t < T) {
+      const int ei = (E + 31) >> 5;
+      uint32_t allow[2] = {0u, 0u};
+#pragma unroll 1
+      for (int i = 0; i < ei; ++i) {
+        const int e = lane + 32 * i;
+        if (e < E) {
+          allow[0] |= 1u << i;
+          if (R->e2s[e] >= 0) allow[1] |= 1u << i;
+        }
+      }
+      int se[2][kMaxTopK];
+      float sg[2][kMaxTopK];
+      dec_topk_gate2(slog + t * (kMaxE + 1), allow, ei, k, a.renorm, lane, se, sg);
+      if (lane == 0) {
+        const float xn = Q->xn[t];
+#pragma unroll
+        for (int j = 0; j < kMaxTopK; ++j) {
+          if (j < k) {
+            const int p = t * k + j;
+            const size_t gp = (size_t)(tok0 + t) * k + j;
+            const float gu = alive ? sg[0][j] : 0.f, gm = alive ? sg[1][j] : 0.f;
+            const int sl = R->e2s[se[1][j]];
+            Q->ue[p] = se[0][j];
+            a.uidx[gp] = se[0][j]; a.ugate[gp] = gu;
+            Q->pt[p] = xn * fabsf(gu) * Q->enorm[se[0][j]];
+            Q->sl[p] = sl;
+            a.midx[gp] = se[1][j]; a.mgate[gp] = gm; a.slot[gp] = sl;
+            Q->pm[p] = xn * fabsf(gm) * Q->enorm[se[1][j]];
+          }
+        }
+        a.xnorm[tok0 + t] = xn;
+      }
+    }
+  } else {
   // gates: task = (token, pass); pass 0 the off-the-shelf gate, pass 1 the masked one; 2 TOK tasks over 16 warps
 #pragma unroll 1
   for (int task = warp; task < 2 * TOK; task += kDecWarps) {
@@ -240,6 +278,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
       }
       if (pass == 0) a.xnorm[tok0 + t] = xn;
     }
+  }
   }
 #pragma unroll 1
   for (int i = tid; i < T * E; i += kDecThreads) {
