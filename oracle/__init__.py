@@ -134,6 +134,20 @@ def topk_importance(imp, K):
     return out
 
 
+def expert_hidden(x, slot, phys_slot, arena_in, *, k, act, token_subset=None):
+    """h[p, :] = act(W_in[slot[p]] x[p // k]) for every pair p in flat (token, j) order; rows of
+    tokens outside ``token_subset`` stay zero."""
+    x, arena_in = _f32(x), _f32(arena_in)
+    T, d = x.shape
+    f = arena_in.shape[2]
+    slot, phys = _i32(slot).reshape(-1), _i32(phys_slot)
+    sub = _i32(token_subset)
+    h = np.zeros((T * k, f), np.float64)
+    lib().oracle_expert_hidden(_p(x), T, d, f, int(k), int(act), _p(slot), _p(phys), _p(arena_in),
+                               _p(sub), 0 if sub is None else sub.size, _p(h))
+    return h
+
+
 def forward(x, Wr, enorm, slot_to_expert, arena_in, arena_out, *, k, act, renorm,
             phys_slot=None, ext_logits=None, token_subset=None, imp=None, want_y=False):
     """Run the whole layer; returns a dict of every intermediate and the output.

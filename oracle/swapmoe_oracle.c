@@ -21,7 +21,7 @@
  * is the method as read from Sections 2, 3.1 and the Masked-Gating caption of
  * Figure 4.
  *
- * Readings taken where the paper is silent (each also listed in the design notes):
+ * Readings taken where the paper is silent:
  *   - Masked Gating (Fig. 4): non-resident experts get logit -inf before the
  *     softmax, so the gate is a softmax over the resident set.
  *   - Eq. (1) uses the UNMASKED routing for the token set X_i (otherwise an
@@ -201,6 +201,40 @@ void oracle_expert_outputs(const float* x, int T, int d, int f, int k, int act,
       }
     }
     free(h);
+  }
+}
+
+/*
+ * Section 2, the inner half of E_i(x) on its own: h[p,:] = act(W_in[slot[p]] * x[p div k,:])
+ * for every pair p in flat (token, j) order, so that the first grouped product of an
+ * implementation can be compared by itself.  Same definitions as expert_ffn:
+ * ReLU max(0, W_in x); SwiGLU silu(W_1 x) .* (W_3 x).  token_subset as above.
+ */
+void oracle_expert_hidden(const float* x, int T, int d, int f, int k, int act,
+                          const int32_t* slot, const int32_t* phys_slot, const float* arena_in,
+                          const int32_t* token_subset, int n_subset, double* h) {
+  const int nin = (act == ORACLE_ACT_SWIGLU) ? 2 : 1;
+  const int n = token_subset ? n_subset : T;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int i = 0; i < n; ++i) {
+    const int t = token_subset ? token_subset[i] : i;
+    const float* xt = x + (size_t)t * d;
+    for (int j = 0; j < k; ++j) {
+      const size_t p = (size_t)t * k + j;
+      const float* w1 = arena_in + (size_t)phys_slot[slot[p]] * nin * f * d;
+      const float* w3 = w1 + (size_t)f * d;
+      for (int r = 0; r < f; ++r) {
+        double a = 0.0;
+        for (int c = 0; c < d; ++c) a += (double)w1[(size_t)r * d + c] * (double)xt[c];
+        if (act == ORACLE_ACT_SWIGLU) {
+          double b = 0.0;
+          for (int c = 0; c < d; ++c) b += (double)w3[(size_t)r * d + c] * (double)xt[c];
+          h[p * f + r] = (a / (1.0 + exp(-a))) * b;
+        } else {
+          h[p * f + r] = a > 0.0 ? a : 0.0;
+        }
+      }
+    }
   }
 }
 

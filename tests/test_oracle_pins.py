@@ -117,6 +117,35 @@ def test_full_budget_equals_unrestricted_layer(act, k, renorm):
     assert np.max(np.abs(r["ugate"] - r["mgate"])) == 0.0
 
 
+@pytest.mark.parametrize("case", CASES[:4])
+def test_expert_hidden_is_the_inner_half_of_the_expert(case):
+    """oracle.expert_hidden against numpy: row p is act(W_in x) of pair p's token under pair p's
+    expert (dense evaluation of every resident expert, then picked), and W_out applied to it
+    reproduces the expert outputs the layer's own evaluation returns."""
+    seed, T, d, f, E, k, K, act, renorm = case
+    cfg, x, Wr, experts, enorm, s2e, phys, a_in, a_out = _tiny(seed, T, d, f, E, k, K, act, renorm)
+    r = oracle.forward(x, Wr, enorm, s2e, a_in, a_out, k=k, act=act, renorm=renorm, phys_slot=phys,
+                       want_y=True)
+    h = oracle.expert_hidden(x, r["slot"], phys, a_in, k=k, act=act)
+    x64 = x.astype(np.float64)
+    for t in range(T):
+        for j in range(k):
+            w_in, w_out = experts[r["midx"][t, j]]
+            a = w_in[0].astype(np.float64) @ x64[t]
+            ref = a / (1 + np.exp(-a)) * (w_in[1].astype(np.float64) @ x64[t]) if act == I.ACT_SWIGLU \
+                else np.maximum(a, 0)
+            assert np.max(np.abs(h[t * k + j] - ref)) <= 1e-12 * max(1.0, np.max(np.abs(ref)))
+            y = w_out.astype(np.float64) @ h[t * k + j]
+            assert np.max(np.abs(y - r["y"][t * k + j])) <= 1e-12 * max(1.0, np.max(np.abs(y)))
+    # a token subset leaves the other rows at zero and changes nothing else
+    sub = np.array([1, 4, 7], np.int32)
+    hs = oracle.expert_hidden(x, r["slot"], phys, a_in, k=k, act=act, token_subset=sub)
+    rows = (sub[:, None] * k + np.arange(k)[None, :]).reshape(-1)
+    assert np.array_equal(hs[rows], h[rows])
+    mask = np.ones(T * k, bool); mask[rows] = False
+    assert not hs[mask].any()
+
+
 @pytest.mark.parametrize("act", [I.ACT_RELU, I.ACT_SWIGLU])
 def test_single_expert_is_a_dense_mlp(act):
     """E = K = 1: gate is exactly 1 and the layer is W_out * act(W_in * x)."""
