@@ -49,7 +49,8 @@ enum {
   SWAPMOE_ERR_BAD_SLOT_TABLE = -4,  /* expert out of range / listed twice / bad phys    */
   SWAPMOE_ERR_CUDA = -5,            /* a CUDA runtime or driver call failed             */
   SWAPMOE_ERR_DEVICE_TIMEOUT = -6,  /* a bounded in-kernel wait gave up                 */
-  SWAPMOE_ERR_UNSUPPORTED = -7      /* shape outside what the kernels are built for     */
+  SWAPMOE_ERR_UNSUPPORTED = -7,     /* shape outside what the kernels are built for     */
+  SWAPMOE_ERR_NO_MEMORY = -8        /* a host or device allocation failed (create only) */
 };
 
 /* Limits of this build: E <= 256, K + spare_slots <= 64, top_k <= 4,
@@ -82,7 +83,15 @@ enum {
   SWAPMOE_TAP_OFFSET = 7, /* int32 [K+1]                                         */
   SWAPMOE_TAP_PERM = 8,   /* int32 [T*k]   position -> flat pair index t*k+j     */
   SWAPMOE_TAP_INV = 9,    /* int32 [T*k]   flat pair index -> position           */
-  SWAPMOE_TAP_XNORM = 10  /* fp32 [T]      L2 norm of every token                */
+  SWAPMOE_TAP_XNORM = 10, /* fp32 [T]      L2 norm of every token                */
+  /* The next two deliver the T*k occupied rows in POSITION order (row pos belongs to the pair
+   * perm[pos]; Section 2, E_i(x) = W_out act(W_in x)).  They exist only when the last forward
+   * left them in HBM: H after every forward but the one-launch decode step; Y when GEMM-2 wrote
+   * the expert outputs unweighted in one piece, i.e. top_k > 1 on the tensor-core path, or an
+   * unsliced contraction on the other paths (top-1 tensor-core layers fold gate * y into `out`).
+   * Otherwise the call returns SWAPMOE_ERR_UNSUPPORTED. */
+  SWAPMOE_TAP_H = 11,     /* layer dtype [T*k, d_ff]  act(W_in x) of every pair        */
+  SWAPMOE_TAP_Y = 12      /* fp32 [T*k, d_model]      W_out h of every pair            */
 };
 
 /*
@@ -90,7 +99,8 @@ enum {
  * resident slots.  Allocates the layer's device workspace (sized for
  * cfg->max_tokens) on the CURRENT CUDA device and zeroes the importance
  * accumulator.  *out is written only on success.  Errors: INVALID_ARG
- * (null, K < top_k, K > E, sizes out of the limits above), UNSUPPORTED, CUDA.
+ * (null, K < top_k, K > E, sizes out of the limits above), UNSUPPORTED, CUDA,
+ * NO_MEMORY (the workspace did not fit).
  */
 int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg);
 
@@ -168,7 +178,9 @@ int32_t swapmoe_forward_timed(swapmoe_layer_t* layer, const void* x_dev, void* o
 /* End-to-end form with HOST buffers: copies x_host [n_tokens, d_model] to the
  * device, runs swapmoe_forward, copies the result to out_host, and returns after
  * `stream` has completed.  Pinned host memory makes the copies asynchronous
- * with respect to other streams; pageable memory works but is slower. */
+ * with respect to other streams; pageable memory works but is slower.  It shares
+ * the layer's staging buffers with swapmoe_forward_host_async and is ordered
+ * behind that call's outstanding work on this layer. */
 int32_t swapmoe_forward_host(swapmoe_layer_t* layer, const void* x_host, void* out_host,
                              int32_t n_tokens, void* stream);
 
@@ -206,6 +218,16 @@ enum { SWAPMOE_IMP_EQ1 = 0, SWAPMOE_IMP_COUNT = 1, SWAPMOE_IMP_EQ1_MASKED = 2 };
 int32_t swapmoe_read_importance_kind(swapmoe_layer_t* layer, int32_t kind, float* imp_host,
                                      int32_t reset, void* stream);
 
+/*
+ * Measurement aid (Section 3.3 profiles an expert's memory traffic; here it is counted): the number
+ * of Virtual-Expert slots that received at least one (token, j) pair, summed over every forward
+ * since the last reset - i.e. how many experts' weights the layer had to read, the algorithmic
+ * weight traffic of the path.  Waits for `stream`; reset != 0 zeroes the counter (ordered on
+ * `stream`).
+ */
+int32_t swapmoe_read_touched_slots(swapmoe_layer_t* layer, int64_t* total_host, int32_t reset,
+                                   void* stream);
+
 /* Sections 3.1-3.2: the K most important experts, by descending importance, ties
  * to the lowest index.  Pure host function (E <= 256 floats). */
 int32_t swapmoe_topk_importance(const float* imp_host, int32_t E, int32_t K,
@@ -216,14 +238,18 @@ int32_t swapmoe_topk_importance(const float* imp_host, int32_t E, int32_t K,
  * one expert's matrices from PINNED host memory into arena entry `phys` of the
  * arenas last given to set_resident (in_host_pinned: [nin, d_ff, d_model],
  * out_host_pinned: [d_model, d_ff]), then record `done_event` (may be NULL) on
- * side_stream.  `phys` must not back any logical slot of the current table
- * (-> BAD_SLOT_TABLE), so a running forward never reads memory being written.
- * The caller later makes its compute stream wait on done_event and calls
- * set_resident with a table that uses `phys`.
+ * side_stream.  `phys` must not back any logical slot of the table given by the
+ * LATEST set_resident (-> BAD_SLOT_TABLE).  Forwards enqueued under an earlier
+ * table may still read that entry, so the copy is ordered behind everything
+ * enqueued so far on `compute_stream` (the stream the layer's forwards and
+ * set_resident calls run on; the call records an event there and makes
+ * side_stream wait for it): a forward never reads memory being written.
+ * compute_stream must not be capturing.  The caller later makes its compute
+ * stream wait on done_event and calls set_resident with a table that uses `phys`.
  */
 int32_t swapmoe_load_slot_async(swapmoe_layer_t* layer, int32_t phys, const void* in_host_pinned,
-                                const void* out_host_pinned, void* side_stream,
-                                void* done_event);
+                                const void* out_host_pinned, void* compute_stream,
+                                void* side_stream, void* done_event);
 
 /* Copies one intermediate of the last forward to the host after waiting for
  * `stream`.  `bytes` must equal the tap's size for the last n_tokens. */
@@ -250,8 +276,9 @@ int64_t swapmoe_launch_count(const swapmoe_layer_t* layer);
 int64_t swapmoe_workspace_bytes(const swapmoe_layer_t* layer);
 
 /* Selects the grouped-GEMM implementation for later forwards (test / benchmark
- * hook): 0 = automatic, 1 = CUDA-core FFMA tiles, 2 = tcgen05 tensor-core tiles
- * (bf16 only; UNSUPPORTED otherwise). */
+ * hook): 0 = automatic, 1 = warp-level mma tiles (the kernels that serve shapes
+ * the tcgen05 kernels do not take), 2 = tcgen05 tensor-core tiles (bf16 only;
+ * UNSUPPORTED otherwise). */
 int32_t swapmoe_set_gemm_path(swapmoe_layer_t* layer, int32_t path);
 
 /*
@@ -272,7 +299,7 @@ int32_t swapmoe_set_gemm_path(swapmoe_layer_t* layer, int32_t path);
  * allocating library routine.
  *
  * The price of the fixed array: every GPU that loads the library holds it
- * (about 0.4 MB) until the process exits; n_tokens is limited to
+ * (about 0.35 MB) until the process exits; n_tokens is limited to
  * SWAPMOE_ROUTE_STATIC_MAX_TOKENS (more -> SWAPMOE_ERR_TOO_MANY_TOKENS, E > 256,
  * K > 64, top_k > 4 or d_model not a multiple of 64 -> SWAPMOE_ERR_UNSUPPORTED);
  * and all calls on one GPU share it, so two calls whose kernels may overlap on

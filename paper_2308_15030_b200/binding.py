@@ -25,6 +25,7 @@ TAPS = {
     "midx": (3, np.int32), "mgate": (4, np.float32), "slot": (5, np.int32),
     "count": (6, np.int32), "offset": (7, np.int32), "perm": (8, np.int32),
     "inv": (9, np.int32), "xnorm": (10, np.float32),
+    "h": (11, None), "y": (12, np.float32),       # h comes in the layer's dtype (bf16 as uint16 bit patterns)
 }
 
 EXPORTS = [
@@ -34,7 +35,7 @@ EXPORTS = [
     "swapmoe_read_importance", "swapmoe_read_importance_kind", "swapmoe_topk_importance", "swapmoe_load_slot_async",
     "swapmoe_debug_copy", "swapmoe_device_status", "swapmoe_launch_count",
     "swapmoe_workspace_bytes", "swapmoe_set_gemm_path", "swapmoe_status_string",
-    "swapmoe_route_static", "swapmoe_selftest_bounded_wait",
+    "swapmoe_route_static", "swapmoe_selftest_bounded_wait", "swapmoe_read_touched_slots",
 ]
 
 
@@ -76,7 +77,7 @@ def lib() -> ctypes.CDLL:
         L.swapmoe_read_importance.argtypes = [vp, vp, i32, vp]
         L.swapmoe_read_importance_kind.argtypes = [vp, i32, vp, i32, vp]
         L.swapmoe_topk_importance.argtypes = [vp, i32, i32, vp]
-        L.swapmoe_load_slot_async.argtypes = [vp, i32, vp, vp, vp, vp]
+        L.swapmoe_load_slot_async.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.swapmoe_debug_copy.argtypes = [vp, i32, vp, ctypes.c_size_t, vp]
         L.swapmoe_device_status.argtypes = [vp, vp, vp]
         L.swapmoe_launch_count.argtypes = [vp]
@@ -86,6 +87,7 @@ def lib() -> ctypes.CDLL:
         L.swapmoe_set_gemm_path.argtypes = [vp, i32]
         L.swapmoe_route_static.argtypes = [vp] * 4 + [i32] * 7 + [vp] * 11
         L.swapmoe_selftest_bounded_wait.argtypes = [vp, i32, vp]
+        L.swapmoe_read_touched_slots.argtypes = [vp, vp, i32, vp]
         L.swapmoe_status_string.argtypes = [i32]
         L.swapmoe_status_string.restype = ctypes.c_char_p
         for n in EXPORTS:
@@ -243,6 +245,13 @@ class Layer:
                                              _stream_ptr(stream)), "swapmoe_read_importance")
         return imp
 
+    def read_touched_slots(self, reset: bool = False, stream=None) -> int:
+        """Slots that received at least one pair, summed over the forwards since the last reset."""
+        v = ctypes.c_int64(0)
+        _check(lib().swapmoe_read_touched_slots(self._h, ctypes.byref(v), int(bool(reset)), _stream_ptr(stream)),
+               "swapmoe_read_touched_slots")
+        return int(v.value)
+
     def read_score(self, kind: str, reset: bool = False, stream=None) -> np.ndarray:
         """kind: "eq1" (Eq. 1, unmasked routing), "count" (token counts), "eq1_masked"."""
         k = {"eq1": 0, "count": 1, "eq1_masked": 2}[kind]
@@ -251,21 +260,25 @@ class Layer:
                                                   _stream_ptr(stream)), "swapmoe_read_importance_kind")
         return out
 
-    def load_slot_async(self, phys: int, in_host_pinned, out_host_pinned, side_stream,
+    def load_slot_async(self, phys: int, in_host_pinned, out_host_pinned, compute_stream, side_stream,
                         done_event=None) -> None:
+        """The copy runs on side_stream behind everything enqueued so far on compute_stream."""
         if done_event is not None and not done_event.cuda_event:
             done_event.record(side_stream)      # torch creates the CUDA event on its first record
         ev = None if done_event is None else done_event.cuda_event
         _check(lib().swapmoe_load_slot_async(self._h, int(phys), in_host_pinned.data_ptr(),
-                                             out_host_pinned.data_ptr(), _stream_ptr(side_stream),
-                                             ev), "swapmoe_load_slot_async")
+                                             out_host_pinned.data_ptr(), _stream_ptr(compute_stream),
+                                             _stream_ptr(side_stream), ev), "swapmoe_load_slot_async")
 
     # -- inspection
     def tap(self, name: str, stream=None) -> np.ndarray:
         which, dt = TAPS[name]
         c, T = self.cfg, self.last_T
+        if dt is None:
+            dt = np.uint16 if c.dtype == BF16 else np.float32
         shape = {"logits": (T, c.E), "count": (c.K,), "offset": (c.K + 1,), "perm": (T * c.top_k,),
-                 "inv": (T * c.top_k,), "xnorm": (T,)}.get(name, (T, c.top_k))
+                 "inv": (T * c.top_k,), "xnorm": (T,), "h": (T * c.top_k, c.d_ff),
+                 "y": (T * c.top_k, c.d_model)}.get(name, (T, c.top_k))
         a = np.empty(shape, dtype=dt)
         _check(lib().swapmoe_debug_copy(self._h, which, _np_ptr(a), a.nbytes, _stream_ptr(stream)),
                "swapmoe_debug_copy")

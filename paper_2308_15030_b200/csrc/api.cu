@@ -13,9 +13,8 @@
 
 #include "common.cuh"
 #include "decode_fused.cuh"
-#include "gemm_simt.cuh"
+#include "gemm_mma.cuh"
 #include "gemm_tc.cuh"
-#include "ffn_fused.cuh"
 #include "gemm_tc_f32.cuh"
 #include "gemm_tc_pair.cuh"
 #include "gemm_tc_small.cuh"
@@ -39,9 +38,7 @@ struct swapmoe_layer {
   int32_t *uidx, *midx, *slot, *cta_hist, *cta_base, *count, *offset, *pad_offset;
   int32_t *perm, *inv, *inv_pad, *row_pair, *n_tiles, *e2s, *phys, *s2e, *status;
   unsigned* ticket;
-  int32_t* done;               // per-row-tile counters of the fused FFN kernel
-  int32_t n_done;
-  bool fused_ffn;              // both grouped GEMMs in one launch
+  unsigned long long* touched; // running total of slots that received at least one pair (device)
   bool small_path;             // small-batch GEMM kernels for <= 64 pairs
   TcSmallCache small;
   TileDesc* tiles;
@@ -66,12 +63,14 @@ struct swapmoe_layer {
   float* dec_ws;               // its partial-row workspace
   unsigned* dec_tickets;
   CUtensorMap dec_map_wo;      // W_out viewed for the decode kernel's column-slice loads
-  bool fp32_ffma;              // CUDA-core FFMA grouped GEMM instead of the split-TF32 tensor-core one
+  int row_group;               // row tiles per scheduling group of the grouped GEMMs (0: automatic; SWAPMOE_ROW_GROUP)
+  bool h_valid, y_valid;       // whether the last forward left h / y in the workspace (debug taps)
+  int32_t y_split_last;        // copies of y the last forward's GEMM-2 wrote (slices of its contraction)
   int32_t y_copies;            // copies of y in the workspace (slices of a split contraction)
   int32_t sm_count;
   bool use_pdl;                // programmatic dependent launch between the kernels of a forward
   cudaStream_t s_in, s_out;    // private copy streams of the asynchronous host path
-  cudaEvent_t ev_in, ev_comp, ev_out;
+  cudaEvent_t ev_in, ev_comp, ev_out, ev_load;
   int32_t router_tok;          // 0 = automatic token-tile size of the tensor-core router, else 32/64/128
   bool prefetch;               // pull resident weights into L2 from the router kernel
   long long l2_prefetch_bytes; // how much of them (L2 capacity minus head room)
@@ -129,7 +128,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     da.inv = L->inv; da.imp = L->imp; da.cnt = L->cnt; da.mimp = L->mimp;
     const size_t n_jb = c.d_ff / kDecJB;
     da.ypart = L->dec_ws; da.gpart = L->dec_ws + n_jb * (size_t)(kDecMaxTokens * c.top_k) * c.d_model;
-    da.tickets = L->dec_tickets; da.out = static_cast<bf16*>(out); da.status = L->status;
+    da.tickets = L->dec_tickets; da.out = static_cast<bf16*>(out); da.status = L->status; da.touched = L->touched;
     da.T = T; da.d = c.d_model; da.f = c.d_ff; da.E = c.E; da.k = c.top_k; da.K = c.K; da.renorm = c.renorm_topk;
     da.swiglu = c.act == SWAPMOE_ACT_SWIGLU;
     mark(L, 0, st);
@@ -137,6 +136,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
                       L->dec_map_wo, da) != cudaSuccess)
       return SWAPMOE_ERR_CUDA;
     L->launches++;
+    L->h_valid = L->y_valid = false;          // the one-launch kernel keeps both in shared memory
     for (int i = 1; i <= 6; ++i) mark(L, i, st);
     return check_launch();
   }
@@ -157,7 +157,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   const bool use_pairs = use_tc && tc_use_pairs(c, T, L->gemm_pairs, L->pair_min_rows);
   const int mt = use_tc ? tc_row_subtiles(c, T, use_pairs) : 1;
   const bool use_tc32 = !use_tc && L->tc32.enabled && L->tc32.arena_bound;
-  const int tile_rows = use_tc ? kTcBM * mt : (use_tc32 ? kTcBM : kSimtBM);
+  const int tile_rows = use_tc ? kTcBM * mt : (use_tc32 ? kTcBM : kMmaBM);
   const int max_tiles = (n_pairs + tile_rows - 1) / tile_rows + c.K;
 
   RouterArgs ra;
@@ -169,11 +169,15 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   ra.T = T; ra.d = c.d_model; ra.E = c.E; ra.k = c.top_k; ra.K = c.K; ra.renorm = c.renorm_topk;
   ScanArgs& sa = ra.scan;
   sa.cta_hist = L->cta_hist; sa.cta_imp = L->cta_imp; sa.phys_slot = L->phys;
-  sa.cta_base = L->cta_base; sa.count = L->count; sa.offset = L->offset;
+  // Up to 256 router CTAs the router only leaves its per-CTA histograms and the permute kernel sums them itself
+  // (every CTA its own base counts, one CTA the Eq. (1) partials); beyond that the last router CTA to finish scans
+  // (re-reading all rows in every permute CTA would then cost more than its serial walk).
+  const bool own_scan = n_cta <= 256;
+  sa.cta_base = own_scan ? nullptr : L->cta_base; sa.count = L->count; sa.offset = L->offset;
   sa.pad_offset = L->pad_offset; sa.tiles = L->tiles; sa.n_tiles = L->n_tiles; sa.imp = L->imp;
   sa.cta_cnt = L->cta_cnt; sa.cta_mimp = L->cta_mimp; sa.s2e = L->s2e; sa.cnt = L->cnt; sa.mimp = L->mimp;
-  sa.ticket = L->ticket;
-  sa.done = L->done; sa.n_done = L->n_done;
+  sa.ticket = own_scan ? nullptr : L->ticket;
+  sa.touched = L->touched;
   sa.n_cta = n_cta; sa.K = c.K; sa.E = c.E; sa.tile_rows = tile_rows;
   // GEMM-2 with two row sub-tiles per CTA walks 256-row tiles; GEMM-1 then gets its own compact
   // list of 128-row tiles (walking the 256-row list as pairs would leave holes in its schedule).
@@ -237,13 +241,16 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   pa.pad_offset = L->pad_offset; pa.perm = L->perm; pa.inv = L->inv; pa.inv_pad = L->inv_pad;
   pa.row_pair = L->row_pair;
   pa.xp = L->xp; pa.T = T; pa.d = c.d_model; pa.k = c.top_k; pa.K = c.K; pa.tok_tile = tok_tile;
+  pa.own_scan = own_scan ? 1 : 0;
+  pa.scan = sa;
   mark(L, 2, st);
   // enough CTAs to fill the GPU: every row-group of a token tile gets its own CTA
   int groups = (2 * L->sm_count + n_cta - 1) / n_cta;
   const int max_groups = (tok_tile * c.top_k + 7) / 8;
   if (groups > max_groups) groups = max_groups;
   if (groups < 1) groups = 1;
-  if (launch_kernel(permute_gather_kernel<DT>, dim3(n_cta, groups), dim3(kPermThreads), 0, st, pdl, pa) !=
+  // own_scan: one extra column of CTAs, whose first CTA reduces the Eq. (1) partials
+  if (launch_kernel(permute_gather_kernel<DT>, dim3(n_cta + (own_scan ? 1 : 0), groups), dim3(kPermThreads), 0, st, pdl, pa) !=
       cudaSuccess)
     return SWAPMOE_ERR_CUDA;
   L->launches++;
@@ -257,20 +264,16 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
       rc = tc_ffn_small(L->tc, L->small, c, L->xp, L->h, L->y, out, L->rows_pad_max, L->arena_in, L->arena_out,
                         L->tiles, L->n_tiles, L->row_pair, L->mgate, max_tiles, T, L->status, st, pdl,
                         &L->launches, &combined, mid);
-    } else if (L->fused_ffn && mt == 1) {
-      rc = tc_ffn_fused(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->done, L->row_pair, L->mgate, max_tiles,
-                        L->status, st, pdl, &L->launches, &combined);
-      if (mid) cudaEventRecord(mid, st);      // one kernel: the GEMM-2 stage reads as zero
     } else if (mt == 2 && L->gemm_pairs > 0 && c.d_ff % 256 == 0) {
       // 256-row tiles: GEMM-1 always on CTA pairs (its one-CTA form pulls 48 KB per k-block); GEMM-2 on pairs for
       // very large slots, else on one CTA with two row sub-tiles (same bytes per flop, and a tile whose second
       // half is empty costs half; cfg3: 128.6 -> 126.8 us)
       rc = tc_ffn_pair(L->tc, L->gemm_pairs, c, L->h, L->y, out, L->tiles, L->n_tiles, L->row_pair, L->mgate, max_tiles,
-                       T, L->status, st, pdl, &L->launches, &combined, mid, use_pairs);
+                       T, L->status, st, pdl, &L->launches, &combined, mid, use_pairs, L->row_group);
     } else {
       rc = tc_ffn(L->tc, c, L->h, L->y, out, L->tiles, L->n_tiles, L->tiles_b, L->n_tiles_b, L->row_pair, L->mgate,
                   max_tiles, mt, T,
-                  L->status, st, pdl, &L->launches, &combined, mid);
+                  L->status, st, pdl, &L->launches, &combined, mid, L->row_group);
     }
     if (rc != SWAPMOE_OK) return rc;
   } else if (use_tc32) {
@@ -279,42 +282,33 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
                                   L->n_tiles, max_tiles, T, L->status, st, pdl, &L->launches, &y_split, mid);
     if (rc != SWAPMOE_OK) return rc;
   } else {
-    SimtGemmArgs g1;
+    MmaGemmArgs g1;
     g1.A = L->xp; g1.W = L->arena_in; g1.C = L->h; g1.tiles = L->tiles; g1.n_tiles = L->n_tiles;
     g1.slot_stride = (long long)L->nin * c.d_ff * c.d_model;
     g1.gate_offset = (long long)c.d_ff * c.d_model;
     g1.N = c.d_ff; g1.Kdim = c.d_model; g1.split_stride = 0;
-    const dim3 grid1(c.d_ff / kSimtBN, max_tiles);
-    cudaError_t e;
-    if (L->fp32_ffma) {
-      if (c.act == SWAPMOE_ACT_SWIGLU)
-        e = launch_kernel(gemm_simt_kernel<DT, DT, DT, kEpiSwiglu>, grid1, dim3(kSimtThreads), 0, st, pdl, g1);
-      else
-        e = launch_kernel(gemm_simt_kernel<DT, DT, DT, kEpiRelu>, grid1, dim3(kSimtThreads), 0, st, pdl, g1);
-    } else {
-      if (c.act == SWAPMOE_ACT_SWIGLU)
-        e = launch_kernel(gemm_tf32x3_kernel<DT, DT, DT, kEpiSwiglu>, grid1, dim3(kSimtThreads), 0, st, pdl, g1);
-      else
-        e = launch_kernel(gemm_tf32x3_kernel<DT, DT, DT, kEpiRelu>, grid1, dim3(kSimtThreads), 0, st, pdl, g1);
-    }
+    const dim3 grid1(c.d_ff / kMmaBN, max_tiles);
+    const cudaError_t e =
+        c.act == SWAPMOE_ACT_SWIGLU
+            ? launch_kernel(gemm_tf32x3_kernel<DT, DT, DT, kEpiSwiglu>, grid1, dim3(kMmaThreads), 0, st, pdl, g1)
+            : launch_kernel(gemm_tf32x3_kernel<DT, DT, DT, kEpiRelu>, grid1, dim3(kMmaThreads), 0, st, pdl, g1);
     if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
     L->launches++;
     mark(L, 4, st);
-    SimtGemmArgs g2;
+    MmaGemmArgs g2;
     g2.A = L->h; g2.W = L->arena_out; g2.C = L->y; g2.tiles = L->tiles; g2.n_tiles = L->n_tiles;
     g2.slot_stride = (long long)c.d_ff * c.d_model;
     g2.gate_offset = 0;
     g2.N = c.d_model; g2.Kdim = c.d_ff;
     // Few output tiles and a long contraction: slice the contraction so that every SM has work.
     // The slices land in separate copies of y and the combine kernel adds them in order.
-    const long long tiles_est = ((long long)n_pairs / kSimtBM + (n_pairs < c.K ? n_pairs : c.K) / 2 + 1) *
-                                (c.d_model / kSimtBN);
-    y_split = simt_pick_split(tiles_est, L->sm_count, c.d_ff, L->y_copies);
+    const long long tiles_est = ((long long)n_pairs / kMmaBM + (n_pairs < c.K ? n_pairs : c.K) / 2 + 1) *
+                                (c.d_model / kMmaBN);
+    y_split = mma_pick_split(tiles_est, L->sm_count, c.d_ff, L->y_copies);
     g2.split_stride = (long long)L->rows_pad_max * c.d_model;
-    const dim3 grid2(c.d_model / kSimtBN, max_tiles, y_split);
-    if ((L->fp32_ffma ? launch_kernel(gemm_simt_kernel<DT, DT, float, kEpiNone>, grid2, dim3(kSimtThreads), 0, st, pdl, g2)
-                      : launch_kernel(gemm_tf32x3_kernel<DT, DT, float, kEpiNone>, grid2, dim3(kSimtThreads), 0, st, pdl,
-                                      g2)) != cudaSuccess)
+    const dim3 grid2(c.d_model / kMmaBN, max_tiles, y_split);
+    if (launch_kernel(gemm_tf32x3_kernel<DT, DT, float, kEpiNone>, grid2, dim3(kMmaThreads), 0, st, pdl, g2) !=
+        cudaSuccess)
       return SWAPMOE_ERR_CUDA;
     L->launches++;
   }
@@ -332,6 +326,10 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     L->launches++;
   }
   mark(L, 6, st);
+  // what the debug taps may read back: h unless the small-batch kernels kept it on chip, y when GEMM-2 wrote it
+  L->h_valid = true;
+  L->y_valid = !combined;
+  L->y_split_last = y_split;
   return check_launch();
 }
 
@@ -347,6 +345,34 @@ int32_t forward_checked(swapmoe_layer* L, const void* x, const float* ext, void*
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (L->cfg.dtype == SWAPMOE_BF16) return forward_impl<bf16>(L, x, ext, out, T, st);
   return forward_impl<float>(L, x, ext, out, T, st);
+}
+
+// H / Y taps: the hidden activations and the expert outputs live in the padded workspace (slot
+// segments start at multiples of 128 rows); the tap delivers the T*k occupied rows in position
+// order (row `pos` belongs to pair perm[pos]), one copy per slot segment.
+int32_t debug_copy_rows(swapmoe_layer* L, int32_t which, void* host, size_t bytes, cudaStream_t st) {
+  const swapmoe_config_t& c = L->cfg;
+  const size_t P = (size_t)L->last_T * c.top_k;
+  const bool is_h = which == SWAPMOE_TAP_H;
+  if (is_h ? !L->h_valid : (!L->y_valid || L->y_split_last != 1)) return SWAPMOE_ERR_UNSUPPORTED;
+  const size_t row_bytes = is_h ? (size_t)c.d_ff * L->elem : (size_t)c.d_model * sizeof(float);
+  if (bytes != P * row_bytes) return SWAPMOE_ERR_INVALID_ARG;
+  if (P == 0) return SWAPMOE_OK;
+  int32_t count[kMaxSlots], pad[kMaxSlots + 1];
+  if (!cuda_ok(cudaMemcpyAsync(count, L->count, sizeof(int32_t) * c.K, cudaMemcpyDeviceToHost, st)) ||
+      !cuda_ok(cudaMemcpyAsync(pad, L->pad_offset, sizeof(int32_t) * (c.K + 1), cudaMemcpyDeviceToHost, st)) ||
+      !cuda_ok(cudaStreamSynchronize(st)))
+    return SWAPMOE_ERR_CUDA;
+  const char* base = is_h ? static_cast<const char*>(L->h) : reinterpret_cast<const char*>(L->y);
+  char* dst = static_cast<char*>(host);
+  for (int s = 0; s < c.K; ++s) {
+    if (count[s] == 0) continue;
+    if (!cuda_ok(cudaMemcpyAsync(dst, base + (size_t)pad[s] * row_bytes, (size_t)count[s] * row_bytes,
+                                 cudaMemcpyDeviceToHost, st)))
+      return SWAPMOE_ERR_CUDA;
+    dst += (size_t)count[s] * row_bytes;
+  }
+  return cuda_ok(cudaStreamSynchronize(st)) ? SWAPMOE_OK : SWAPMOE_ERR_CUDA;
 }
 
 }  // namespace
@@ -374,7 +400,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   if (prop.major != 10) return SWAPMOE_ERR_UNSUPPORTED;  // kernels are built for sm_100a only
 
   swapmoe_layer* L = new (std::nothrow) swapmoe_layer();
-  if (!L) return SWAPMOE_ERR_INVALID_ARG;
+  if (!L) return SWAPMOE_ERR_NO_MEMORY;
   std::memset(L, 0, sizeof(*L));
   L->cfg = c;
   L->device = dev;
@@ -382,15 +408,13 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   {
     const char* env = std::getenv("SWAPMOE_PDL");      // SWAPMOE_PDL=0 launches every kernel fully serialised
     L->use_pdl = !(env && env[0] == '0');
-    env = std::getenv("SWAPMOE_FUSED_FFN");             // SWAPMOE_FUSED_FFN=1: both grouped GEMMs in one launch
-    L->fused_ffn = env && env[0] == '1';                // off by default: measured slower than two launches
     env = std::getenv("SWAPMOE_ROUTER_TOK");            // force the router's token tile (32, 64 or 128)
     L->router_tok = env ? std::atoi(env) : 0;
     if (L->router_tok != 32 && L->router_tok != 64 && L->router_tok != 128) L->router_tok = 0;
     env = std::getenv("SWAPMOE_SMALL_PATH");            // SWAPMOE_SMALL_PATH=0: general GEMM kernels for small batches too
     L->small_path = !(env && env[0] == '0');
-    env = std::getenv("SWAPMOE_FP32_FFMA");             // SWAPMOE_FP32_FFMA=1: FFMA form of the non-tcgen05 grouped GEMM
-    L->fp32_ffma = env && env[0] == '1';
+    env = std::getenv("SWAPMOE_ROW_GROUP");             // row tiles per scheduling group of the grouped GEMMs
+    L->row_group = env && std::atoi(env) > 0 ? std::atoi(env) : 0;
     env = std::getenv("SWAPMOE_PREFETCH");              // SWAPMOE_PREFETCH=0 disables the L2 weight prefetch
     L->prefetch = !(env && env[0] == '0');
     // The prefetch must drain while the router runs (about 15 us on 16-64 SMs): what HBM delivers
@@ -418,7 +442,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
     if (c.dtype == SWAPMOE_F32 && f32small > n_cta) n_cta = f32small;
   }
   const size_t rows_pad = align_up(P + (size_t)c.K * kSegAlign, kSegAlign);
-  const size_t max_tiles = (P + kSimtBM - 1) / kSimtBM + c.K;
+  const size_t max_tiles = (P + kMmaBM - 1) / kMmaBM + c.K;
   L->rows_pad_max = (int32_t)rows_pad;
 
   Carver cv;
@@ -438,7 +462,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_phys = cv.take<int32_t>(kMaxSlots), o_s2e = cv.take<int32_t>(kMaxSlots);
   const size_t o_status = cv.take<int32_t>(4);
   const size_t o_ticket = cv.take<unsigned>(4);
-  const size_t o_done = cv.take<int32_t>(max_tiles);
+  const size_t o_touched = cv.take<unsigned long long>(2);
   const size_t o_tiles = cv.take<TileDesc>(max_tiles);
   const size_t o_tiles_b = cv.take<TileDesc>(max_tiles), o_ntiles_b = cv.take<int32_t>(4);
   const size_t o_xp = cv.take<char>(rows_pad * c.d_model * L->elem);
@@ -462,7 +486,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_dec_ws = cv.take<float>(L->decode_path ? decode_ws_floats(c.d_model, c.d_ff, c.top_k) : 1);
   const size_t o_dec_tk = cv.take<unsigned>(L->decode_path ? decode_ticket_count(c.d_ff, c.K) : 1);
   L->ws_bytes = cv.off;
-  if (!cuda_ok(cudaMalloc(&L->ws_base, L->ws_bytes))) { cudaGetLastError(); delete L; return SWAPMOE_ERR_CUDA; }
+  if (!cuda_ok(cudaMalloc(&L->ws_base, L->ws_bytes))) { cudaGetLastError(); delete L; return SWAPMOE_ERR_NO_MEMORY; }
   char* b = L->ws_base;
   L->logits = (float*)(b + o_logits); L->ugate = (float*)(b + o_ugate); L->mgate = (float*)(b + o_mgate);
   L->xnorm = (float*)(b + o_xnorm); L->cta_imp = (float*)(b + o_cta_imp); L->imp = (float*)(b + o_imp);
@@ -477,8 +501,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   L->n_tiles = (int32_t*)(b + o_ntiles); L->e2s = (int32_t*)(b + o_e2s); L->phys = (int32_t*)(b + o_phys);
   L->s2e = (int32_t*)(b + o_s2e); L->status = (int32_t*)(b + o_status);
   L->ticket = (unsigned*)(b + o_ticket);
-  L->done = (int32_t*)(b + o_done);
-  L->n_done = (int32_t)max_tiles;
+  L->touched = (unsigned long long*)(b + o_touched);
   L->tiles = (TileDesc*)(b + o_tiles);
   L->tiles_b = (TileDesc*)(b + o_tiles_b); L->n_tiles_b = (int32_t*)(b + o_ntiles_b);
   L->xp = b + o_xp; L->h = b + o_h; L->y = (float*)(b + o_y);
@@ -490,6 +513,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   ok = ok && cuda_ok(cudaMemset(L->mimp, 0, sizeof(float) * c.E));
   ok = ok && cuda_ok(cudaMemset(L->status, 0, sizeof(int32_t) * 4));
   ok = ok && cuda_ok(cudaMemset(L->ticket, 0, sizeof(unsigned) * 4));
+  ok = ok && cuda_ok(cudaMemset(L->touched, 0, sizeof(unsigned long long) * 2));
   if (L->decode_path) {
     ok = ok && cuda_ok(cudaMemset(L->dec_tickets, 0, sizeof(unsigned) * decode_ticket_count(c.d_ff, c.K)));
     ok = ok && cuda_ok(decode_fused_set_smem_limit((int)decode_smem_bytes(c.d_model)));
@@ -505,7 +529,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   L->encode32 = nullptr;
   {
     const char* env = std::getenv("SWAPMOE_FP32_TC");        // SWAPMOE_FP32_TC=0: warp-level mma (or FFMA) for fp32 layers
-    if (ok && c.dtype == SWAPMOE_F32 && !L->fp32_ffma && !(env && env[0] == '0')) {
+    if (ok && c.dtype == SWAPMOE_F32 && !(env && env[0] == '0')) {
       L->encode32 = tc_get_encoder();
       ok = tc_f32_init(L->tc32, L->encode32, c, L->xp, L->h, L->rows_pad_max, L->sm_count) == SWAPMOE_OK;
     }
@@ -546,7 +570,8 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_in, cudaEventDisableTiming));
   ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_comp, cudaEventDisableTiming));
   ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_out, cudaEventDisableTiming));
-  if (!ok) { cudaGetLastError(); cudaFree(L->ws_base); delete L; return SWAPMOE_ERR_CUDA; }
+  ok = ok && cuda_ok(cudaEventCreateWithFlags(&L->ev_load, cudaEventDisableTiming));
+  if (!ok) { cudaGetLastError(); swapmoe_destroy(L); return SWAPMOE_ERR_CUDA; }   // frees whatever was created
   *out = L;
   return SWAPMOE_OK;
 }
@@ -558,6 +583,7 @@ int32_t swapmoe_destroy(swapmoe_layer_t* L) {
   if (L->ev_in) cudaEventDestroy(L->ev_in);
   if (L->ev_comp) cudaEventDestroy(L->ev_comp);
   if (L->ev_out) cudaEventDestroy(L->ev_out);
+  if (L->ev_load) cudaEventDestroy(L->ev_load);
   cudaFree(L->ws_base);
   delete L;
   return SWAPMOE_OK;
@@ -651,6 +677,10 @@ int32_t swapmoe_forward_host(swapmoe_layer_t* L, const void* x_host, void* out_h
   if (T > L->cfg.max_tokens) return SWAPMOE_ERR_TOO_MANY_TOKENS;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t bytes = (size_t)T * L->cfg.d_model * L->elem;
+  // the staging buffers are shared with the pipelined entry point: wait for its last forward (which
+  // reads x_stage) and its last copy-out (which reads out_stage); no-ops when it was never used
+  if (!cuda_ok(cudaStreamWaitEvent(st, L->ev_comp, 0)) || !cuda_ok(cudaStreamWaitEvent(st, L->ev_out, 0)))
+    return SWAPMOE_ERR_CUDA;
   if (!cuda_ok(cudaMemcpyAsync(L->x_stage, x_host, bytes, cudaMemcpyHostToDevice, st))) return SWAPMOE_ERR_CUDA;
   const int32_t rc = forward_checked(L, L->x_stage, nullptr, L->out_stage, T, stream);
   if (rc != SWAPMOE_OK) return rc;
@@ -709,6 +739,17 @@ int32_t swapmoe_read_importance(swapmoe_layer_t* L, float* imp_host, int32_t res
   return swapmoe_read_importance_kind(L, SWAPMOE_IMP_EQ1, imp_host, reset, stream);
 }
 
+int32_t swapmoe_read_touched_slots(swapmoe_layer_t* L, int64_t* total_host, int32_t reset, void* stream) {
+  if (!L || !total_host) return SWAPMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned long long v = 0;
+  if (!cuda_ok(cudaMemcpyAsync(&v, L->touched, sizeof(v), cudaMemcpyDeviceToHost, st))) return SWAPMOE_ERR_CUDA;
+  if (reset && !cuda_ok(cudaMemsetAsync(L->touched, 0, sizeof(v), st))) return SWAPMOE_ERR_CUDA;
+  if (!cuda_ok(cudaStreamSynchronize(st))) return SWAPMOE_ERR_CUDA;
+  *total_host = (int64_t)v;
+  return SWAPMOE_OK;
+}
+
 int32_t swapmoe_topk_importance(const float* imp, int32_t E, int32_t K, int32_t* out_idx) {
   if (!imp || !out_idx || E < 1 || K < 1 || K > E || E > kMaxE) return SWAPMOE_ERR_INVALID_ARG;
   bool taken[kMaxE];
@@ -726,7 +767,7 @@ int32_t swapmoe_topk_importance(const float* imp, int32_t E, int32_t K, int32_t*
 }
 
 int32_t swapmoe_load_slot_async(swapmoe_layer_t* L, int32_t phys, const void* in_host, const void* out_host,
-                                void* side_stream, void* done_event) {
+                                void* compute_stream, void* side_stream, void* done_event) {
   if (!L || !in_host || !out_host) return SWAPMOE_ERR_INVALID_ARG;
   if (!L->resident_set) return SWAPMOE_ERR_NOT_READY;
   const swapmoe_config_t& c = L->cfg;
@@ -734,6 +775,14 @@ int32_t swapmoe_load_slot_async(swapmoe_layer_t* L, int32_t phys, const void* in
   for (int s = 0; s < c.K; ++s)
     if (L->h_phys[s] == phys) return SWAPMOE_ERR_BAD_SLOT_TABLE;
   cudaStream_t st = static_cast<cudaStream_t>(side_stream);
+  // Forwards enqueued under an EARLIER table may still read entry `phys` (it is spare only in the
+  // latest table), and the grouped GEMMs request weight boxes before their dependent-launch wait:
+  // the copy is ordered behind everything enqueued so far on the stream the forwards run on.
+  if (side_stream != compute_stream) {
+    if (!cuda_ok(cudaEventRecord(L->ev_load, static_cast<cudaStream_t>(compute_stream))) ||
+        !cuda_ok(cudaStreamWaitEvent(st, L->ev_load, 0)))
+      return SWAPMOE_ERR_CUDA;
+  }
   const size_t in_bytes = (size_t)L->nin * c.d_ff * c.d_model * L->elem;
   const size_t out_bytes = (size_t)c.d_ff * c.d_model * L->elem;
   char* din = static_cast<char*>(const_cast<void*>(L->arena_in)) + (size_t)phys * in_bytes;
@@ -762,6 +811,8 @@ int32_t swapmoe_debug_copy(swapmoe_layer_t* L, int32_t which, void* host, size_t
     case SWAPMOE_TAP_PERM: src = L->perm; need = P * 4; break;
     case SWAPMOE_TAP_INV: src = L->inv; need = P * 4; break;
     case SWAPMOE_TAP_XNORM: src = L->xnorm; need = T * 4; break;
+    case SWAPMOE_TAP_H:
+    case SWAPMOE_TAP_Y: return debug_copy_rows(L, which, host, bytes, static_cast<cudaStream_t>(stream));
     default: return SWAPMOE_ERR_INVALID_ARG;
   }
   if (bytes != need) return SWAPMOE_ERR_INVALID_ARG;
@@ -791,10 +842,26 @@ int32_t swapmoe_selftest_bounded_wait(swapmoe_layer_t* L, int32_t limit_ms, void
   return check_launch();
 }
 
+#ifdef SWAPMOE_TRACE
+// Tracing builds only: copies the kernels' %globaltimer stamps ([4 kernels][160 CTAs][16 slots] uint64) to the host.
+int32_t swapmoe_debug_trace(unsigned long long* host, int32_t clear) {
+  if (!host) return SWAPMOE_ERR_INVALID_ARG;
+  if (!cuda_ok(cudaDeviceSynchronize()) || !cuda_ok(cudaMemcpyFromSymbol(host, swapmoe::g_trace, sizeof(swapmoe::g_trace))))
+    return SWAPMOE_ERR_CUDA;
+  if (clear) {
+    void* p = nullptr;
+    if (!cuda_ok(cudaGetSymbolAddress(&p, swapmoe::g_trace)) || !cuda_ok(cudaMemset(p, 0, sizeof(swapmoe::g_trace))))
+      return SWAPMOE_ERR_CUDA;
+  }
+  return SWAPMOE_OK;
+}
+#endif
+
 int64_t swapmoe_launch_count(const swapmoe_layer_t* L) { return L ? L->launches : 0; }
 int64_t swapmoe_workspace_bytes(const swapmoe_layer_t* L) { return L ? (int64_t)L->ws_bytes : 0; }
 
 int32_t swapmoe_set_gemm_path(swapmoe_layer_t* L, int32_t path) {
+  // 0 = automatic, 1 = warp-level mma kernels (gemm_tf32x3_kernel), 2 = tcgen05 kernels
   if (!L || path < 0 || path > 2) return SWAPMOE_ERR_INVALID_ARG;
   if (path == 2 && !tc_supported(L->cfg)) return SWAPMOE_ERR_UNSUPPORTED;
   L->gemm_path = path;
@@ -811,6 +878,7 @@ const char* swapmoe_status_string(int32_t s) {
     case SWAPMOE_ERR_CUDA: return "CUDA error";
     case SWAPMOE_ERR_DEVICE_TIMEOUT: return "bounded device wait timed out";
     case SWAPMOE_ERR_UNSUPPORTED: return "unsupported shape or device";
+    case SWAPMOE_ERR_NO_MEMORY: return "out of host or device memory";
     default: return "unknown status";
   }
 }

@@ -59,6 +59,24 @@ __device__ __forceinline__ void store8(bf16* p, const float v[8]) {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Timeline tracing (built only with -DSWAPMOE_TRACE, see build.py): a kernel stamps %globaltimer
+// into g_trace[kernel][CTA][slot]; swapmoe_debug_trace copies the table out.  Kernel ids: 0 router,
+// 1 permute, 2 grouped GEMM-1, 3 grouped GEMM-2.  SWAPMOE_STAMP is called by ONE thread of a CTA.
+constexpr int kTraceKernels = 4, kTraceCtas = 160, kTraceSlots = 16;
+#ifdef SWAPMOE_TRACE
+static __device__ unsigned long long g_trace[kTraceKernels][kTraceCtas][kTraceSlots];
+#define SWAPMOE_STAMP(kern, slot)                                                     \
+  do {                                                                                \
+    if (blockIdx.x < kTraceCtas) {                                                    \
+      unsigned long long t_;                                                          \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)::"memory");                \
+      g_trace[kern][blockIdx.x][slot] = t_;                                           \
+    }                                                                                 \
+  } while (0)
+#else
+#define SWAPMOE_STAMP(kern, slot) do { } while (0)
+#endif
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -64,6 +64,7 @@ struct DecodeArgs {
   unsigned* tickets;         // [K * groups + 1], all zero between launches
   bf16* out;                 // [T, d]
   int32_t* status;           // device status words (bounded waits report here)
+  unsigned long long* touched;   // [1] running total of slots that received at least one pair, or nullptr
   int32_t T, d, f, E, k, K, renorm, swiglu;
 };
 
@@ -536,6 +537,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
       for (int p = 0; p < P; ++p) { c += (R->sl[p] == tid); lower += (R->sl[p] < tid); }
       a.offset[tid] = lower;
       if (tid < K) a.count[tid] = c;
+      if (tid < K && c > 0 && a.touched != nullptr) atomicAdd(a.touched, 1ull);   // slots whose weights were read
     }
     if (tid < K) {
       // Eq. (1) under the masked routing, credited to the slot's expert

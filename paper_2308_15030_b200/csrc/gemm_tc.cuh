@@ -47,6 +47,7 @@ struct TcGemmArgs {
   const int32_t* row_pair;  // [rows_pad] pair index of each padded row (scatter epilogue)
   const float* gate;        // [T*k] masked gate values (scatter epilogue)
   int32_t top_k;
+  int32_t early_b;          // 1: the tile list is final when the CTAs start (see the kernel): weights are requested early
 };
 
 // ----------------------------------------------------------------------------- PTX wrappers
@@ -349,8 +350,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   unsigned char* epi_stage = smem + kStages * S::kStageBytes + 1024;   // [4 warps][32 rows][128 bytes]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int kTr = (EPI == kTcEpiReluBf16 || EPI == kTcEpiSwigluBf16) ? 2 : 3;   // trace id: GEMM-1 or GEMM-2
+  (void)kTr;
 
   if (threadIdx.x == 0) {
+    SWAPMOE_STAMP(kTr, 0);
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 128); }
     *abort_flag = 0;
@@ -367,13 +371,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // The tile list was written by the router, which finished before the kernel in front of this one was
-  // allowed to start (every kernel of the chain triggers its dependents only after its own wait), and the
-  // weights are constants of the layer.  So the producer requests the weight boxes of its first stages
-  // BEFORE the dependent-launch wait; only the activations (written by the kernel in front) have to wait.
+  // The weights are constants of the layer, and for GEMM-2 the tile list is complete long before its CTAs can
+  // start (it is written before GEMM-1's wait returns, and GEMM-2's CTAs are scheduled after that).  So with
+  // `early_b` the producer requests the weight boxes of its first stages BEFORE the dependent-launch wait; only
+  // the activations (written by the kernel in front) have to wait.  GEMM-1 may be scheduled while the kernels
+  // that write the tile list still run, so it asks for nothing early.
   const bool is_producer = warp == 0 && lane == 0;
   int pre = 0;                                   // stages whose weight boxes are already requested
-  if (is_producer) {
+  if (is_producer && a.early_b) {
     const int n_rt = __ldcg(a.n_tiles);
     if ((int)blockIdx.x < n_rt * a.n_col_tiles) {
       int rt, ct;
@@ -392,6 +397,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   }
+  if (is_producer) SWAPMOE_STAMP(kTr, 1);
   pdl_wait();      // the activations come from the preceding kernel
   pdl_trigger();
   const int n_row_tiles = *a.n_tiles;
@@ -400,6 +406,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 0) {
     if (lane == 0) {
       // ------------------------------------------------------------------ TMA producer
+      SWAPMOE_STAMP(kTr, 2);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -428,6 +435,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
+      SWAPMOE_STAMP(kTr, 3);                  // last load requested
       if (!ok) {
         // Give copies that are still in flight time to land before shared memory is released.
         const uint64_t t0 = ptx::globaltimer_ns();
@@ -437,6 +445,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     if (lane == 0) {
       // ------------------------------------------------------------------ MMA issuer
+      bool first_full = true;
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
@@ -454,6 +463,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int kb = 0; kb < a.k_blocks; ++kb) {
           ok = bounded_wait(&full[stage], phase, abort_flag, a.status, 3);
           if (!ok) break;
+          if (first_full) { SWAPMOE_STAMP(kTr, 4); first_full = false; }
           ptx::tc_fence_after();
           const uint64_t db = make_kmajor_sw128_desc(ptx::smem_u32(sB + stage * S::kBBytes));
           for (int hf = 0; hf < halves; ++hf) {
@@ -472,6 +482,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         ptx::umma_commit(&acc_full[acc]);    // accumulator complete
         if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1u; }
       }
+      SWAPMOE_STAMP(kTr, 5);                  // last MMA issued
     }
   } else if (warp >= 4) {
     // -------------------------------------------------------------------- epilogue
@@ -530,6 +541,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       ptx::mbar_arrive(&acc_empty[acc]);       // 128 arrivals hand the buffer back to the MMA warp
       if (++acc == kAccBufs) { acc = 0; acc_phase ^= 1u; }
     }
+    if (threadIdx.x == 128) SWAPMOE_STAMP(kTr, 6);   // this CTA's last epilogue done
   }
   ptx::tc_fence_before();
   __syncthreads();
@@ -707,7 +719,7 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
                       const int32_t* n_tiles, const TileDesc* tiles128, const int32_t* n_tiles128,
                       const int32_t* row_pair, const float* mgate, int max_tiles, int mt,
                       int n_tokens, int32_t* status, cudaStream_t st, bool pdl, int64_t* launches, bool* combined,
-                      cudaEvent_t between = nullptr) {
+                      cudaEvent_t between = nullptr, int row_group_forced = 0) {
   if (!s.enabled || !s.arena_bound) return SWAPMOE_ERR_NOT_READY;
   const bool swiglu = c.act == SWAPMOE_ACT_SWIGLU;
   const bool scatter = c.top_k == 1;
@@ -726,11 +738,8 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
   // Large activation matrices (tens of MB) are walked in groups of 32 row tiles so that a group's
   // rows stay in L2 across its column tiles; small ones are a single group.
   int row_group = 1 << 30;
-  {
-    const char* env = std::getenv("SWAPMOE_ROW_GROUP");
-    if (env) row_group = std::atoi(env) > 0 ? std::atoi(env) : row_group;
-    else if (pairs * (long long)c.d_model * 2 > (48ll << 20)) row_group = 32;
-  }
+  if (row_group_forced > 0) row_group = row_group_forced;
+  else if (pairs * (long long)c.d_model * 2 > (48ll << 20)) row_group = 32;
   // ---- GEMM-1: h = act(xp * W_in^T).  Its k-loop is short (d_model / 64 blocks), so its epilogue must
   // overlap the next tile's MMAs: always one sub-tile per CTA with two TMEM buffers.
   const int i1 = tc_pick_bn(kBn1Options, 3, c.d_ff, row_tiles_est * mt, s.sm_count, a_box_bytes, swiglu ? 64 : 32);
@@ -748,6 +757,7 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
   g1.row_pair = nullptr; g1.gate = nullptr; g1.top_k = c.top_k;
   g1.row_group = row_group;
   g1.a_box_bytes = a_box_bytes;
+  g1.early_b = 0;
   long long work = (long long)max_tiles * mt * g1.n_col_tiles;
   int grid = work > s.sm_count ? s.sm_count : (int)work;
   static const TcGemmKernel k1[2][3] = {
@@ -775,6 +785,7 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
   g2.row_pair = row_pair; g2.gate = mgate; g2.top_k = c.top_k;
   g2.row_group = row_group;
   g2.a_box_bytes = a_box_bytes;
+  g2.early_b = 1;
   work = (long long)max_tiles * g2.n_col_tiles;
   grid = work > s.sm_count ? s.sm_count : (int)work;
   const bool pdl2 = pdl && between == nullptr;

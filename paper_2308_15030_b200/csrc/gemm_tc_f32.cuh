@@ -50,6 +50,7 @@ struct TcF32Args {
   long long split_stride;   // elements between the copies of C
   int32_t ldc, n_col_tiles, k_blocks, n_split;   // k_blocks per slice
   int32_t b_rows_per_phys, b_rows_gate;
+  int32_t early_b;          // 1: the tile list is final when the CTAs start: weights are requested before the wait
 };
 
 namespace ptx {
@@ -160,11 +161,10 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // As in tc_gemm_kernel: the tile list (written by the router, two or more kernels back) and the weights do not
-  // depend on the kernel in front, so the producer requests the weight boxes of its first stages before the
-  // dependent-launch wait; only the activations have to wait.
+  // As in tc_gemm_kernel: with `early_b` (GEMM-2: the tile list is final long before its CTAs start) the producer
+  // requests the weight boxes of its first stages before the dependent-launch wait; only the activations have to wait.
   int pre = 0;
-  if (warp == 0 && lane == 0) {
+  if (warp == 0 && lane == 0 && a.early_b) {
     const int n_rt = __ldcg(a.n_tiles);
     const int per = n_rt * a.n_col_tiles;
     if ((int)blockIdx.x < per * a.n_split) {
@@ -439,6 +439,7 @@ inline int32_t tc_ffn_f32(TcF32State& s, const swapmoe_config_t& c, void* h, flo
   g1.ldc = c.d_ff; g1.n_col_tiles = c.d_ff / out1; g1.k_blocks = c.d_model / kF32BK; g1.n_split = 1;
   g1.b_rows_per_phys = swiglu ? 2 * c.d_ff : c.d_ff;
   g1.b_rows_gate = swiglu ? c.d_ff : 0;
+  g1.early_b = 0;
   long long work = (long long)max_tiles * g1.n_col_tiles;
   int grid = work > s.sm_count ? s.sm_count : (int)work;
   cudaError_t e = swiglu ? launch_kernel(tc_gemm_f32_kernel<kTcEpiSwigluF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes,
@@ -463,6 +464,7 @@ inline int32_t tc_ffn_f32(TcF32State& s, const swapmoe_config_t& c, void* h, flo
   g2.C = y; g2.tiles = tiles; g2.n_tiles = n_tiles; g2.status = status; g2.split_stride = y_copy_stride;
   g2.ldc = c.d_model; g2.n_col_tiles = n_col2; g2.k_blocks = c.d_ff / kF32BK / split; g2.n_split = split;
   g2.b_rows_per_phys = c.d_model; g2.b_rows_gate = 0;
+  g2.early_b = 1;
   work = (long long)max_tiles * n_col2 * split;
   grid = work > s.sm_count ? s.sm_count : (int)work;
   e = launch_kernel(tc_gemm_f32_kernel<kTcEpiF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes, st,

@@ -137,10 +137,10 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // As in tc_gemm_kernel: the tile list and the weights do not depend on the kernel in front, so each
-  // producer requests the weight boxes of its first stages before the dependent-launch wait.
+  // As in tc_gemm_kernel: with `early_b` each producer requests the weight boxes of its first stages before the
+  // dependent-launch wait.
   int pre = 0;
-  if (warp == 0 && lane == 0) {
+  if (warp == 0 && lane == 0 && a.early_b) {
     const int n_rt = __ldcg(a.n_tiles);
     if (pair < n_rt * a.n_col_tiles) {
       int rt, ct;
@@ -308,7 +308,8 @@ inline int tc_pair_init(int sm_count) {
 inline int32_t tc_ffn_pair(TcState& s, int n_pairs, const swapmoe_config_t& c, void* h, float* y, void* out,
                            const TileDesc* tiles, const int32_t* n_tiles, const int32_t* row_pair, const float* mgate,
                            int max_tiles, int n_tokens, int32_t* status, cudaStream_t st, bool pdl, int64_t* launches,
-                           bool* combined, cudaEvent_t between = nullptr, bool gemm2_pairs = true) {
+                           bool* combined, cudaEvent_t between = nullptr, bool gemm2_pairs = true,
+                           int row_group_forced = 0) {
   if (!s.enabled || !s.arena_bound || n_pairs < 1) return SWAPMOE_ERR_NOT_READY;
   const bool swiglu = c.act == SWAPMOE_ACT_SWIGLU;
   const bool scatter = c.top_k == 1;
@@ -316,11 +317,8 @@ inline int32_t tc_ffn_pair(TcState& s, int n_pairs, const swapmoe_config_t& c, v
   if (c.d_ff % out1 || c.d_model % kPairBN) return SWAPMOE_ERR_UNSUPPORTED;
   const long long pairs = (long long)n_tokens * c.top_k;
   int row_group = 1 << 30;
-  {
-    const char* env = std::getenv("SWAPMOE_ROW_GROUP");
-    if (env) row_group = std::atoi(env) > 0 ? std::atoi(env) : row_group;
-    else if (pairs * (long long)c.d_model * 2 > (48ll << 20)) row_group = 16;   // 16 tiles of 256 rows
-  }
+  if (row_group_forced > 0) row_group = row_group_forced;
+  else if (pairs * (long long)c.d_model * 2 > (48ll << 20)) row_group = 16;   // 16 tiles of 256 rows
   TcGemmArgs g1;
   g1.C = h; g1.status = status; g1.ldc = c.d_ff;
   g1.tiles = tiles; g1.n_tiles = n_tiles;
@@ -331,6 +329,7 @@ inline int32_t tc_ffn_pair(TcState& s, int n_pairs, const swapmoe_config_t& c, v
   g1.row_pair = nullptr; g1.gate = nullptr; g1.top_k = c.top_k;
   g1.row_group = row_group;
   g1.a_box_bytes = kPairABytes;
+  g1.early_b = 0;
   long long work = (long long)max_tiles * g1.n_col_tiles;
   int grid = 2 * (work > n_pairs ? n_pairs : (int)work);
   // weight boxes of 128 rows: kBn1Options[1] for one input matrix, kBn1Options[0] / 2 for SwiGLU's two
@@ -353,6 +352,7 @@ inline int32_t tc_ffn_pair(TcState& s, int n_pairs, const swapmoe_config_t& c, v
   g2.row_pair = row_pair; g2.gate = mgate; g2.top_k = c.top_k;
   g2.row_group = row_group;
   g2.a_box_bytes = kPairABytes;
+  g2.early_b = 1;
   work = (long long)max_tiles * g2.n_col_tiles;
   grid = 2 * (work > n_pairs ? n_pairs : (int)work);
   const bool pdl2 = pdl && between == nullptr;

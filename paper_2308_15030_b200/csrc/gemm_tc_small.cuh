@@ -81,10 +81,10 @@ tc_gemm_small_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   const uint32_t tmem_base = *tmem_slot;
 
   const int n_chunks = a.k_blocks / kps;
-  // As in tc_gemm_kernel: the tile list and the weights do not depend on the kernel in front, so the producer
-  // requests the weight boxes of its first stages before the dependent-launch wait.
+  // As in tc_gemm_kernel: with `early_b` the producer requests the weight boxes of its first stages before the
+  // dependent-launch wait.
   int pre = 0;
-  if (warp == 0 && lane == 0) {
+  if (warp == 0 && lane == 0 && a.early_b) {
     const int n_rt = __ldcg(a.n_tiles);
     if ((int)blockIdx.x < n_rt * a.n_col_tiles) {
       const int ct = (int)blockIdx.x / n_rt, rt = (int)blockIdx.x - ct * n_rt;
@@ -329,7 +329,7 @@ inline int32_t tc_ffn_small(TcState& s, TcSmallCache& cache, const swapmoe_confi
   a1.g.C = h; a1.g.tiles = tiles; a1.g.n_tiles = n_tiles; a1.g.status = status; a1.g.ldc = c.d_ff;
   a1.g.n_col_tiles = c.d_ff / cache.g1.bn; a1.g.k_blocks = c.d_model / kTcBK;
   a1.g.b_rows_per_phys = c.d_ff; a1.g.b_rows_gate = 0; a1.g.a_box_bytes = a_tile; a1.g.row_group = 1 << 30;
-  a1.g.row_pair = nullptr; a1.g.gate = nullptr; a1.g.top_k = c.top_k;
+  a1.g.row_pair = nullptr; a1.g.gate = nullptr; a1.g.top_k = c.top_k; a1.g.early_b = 0;
   a1.kps = cache.g1.kps; a1.n_stages = cache.g1.n_stages; a1.a_tile_bytes = a_tile;
   long long work = (long long)max_tiles * a1.g.n_col_tiles;
   int grid = work > s.sm_count ? s.sm_count : (int)work;
@@ -344,7 +344,7 @@ inline int32_t tc_ffn_small(TcState& s, TcSmallCache& cache, const swapmoe_confi
   a2.g.tiles = tiles; a2.g.n_tiles = n_tiles; a2.g.status = status; a2.g.ldc = c.d_model;
   a2.g.n_col_tiles = c.d_model / cache.g2.bn; a2.g.k_blocks = c.d_ff / kTcBK;
   a2.g.b_rows_per_phys = c.d_model; a2.g.b_rows_gate = 0; a2.g.a_box_bytes = a_tile; a2.g.row_group = 1 << 30;
-  a2.g.row_pair = row_pair; a2.g.gate = mgate; a2.g.top_k = c.top_k;
+  a2.g.row_pair = row_pair; a2.g.gate = mgate; a2.g.top_k = c.top_k; a2.g.early_b = 1;
   a2.kps = cache.g2.kps; a2.n_stages = cache.g2.n_stages; a2.a_tile_bytes = a_tile;
   work = (long long)max_tiles * a2.g.n_col_tiles;
   grid = work > s.sm_count ? s.sm_count : (int)work;

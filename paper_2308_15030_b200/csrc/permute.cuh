@@ -14,26 +14,129 @@ struct ScanArgs {
   float* cnt;                // [E] accumulator of the token counts ("simple scheduling" score)
   float* mimp;               // [E] accumulator of Eq. (1) over the masked routing
   const int32_t* phys_slot;  // [K]
-  int32_t* cta_base;         // [n_cta, K] pairs of the same slot in earlier CTAs
+  int32_t* cta_base;         // [n_cta, K] pairs of the same slot in earlier CTAs (written only by the last-CTA scan)
   int32_t* count;            // [K]
   int32_t* offset;           // [K+1]  exclusive scan of count
   int32_t* pad_offset;       // [K+1]  same with every segment rounded up to kSegAlign rows
   TileDesc* tiles;           // GEMM work list
   int32_t* n_tiles;          // [1]
   float* imp;                // [E] accumulator of Eq. (1)
-  unsigned* ticket;          // [1] router CTAs finished so far (returns to 0)
-  int32_t* done;             // [n_done] per-row-tile progress counters of the fused FFN kernel (zeroed here)
+  unsigned* ticket;          // [1] router CTAs finished so far (returns to 0); nullptr: the router CTAs do not
+                             // scan at all - the permute kernel sums the histograms itself (see below)
   TileDesc* tiles_b;         // optional second work list with tile_rows_b rows per tile (or nullptr)
   int32_t* n_tiles_b;
-  int32_t n_cta, K, E, tile_rows, tile_rows_b, n_done;
+  unsigned long long* touched;   // [1] running total of slots that received at least one pair, or nullptr
+  int32_t n_cta, K, E, tile_rows, tile_rows_b;
 };
 
-// Work of the LAST router CTA to finish (all of its threads call this).  The per-CTA
-// histograms and importance partials written by the other CTAs are first staged into shared
-// memory with coalesced L1-bypassing loads (one latency for everything) when `stage` is large
-// enough, else read in place.  Then thread s walks slot s over the router CTAs in order and lays
-// out the slot (offsets, padded offsets, tile list); thread e adds expert e's partials in CTA
-// order, which fixes the summation order of Eq. (1) run to run.
+// Eq. (1) partial sums are added with ONE association wherever they are reduced: the router CTAs
+// are cut into shares of kRedShare consecutive CTAs, a share is summed in CTA order, and the shares
+// are added in order.  Whether one thread walks a column alone or the shares are summed side by
+// side, the result is the same to the last bit, run to run and path to path.
+constexpr int kRedShare = 16;
+
+__device__ __forceinline__ float reduce_column_serial(const float* src, int n_rows, int C, int col) {
+  float total = 0.f;
+  for (int r0 = 0; r0 < n_rows; r0 += kRedShare) {
+    const int r1 = min(n_rows, r0 + kRedShare);
+    float acc = 0.f;
+#pragma unroll 8
+    for (int r = r0; r < r1; ++r) acc += src[(size_t)r * C + col];
+    total += acc;
+  }
+  return total;
+}
+
+// Slot layout by one warp from the per-slot counts in shared memory: lane l owns slots l and l + 32
+// (K <= 64); offsets, padded offsets and first-tile indices are exclusive prefix sums over the slots,
+// taken with warp scans (tile heights are powers of two: shifts, no divisions - this code runs once,
+// every dependent instruction counts).  s_off / s_pad (shared, may be nullptr) receive the exclusive
+// offsets; with `write_global` the warp also writes count / offset / pad_offset and the tile lists.
+__device__ __forceinline__ void slot_layout_warp(const ScanArgs& a, const int32_t* s_count, int32_t* s_off,
+                                                 int32_t* s_pad, bool write_global) {
+  const int lane = threadIdx.x & 31;
+  const int sh_a = 31 - __clz(a.tile_rows);
+  const bool two_lists = write_global && a.tiles_b != nullptr;
+  const int sh_b = two_lists ? 31 - __clz(a.tile_rows_b) : 0;
+  int c[2], off[2], pad[2], ta[2], tb[2], ph[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int s = lane + 32 * h;
+    c[h] = s < a.K ? s_count[s] : 0;
+    ph[h] = (write_global && s < a.K) ? a.phys_slot[s] : 0;     // issued early: its latency hides behind the scans
+    off[h] = c[h];
+    pad[h] = (c[h] + kSegAlign - 1) & ~(kSegAlign - 1);
+    ta[h] = (c[h] + a.tile_rows - 1) >> sh_a;
+    tb[h] = two_lists ? (c[h] + a.tile_rows_b - 1) >> sh_b : 0;
+  }
+  {
+    // slots whose weights this forward reads: the algorithmic weight traffic of the layer
+    const int nz = __popc(__ballot_sync(0xffffffffu, c[0] > 0)) + __popc(__ballot_sync(0xffffffffu, c[1] > 0));
+    if (write_global && lane == 0 && a.touched != nullptr) atomicAdd(a.touched, (unsigned long long)nz);
+  }
+  // inclusive scans of the four quantities over 64 slots
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u0 = __shfl_up_sync(0xffffffffu, off[h], o), u1 = __shfl_up_sync(0xffffffffu, pad[h], o);
+      const int u2 = __shfl_up_sync(0xffffffffu, ta[h], o), u3 = __shfl_up_sync(0xffffffffu, tb[h], o);
+      if (lane >= o) { off[h] += u0; pad[h] += u1; ta[h] += u2; tb[h] += u3; }
+    }
+  }
+  {
+    const int t0 = __shfl_sync(0xffffffffu, off[0], 31), t1 = __shfl_sync(0xffffffffu, pad[0], 31);
+    const int t2 = __shfl_sync(0xffffffffu, ta[0], 31), t3 = __shfl_sync(0xffffffffu, tb[0], 31);
+    off[1] += t0; pad[1] += t1; ta[1] += t2; tb[1] += t3;
+  }
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int s = lane + 32 * h;
+    if (s < a.K) {
+      const int cnt = c[h];
+      const int padded = (cnt + kSegAlign - 1) & ~(kSegAlign - 1);
+      const int nt = (cnt + a.tile_rows - 1) >> sh_a;
+      const int o_excl = off[h] - cnt, p_excl = pad[h] - padded, t_excl = ta[h] - nt;
+      if (s_off != nullptr) { s_off[s] = o_excl; s_pad[s] = p_excl; }
+      if (!write_global) continue;
+      a.count[s] = cnt;
+      a.offset[s] = o_excl;
+      a.pad_offset[s] = p_excl;
+      for (int i = 0; i < nt; ++i) {
+        TileDesc td;
+        td.phys = ph[h];
+        td.row0 = p_excl + i * a.tile_rows;
+        td.rows = min(a.tile_rows, cnt - i * a.tile_rows);
+        td.slot = s;
+        a.tiles[t_excl + i] = td;
+      }
+      if (s == a.K - 1) {
+        a.offset[a.K] = off[h];
+        a.pad_offset[a.K] = pad[h];
+        *a.n_tiles = ta[h];
+      }
+      if (two_lists) {                         // same segments cut into tiles of another height
+        const int ntb = (cnt + a.tile_rows_b - 1) >> sh_b;
+        const int tb_excl = tb[h] - ntb;
+        for (int i = 0; i < ntb; ++i) {
+          TileDesc td;
+          td.phys = ph[h];
+          td.row0 = p_excl + i * a.tile_rows_b;
+          td.rows = min(a.tile_rows_b, cnt - i * a.tile_rows_b);
+          td.slot = s;
+          a.tiles_b[tb_excl + i] = td;
+        }
+        if (s == a.K - 1) *a.n_tiles_b = tb[h];
+      }
+    }
+  }
+}
+
+// Last-CTA form of the scan (routing without a permutation: swapmoe_route_static; grids of more
+// than 256 router CTAs).  All threads of the LAST router CTA to finish call this: thread s walks
+// slot s over the router CTAs in order (writing the running counts, `cta_base`, when asked), thread
+// e adds expert e's Eq. (1) partials, then warp 0 lays out the slots.  The per-CTA arrays are first
+// staged into shared memory with L1-bypassing copies when `stage` is large enough.
 __device__ __forceinline__ void scan_reduce_block(const ScanArgs& a, void* stage, int stage_bytes) {
   __shared__ int32_t s_count[kMaxSlots];
   const int tid = threadIdx.x;
@@ -87,113 +190,29 @@ __device__ __forceinline__ void scan_reduce_block(const ScanArgs& a, void* stage
 #pragma unroll 16
       for (int c = 0; c < a.n_cta; ++c) {
         const int v = hist[(size_t)c * a.K + s];
-        a.cta_base[(size_t)c * a.K + s] = running;
+        if (a.cta_base != nullptr) a.cta_base[(size_t)c * a.K + s] = running;
         running += v;
       }
       s_count[s] = running;
     }
   }
-  for (int i = tid; i < a.n_done; i += blockDim.x) a.done[i] = 0;
   if (own_e) {
-    const int e = tid;
-    float acc = 0.f;
-#pragma unroll 16
-    for (int c = 0; c < a.n_cta; ++c) acc += impp[(size_t)c * a.E + e];
-    a.imp[e] = old_imp + acc;
-    if (a.cta_cnt != nullptr) {            // token counts: small integers, exact in fp32
-      float n = 0.f;
-#pragma unroll 16
-      for (int c = 0; c < a.n_cta; ++c) n += cntp[(size_t)c * a.E + e];
-      a.cnt[e] = old_cnt + n;
-    }
+    a.imp[tid] = old_imp + reduce_column_serial(impp, a.n_cta, a.E, tid);
+    if (a.cta_cnt != nullptr)                // token counts: small integers, exact in fp32
+      a.cnt[tid] = old_cnt + reduce_column_serial(cntp, a.n_cta, a.E, tid);
   }
-  if (own_s && a.cta_mimp != nullptr) {
-    const int sl = tid;
-    float acc = 0.f;
-#pragma unroll 16
-    for (int c = 0; c < a.n_cta; ++c) acc += mimpp[(size_t)c * a.K + sl];
-    a.mimp[my_expert] += acc;              // slots map to distinct experts: no two threads share a target
-  }
+  if (own_s && a.cta_mimp != nullptr)        // slots map to distinct experts: no two threads share a target
+    a.mimp[my_expert] += reduce_column_serial(mimpp, a.n_cta, a.K, tid);
   __syncthreads();
-  // Slot layout by the first warp: lane l owns slots l and l + 32 (K <= 64); offsets, padded
-  // offsets and first-tile indices are exclusive prefix sums over the slots, taken with warp scans
-  // (tile heights are powers of two: shifts, no divisions — this code runs once, every dependent
-  // instruction counts).
-  if (tid < 32) {
-    const int lane = tid;
-    const int sh_a = 31 - __clz(a.tile_rows);
-    const int sh_b = a.tiles_b != nullptr ? 31 - __clz(a.tile_rows_b) : 0;
-    int c[2], off[2], pad[2], ta[2], tb[2];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int s = lane + 32 * h;
-      c[h] = s < a.K ? s_count[s] : 0;
-      off[h] = c[h];
-      pad[h] = (c[h] + kSegAlign - 1) & ~(kSegAlign - 1);
-      ta[h] = (c[h] + a.tile_rows - 1) >> sh_a;
-      tb[h] = a.tiles_b != nullptr ? (c[h] + a.tile_rows_b - 1) >> sh_b : 0;
-    }
-    // inclusive scans of the four quantities over 64 slots
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int u0 = __shfl_up_sync(0xffffffffu, off[h], o), u1 = __shfl_up_sync(0xffffffffu, pad[h], o);
-        const int u2 = __shfl_up_sync(0xffffffffu, ta[h], o), u3 = __shfl_up_sync(0xffffffffu, tb[h], o);
-        if (lane >= o) { off[h] += u0; pad[h] += u1; ta[h] += u2; tb[h] += u3; }
-      }
-    }
-    {
-      const int t0 = __shfl_sync(0xffffffffu, off[0], 31), t1 = __shfl_sync(0xffffffffu, pad[0], 31);
-      const int t2 = __shfl_sync(0xffffffffu, ta[0], 31), t3 = __shfl_sync(0xffffffffu, tb[0], 31);
-      off[1] += t0; pad[1] += t1; ta[1] += t2; tb[1] += t3;
-    }
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int s = lane + 32 * h;
-      if (s < a.K) {
-        const int cnt = c[h];
-        const int padded = (cnt + kSegAlign - 1) & ~(kSegAlign - 1);
-        const int nt = (cnt + a.tile_rows - 1) >> sh_a;
-        const int o_excl = off[h] - cnt, p_excl = pad[h] - padded, t_excl = ta[h] - nt;
-        a.count[s] = cnt;
-        a.offset[s] = o_excl;
-        a.pad_offset[s] = p_excl;
-        const int ph = a.phys_slot[s];
-        for (int i = 0; i < nt; ++i) {
-          TileDesc td;
-          td.phys = ph;
-          td.row0 = p_excl + i * a.tile_rows;
-          td.rows = min(a.tile_rows, cnt - i * a.tile_rows);
-          td.slot = s;
-          a.tiles[t_excl + i] = td;
-        }
-        if (s == a.K - 1) {
-          a.offset[a.K] = off[h];
-          a.pad_offset[a.K] = pad[h];
-          *a.n_tiles = ta[h];
-        }
-        if (a.tiles_b != nullptr) {            // same segments cut into tiles of another height
-          const int ntb = (cnt + a.tile_rows_b - 1) >> sh_b;
-          const int tb_excl = tb[h] - ntb;
-          for (int i = 0; i < ntb; ++i) {
-            TileDesc td;
-            td.phys = ph;
-            td.row0 = p_excl + i * a.tile_rows_b;
-            td.rows = min(a.tile_rows_b, cnt - i * a.tile_rows_b);
-            td.slot = s;
-            a.tiles_b[tb_excl + i] = td;
-          }
-          if (s == a.K - 1) *a.n_tiles_b = tb[h];
-        }
-      }
-    }
-  }
+  if (tid < 32) slot_layout_warp(a, s_count, nullptr, nullptr, true);
 }
 
-// Called by every thread of a router CTA after its partials are written: the CTA
-// that draws the last ticket runs the scan.  No CTA waits for another.
+// Called by every thread of a router CTA after its partials are written.  With a ticket counter the
+// CTA that draws the last ticket runs the scan (no CTA waits for another); without one the router
+// CTAs are done: the permute kernel sums the per-CTA histograms itself.
 __device__ __forceinline__ void finish_router_cta(const ScanArgs& a, void* stage = nullptr, int stage_bytes = 0) {
+  if (threadIdx.x == 0) SWAPMOE_STAMP(0, 7);
+  if (a.ticket == nullptr) return;
   __shared__ int s_last;
   __threadfence();
   __syncthreads();
@@ -206,39 +225,113 @@ __device__ __forceinline__ void finish_router_cta(const ScanArgs& a, void* stage
     __threadfence();
     scan_reduce_block(a, stage, stage_bytes);
     if (threadIdx.x == 0) *a.ticket = 0u;
+    if (threadIdx.x == 0) SWAPMOE_STAMP(0, 9);
   }
 }
 
 struct PermuteArgs {
   const void* x;              // [T, d]
   const int32_t* slot;        // [T*k]
-  const int32_t* cta_base;    // [n_cta, K]
-  const int32_t* offset;      // [K+1]
-  const int32_t* pad_offset;  // [K+1]
+  const int32_t* cta_base;    // [n_cta, K] pairs of the same slot in earlier router CTAs  } read when the router's
+  const int32_t* offset;      // [K+1]                                                      } last CTA scanned
+  const int32_t* pad_offset;  // [K+1]                                                      } (own_scan == 0)
   int32_t* perm;              // [T*k]
   int32_t* inv;               // [T*k]
   int32_t* inv_pad;           // [T*k] row of the pair in the padded workspace
   int32_t* row_pair;          // [rows_pad] flat pair index stored in each occupied padded row
   void* xp;                   // [rows_pad, d]
   int32_t T, d, k, K, tok_tile;
+  int32_t own_scan;           // 1: this kernel sums the router's per-CTA histograms itself (scan.*), CTA (0, 0)
+                              // publishes count / offset / pad_offset / tile lists, and the extra CTA column
+                              // blockIdx.x == scan.n_cta reduces the Eq. (1) partials
+  ScanArgs scan;
 };
 
 constexpr int kPermThreads = 512;
 
+// The Eq. (1) reduction of the forward (one CTA of the permute kernel, off everybody's critical path):
+// work item (share, column) sums its kRedShare router CTAs in order; thread `column` then adds the
+// shares in order - the association of reduce_column_serial.
+__device__ __forceinline__ float reduce_columns_parallel(const float* src, int n_rows, int C, float* s_red,
+                                                         int cap_floats) {
+  const int tid = threadIdx.x;
+  const int n_share = (n_rows + kRedShare - 1) / kRedShare;
+  const int cols_per_pass = max(1, min(C, cap_floats / n_share));    // columns whose shares fit the buffer at once
+  float total = 0.f;
+  for (int c0 = 0; c0 < C; c0 += cols_per_pass) {
+    const int nc = min(cols_per_pass, C - c0);
+    for (int w = tid; w < n_share * nc; w += kPermThreads) {
+      const int sh = w / nc, col = c0 + (w - sh * nc);
+      const int r0 = sh * kRedShare, r1 = min(n_rows, r0 + kRedShare);
+      float v[kRedShare];
+#pragma unroll
+      for (int u = 0; u < kRedShare; ++u) v[u] = r0 + u < r1 ? src[(size_t)(r0 + u) * C + col] : 0.f;   // all in flight together
+      float acc = 0.f;
+#pragma unroll
+      for (int u = 0; u < kRedShare; ++u) acc += v[u];       // adding 0.f beyond the last row changes nothing
+      s_red[w] = acc;
+    }
+    __syncthreads();
+    if (tid >= c0 && tid < c0 + nc)
+      for (int sh = 0; sh < n_share; ++sh) total += s_red[sh * nc + (tid - c0)];
+    __syncthreads();
+  }
+  return total;
+}
+
 // One CTA = the pairs of tok_tile (<= 128) tokens in flat order p = t*k + j.  The rank of a
-// pair among the pairs of the same slot is: pairs in earlier CTAs (cta_base) +
+// pair among the pairs of the same slot is: pairs in earlier CTAs +
 // pairs in earlier warps of this CTA + earlier lanes of this warp (match + popc),
 // which is exactly a stable counting sort.  gridDim.y CTAs share one token tile: each
 // recomputes the (cheap) positions and copies every gridDim.y-th row of the tile.
 // The kernel is a chain of memory round trips, so the independent ones are started together:
 // the token rows (inputs of the layer, so even before the wait on the predecessor) go to
-// registers while the slots, the CTA's base counts and the offsets are fetched.
+// registers while the slots and the histograms are fetched.
+//
+// own_scan: the router CTAs only left their per-CTA slot histograms [n_cta, K].  Every CTA here adds
+// the rows of all router CTAs (slot totals -> offsets) and of the router CTAs in front of its token
+// tile (its base counts): thread (share, slot) adds a contiguous share of the rows, thread `slot` adds
+// the shares.  That is 8 KB of L2 reads per CTA at 2048 tokens, in place of a serial scan by the last
+// router CTA that kept every other SM waiting for a third of the router's duration.
 template <typename T>
 __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const PermuteArgs a) {
-  __shared__ int32_t wcount[kPermThreads / 32][kMaxSlots];
-  __shared__ int32_t dst_row[kPermThreads];
-  __shared__ int32_t s_base[kMaxSlots], s_off[kMaxSlots], s_pad[kMaxSlots];
+  // 11 KB of shared memory, so that these CTAs fit beside a router CTA (over 210 KB) and are already
+  // waiting when the router finishes.  The reducing CTAs use the same bytes for their shares.
+  constexpr int kRawBytes = (kPermThreads / 32) * kMaxSlots * 4 + kPermThreads * 4 + 4 * kMaxSlots * 4 + 2 * kPermThreads * 4;
+  __shared__ __align__(16) unsigned char s_raw[kRawBytes];
+  int32_t (*wcount)[kMaxSlots] = reinterpret_cast<int32_t (*)[kMaxSlots]>(s_raw);
+  int32_t* dst_row = reinterpret_cast<int32_t*>(s_raw + (kPermThreads / 32) * kMaxSlots * 4);
+  int32_t* s_base = dst_row + kPermThreads;
+  int32_t* s_off = s_base + kMaxSlots;
+  int32_t* s_pad = s_off + kMaxSlots;
+  int32_t* s_tot = s_pad + kMaxSlots;
+  int32_t (*s_part)[kPermThreads] = reinterpret_cast<int32_t (*)[kPermThreads]>(s_tot + kMaxSlots);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // the next kernel's CTAs may be scheduled at once: they stop at their own wait, and until then they
+  // touch nothing this kernel or the router writes
+  pdl_trigger();
+  if (a.own_scan && (int)blockIdx.x == a.scan.n_cta) {
+    // ---- the Eq. (1) reductions: CTA y of this extra column takes the scores y, y + gridDim.y, ... of
+    // {Eq. (1), token counts, Eq. (1) over the masked routing}, so that each is done long before the copying CTAs are
+    const ScanArgs& sc = a.scan;
+    pdl_wait();
+    if (tid == 0) SWAPMOE_STAMP(1, 4 + 2 * min((int)blockIdx.y, 2));
+    float* s_red = reinterpret_cast<float*>(s_raw);
+    for (int which = (int)blockIdx.y; which < 3; which += (int)gridDim.y) {
+      const float* src = which == 0 ? sc.cta_imp : which == 1 ? sc.cta_cnt : sc.cta_mimp;
+      if (src == nullptr) continue;
+      const int C = which == 2 ? sc.K : sc.E;
+      float* acc = which == 0 ? sc.imp : which == 1 ? sc.cnt : sc.mimp;
+      // thread c owns column c: expert c, or for the masked score the expert that slot c serves
+      const int target = tid < C ? (which == 2 ? sc.s2e[tid] : tid) : 0;
+      const float old = tid < C ? acc[target] : 0.f;
+      const float v = reduce_columns_parallel(src, sc.n_cta, C, s_red, kRawBytes / 4);
+      if (tid < C) acc[target] = old + v;
+    }
+    if (tid == 0) SWAPMOE_STAMP(1, 5 + 2 * min((int)blockIdx.y, 2));
+    return;
+  }
+  if (tid == 0 && blockIdx.y == 0) SWAPMOE_STAMP(1, 0);
   const int npair = a.tok_tile * a.k;          // <= 512
   const int nwarp_p = (npair + 31) >> 5;
   const int p0 = blockIdx.x * npair;
@@ -263,11 +356,40 @@ __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const Perm
     }
   }
   pdl_wait();
-  pdl_trigger();
+  if (tid == 0 && blockIdx.y == 0) SWAPMOE_STAMP(1, 1);
   int s = -1, rank = 0;
   const int p = p0 + tid;
   if (tid < npair && p < n_total) s = a.slot[p];
-  if (tid < a.K) {
+  if (a.own_scan) {
+    // thread (share, slot): the histogram rows of a contiguous share of the router CTAs, all loads in flight together
+    const int K = a.K, n_cta = a.scan.n_cta, n_before = (int)blockIdx.x;
+    const int PK = kPermThreads / K;                       // shares per slot
+    const int R = (n_cta + PK - 1) / PK;                   // router CTAs per share (<= 8 up to 256 CTAs, K = 16)
+    const int sh = tid / K, col = tid - sh * K;
+    if (sh < PK) {
+      int tot = 0, before = 0;
+      const int c0 = sh * R, c1 = min(n_cta, c0 + R);
+      for (int cb = c0; cb < c1; cb += 8) {
+        int v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = cb + u < c1 ? a.scan.cta_hist[(size_t)(cb + u) * K + col] : 0;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { tot += v[u]; before += cb + u < n_before ? v[u] : 0; }
+      }
+      s_part[0][tid] = tot;
+      s_part[1][tid] = before;
+    }
+    __syncthreads();
+    if (tid < K) {
+      int tot = 0, before = 0;
+#pragma unroll 8
+      for (int q = 0; q < PK; ++q) { tot += s_part[0][q * K + tid]; before += s_part[1][q * K + tid]; }
+      s_tot[tid] = tot;
+      s_base[tid] = before;
+    }
+    __syncthreads();
+    if (warp == 0) slot_layout_warp(a.scan, s_tot, s_off, s_pad, blockIdx.x == 0 && blockIdx.y == 0);
+  } else if (tid < a.K) {
     s_base[tid] = a.cta_base[(size_t)blockIdx.x * a.K + tid];
     s_off[tid] = a.offset[tid];
     s_pad[tid] = a.pad_offset[tid];
@@ -296,6 +418,7 @@ __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const Perm
     dst_row[tid] = -1;
   }
   __syncthreads();
+  if (tid == 0 && blockIdx.y == 0) SWAPMOE_STAMP(1, 2);
   // Gather: copy each pair's token row into its slot segment, 16 bytes per access.
   uint4* dst = static_cast<uint4*>(a.xp);
 #pragma unroll
@@ -316,6 +439,7 @@ __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const Perm
       dst[(size_t)row * vec_per_row + v] = src[(size_t)t * vec_per_row + v];
     }
   }
+  if (tid == 0 && blockIdx.y == 0) SWAPMOE_STAMP(1, 3);
 }
 
 struct CombineArgs {

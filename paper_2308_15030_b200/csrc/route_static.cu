@@ -18,8 +18,8 @@ namespace {
 constexpr int kStaticMaxTokens = SWAPMOE_ROUTE_STATIC_MAX_TOKENS;
 constexpr int kStaticMaxCta = (kStaticMaxTokens + kTokTile - 1) / kTokTile;
 constexpr int kStaticMaxPairs = kStaticMaxTokens * kMaxTopK;
-constexpr int kSimtBMStatic = 64;   // row-tile height used for the (unused) tile list
-constexpr int kStaticMaxTiles = kStaticMaxPairs / kSimtBMStatic + kMaxSlots;
+constexpr int kStaticTileRows = 64;   // row-tile height used for the (unused) tile list
+constexpr int kStaticMaxTiles = kStaticMaxPairs / kStaticTileRows + kMaxSlots;
 
 // Layout of the scratch array (all offsets multiples of 256 bytes).
 constexpr size_t kOffTicket = 0;                                          // unsigned [1]
@@ -27,12 +27,11 @@ constexpr size_t kOffPhys = 256;                                          // int
 constexpr size_t kOffNTiles = kOffPhys + 256;                             // int32 [1]
 constexpr size_t kOffPad = kOffNTiles + 256;                              // int32 [kMaxSlots + 1]
 constexpr size_t kOffHist = kOffPad + 512;                                // int32 [cta][K]
-constexpr size_t kOffBase = kOffHist + sizeof(int32_t) * kStaticMaxCta * kMaxSlots;
-constexpr size_t kOffImp = kOffBase + sizeof(int32_t) * kStaticMaxCta * kMaxSlots;   // float [cta][E]
+constexpr size_t kOffImp = kOffHist + sizeof(int32_t) * kStaticMaxCta * kMaxSlots;   // float [cta][E]
 constexpr size_t kOffTiles = kOffImp + sizeof(float) * kStaticMaxCta * kMaxE;        // TileDesc [tiles]
 constexpr size_t kScratchBytes = kOffTiles + ((sizeof(TileDesc) * kStaticMaxTiles + 255) / 256) * 256;
 
-// Every GPU that loads this library holds this array (about 0.4 MB) until the process exits.
+// Every GPU that loads this library holds this array (about 0.35 MB) until the process exits.
 static __device__ __align__(256) unsigned char g_route_scratch[kScratchBytes];
 
 // In host code `g_route_scratch` is only a host-side stand-in for the symbol, not a
@@ -98,17 +97,16 @@ extern "C" int32_t swapmoe_route_static(const void* x_dev, const void* Wr_dev, c
   ScanArgs& sa = ra.scan;
   sa.cta_hist = ra.cta_hist; sa.cta_imp = ra.cta_imp;
   sa.phys_slot = reinterpret_cast<const int32_t*>(s + kOffPhys);
-  sa.cta_base = reinterpret_cast<int32_t*>(s + kOffBase);
+  sa.cta_base = nullptr;                       // per-CTA running counts: only a permutation would need them
   sa.count = count_dev; sa.offset = offset_dev;
   sa.pad_offset = reinterpret_cast<int32_t*>(s + kOffPad);
   sa.tiles = reinterpret_cast<TileDesc*>(s + kOffTiles);
   sa.n_tiles = reinterpret_cast<int32_t*>(s + kOffNTiles);
   sa.imp = imp_dev;
   sa.ticket = reinterpret_cast<unsigned*>(s + kOffTicket);
-  sa.done = nullptr; sa.n_done = 0;
-  sa.tiles_b = nullptr; sa.n_tiles_b = nullptr; sa.tile_rows_b = 0;
+  sa.tiles_b = nullptr; sa.n_tiles_b = nullptr; sa.tile_rows_b = 0; sa.touched = nullptr;
   sa.cta_cnt = nullptr; sa.cta_mimp = nullptr; sa.s2e = nullptr; sa.cnt = nullptr; sa.mimp = nullptr;
-  sa.n_cta = n_cta; sa.K = K; sa.E = E; sa.tile_rows = kSimtBMStatic;
+  sa.n_cta = n_cta; sa.K = K; sa.E = E; sa.tile_rows = kStaticTileRows;
   if (dtype == SWAPMOE_BF16)
     router_gate_fn<bf16>(E)<<<n_cta, 256, router_smem_bytes(E), st>>>(ra);
   else

@@ -4,7 +4,7 @@
 #pragma once
 #include "common.cuh"
 #include "gate_epilogue.cuh"
-#include "gemm_simt.cuh"
+#include "gemm_mma.cuh"
 #include "permute.cuh"
 #include "router_args.cuh"
 

@@ -109,6 +109,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
     router_prefetch_role(a, a.scan.n_cta);
     return;
   }
+  if (threadIdx.x == 0) SWAPMOE_STAMP(0, 0);
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -152,6 +153,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
   }
   pdl_wait();
   pdl_trigger();
+  if (tid == 0) SWAPMOE_STAMP(0, 1);
   {
     // token t is copied by the kDecWarps / TOK warps t, t + TOK, ...; four independent loads per lane and round
     constexpr int kWpt = kDecWarps / TOK;                   // warps per token: 2 or 1
@@ -190,6 +192,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
     ss = warp_sum(ss);
     if (lane == 0) Q->xn[warp] = sqrtf(ss);
   }
+  if (tid == 0) SWAPMOE_STAMP(0, 2);
   bool alive = true;
 #pragma unroll 1
   for (int w = 0; w < n_rw; ++w) {
@@ -203,6 +206,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
   if (!alive)
     for (int i = tid; i < TOK * (kMaxE + 1); i += kDecThreads) slog[i] = 0.f;
   __syncthreads();
+  if (tid == 0) SWAPMOE_STAMP(0, 3);
   if constexpr (NT == 2) {
     // sixteen tokens, sixteen warps: a warp computes both gates of its token in one interleaved pass
     const int t = warp;
@@ -280,12 +284,14 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
     }
   }
   }
+  if (tid == 0) SWAPMOE_STAMP(0, 4);
 #pragma unroll 1
   for (int i = tid; i < T * E; i += kDecThreads) {
     const int t = i / E, e = i - t * E;
     a.logits[(size_t)(tok0 + t) * E + e] = alive ? slog[t * (kMaxE + 1) + e] : 0.f;
   }
   __syncthreads();
+  if (tid == 0) SWAPMOE_STAMP(0, 5);
   // per-CTA partial sums in pair order (at most 32 pairs): fixed order, run to run
   if (tid < E) {
     float s = 0.f;
@@ -311,7 +317,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
     const uint64_t t0 = ptx::globaltimer_ns();
     while (ptx::globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
   }
+  if (tid == 0) SWAPMOE_STAMP(0, 6);
   finish_router_cta(a.scan, ring, 2 * kDecHalfBytes);       // the wave buffers are free: stage the scan inputs there
+  if (tid == 0) SWAPMOE_STAMP(0, 10);
 }
 
 }  // namespace swapmoe

@@ -10,7 +10,7 @@
 #include "permute.cuh"
 #include "router_args.cuh"
 #include "router_small.cuh"
-#include "gemm_simt.cuh"
+#include "gemm_mma.cuh"
 
 namespace swapmoe {
 

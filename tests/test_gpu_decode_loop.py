@@ -13,7 +13,8 @@ from paper_2308_15030_b200 import inputs as I
 pytestmark = pytest.mark.gpu
 
 
-def _build(cfg, L, B, steps, frequency, lag, spare, loads_per_step=1):
+def _build(cfg, L, B, steps, frequency, lag, spare, loads_per_step=1, Ks=None, **stack_kw):
+    """Ks: per-layer resident budgets (default cfg.K everywhere); stack_kw goes to DecodeStack."""
     import torch
     from harness import to_device
     from paper_2308_15030_b200 import binding
@@ -21,8 +22,10 @@ def _build(cfg, L, B, steps, frequency, lag, spare, loads_per_step=1):
     host = []
     states = []
     tdt = torch.bfloat16 if cfg.dtype == I.BF16 else torch.float32
+    Ks = [cfg.K] * L if Ks is None else list(Ks)
     for l in range(L):
         c = cfg.scaled(seed=1000 + l)
+        K = Ks[l]
         Wr, enorm = I.make_router(c), I.make_enorm(c)
         w_in = np.empty((cfg.E, cfg.nin, cfg.f, cfg.d), np.float32)
         w_out = np.empty((cfg.E, cfg.d, cfg.f), np.float32)
@@ -33,23 +36,33 @@ def _build(cfg, L, B, steps, frequency, lag, spare, loads_per_step=1):
             h_out = torch.from_numpy(I.bf16_bits(w_out).view(np.int16)).view(torch.bfloat16).pin_memory()
         else:
             h_in, h_out = torch.from_numpy(w_in).pin_memory(), torch.from_numpy(w_out).pin_memory()
-        P = cfg.K + spare
+        P = K + spare
         a_in = torch.zeros((P, cfg.nin, cfg.f, cfg.d), dtype=tdt, device="cuda")
         a_out = torch.zeros((P, cfg.d, cfg.f), dtype=tdt, device="cuda")
-        s2e = np.arange(cfg.K, dtype=np.int32)                  # arbitrary initial resident set
-        a_in[: cfg.K].copy_(h_in[: cfg.K]); a_out[: cfg.K].copy_(h_out[: cfg.K])
-        layer = binding.Layer(cfg.E, cfg.d, cfg.f, cfg.k, cfg.K, cfg.dtype, cfg.act, cfg.renorm,
+        s2e = np.arange(K, dtype=np.int32)                      # arbitrary initial resident set
+        a_in[:K].copy_(h_in[:K]); a_out[:K].copy_(h_out[:K])
+        layer = binding.Layer(cfg.E, cfg.d, cfg.f, cfg.k, K, cfg.dtype, cfg.act, cfg.renorm,
                               max_tokens=B, spare_slots=spare)
         d_Wr = to_device(Wr, cfg.dtype)
         layer.set_router(d_Wr, enorm)
-        states.append(LayerState(layer, s2e, np.arange(cfg.K, dtype=np.int32), list(range(cfg.K, P)),
-                                 a_in, a_out, h_in, h_out))
+        states.append(LayerState(layer, s2e, np.arange(K, dtype=np.int32), list(range(K, P)),
+                                 a_in, a_out, h_in, h_out, enorm=enorm))
         host.append(dict(Wr=Wr, enorm=enorm, w_in=w_in, w_out=w_out, d_Wr=d_Wr))
     x = I.make_decode_tokens(cfg, [h["Wr"] for h in host], B, steps)      # [steps, L, B, d]
     d_x = to_device(x.reshape(-1, cfg.d), cfg.dtype).reshape(steps, L, B, cfg.d)
     torch.cuda.synchronize()
-    stack = DecodeStack(states, frequency=frequency, loads_per_step=loads_per_step, lag=lag)
+    stack = DecodeStack(states, frequency=frequency, loads_per_step=loads_per_step, lag=lag, **stack_kw)
     return stack, host, x, d_x
+
+
+def _check_replay(cfg, stack, host, x, outs):
+    from harness import TOL_OUT
+    for entry in stack.trace:
+        s, l, s2e, phys = entry
+        assert len(set(phys.tolist())) == len(phys) and len(set(s2e.tolist())) == len(s2e)
+        ref = _replay(cfg, host, x, entry)["out"]
+        err = np.max(np.abs(outs[s, l] - ref)) / max(1e-30, np.max(np.abs(ref)))
+        assert err <= TOL_OUT[cfg.dtype], (s, l, err)
 
 
 def _run(stack, d_x, cfg, steps, L, B):
@@ -164,3 +177,78 @@ def test_decode_loop_through_cuda_graph_matches_replay():
         ref = _replay(cfg, host, x, entry)["out"]
         err = np.max(np.abs(outs[s, l] - ref)) / max(1e-30, np.max(np.abs(ref)))
         assert err <= TOL_OUT[cfg.dtype], (s, l, err)
+
+
+def test_commit_when_ready_with_a_global_load_budget():
+    """Fig. 5 (ii), amortised + asynchronous: at most two loads per step over all layers, and a slot flips
+    only once its copy has landed (nothing ever waits for a copy); the recorded tables replay exactly."""
+    from harness import to_host_f32
+    cfg = I.LayerConfig("decr", I.BF16, T=6, d=128, f=256, E=16, k=1, K=4, zipf_s=1.1, seed=7)
+    L, B, steps = 4, 6, 48
+    stack, host, x, d_x = _build(cfg, L, B, steps, frequency=4, lag=1, spare=2, step_budget=2, commit="ready")
+    outs = to_host_f32(_run(stack, d_x, cfg, steps, L, B).reshape(-1, cfg.d)).reshape(steps, L, B, cfg.d)
+    assert stack.loads > 0 and stack.commits > 0 and stack.stalls == 0
+    assert stack.commits + sum(len(st.pending) for st in stack.layers) == stack.loads
+    _check_replay(cfg, stack, host, x, outs)
+    assert any(set(t[2].tolist()) != set(range(cfg.K)) for t in stack.trace if t[0] == steps - 1)
+
+
+def test_static_pruning_policy():
+    """Section 4.1 "Pruning": the K experts with the largest ||E_i|| are installed once and never change."""
+    import oracle
+    from harness import to_host_f32
+    cfg = I.LayerConfig("decp", I.BF16, T=5, d=128, f=256, E=16, k=1, K=4, zipf_s=1.1, seed=8)
+    L, B, steps = 2, 5, 10
+    stack, host, x, d_x = _build(cfg, L, B, steps, frequency=2, lag=0, spare=1, policy="static_pruning")
+    loads0 = stack.loads
+    outs = to_host_f32(_run(stack, d_x, cfg, steps, L, B).reshape(-1, cfg.d)).reshape(steps, L, B, cfg.d)
+    assert stack.loads == loads0 and not stack.decisions          # no updates during the loop
+    for s, l, s2e, _ in stack.trace:
+        assert set(s2e.tolist()) == set(oracle.topk_importance(host[l]["enorm"], cfg.K).tolist())
+    _check_replay(cfg, stack, host, x, outs)
+
+
+def test_on_demand_policy():
+    """Section 2.1 / 4.1 "On demand": an expert the off-the-shelf gate asks for is loaded before the layer
+    runs (blocking), so with no more distinct requests than slots the output is the unrestricted layer's."""
+    import oracle
+    from harness import to_host_f32, TOL_OUT
+    cfg = I.LayerConfig("deco", I.BF16, T=3, d=128, f=256, E=16, k=1, K=4, zipf_s=1.1, seed=9)
+    L, B, steps = 2, 3, 16
+    stack, host, x, d_x = _build(cfg, L, B, steps, frequency=1 << 30, lag=0, spare=1, policy="on_demand")
+    outs = to_host_f32(_run(stack, d_x, cfg, steps, L, B).reshape(-1, cfg.d)).reshape(steps, L, B, cfg.d)
+    assert stack.blocking_loads > 0 and stack.misses >= stack.blocking_loads and stack.requests == steps * L * B
+    _check_replay(cfg, stack, host, x, outs)
+    for s, l, s2e, _ in stack.trace:
+        h = host[l]
+        uidx, _ = oracle.gate(oracle.logits(x[s, l], h["Wr"]), cfg.k, cfg.renorm)
+        assert set(uidx.reshape(-1).tolist()) <= set(s2e.tolist())          # B <= K: every request is served
+        full = oracle.forward(x[s, l], h["Wr"], h["enorm"], np.arange(cfg.E), h["w_in"], h["w_out"],
+                              k=cfg.k, act=cfg.act, renorm=cfg.renorm)      # all experts resident
+        # the gate value differs (softmax over the resident set, not over all experts); the expert does not
+        r = _replay(cfg, host, x, (s, l, s2e, None))
+        assert np.array_equal(r["midx"], full["midx"])
+
+
+def test_heterogeneous_budgets_in_one_graph():
+    """Section 3.3: the configuration is {frequency, #experts_1..L}.  Layers with K = 8, 12, 16, 24 slots run as
+    ONE CUDA graph per step; tables flip outside the graph; every (step, layer) output replays."""
+    import torch
+    from harness import to_host_f32
+    cfg = I.LayerConfig("dech", I.BF16, T=16, d=128, f=256, E=32, k=1, K=8, zipf_s=1.1, seed=10)
+    Ks = [8, 12, 16, 24] * 3
+    L, B, steps = len(Ks), 16, 12
+    stack, host, x, d_x = _build(cfg, L, B, steps, frequency=4, lag=1, spare=2, Ks=Ks, step_budget=3,
+                                 commit="ready")
+    xbuf = torch.empty((L, B, cfg.d), dtype=d_x.dtype, device="cuda")
+    obuf = torch.empty_like(xbuf)
+    stack.graph_buffers = (xbuf, obuf)
+    outs = torch.empty((steps, L, B, cfg.d), dtype=d_x.dtype, device="cuda")
+    for s in range(steps):
+        stack.step_graph(d_x[s], record=True)
+        outs[s].copy_(obuf)
+    torch.cuda.synchronize()
+    outs = to_host_f32(outs.reshape(-1, cfg.d)).reshape(steps, L, B, cfg.d)
+    assert stack.loads > 0
+    assert [len(t[2]) for t in stack.trace[:L]] == Ks
+    _check_replay(cfg, stack, host, x, outs)

@@ -38,7 +38,7 @@ def test_small_shapes(cfg):
 @pytest.mark.parametrize("act,k,renorm", [(I.ACT_RELU, 1, 0), (I.ACT_SWIGLU, 2, 1)])
 @pytest.mark.parametrize("path", [1, 2])
 def test_both_gemm_paths(path, act, k, renorm):
-    """The CUDA-core and the tcgen05 grouped GEMM must both match the oracle."""
+    """The warp-level mma and the tcgen05 grouped GEMM must both match the oracle."""
     from harness import Case, check_against_oracle
     cfg = _cfg(T=700, d=256, f=512, E=16, K=6, k=k, act=act, renorm=renorm, zipf_s=1.1)
     case = Case(cfg)
@@ -138,16 +138,14 @@ def test_error_codes():
 
 
 # ------------------------------------------------------------------ the named configurations
-@pytest.mark.parametrize("path", ["tcgen05", "mma", "ffma"])
+@pytest.mark.parametrize("path", ["tcgen05", "mma"])
 def test_fp32_gemm_paths(monkeypatch, path):
-    """fp32 layers: split-TF32 on tcgen05 (default), the warp-level mma form (SWAPMOE_FP32_TC=0) and the
-    FFMA form (SWAPMOE_FP32_FFMA=1) all hold the fp32 tolerance; ReLU top-1 with a sliced GEMM-2 and
-    SwiGLU top-2, slots above and below one 128-row tile."""
+    """fp32 layers: split-TF32 on tcgen05 (default) and the warp-level mma form (SWAPMOE_FP32_TC=0) both
+    hold the fp32 tolerance; ReLU top-1 with a sliced GEMM-2 and SwiGLU top-2, slots above and below one
+    128-row tile."""
     from harness import Case, check_against_oracle
     if path == "mma":
         monkeypatch.setenv("SWAPMOE_FP32_TC", "0")
-    if path == "ffma":
-        monkeypatch.setenv("SWAPMOE_FP32_FFMA", "1")
     for cfg in (_cfg(T=700, dtype=I.F32, d=256, f=512, E=8, K=3, zipf_s=1.2),
                 _cfg(T=300, dtype=I.F32, d=128, f=384, E=16, K=5, k=2, act=I.ACT_SWIGLU, renorm=1)):
         case = Case(cfg)
@@ -193,25 +191,90 @@ def test_cfg3_prefill_and_topk_update():
 def test_cfg5_mixtral_shape_sampled():
     """Full-size routing parity on all 4096 tokens; FFN values on a seeded token sample."""
     from harness import Case, check_against_oracle
+    import oracle
     cfg = I.CONFIGS["cfg5"]
     case = Case(cfg)
     out = case.run()
-    sub = np.sort(np.random.default_rng(5).choice(cfg.T, size=48, replace=False)).astype(np.int32)
+    # 256 tokens, stratified over the grouped GEMM's tiles: the oracle's routing (from the GPU's logits)
+    # gives every pair's position; every 128-row half of every 256-row tile of every slot segment gets
+    # at least two checked pairs (a mis-ordered or skipped tile then cannot pass), the rest is random.
+    lg = case.layer.tap("logits")
+    res = np.zeros(cfg.E, bool); res[case.s2e] = True
+    midx, _ = oracle.gate(lg, cfg.k, cfg.renorm, allowed=res.astype(np.int32))
+    slot = oracle.invert_slot_table(case.s2e, cfg.E)[midx]
+    count, offset, perm, _ = oracle.permute(slot, cfg.K)
+    rng = np.random.default_rng(5)
+    picked = set()
+    for s_ in range(cfg.K):
+        for h0 in range(0, int(count[s_]), 128):
+            seg = perm[offset[s_] + h0: offset[s_] + min(h0 + 128, int(count[s_]))]
+            for p in rng.choice(seg, size=min(2, seg.size), replace=False):
+                picked.add(int(p) // cfg.k)
+    n_strat = len(picked)
+    rest = [t for t in rng.permutation(cfg.T) if int(t) not in picked]
+    picked.update(int(t) for t in rest[: max(0, 256 - n_strat)])
+    sub = np.array(sorted(picked), np.int32)
+    assert sub.size >= 256
+    chosen = np.zeros(cfg.T, bool); chosen[sub] = True
+    for s_ in range(cfg.K):
+        for h0 in range(0, int(count[s_]), 128):
+            seg = perm[offset[s_] + h0: offset[s_] + min(h0 + 128, int(count[s_]))]
+            assert int(chosen[seg // cfg.k].sum()) >= min(2, seg.size)
     check_against_oracle(case, out, token_subset=sub)
     assert np.all(np.isfinite(out))
 
 
-def test_fused_ffn_kernel_option(monkeypatch):
-    """SWAPMOE_FUSED_FFN=1 runs both grouped GEMMs in one persistent launch; results must not change."""
+@pytest.mark.parametrize("pair_gemm", ["1", "0"])
+@pytest.mark.parametrize("k,act,renorm,T,K", [(1, I.ACT_RELU, 0, 1500, 5), (2, I.ACT_SWIGLU, 1, 800, 5),
+                                              (1, I.ACT_RELU, 0, 700, 6)])
+def test_grouped_tile_order_forced(monkeypatch, pair_gemm, k, act, renorm, T, K):
+    """The grouped GEMMs walk large activation matrices in groups of row tiles (row tiles fastest inside a
+    group, then column tiles, then the next group).  SWAPMOE_ROW_GROUP=2 forces that order on shapes the
+    oracle checks in full: 256-row tiles on CTA pairs (pairs for both GEMMs: SWAPMOE_PAIR_MIN_ROWS=160) and
+    on one CTA per tile (SWAPMOE_PAIR_GEMM=0), 128-row tiles (the third shape), an odd number of row tiles
+    (ragged last group)."""
     from harness import Case, check_against_oracle
-    monkeypatch.setenv("SWAPMOE_FUSED_FFN", "1")
-    for k, act, renorm in ((1, I.ACT_RELU, 0), (2, I.ACT_SWIGLU, 1)):
-        cfg = _cfg(T=900 // k, d=256, f=512, E=16, K=6, k=k, act=act, renorm=renorm, zipf_s=1.1)
-        case = Case(cfg)
-        n0 = case.layer.launch_count
-        out = case.run()
-        assert case.layer.launch_count - n0 == (3 if k == 1 else 4)
-        check_against_oracle(case, out)
+    monkeypatch.setenv("SWAPMOE_ROW_GROUP", "2")
+    monkeypatch.setenv("SWAPMOE_PAIR_GEMM", pair_gemm)
+    monkeypatch.setenv("SWAPMOE_PAIR_MIN_ROWS", "160")
+    cfg = _cfg(T=T, d=256, f=512, E=12, K=K, k=k, act=act, renorm=renorm, zipf_s=1.3)
+    case = Case(cfg)
+    res = check_against_oracle(case, case.run())
+    cnt = res["oracle"]["count"]
+    tile = 256 if T * k // K >= 160 else 128
+    assert int(np.sum((cnt + tile - 1) // tile)) >= 5           # several groups of two row tiles
+
+
+@pytest.mark.parametrize("dtype,k,act,renorm", [(I.BF16, 2, I.ACT_SWIGLU, 1), (I.BF16, 1, I.ACT_RELU, 0),
+                                                (I.F32, 2, I.ACT_RELU, 0)])
+def test_hidden_and_expert_output_taps(monkeypatch, dtype, k, act, renorm):
+    """Stage-by-stage comparison: the hidden activations h = act(W_in x) and the expert outputs
+    y = W_out h of every pair, as the grouped GEMMs left them in HBM, against the oracle's."""
+    import oracle
+    from harness import Case, check_against_oracle, TOL_OUT
+    from paper_2308_15030_b200 import binding
+    if dtype == I.F32:
+        monkeypatch.setenv("SWAPMOE_FP32_TC", "0")     # the warp-level kernels leave y in one piece at this size
+    cfg = _cfg(T=12000 if dtype == I.F32 else 600, dtype=dtype, d=128, f=256, E=8, K=4, k=k, act=act, renorm=renorm,
+               zipf_s=1.1)
+    case = Case(cfg)
+    out = case.run()
+    h = case.layer.tap("h")
+    if dtype == I.BF16:
+        h = I.bits_to_f32(h)
+    r = check_against_oracle(case, out)["oracle"]
+    ref_h = oracle.expert_hidden(case.x, r["slot"], case.phys, case.a_in, k=k, act=act)[r["perm"]]
+    assert np.max(np.abs(h - ref_h)) <= TOL_OUT[dtype] * np.max(np.abs(ref_h))
+    if k > 1:
+        y = case.layer.tap("y")
+        ref_y = oracle.forward(case.x, case.Wr, case.enorm, case.s2e, case.a_in, case.a_out, k=k, act=act,
+                               renorm=renorm, phys_slot=case.phys, ext_logits=case.layer.tap("logits"),
+                               want_y=True)["y"][r["perm"]]
+        assert np.max(np.abs(y - ref_y)) <= TOL_OUT[dtype] * np.max(np.abs(ref_y))
+    else:
+        with pytest.raises(binding.SwapMoEError) as e:      # top-1: gate * y went straight into `out`
+            case.layer.tap("y")
+        assert e.value.status == -7
 
 
 def test_two_row_subtiles_per_cta():

@@ -10,6 +10,9 @@ its taps) on the same inputs.  fp32 layers run the same router kernel on both si
 everything must agree to the last bit; bf16 layers route through the tensor-core router
 on the regular path, so logits and gates agree to the tolerances of the parity tests
 and indices are compared wherever the deciding logit margin is not a near-tie.
+Each call's outputs are also held against the CPU oracle (fed the call's own logits):
+indices, counts and offsets bit for bit, gate values, token norms and Eq. (1) within
+the tolerances of the parity tests.
 """
 import numpy as np
 import pytest
@@ -46,7 +49,31 @@ def _route_static(case, T):
     return {k: v.cpu().numpy() for k, v in t.items()}
 
 
+def _compare_with_oracle(case, T, got):
+    """The arithmetic itself: logits against the fp64 product, then routing from those very logits."""
+    import oracle
+    from harness import TOL_GATE_ABS, TOL_IMP_REL, TOL_LOGIT_REL
+    cfg = case.cfg
+    x = case.x[:T]
+    ref_l = oracle.logits(x, case.Wr)
+    assert np.max(np.abs(got["logits"] - ref_l)) <= TOL_LOGIT_REL * np.max(np.abs(ref_l))
+    uidx, ugate = oracle.gate(got["logits"], cfg.k, cfg.renorm)
+    res = np.zeros(cfg.E, np.int32); res[case.s2e] = 1
+    midx, mgate = oracle.gate(got["logits"], cfg.k, cfg.renorm, allowed=res)
+    slot = oracle.invert_slot_table(case.s2e, cfg.E)[midx]
+    count, offset, _, _ = oracle.permute(slot, cfg.K)
+    for name, ref in (("uidx", uidx), ("midx", midx), ("slot", slot), ("count", count), ("offset", offset)):
+        assert np.array_equal(got[name], ref.reshape(got[name].shape)), name
+    assert np.max(np.abs(got["ugate"] - ugate)) <= TOL_GATE_ABS
+    assert np.max(np.abs(got["mgate"] - mgate)) <= TOL_GATE_ABS
+    xn = np.linalg.norm(x.astype(np.float64), axis=1)
+    assert np.max(np.abs(got["xnorm"] - xn)) <= 1e-5 * max(1.0, xn.max())
+    imp = oracle.importance(x, uidx, ugate, case.enorm)
+    assert np.max(np.abs(got["imp"] - imp)) <= TOL_IMP_REL * imp.max()
+
+
 def _compare(case, T, got, exact):
+    _compare_with_oracle(case, T, got)
     L = case.layer
     L.read_importance(reset=True)
     L.forward(case.d_x, case.d_out, n_tokens=T)
