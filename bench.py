@@ -463,6 +463,7 @@ def run_per_config(args, peaks):
         torch.cuda.empty_cache()
     dargs = argparse.Namespace(**vars(args))
     dargs.steps, dargs.batches, dargs.sweep_frequency, dargs.sweep_budget, dargs.policies = None, [1, 16, 64], None, None, False
+    dargs.cfg4_variant = "full"
     d = run_decode(dargs, I.CONFIGS["cfg4"])
     out["cfg4"] = {"workload": d["config"]["workload"], "pcie_probe_GBps": d["pcie_probe_GBps"],
                    "per_batch": d["per_batch"], "clocks": d.get("clocks")}
@@ -551,7 +552,8 @@ def run_decode(args, cfg):
             torch.cuda.synchronize()
             for st in stack.layers:
                 st.layer.read_touched_slots(reset=True)
-            base = dict(loads=stack.loads, bytes=stack.bytes_loaded, stalls=stack.stalls, deferred=stack.deferred,
+                st.layer.read_decode_prefetch(reset=True)
+            base = dict(host=stack.host_seconds, waits=stack.throttle_waits, loads=stack.loads, bytes=stack.bytes_loaded, stalls=stack.stalls, deferred=stack.deferred,
                         commits=stack.commits, hits=stack.hits, asked=stack.asked, misses=stack.misses,
                         blocking=stack.blocking_loads, requests=stack.requests, n_ev=len(stack.load_events),
                         launches=sum(st.layer.launch_count for st in stack.layers))
@@ -564,6 +566,7 @@ def run_decode(args, cfg):
             e1.record(); torch.cuda.synchronize()
             ms = e0.elapsed_time(e1)
             touched = sum(st.layer.read_touched_slots(reset=True) for st in stack.layers)
+            pf = [st.layer.read_decode_prefetch(reset=True) for st in stack.layers]
             status = [st.layer.device_status() for st in stack.layers]
             assert all(s_ == (0, 0) for s_ in status), status
             bytes_alg = touched * expert_bytes + steps * L * (2 * B * cfg.d * cfg.nb + cfg.E * cfg.d * cfg.nb)
@@ -577,7 +580,13 @@ def run_decode(args, cfg):
                  "loads": stack.loads - base["loads"], "loaded_GB": nbytes / 1e9,
                  "commits": stack.commits - base["commits"], "stalls": stack.stalls - base["stalls"],
                  "deferred_commits": stack.deferred - base["deferred"],
-                 "pcie_seconds_needed": nbytes / (pcie_gbs * 1e9), "loop_seconds": ms * 1e-3}
+                 "pcie_seconds_needed": nbytes / (pcie_gbs * 1e9), "loop_seconds": ms * 1e-3,
+                 # host time per step spent preparing and enqueuing (waiting for the device excluded), and the share
+                 # of steps before which the device was still busy (else the loop is bound by the host)
+                 "host_ms_per_step": (stack.host_seconds - base["host"]) / steps * 1e3,
+                 "steps_host_waited_for_device": (stack.throttle_waits - base["waits"]) / steps}
+            if sum(t_ for _, t_ in pf) > 0:      # one-launch decode steps: L2 prefetch of the recently served experts
+                r["decode_prefetch_hit_rate"] = sum(h_ for h_, _ in pf) / sum(t_ for _, t_ in pf)
             if load_s > 0:
                 r["loader_GBps"] = nbytes / load_s / 1e9
                 r["loader_frac_of_pcie_probe"] = nbytes / load_s / 1e9 / pcie_gbs
@@ -589,11 +598,15 @@ def run_decode(args, cfg):
             return r
 
         # arm 1: scheduler off (no importance reads, no swaps): what the kernels alone allow
-        no_swap = run_arm(make_stack(frequency=1 << 30))
+        no_swap = run_arm(make_stack(frequency=1 << 30, max_in_flight=3))
         # arm 2: swapping on.  The step's load budget follows the link: what PCIe carries while a step computes.
         budget = suggest_step_budget(no_swap["ms_per_step"] * 1e-3, pcie_gbs, expert_bytes)
+        if args.cfg4_variant == "no_loads":          # diagnostic: decisions only
+            budget = 0.0
         swap = run_arm(make_stack(frequency=args.frequency, loads_per_step=1, step_budget=budget, commit="ready",
-                                  time_loads=True, track_hits=True))
+                                  lag=(10 ** 9 if args.cfg4_variant == "no_commits" else 2),
+                                  time_loads=(B == max(args.batches)), track_hits=True, async_decide=True,
+                                  max_in_flight=3))
         swap["step_budget"] = budget
         swap["slowdown_vs_no_swap"] = swap["us_per_layer"] / no_swap["us_per_layer"]
         entry = {"swap": swap, "no_swap": no_swap}
@@ -602,11 +615,12 @@ def run_decode(args, cfg):
         if args.sweep_frequency and big:
             entry["frequency_sweep"] = {
                 str(fr): run_arm(make_stack(frequency=fr, loads_per_step=1, step_budget=budget, commit="ready",
-                                            track_hits=True)) for fr in args.sweep_frequency}
+                                            track_hits=True, async_decide=True, max_in_flight=3)) for fr in args.sweep_frequency}
         if args.sweep_budget and big:
             entry["budget_sweep"] = {
                 str(bu): run_arm(make_stack(frequency=args.frequency, loads_per_step=max(1, -(-bu // L)), step_budget=bu,
-                                            commit="wait" if args.sweep_commit == "wait" else "ready", track_hits=True))
+                                            commit="wait" if args.sweep_commit == "wait" else "ready", track_hits=True,
+                                            async_decide=True))
                 for bu in args.sweep_budget}
         # Section 4.1 baselines as policies over the same kernels, and per-layer budgets (Section 3.3)
         if args.policies and big:
@@ -615,13 +629,14 @@ def run_decode(args, cfg):
                 Ks = [K] * L
                 pol["K=%d" % K] = {
                     "swap": run_arm(make_stack(Ks, frequency=args.frequency, loads_per_step=1, step_budget=budget,
-                                               commit="ready", track_hits=True)),
+                                               commit="ready", track_hits=True, async_decide=True, max_in_flight=3)),
                     "static_pruning": run_arm(make_stack(Ks, policy="static_pruning")),
                     "on_demand": run_arm(make_stack(Ks, policy="on_demand", lag=0), graph=False)}
             entry["policies_vs_K"] = pol
             Ks = [8, 12, 16, 24] * (L // 4) + [16] * (L % 4)
             entry["per_layer_K"] = dict(run_arm(make_stack(Ks, frequency=args.frequency, loads_per_step=1,
-                                                           step_budget=budget, commit="ready", track_hits=True)), Ks=Ks)
+                                                           step_budget=budget, commit="ready", track_hits=True,
+                                                           async_decide=True)), Ks=Ks)
         results[str(B)] = entry
     clocks = sampler.stop()
     Bmax = str(max(args.batches))
@@ -717,6 +732,8 @@ def main():
                     help="cfg4: also run the loop (largest batch) with these numbers of expert loads per step")
     ap.add_argument("--sweep-commit", default="ready", choices=["ready", "wait"],
                     help="cfg4 budget sweep: flip when the copy has landed, or wait for it at the commit step")
+    ap.add_argument("--cfg4-variant", default="full", choices=["full", "no_loads", "no_commits"],
+                    help="cfg4 diagnostic: swapping arm without expert copies / with copies that are never committed")
     ap.add_argument("--policies", action="store_true",
                     help="cfg4: also run static pruning / on-demand loading / swapping at K = 4, 8, 16 and per-layer K")
     ap.add_argument("--no-per-config", action="store_true",

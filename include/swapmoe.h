@@ -219,6 +219,27 @@ int32_t swapmoe_read_importance_kind(swapmoe_layer_t* layer, int32_t kind, float
                                      int32_t reset, void* stream);
 
 /*
+ * Section 2.2 (activation locality: successive tokens use consistent experts), used by the one-launch
+ * decode step: while its CTAs route, the kernel pulls the weights of the experts this layer served on
+ * its latest steps towards L2 (environment variable SWAPMOE_DECODE_PREFETCH = 1..4 experts; 0, the default, = off),
+ * so that a step that asks for the same expert again reads it from cache.  This call reports how often
+ * that guess was right: *hits_host of the *touched_host slots served by decode steps since the last reset
+ * held a prefetched expert.  Waits for `stream`; reset != 0 zeroes both (ordered on `stream`).
+ */
+int32_t swapmoe_read_decode_prefetch(swapmoe_layer_t* layer, int64_t* hits_host, int64_t* touched_host,
+                                     int32_t reset, void* stream);
+
+/* The same without the wait, for several scores at once: bit k of kinds_mask selects score k
+ * (SWAPMOE_IMP_EQ1 = bit 0, SWAPMOE_IMP_COUNT = bit 1, SWAPMOE_IMP_EQ1_MASKED = bit 2).  One small kernel
+ * enqueued on `stream` writes score k to scores_host_pinned[k * E .. k * E + E) (PINNED host memory of 3 * E
+ * floats, written directly by the device) and, if reset != 0, zeroes the selected accumulators.  The values
+ * are there once the caller has synchronised with the stream (an event recorded after this call).  A scheduler
+ * can thus read the scores of many layers with one wait, or pick them up a step later without ever stalling
+ * the queue of forwards (Section 3.2: updates must not block inference). */
+int32_t swapmoe_read_scores_async(swapmoe_layer_t* layer, int32_t kinds_mask, float* scores_host_pinned,
+                                  int32_t reset, void* stream);
+
+/*
  * Measurement aid (Section 3.3 profiles an expert's memory traffic; here it is counted): the number
  * of Virtual-Expert slots that received at least one (token, j) pair, summed over every forward
  * since the last reset - i.e. how many experts' weights the layer had to read, the algorithmic

@@ -36,6 +36,7 @@ EXPORTS = [
     "swapmoe_debug_copy", "swapmoe_device_status", "swapmoe_launch_count",
     "swapmoe_workspace_bytes", "swapmoe_set_gemm_path", "swapmoe_status_string",
     "swapmoe_route_static", "swapmoe_selftest_bounded_wait", "swapmoe_read_touched_slots",
+    "swapmoe_read_scores_async", "swapmoe_read_decode_prefetch",
 ]
 
 
@@ -88,6 +89,8 @@ def lib() -> ctypes.CDLL:
         L.swapmoe_route_static.argtypes = [vp] * 4 + [i32] * 7 + [vp] * 11
         L.swapmoe_selftest_bounded_wait.argtypes = [vp, i32, vp]
         L.swapmoe_read_touched_slots.argtypes = [vp, vp, i32, vp]
+        L.swapmoe_read_scores_async.argtypes = [vp, i32, vp, i32, vp]
+        L.swapmoe_read_decode_prefetch.argtypes = [vp, vp, vp, i32, vp]
         L.swapmoe_status_string.argtypes = [i32]
         L.swapmoe_status_string.restype = ctypes.c_char_p
         for n in EXPORTS:
@@ -244,6 +247,22 @@ class Layer:
         _check(lib().swapmoe_read_importance(self._h, _np_ptr(imp), int(bool(reset)),
                                              _stream_ptr(stream)), "swapmoe_read_importance")
         return imp
+
+    def read_scores_async(self, kinds: Sequence[str], out_pinned, reset: bool = False, stream=None) -> None:
+        """Enqueues one small kernel that writes the scores named in `kinds` ("eq1", "count", "eq1_masked") into a
+        pinned float32 tensor [3, E] (row 0 / 1 / 2 for the three scores); no wait - synchronise with the stream
+        before reading it."""
+        mask = sum(1 << {"eq1": 0, "count": 1, "eq1_masked": 2}[k] for k in kinds)
+        assert out_pinned.is_pinned() and out_pinned.numel() >= 3 * self.cfg.E
+        _check(lib().swapmoe_read_scores_async(self._h, mask, out_pinned.data_ptr(), int(bool(reset)),
+                                               _stream_ptr(stream)), "swapmoe_read_scores_async")
+
+    def read_decode_prefetch(self, reset: bool = False, stream=None):
+        """(hits, touched): slots served by one-launch decode steps whose expert had been prefetched to L2, and all."""
+        h, t = ctypes.c_int64(0), ctypes.c_int64(0)
+        _check(lib().swapmoe_read_decode_prefetch(self._h, ctypes.byref(h), ctypes.byref(t), int(bool(reset)),
+                                                  _stream_ptr(stream)), "swapmoe_read_decode_prefetch")
+        return int(h.value), int(t.value)
 
     def read_touched_slots(self, reset: bool = False, stream=None) -> int:
         """Slots that received at least one pair, summed over the forwards since the last reset."""

@@ -38,6 +38,9 @@ struct swapmoe_layer {
   int32_t *uidx, *midx, *slot, *cta_hist, *cta_base, *count, *offset, *pad_offset;
   int32_t *perm, *inv, *inv_pad, *row_pair, *n_tiles, *e2s, *phys, *s2e, *status;
   unsigned* ticket;
+  int32_t* dec_recent;         // one-launch decode path: experts served most recently (device)
+  unsigned long long* dec_pf_stats;   // ... and how often its L2 prefetch of them was right (device)
+  int32_t dec_pf_depth;        // recently served experts to prefetch while routing (SWAPMOE_DECODE_PREFETCH, 0 = off)
   unsigned long long* touched; // running total of slots that received at least one pair (device)
   bool small_path;             // small-batch GEMM kernels for <= 64 pairs
   TcSmallCache small;
@@ -74,6 +77,7 @@ struct swapmoe_layer {
   int32_t router_tok;          // 0 = automatic token-tile size of the tensor-core router, else 32/64/128
   bool prefetch;               // pull resident weights into L2 from the router kernel
   long long l2_prefetch_bytes; // how much of them (L2 capacity minus head room)
+  bool fp32_swap;              // fp32 layers: swapped-operand GEMM for small slots
   int prefetch_min_pairs;      // ... when the batch has at least this many HALF pairs per slot (SWAPMOE_PREFETCH_MIN_PAIRS)
   void* const* stage_events;   // 7 cudaEvent_t of the forward being enqueued, or nullptr
   CUtensorMap map_x;           // TMA view of the last token matrix [T, d]
@@ -99,6 +103,21 @@ struct Carver {
 };
 
 inline bool cuda_ok(cudaError_t e) { return e == cudaSuccess; }
+
+// One small launch copies the selected per-expert scores of a layer into mapped pinned host memory and zeroes
+// them: a pair of tiny memcpy / memset nodes per score costs 10-15 us of stream time each, which a decode step of
+// a few hundred microseconds cannot afford twelve layers at a time.
+struct ScoreSnapshot { float* acc[3]; float* dst; int E, mask, reset; };
+__global__ void snapshot_scores_kernel(const ScoreSnapshot s) {
+  for (int k = 0; k < 3; ++k) {
+    if (!((s.mask >> k) & 1)) continue;
+    for (int e = threadIdx.x; e < s.E; e += blockDim.x) {
+      s.dst[k * s.E + e] = s.acc[k][e];
+      if (s.reset) s.acc[k][e] = 0.f;
+    }
+  }
+  __threadfence_system();
+}
 
 struct EnormTable { float v[kMaxE]; };
 __global__ void set_enorm_kernel(const EnormTable t, int E, float* enorm) {
@@ -129,6 +148,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     const size_t n_jb = c.d_ff / kDecJB;
     da.ypart = L->dec_ws; da.gpart = L->dec_ws + n_jb * (size_t)(kDecMaxTokens * c.top_k) * c.d_model;
     da.tickets = L->dec_tickets; da.out = static_cast<bf16*>(out); da.status = L->status; da.touched = L->touched;
+    da.recent = L->dec_recent; da.pf_stats = L->dec_pf_stats; da.pf_depth = L->dec_pf_depth;
     da.T = T; da.d = c.d_model; da.f = c.d_ff; da.E = c.E; da.k = c.top_k; da.K = c.K; da.renorm = c.renorm_topk;
     da.swiglu = c.act == SWAPMOE_ACT_SWIGLU;
     mark(L, 0, st);
@@ -157,7 +177,10 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   const bool use_pairs = use_tc && tc_use_pairs(c, T, L->gemm_pairs, L->pair_min_rows);
   const int mt = use_tc ? tc_row_subtiles(c, T, use_pairs) : 1;
   const bool use_tc32 = !use_tc && L->tc32.enabled && L->tc32.arena_bound;
-  const int tile_rows = use_tc ? kTcBM * mt : (use_tc32 ? kTcBM : kMmaBM);
+  // fp32 layers whose slots hold well under 128 rows on average: weights on the MMA's rows, the slot's tokens on its
+  // columns (64-token tiles), so that no tensor time goes to empty rows (SWAPMOE_FP32_SWAP=0: never)
+  const bool swap32 = use_tc32 && L->tc32.swap_ok && L->fp32_swap && (long long)n_pairs < 96ll * c.K;
+  const int tile_rows = use_tc ? kTcBM * mt : (use_tc32 ? (swap32 ? kF32SwapTok : kTcBM) : kMmaBM);
   const int max_tiles = (n_pairs + tile_rows - 1) / tile_rows + c.K;
 
   RouterArgs ra;
@@ -236,6 +259,13 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   L->launches++;
   mark(L, 1, st);   // the slot scan and importance reduction run inside the router's last CTA
 
+  // enough permute CTAs to fill the GPU: every row-group of a token tile gets its own CTA
+  int groups_planned = (2 * L->sm_count + n_cta - 1) / n_cta;
+  {
+    const int max_groups = (tok_tile * c.top_k + 7) / 8;
+    if (groups_planned > max_groups) groups_planned = max_groups;
+    if (groups_planned < 1) groups_planned = 1;
+  }
   PermuteArgs pa;
   pa.x = x; pa.slot = L->slot; pa.cta_base = L->cta_base; pa.offset = L->offset;
   pa.pad_offset = L->pad_offset; pa.perm = L->perm; pa.inv = L->inv; pa.inv_pad = L->inv_pad;
@@ -244,13 +274,9 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   pa.own_scan = own_scan ? 1 : 0;
   pa.scan = sa;
   mark(L, 2, st);
-  // enough CTAs to fill the GPU: every row-group of a token tile gets its own CTA
-  int groups = (2 * L->sm_count + n_cta - 1) / n_cta;
-  const int max_groups = (tok_tile * c.top_k + 7) / 8;
-  if (groups > max_groups) groups = max_groups;
-  if (groups < 1) groups = 1;
-  // own_scan: one extra column of CTAs, whose first CTA reduces the Eq. (1) partials
-  if (launch_kernel(permute_gather_kernel<DT>, dim3(n_cta + (own_scan ? 1 : 0), groups), dim3(kPermThreads), 0, st, pdl, pa) !=
+  const int groups = groups_planned;
+  // own_scan: three extra columns of CTAs, whose first CTAs reduce the three per-expert scores
+  if (launch_kernel(permute_gather_kernel<DT>, dim3(n_cta + (own_scan ? 3 : 0), groups), dim3(kPermThreads), 0, st, pdl, pa) !=
       cudaSuccess)
     return SWAPMOE_ERR_CUDA;
   L->launches++;
@@ -279,7 +305,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   } else if (use_tc32) {
     cudaEvent_t mid = L->stage_events ? static_cast<cudaEvent_t>(L->stage_events[4]) : nullptr;
     const int32_t rc = tc_ffn_f32(L->tc32, c, L->h, L->y, (long long)L->rows_pad_max * c.d_model, L->y_copies, L->tiles,
-                                  L->n_tiles, max_tiles, T, L->status, st, pdl, &L->launches, &y_split, mid);
+                                  L->n_tiles, max_tiles, T, L->status, st, pdl, &L->launches, &y_split, mid, swap32);
     if (rc != SWAPMOE_OK) return rc;
   } else {
     MmaGemmArgs g1;
@@ -415,15 +441,14 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
     L->small_path = !(env && env[0] == '0');
     env = std::getenv("SWAPMOE_ROW_GROUP");             // row tiles per scheduling group of the grouped GEMMs
     L->row_group = env && std::atoi(env) > 0 ? std::atoi(env) : 0;
-    env = std::getenv("SWAPMOE_PREFETCH");              // SWAPMOE_PREFETCH=0 disables the L2 weight prefetch
-    L->prefetch = !(env && env[0] == '0');
-    // The prefetch must drain while the router runs (about 15 us on 16-64 SMs): what HBM delivers
-    // in that time, and well under the L2 capacity.  Measured on B200: 56 MB hides fully, 76 MB
-    // stretches the router kernel.
-    const long long l2 = prop.l2CacheSize;
-    L->l2_prefetch_bytes = l2 > (80ll << 20) ? (56ll << 20) : 0;
+    // L2 weight prefetch from the router's idle blocks (SWAPMOE_PREFETCH_MB=<MB> switches it on).  Off by default:
+    // since the slot scan left the router, the router is too short to hide it - every megabyte prefetched slows
+    // the router by about as much as it speeds GEMM-1 up (B200, 2048 tokens: 0 / 24 / 56 MB -> 54.7 / 54.9 / 56.4 us).
     env = std::getenv("SWAPMOE_PREFETCH_MB");
-    if (env) L->l2_prefetch_bytes = std::atoll(env) << 20;
+    L->l2_prefetch_bytes = env ? std::atoll(env) << 20 : 0;
+    L->prefetch = L->l2_prefetch_bytes > 0;
+    env = std::getenv("SWAPMOE_FP32_SWAP");             // SWAPMOE_FP32_SWAP=0: fp32 layers always on 128-token tiles
+    L->fp32_swap = !(env && env[0] == '0');
     env = std::getenv("SWAPMOE_PREFETCH_MIN_PAIRS");
     L->prefetch_min_pairs = env ? std::max(1, std::atoi(env)) : 1;
   }
@@ -463,6 +488,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_status = cv.take<int32_t>(4);
   const size_t o_ticket = cv.take<unsigned>(4);
   const size_t o_touched = cv.take<unsigned long long>(2);
+  const size_t o_dec_stats = cv.take<unsigned long long>(2), o_dec_recent = cv.take<int32_t>(kDecRecent);
   const size_t o_tiles = cv.take<TileDesc>(max_tiles);
   const size_t o_tiles_b = cv.take<TileDesc>(max_tiles), o_ntiles_b = cv.take<int32_t>(4);
   const size_t o_xp = cv.take<char>(rows_pad * c.d_model * L->elem);
@@ -502,6 +528,7 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   L->s2e = (int32_t*)(b + o_s2e); L->status = (int32_t*)(b + o_status);
   L->ticket = (unsigned*)(b + o_ticket);
   L->touched = (unsigned long long*)(b + o_touched);
+  L->dec_pf_stats = (unsigned long long*)(b + o_dec_stats); L->dec_recent = (int32_t*)(b + o_dec_recent);
   L->tiles = (TileDesc*)(b + o_tiles);
   L->tiles_b = (TileDesc*)(b + o_tiles_b); L->n_tiles_b = (int32_t*)(b + o_ntiles_b);
   L->xp = b + o_xp; L->h = b + o_h; L->y = (float*)(b + o_y);
@@ -514,6 +541,17 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   ok = ok && cuda_ok(cudaMemset(L->status, 0, sizeof(int32_t) * 4));
   ok = ok && cuda_ok(cudaMemset(L->ticket, 0, sizeof(unsigned) * 4));
   ok = ok && cuda_ok(cudaMemset(L->touched, 0, sizeof(unsigned long long) * 2));
+  ok = ok && cuda_ok(cudaMemset(L->dec_pf_stats, 0, sizeof(unsigned long long) * 2));
+  ok = ok && cuda_ok(cudaMemset(L->dec_recent, 0xff, sizeof(int32_t) * kDecRecent));      // -1: nothing served yet
+  {
+    // Decode steps: L2 prefetch of the experts the layer served last (activation locality, Section 2.2).  Off by
+    // default: measured on B200 with the synthetic decode traffic (a token keeps its expert of the step before in
+    // 11 % of the steps, one of the last three in 29 %) the step got no faster (18.3 -> 18.6 .. 19.2 us per layer at one
+    // token per step): even a correct guess saves little, because the step is bound by its chain of dependent
+    // phases, not by the 2.6 us its weights take from HBM.
+    const char* envp = std::getenv("SWAPMOE_DECODE_PREFETCH");   // 0 .. 4 recently served experts
+    L->dec_pf_depth = envp ? std::min(std::max(std::atoi(envp), 0), kDecRecent) : 0;
+  }
   if (L->decode_path) {
     ok = ok && cuda_ok(cudaMemset(L->dec_tickets, 0, sizeof(unsigned) * decode_ticket_count(c.d_ff, c.K)));
     ok = ok && cuda_ok(decode_fused_set_smem_limit((int)decode_smem_bytes(c.d_model)));
@@ -735,6 +773,20 @@ int32_t swapmoe_read_importance_kind(swapmoe_layer_t* L, int32_t kind, float* im
   return SWAPMOE_OK;
 }
 
+int32_t swapmoe_read_scores_async(swapmoe_layer_t* L, int32_t kinds_mask, float* scores_host_pinned, int32_t reset,
+                                  void* stream) {
+  if (!L || !scores_host_pinned || kinds_mask < 1 || kinds_mask > 7) return SWAPMOE_ERR_INVALID_ARG;
+  // pinned host memory is mapped into the device's address space: the kernel writes it directly
+  void* dst = nullptr;
+  if (!cuda_ok(cudaHostGetDevicePointer(&dst, scores_host_pinned, 0)) || !dst) { cudaGetLastError(); return SWAPMOE_ERR_INVALID_ARG; }
+  ScoreSnapshot sn;
+  sn.acc[0] = L->imp; sn.acc[1] = L->cnt; sn.acc[2] = L->mimp;
+  sn.dst = static_cast<float*>(dst); sn.E = L->cfg.E; sn.mask = kinds_mask; sn.reset = reset;
+  snapshot_scores_kernel<<<1, 256, 0, static_cast<cudaStream_t>(stream)>>>(sn);
+  L->launches++;
+  return check_launch();
+}
+
 int32_t swapmoe_read_importance(swapmoe_layer_t* L, float* imp_host, int32_t reset, void* stream) {
   return swapmoe_read_importance_kind(L, SWAPMOE_IMP_EQ1, imp_host, reset, stream);
 }
@@ -747,6 +799,19 @@ int32_t swapmoe_read_touched_slots(swapmoe_layer_t* L, int64_t* total_host, int3
   if (reset && !cuda_ok(cudaMemsetAsync(L->touched, 0, sizeof(v), st))) return SWAPMOE_ERR_CUDA;
   if (!cuda_ok(cudaStreamSynchronize(st))) return SWAPMOE_ERR_CUDA;
   *total_host = (int64_t)v;
+  return SWAPMOE_OK;
+}
+
+int32_t swapmoe_read_decode_prefetch(swapmoe_layer_t* L, int64_t* hits_host, int64_t* touched_host, int32_t reset,
+                                     void* stream) {
+  if (!L || !hits_host || !touched_host) return SWAPMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned long long v[2] = {0, 0};
+  if (!cuda_ok(cudaMemcpyAsync(v, L->dec_pf_stats, sizeof(v), cudaMemcpyDeviceToHost, st))) return SWAPMOE_ERR_CUDA;
+  if (reset && !cuda_ok(cudaMemsetAsync(L->dec_pf_stats, 0, sizeof(v), st))) return SWAPMOE_ERR_CUDA;
+  if (!cuda_ok(cudaStreamSynchronize(st))) return SWAPMOE_ERR_CUDA;
+  *hits_host = (int64_t)v[0];
+  *touched_host = (int64_t)v[1];
   return SWAPMOE_OK;
 }
 

@@ -41,6 +41,7 @@ constexpr int kDecJB = 32;            // hidden units per work item
 constexpr int kDecGroup = 16;         // work items per first-step sum
 constexpr int kDecRowPad = 16;        // bytes added to a row's pitch in shared memory
 constexpr int kDecHalfBytes = 66048;  // one wave buffer (32 rows of 2064 bytes; a multiple of 512); there are two
+constexpr int kDecRecent = 4;         // recently served experts remembered per layer
 constexpr int kDecOutRows = 256;      // rows of W_out per TMA box
 constexpr int kDecOutBoxes = 4;       // boxes per W_out wave: 1024 rows
 constexpr int kDecHPitch = 40;        // bf16 elements between the activation rows of two pairs (80 bytes)
@@ -65,6 +66,12 @@ struct DecodeArgs {
   bf16* out;                 // [T, d]
   int32_t* status;           // device status words (bounded waits report here)
   unsigned long long* touched;   // [1] running total of slots that received at least one pair, or nullptr
+  // Activation locality (Section 2.2: successive tokens use consistent experts): the experts this layer
+  // served most recently, most recent first (-1: none).  While the CTAs route, the first pf_depth of them
+  // that are still resident are pulled towards L2; the reporting CTA then updates the list.
+  int32_t* recent;               // [kDecRecent]
+  unsigned long long* pf_stats;  // [2]: touched slots whose expert had been prefetched, touched slots
+  int32_t pf_depth;              // 0: no prefetch
   int32_t T, d, f, E, k, K, renorm, swiglu;
 };
 
@@ -84,6 +91,16 @@ __host__ __device__ inline int decode_rows_per_wave(int d) {
   return rp;
 }
 
+// Order-preserving integer key of a logit: a > b  <=>  key(a) > key(b), equal logits (-0 and +0 included) have
+// equal keys, and no finite or infinite logit maps to 0, which stands for "nothing available".
+__device__ __forceinline__ uint32_t gate_key(float x) {
+  const uint32_t b = __float_as_uint(x + 0.f);              // -0 becomes +0
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float gate_key_value(uint32_t key) {
+  return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+
 // Top-k of one token's logits by a whole warp: row[e] is the logit of expert e (shared memory), lane l looks
 // at experts l, l + 32, ... of the `ei` 32-expert groups that exist; allow bit i says whether expert l + 32 i
 // may be chosen; ties go to the lowest expert index.  Gate values are the softmax over the allowed experts (or
@@ -99,22 +116,20 @@ __device__ __forceinline__ void dec_topk_gate(const float* row, uint32_t allow, 
   for (int j = 0; j < kMaxTopK; ++j) {
     sel_e[j] = 0; sel_g[j] = 0.f; sel_v[j] = 0.f;
     if (j < k) {
-      float bv = -INFINITY;
+      // the lane's best available logit as an order-preserving integer key (0: none; the first of equals
+      // wins locally), then two warp reductions: the largest key, and the lowest index that holds it
+      uint32_t bk = 0u;
       int be = 0x7fffffff;
 #pragma unroll 1
       for (int i = 0; i < ei; ++i) {
         if ((avail >> i) & 1u) {
-          const float x = row[lane + 32 * i];
-          if (be == 0x7fffffff || x > bv) { bv = x; be = lane + 32 * i; }
+          const uint32_t key = gate_key(row[lane + 32 * i]);
+          if (key > bk) { bk = key; be = lane + 32 * i; }
         }
       }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int oe = __shfl_xor_sync(0xffffffffu, be, o);
-        if (oe != 0x7fffffff && (be == 0x7fffffff || ov > bv || (ov == bv && oe < be))) { bv = ov; be = oe; }
-      }
-      sel_e[j] = be; sel_v[j] = bv;
+      const uint32_t kmax = __reduce_max_sync(0xffffffffu, bk);
+      be = __reduce_min_sync(0xffffffffu, bk == kmax ? be : 0x7fffffff);
+      sel_e[j] = be; sel_v[j] = gate_key_value(kmax);
       if ((be & 31) == lane) avail &= ~(1u << (be >> 5));
     }
   }
@@ -147,33 +162,20 @@ __device__ __forceinline__ void dec_topk_gate2(const float* row, const uint32_t 
 #pragma unroll
     for (int p = 0; p < 2; ++p) { sel_e[p][j] = 0; sel_g[p][j] = 0.f; sel_v[p][j] = 0.f; }
     if (j < k) {
-      float bv[2] = {-INFINITY, -INFINITY};
+      uint32_t bk[2] = {0u, 0u};
       int be[2] = {0x7fffffff, 0x7fffffff};
 #pragma unroll 1
       for (int i = 0; i < ei; ++i) {
-        const float x = row[lane + 32 * i];
+        const uint32_t key = gate_key(row[lane + 32 * i]);
 #pragma unroll
         for (int p = 0; p < 2; ++p)
-          if (((avail[p] >> i) & 1u) && (be[p] == 0x7fffffff || x > bv[p])) { bv[p] = x; be[p] = lane + 32 * i; }
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        float ov[2];
-        int oe[2];
-#pragma unroll
-        for (int p = 0; p < 2; ++p) {
-          ov[p] = __shfl_xor_sync(0xffffffffu, bv[p], o);
-          oe[p] = __shfl_xor_sync(0xffffffffu, be[p], o);
-        }
-#pragma unroll
-        for (int p = 0; p < 2; ++p)
-          if (oe[p] != 0x7fffffff && (be[p] == 0x7fffffff || ov[p] > bv[p] || (ov[p] == bv[p] && oe[p] < be[p]))) {
-            bv[p] = ov[p]; be[p] = oe[p];
-          }
+          if (((avail[p] >> i) & 1u) && key > bk[p]) { bk[p] = key; be[p] = lane + 32 * i; }
       }
 #pragma unroll
       for (int p = 0; p < 2; ++p) {
-        sel_e[p][j] = be[p]; sel_v[p][j] = bv[p];
+        const uint32_t kmax = __reduce_max_sync(0xffffffffu, bk[p]);
+        be[p] = __reduce_min_sync(0xffffffffu, bk[p] == kmax ? be[p] : 0x7fffffff);
+        sel_e[p][j] = be[p]; sel_v[p][j] = gate_key_value(kmax);
         if ((be[p] & 31) == lane) avail[p] &= ~(1u << (be[p] >> 5));
       }
     }
@@ -353,6 +355,10 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
     if (n_rw > 0) issue_rows(0, a.Wr, min(RW, E));
     if (n_rw > 1) issue_rows(1, a.Wr + (size_t)RW * d, min(RW, E - RW));
   }
+  // The list of recently served experts was written by this layer's previous forward, which is long complete
+  // (every kernel of the stream waits for the one in front of it): it may be read before the wait.
+  int recent_e = -1;
+  if (warp == kDecWarps - 1 && lane < a.pf_depth) recent_e = __ldcg(a.recent + lane);
   pdl_wait();
   pdl_trigger();
   // ------------------------------------------------------------------ routing, in every CTA
@@ -378,6 +384,25 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
   if (tid < K) R->phys[tid] = a.phys[tid];
   if (tid < kDecMaxTokens) R->tok[tid] = min(tid, T - 1);
   __syncthreads();
+  if (warp == kDecWarps - 1 && a.pf_depth > 0) {
+    // L2 prefetch of the recently served experts that are resident: 16 KB chunks of both matrices, dealt over
+    // the CTAs (chunk c of a slot goes to CTA c mod grid), so every SM issues a handful of requests
+    constexpr int kChunk = 16384;
+    const int n_in = (int)(a.in_stride * 2 / kChunk), n_out = (int)(a.out_stride * 2 / kChunk);
+#pragma unroll 1
+    for (int h = 0; h < a.pf_depth; ++h) {
+      const int e = __shfl_sync(0xffffffffu, recent_e, h);
+      const int sl = (e >= 0 && e < E) ? R->e2s[e] : -1;
+      if (sl < 0) continue;
+      const int ph = R->phys[sl];
+      for (int c = (int)blockIdx.x + (int)gridDim.x * lane; c < n_in + n_out; c += (int)gridDim.x * 32) {
+        const char* src = c < n_in
+            ? reinterpret_cast<const char*>(a.arena_in + (size_t)ph * a.in_stride) + (size_t)c * kChunk
+            : reinterpret_cast<const char*>(a.arena_out + (size_t)ph * a.out_stride) + (size_t)(c - n_in) * kChunk;
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"((unsigned)kChunk) : "memory");
+      }
+    }
+  }
   if (warp < T && blockIdx.x == gridDim.x - 1) {     // ||x_t||: only the reporting CTA needs it
     float ss = 0.f;
 #pragma unroll 1
@@ -546,6 +571,34 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
       for (int p = 0; p < P; ++p)
         if (R->sl[p] == tid) m += R->xn[p / k] * fabsf(R->mg[p]) * a.enorm[R->me[p]];
       a.mimp[a.s2e[tid]] += m;
+    }
+    if (tid == kDecThreads - 1 && a.recent != nullptr) {
+      // most-recent-first list of served experts: this step's (in slot order), then the older ones
+      int old[kDecRecent], nw[kDecRecent];
+#pragma unroll
+      for (int h = 0; h < kDecRecent; ++h) { old[h] = a.recent[h]; nw[h] = -1; }
+      int n = 0, hits = 0;
+      for (int i = 0; i < R->n_touched; ++i) {
+        const int e = R->me[R->pair_at[R->toffset[i]]];
+        bool predicted = false;
+#pragma unroll
+        for (int h = 0; h < kDecRecent; ++h) predicted = predicted || (h < a.pf_depth && old[h] == e);
+        hits += predicted ? 1 : 0;
+        if (n < kDecRecent) nw[n++] = e;
+      }
+#pragma unroll
+      for (int h = 0; h < kDecRecent; ++h) {
+        bool dup = old[h] < 0;
+#pragma unroll
+        for (int q = 0; q < kDecRecent; ++q) dup = dup || (q < n && nw[q] == old[h]);
+        if (!dup && n < kDecRecent) nw[n++] = old[h];
+      }
+#pragma unroll
+      for (int h = 0; h < kDecRecent; ++h) a.recent[h] = nw[h];
+      if (a.pf_stats != nullptr) {
+        atomicAdd(a.pf_stats, (unsigned long long)hits);
+        atomicAdd(a.pf_stats + 1, (unsigned long long)R->n_touched);
+      }
     }
     if (tid < E) {
       // Eq. (1): terms of the off-the-shelf routing, added in pair order

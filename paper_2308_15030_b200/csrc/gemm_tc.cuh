@@ -713,6 +713,43 @@ inline int tc_pick_bn(const int* options, int n_options, int n, long long row_ti
 
 typedef void (*TcGemmKernel)(const CUtensorMap, const CUtensorMap, const TcGemmArgs);
 
+// How tc_ffn launches GEMM-1 for a forward of n_tokens.
+struct TcGemm1Plan {
+  int i1, bn1, out1;        // index into kBn1Options, tile width, output columns per tile
+  int n_col_tiles, grid, row_group, ia, a_box_bytes, stages;
+  long long row_tiles_est;
+};
+inline bool tc_plan_gemm1(const TcState& s, const swapmoe_config_t& c, int n_tokens, int mt, int max_tiles,
+                          int row_group_forced, TcGemm1Plan* p) {
+  const bool swiglu = c.act == SWAPMOE_ACT_SWIGLU;
+  // row tiles expected: every touched slot (at most min(pairs, K)) has at least one, and large slots
+  // have pairs / 128 in total plus on average half a ragged tile each
+  const long long pairs = (long long)n_tokens * c.top_k;
+  const long long touched = pairs < c.K ? pairs : c.K;
+  const long long by_rows = pairs / kTcBM + touched / 2;
+  p->row_tiles_est = touched > by_rows ? touched : by_rows;
+  // no tile holds more rows than there are pairs: small batches fetch only the rows that can be valid
+  int ia = 0;
+  while (ia < 3 && (kTcBM >> (ia + 1)) >= pairs) ++ia;
+  if (mt == 2) ia = 0;
+  p->ia = ia;
+  p->a_box_bytes = (kTcBM >> ia) * kTcBK * 2;
+  // Large activation matrices (tens of MB) are walked in groups of 32 row tiles so that a group's
+  // rows stay in L2 across its column tiles; small ones are a single group.
+  p->row_group = 1 << 30;
+  if (row_group_forced > 0) p->row_group = row_group_forced;
+  else if (pairs * (long long)c.d_model * 2 > (48ll << 20)) p->row_group = 32;
+  p->i1 = tc_pick_bn(kBn1Options, 3, c.d_ff, p->row_tiles_est * mt, s.sm_count, p->a_box_bytes, swiglu ? 64 : 32);
+  if (p->i1 < 0) return false;
+  p->bn1 = kBn1Options[p->i1];
+  p->out1 = swiglu ? p->bn1 / 2 : p->bn1;
+  p->n_col_tiles = c.d_ff / p->out1;
+  const long long work = (long long)max_tiles * mt * p->n_col_tiles;
+  p->grid = work > s.sm_count ? s.sm_count : (int)work;
+  p->stages = (kTcSmemBudget - 2048) / (kTcBM * kTcBK * 2 + p->bn1 * kTcBK * 2);
+  return true;
+}
+
 // Runs both grouped GEMMs.  With top_k == 1 the second GEMM writes gate * y straight into
 // `out` (*combined = true) and no combine kernel is needed.
 inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, void* out, const TileDesc* tiles,
@@ -723,29 +760,13 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
   if (!s.enabled || !s.arena_bound) return SWAPMOE_ERR_NOT_READY;
   const bool swiglu = c.act == SWAPMOE_ACT_SWIGLU;
   const bool scatter = c.top_k == 1;
-  // row tiles expected: every touched slot (at most min(pairs, K)) has at least one, and large slots
-  // have pairs / 128 in total plus on average half a ragged tile each
-  const long long pairs = (long long)n_tokens * c.top_k;
-  const long long touched = pairs < c.K ? pairs : c.K;
-  const long long by_rows = pairs / kTcBM + touched / 2;
-  const long long row_tiles_est = touched > by_rows ? touched : by_rows;
-  // no tile holds more rows than there are pairs: small batches fetch only the rows that can be valid
-  int ia = 0;
-  while (ia < 3 && (kTcBM >> (ia + 1)) >= pairs) ++ia;
-  if (mt == 2) ia = 0;
-  const int a_box_bytes = (kTcBM >> ia) * kTcBK * 2;
-
-  // Large activation matrices (tens of MB) are walked in groups of 32 row tiles so that a group's
-  // rows stay in L2 across its column tiles; small ones are a single group.
-  int row_group = 1 << 30;
-  if (row_group_forced > 0) row_group = row_group_forced;
-  else if (pairs * (long long)c.d_model * 2 > (48ll << 20)) row_group = 32;
   // ---- GEMM-1: h = act(xp * W_in^T).  Its k-loop is short (d_model / 64 blocks), so its epilogue must
   // overlap the next tile's MMAs: always one sub-tile per CTA with two TMEM buffers.
-  const int i1 = tc_pick_bn(kBn1Options, 3, c.d_ff, row_tiles_est * mt, s.sm_count, a_box_bytes, swiglu ? 64 : 32);
-  if (i1 < 0) return SWAPMOE_ERR_UNSUPPORTED;
-  const int bn1 = kBn1Options[i1];
-  const int out1 = swiglu ? bn1 / 2 : bn1;      // output columns per tile
+  TcGemm1Plan plan;
+  if (!tc_plan_gemm1(s, c, n_tokens, mt, max_tiles, row_group_forced, &plan)) return SWAPMOE_ERR_UNSUPPORTED;
+  const long long row_tiles_est = plan.row_tiles_est;
+  const int ia = plan.ia, a_box_bytes = plan.a_box_bytes, row_group = plan.row_group;
+  const int i1 = plan.i1, out1 = plan.out1;     // output columns per tile
   TcGemmArgs g1;
   g1.C = h; g1.status = status; g1.ldc = c.d_ff;
   g1.tiles = mt == 2 ? tiles128 : tiles;          // always a list of 128-row tiles
@@ -759,7 +780,7 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
   g1.a_box_bytes = a_box_bytes;
   g1.early_b = 0;
   long long work = (long long)max_tiles * mt * g1.n_col_tiles;
-  int grid = work > s.sm_count ? s.sm_count : (int)work;
+  int grid = plan.grid;
   static const TcGemmKernel k1[2][3] = {
       {tc_gemm_kernel<256, kTcEpiReluBf16>, tc_gemm_kernel<128, kTcEpiReluBf16>, tc_gemm_kernel<64, kTcEpiReluBf16>},
       {tc_gemm_kernel<256, kTcEpiSwigluBf16>, tc_gemm_kernel<128, kTcEpiSwigluBf16>,

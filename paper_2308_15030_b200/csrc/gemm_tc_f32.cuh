@@ -36,6 +36,9 @@ constexpr int kF32StageBytes = kF32ABytes + kF32BBytes;
 constexpr int kF32Stages = 5;                       // raw stages (TMA targets; the B half holds the hi parts after conversion)
 constexpr int kF32LoSlots = 2;                      // lo parts of B in shared memory; hi and lo of A in tensor memory
 constexpr int kF32SmemBytes = kF32Stages * kF32StageBytes + kF32LoSlots * kF32BBytes + 2048 + kTcEpiStageBytes;
+// Swapped form for small slots: the 128 rows of the MMA (and of tensor memory) are WEIGHT rows, the accumulator's
+// columns are the tokens of a slot tile (kF32SwapTok of them).
+constexpr int kF32SwapTok = 64;                     // token rows per tile = accumulator columns
 constexpr int kF32TmemAcc = 2 * kF32BN;             // columns of the two accumulator sets
 constexpr int kF32TmemCols = 512;                   // + 2 slots x (hi 32 + lo 32) columns of A, rounded up to a power of two
 
@@ -116,14 +119,20 @@ __device__ __forceinline__ void epi_load_pieces_f32(uint32_t taddr, int c0, int 
   for (int i = 0; i < 8; ++i) pc[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
 }
 
-template <int EPI>
+// kSwap = false: A (128 rows, split into tensor memory) = token rows of a slot tile, B (shared memory) = 128 weight
+// rows; C tile = [128 tokens, 128 outputs].  kSwap = true (ReLU / plain epilogues): A = 128 weight rows, B = the
+// kF32SwapTok token rows of a slot tile; the accumulator holds C^T, lane = output column, column = token.
+template <int EPI, bool kSwap = false>
 __global__ void __launch_bounds__(kF32Threads, 1)
 tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcF32Args a) {
+  static_assert(!(kSwap && EPI == kTcEpiSwigluF32), "the swapped form has no SwiGLU epilogue");
   constexpr int kNB = (EPI == kTcEpiSwigluF32) ? 2 : 1;     // weight boxes per stage
   constexpr int kBoxRows = kF32BN / kNB;
   constexpr int kOutCols = kF32BN / kNB;
+  constexpr int kNRows = kSwap ? kF32SwapTok : kF32BN;      // rows of the B operand = accumulator columns
+  constexpr int kBBytesK = kNRows * kF32BK * 4;             // bytes of the B operand per k-block
   constexpr uint32_t kTmemCols = kF32TmemCols;
-  constexpr uint32_t kIdesc = make_idesc_tf32(kTcBM, kF32BN);
+  constexpr uint32_t kIdesc = make_idesc_tf32(kTcBM, kNRows);
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
@@ -175,11 +184,15 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       const int brow = td.phys * a.b_rows_per_phys + ct * kBoxRows;
       pre = a.k_blocks < kF32Stages ? a.k_blocks : kF32Stages;
       for (int kb = 0; kb < pre; ++kb) {
-        ptx::mbar_expect_tx(&full[kb], (uint32_t)kF32StageBytes);
+        ptx::mbar_expect_tx(&full[kb], (uint32_t)(kF32ABytes + kBBytesK));
+        if (kSwap) {
+          ptx::tma_load_2d(raw + kb * kF32StageBytes, &tmA, &full[kb], (z * a.k_blocks + kb) * kF32BK, brow);
+        } else {
 #pragma unroll
-        for (int j = 0; j < kNB; ++j)
-          ptx::tma_load_2d(raw + kb * kF32StageBytes + kF32ABytes + j * kBoxRows * kF32BK * 4, &tmB, &full[kb],
-                           (z * a.k_blocks + kb) * kF32BK, brow + j * a.b_rows_gate);
+          for (int j = 0; j < kNB; ++j)
+            ptx::tma_load_2d(raw + kb * kF32StageBytes + kF32ABytes + j * kBoxRows * kF32BK * 4, &tmB, &full[kb],
+                             (z * a.k_blocks + kb) * kF32BK, brow + j * a.b_rows_gate);
+        }
       }
     }
   }
@@ -207,14 +220,20 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           if (!early) {
             ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 31);
             if (!ok) break;
-            ptx::mbar_expect_tx(&full[stage], (uint32_t)kF32StageBytes);
+            ptx::mbar_expect_tx(&full[stage], (uint32_t)(kF32ABytes + kBBytesK));
           }
-          ptx::tma_load_2d(sA, &tmA, &full[stage], (kb0 + kb) * kF32BK, td.row0);
-          if (!early) {
+          if (kSwap) {
+            // tokens are the B operand, weights the A operand (the one that may have been requested early)
+            ptx::tma_load_2d(sA + kF32ABytes, &tmB, &full[stage], (kb0 + kb) * kF32BK, td.row0);
+            if (!early) ptx::tma_load_2d(sA, &tmA, &full[stage], (kb0 + kb) * kF32BK, brow);
+          } else {
+            ptx::tma_load_2d(sA, &tmA, &full[stage], (kb0 + kb) * kF32BK, td.row0);
+            if (!early) {
 #pragma unroll
-            for (int j = 0; j < kNB; ++j)
-              ptx::tma_load_2d(sA + kF32ABytes + j * kBoxRows * kF32BK * 4, &tmB, &full[stage], (kb0 + kb) * kF32BK,
-                               brow + j * a.b_rows_gate);
+              for (int j = 0; j < kNB; ++j)
+                ptx::tma_load_2d(sA + kF32ABytes + j * kBoxRows * kF32BK * 4, &tmB, &full[stage], (kb0 + kb) * kF32BK,
+                                 brow + j * a.b_rows_gate);
+            }
           }
           if (++stage == kF32Stages) { stage = 0; phase ^= 1u; }
         }
@@ -235,7 +254,7 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         ok = bounded_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, a.status, 32);
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * kF32BN);
+        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * kNRows);
         for (int kb = 0; kb < a.k_blocks; ++kb) {
           ok = bounded_wait(&conv_done[slot], slot_phase, abort_flag, a.status, 33);
           if (!ok) break;
@@ -302,7 +321,7 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         uint4* src = reinterpret_cast<uint4*>(raw + stage * kF32StageBytes + kF32ABytes);
         uint4* dst = reinterpret_cast<uint4*>(lo + slot * kF32BBytes);
 #pragma unroll 4
-        for (int i = ctid; i < kF32BBytes / 16; i += 128) {
+        for (int i = ctid; i < kBBytesK / 16; i += 128) {
           const uint4 x = src[i];
           uint4 h, l;
           h.x = x.x & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(x.x) - __uint_as_float(h.x));
@@ -331,6 +350,28 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       const int z = t / per_slice, u = t - z * per_slice;
       const int ct = u / n_row_tiles, rt = u - ct * n_row_tiles;
       const TileDesc td = a.tiles[rt];
+      if constexpr (kSwap) {
+        // lane r holds output column ct * 128 + r of every token of the tile: a warp's 32 lanes store 128
+        // contiguous bytes of one token row per instruction
+        float* crow = static_cast<float*>(a.C) + (size_t)z * a.split_stride + (size_t)td.row0 * a.ldc +
+                      (size_t)ct * kF32BN + r;
+        ok = bounded_wait(&acc_full[acc], acc_phase, abort_flag, a.status, 36);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kNRows);
+#pragma unroll 1
+        for (int c0 = 0; c0 < kNRows; c0 += 32) {
+          uint32_t v[32];
+          ptx::tmem_ld32(taddr + (uint32_t)c0, v);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            float f = __uint_as_float(v[i]);
+            if (EPI == kTcEpiReluF32) f = fmaxf(f, 0.f);
+            if (c0 + i < td.rows) crow[(size_t)(c0 + i) * a.ldc] = f;
+          }
+        }
+      } else {
       const int drow = r < td.rows ? td.row0 + r : -1;
       unsigned char* dst[8];
       epi_row_pointers(dst, drow, lane, static_cast<float*>(a.C) + (size_t)z * a.split_stride, (size_t)a.ldc,
@@ -344,6 +385,7 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         uint4 pc[8];
         epi_load_pieces_f32<EPI>(taddr, c0, kOutCols, pc);
         epi_store_chunk(epi_stage + q * kTcEpiWarpStage, pc, lane, dst, c0 * 4);
+      }
       }
       ptx::tc_fence_before();
       ptx::mbar_arrive(&acc_empty[acc]);
@@ -364,6 +406,8 @@ struct TcF32State {
   int sm_count;
   CUtensorMap map_xp, map_h;          // activations, box 32 x 128
   CUtensorMap map_win, map_wout;      // weights flattened to 2D; box 32 x 128 (64 for SwiGLU's W1 / W3)
+  CUtensorMap map_xp_tok, map_h_tok;  // activations, box 32 x kF32SwapTok (swapped form)
+  bool swap_ok;                       // the swapped form is available (ReLU layers)
 };
 
 // The driver's tensor-map encoder (nullptr when it cannot be had).
@@ -400,7 +444,16 @@ inline int32_t tc_f32_init(TcF32State& s, PFN_encodeTiled enc, const swapmoe_con
   s.sm_count = sm_count;
   if (!enc || !tc_f32_supported(c)) return SWAPMOE_OK;
   if (!tc_encode_2d_f32(enc, &s.map_xp, xp, (uint64_t)rows_pad, (uint64_t)c.d_model, kTcBM) ||
-      !tc_encode_2d_f32(enc, &s.map_h, h, (uint64_t)rows_pad, (uint64_t)c.d_ff, kTcBM))
+      !tc_encode_2d_f32(enc, &s.map_h, h, (uint64_t)rows_pad, (uint64_t)c.d_ff, kTcBM) ||
+      !tc_encode_2d_f32(enc, &s.map_xp_tok, xp, (uint64_t)rows_pad, (uint64_t)c.d_model, kF32SwapTok) ||
+      !tc_encode_2d_f32(enc, &s.map_h_tok, h, (uint64_t)rows_pad, (uint64_t)c.d_ff, kF32SwapTok))
+    return SWAPMOE_ERR_CUDA;
+  s.swap_ok = c.act == SWAPMOE_ACT_RELU;
+  if (s.swap_ok &&
+      (cudaFuncSetAttribute(tc_gemm_f32_kernel<kTcEpiReluF32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                            kF32SmemBytes) != cudaSuccess ||
+       cudaFuncSetAttribute(tc_gemm_f32_kernel<kTcEpiF32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                            kF32SmemBytes) != cudaSuccess))
     return SWAPMOE_ERR_CUDA;
   if (cudaFuncSetAttribute(tc_gemm_f32_kernel<kTcEpiReluF32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kF32SmemBytes) != cudaSuccess ||
@@ -430,9 +483,11 @@ inline int32_t tc_f32_bind_arena(TcF32State& s, PFN_encodeTiled enc, const swapm
 inline int32_t tc_ffn_f32(TcF32State& s, const swapmoe_config_t& c, void* h, float* y, long long y_copy_stride,
                           int y_copies, const TileDesc* tiles, const int32_t* n_tiles, int max_tiles, int n_tokens,
                           int32_t* status, cudaStream_t st, bool pdl, int64_t* launches, int* y_split,
-                          cudaEvent_t between = nullptr) {
+                          cudaEvent_t between = nullptr, bool swapped = false) {
   if (!s.enabled || !s.arena_bound) return SWAPMOE_ERR_NOT_READY;
   const bool swiglu = c.act == SWAPMOE_ACT_SWIGLU;
+  if (swapped && (swiglu || !s.swap_ok)) return SWAPMOE_ERR_UNSUPPORTED;
+  const int tile_rows = swapped ? kF32SwapTok : kTcBM;
   const int out1 = swiglu ? kF32BN / 2 : kF32BN;
   TcF32Args g1;
   g1.C = h; g1.tiles = tiles; g1.n_tiles = n_tiles; g1.status = status; g1.split_stride = 0;
@@ -442,10 +497,13 @@ inline int32_t tc_ffn_f32(TcF32State& s, const swapmoe_config_t& c, void* h, flo
   g1.early_b = 0;
   long long work = (long long)max_tiles * g1.n_col_tiles;
   int grid = work > s.sm_count ? s.sm_count : (int)work;
-  cudaError_t e = swiglu ? launch_kernel(tc_gemm_f32_kernel<kTcEpiSwigluF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes,
-                                         st, pdl, s.map_xp, s.map_win, g1)
-                         : launch_kernel(tc_gemm_f32_kernel<kTcEpiReluF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes,
-                                         st, pdl, s.map_xp, s.map_win, g1);
+  // (swapped form: the weight map is the A operand's, the token map with kF32SwapTok-row boxes the B operand's)
+  cudaError_t e = swapped ? launch_kernel(tc_gemm_f32_kernel<kTcEpiReluF32, true>, dim3(grid), dim3(kF32Threads),
+                                          kF32SmemBytes, st, pdl, s.map_win, s.map_xp_tok, g1)
+                  : swiglu ? launch_kernel(tc_gemm_f32_kernel<kTcEpiSwigluF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes,
+                                           st, pdl, s.map_xp, s.map_win, g1)
+                           : launch_kernel(tc_gemm_f32_kernel<kTcEpiReluF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes,
+                                           st, pdl, s.map_xp, s.map_win, g1);
   if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
   ++*launches;
   if (between) cudaEventRecord(between, st);
@@ -453,7 +511,7 @@ inline int32_t tc_ffn_f32(TcF32State& s, const swapmoe_config_t& c, void* h, flo
   // GEMM-2: few output tiles, long contraction: slice it until every SM has an item
   const long long pairs = (long long)n_tokens * c.top_k;
   const long long touched = pairs < c.K ? pairs : c.K;
-  const long long by_rows = pairs / kTcBM + touched / 2;
+  const long long by_rows = pairs / tile_rows + touched / 2;
   const long long row_tiles_est = touched > by_rows ? touched : by_rows;
   const int n_col2 = c.d_model / kF32BN;
   int split = 1;
@@ -467,8 +525,10 @@ inline int32_t tc_ffn_f32(TcF32State& s, const swapmoe_config_t& c, void* h, flo
   g2.early_b = 1;
   work = (long long)max_tiles * n_col2 * split;
   grid = work > s.sm_count ? s.sm_count : (int)work;
-  e = launch_kernel(tc_gemm_f32_kernel<kTcEpiF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes, st,
-                    pdl && between == nullptr, s.map_h, s.map_wout, g2);
+  e = swapped ? launch_kernel(tc_gemm_f32_kernel<kTcEpiF32, true>, dim3(grid), dim3(kF32Threads), kF32SmemBytes, st,
+                              pdl && between == nullptr, s.map_wout, s.map_h_tok, g2)
+              : launch_kernel(tc_gemm_f32_kernel<kTcEpiF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes, st,
+                              pdl && between == nullptr, s.map_h, s.map_wout, g2);
   if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
   ++*launches;
   *y_split = split;

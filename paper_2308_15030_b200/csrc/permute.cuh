@@ -310,16 +310,18 @@ __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const Perm
   // the next kernel's CTAs may be scheduled at once: they stop at their own wait, and until then they
   // touch nothing this kernel or the router writes
   pdl_trigger();
-  if (a.own_scan && (int)blockIdx.x == a.scan.n_cta) {
-    // ---- the Eq. (1) reductions: CTA y of this extra column takes the scores y, y + gridDim.y, ... of
-    // {Eq. (1), token counts, Eq. (1) over the masked routing}, so that each is done long before the copying CTAs are
+  if (a.own_scan && (int)blockIdx.x >= a.scan.n_cta) {
+    // ---- the three extra columns of CTAs: the first CTA of column n_cta + w reduces score w of {Eq. (1), token
+    // counts, Eq. (1) over the masked routing}: each is done before the copying CTAs are, none delays the grid
+    if (blockIdx.y != 0) return;
     const ScanArgs& sc = a.scan;
     pdl_wait();
-    if (tid == 0) SWAPMOE_STAMP(1, 4 + 2 * min((int)blockIdx.y, 2));
     float* s_red = reinterpret_cast<float*>(s_raw);
-    for (int which = (int)blockIdx.y; which < 3; which += (int)gridDim.y) {
+    {
+      const int which = (int)blockIdx.x - sc.n_cta;
+      if (tid == 0) SWAPMOE_STAMP(1, 4 + 2 * which);
       const float* src = which == 0 ? sc.cta_imp : which == 1 ? sc.cta_cnt : sc.cta_mimp;
-      if (src == nullptr) continue;
+      if (src == nullptr) return;
       const int C = which == 2 ? sc.K : sc.E;
       float* acc = which == 0 ? sc.imp : which == 1 ? sc.cnt : sc.mimp;
       // thread c owns column c: expert c, or for the masked score the expert that slot c serves
@@ -327,8 +329,8 @@ __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const Perm
       const float old = tid < C ? acc[target] : 0.f;
       const float v = reduce_columns_parallel(src, sc.n_cta, C, s_red, kRawBytes / 4);
       if (tid < C) acc[target] = old + v;
+      if (tid == 0) SWAPMOE_STAMP(1, 5 + 2 * which);
     }
-    if (tid == 0) SWAPMOE_STAMP(1, 5 + 2 * min((int)blockIdx.y, 2));
     return;
   }
   if (tid == 0 && blockIdx.y == 0) SWAPMOE_STAMP(1, 0);
@@ -337,7 +339,8 @@ __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const Perm
   const int p0 = blockIdx.x * npair;
   const int n_total = a.T * a.k;
 
-  for (int i = tid; i < (kPermThreads / 32) * kMaxSlots; i += kPermThreads) (&wcount[0][0])[i] = 0;
+  for (int i = lane; i < kMaxSlots; i += 32) wcount[warp][i] = 0;     // each warp clears (and later fills) its own row
+  __syncwarp();
   // this CTA's rows: local pair pl = ri * gridDim.y + blockIdx.y; the first kPre 16-byte pieces per
   // thread are fetched now
   constexpr int kPre = 4;
@@ -379,6 +382,11 @@ __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const Perm
       s_part[0][tid] = tot;
       s_part[1][tid] = before;
     }
+    if (warp < nwarp_p) {                      // ranks inside the warp need only the pairs' slots
+      const uint32_t same = __match_any_sync(0xffffffffu, s);
+      rank = __popc(same & ((1u << lane) - 1u));
+      if (s >= 0 && rank == 0) wcount[warp][s] = __popc(same);
+    }
     __syncthreads();
     if (tid < K) {
       int tot = 0, before = 0;
@@ -389,16 +397,17 @@ __global__ void __launch_bounds__(kPermThreads) permute_gather_kernel(const Perm
     }
     __syncthreads();
     if (warp == 0) slot_layout_warp(a.scan, s_tot, s_off, s_pad, blockIdx.x == 0 && blockIdx.y == 0);
-  } else if (tid < a.K) {
-    s_base[tid] = a.cta_base[(size_t)blockIdx.x * a.K + tid];
-    s_off[tid] = a.offset[tid];
-    s_pad[tid] = a.pad_offset[tid];
-  }
-  __syncthreads();
-  if (warp < nwarp_p) {
-    const uint32_t same = __match_any_sync(0xffffffffu, s);
-    rank = __popc(same & ((1u << lane) - 1u));
-    if (s >= 0 && rank == 0) wcount[warp][s] = __popc(same);
+  } else {
+    if (tid < a.K) {
+      s_base[tid] = a.cta_base[(size_t)blockIdx.x * a.K + tid];
+      s_off[tid] = a.offset[tid];
+      s_pad[tid] = a.pad_offset[tid];
+    }
+    if (warp < nwarp_p) {
+      const uint32_t same = __match_any_sync(0xffffffffu, s);
+      rank = __popc(same & ((1u << lane) - 1u));
+      if (s >= 0 && rank == 0) wcount[warp][s] = __popc(same);
+    }
   }
   __syncthreads();
   if (s >= 0) {

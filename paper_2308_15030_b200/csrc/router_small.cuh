@@ -100,6 +100,71 @@ __device__ __forceinline__ void rs_wave_dots(const unsigned char* st, int rows, 
   __syncthreads();
 }
 
+// All logits of the CTA in ONE pass when the router matrix fits the two wave buffers (E <= 2 waves of rows):
+// the output is cut into tiles of 16 experts x 8 tokens (at most 4 x NT of them), a warp owns one tile and a
+// contiguous share of the contraction, and the 16 / tiles shares of a tile are added in order.  Per CTA that is
+// one pair of barriers and a 2-way sum for 64 experts x 16 tokens, where the wave-by-wave form (every wave's
+// contraction split over all 16 warps) pays a 16-way sum and two barriers per wave.
+// slog[token * (kMaxE + 1) + expert] receives the logits.
+template <int NT>
+__device__ __forceinline__ void rs_dots_resident(const unsigned char* ring, int E, int RW, int d, const unsigned char* xs,
+                                                 int n_tok, float* red, float* slog) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int pitch = d * 2 + kDecRowPad;
+  const int MT = (E + 15) >> 4;                 // 16-expert row tiles (<= 4)
+  const int n_tiles = MT * NT;                  // <= 8
+  int tiles_p2 = 1;
+  while (tiles_p2 < n_tiles) tiles_p2 <<= 1;
+  const int S = kDecWarps / tiles_p2;           // shares of the contraction per tile
+  const int tile = warp & (tiles_p2 - 1), part = warp / tiles_p2;
+  if (tile < n_tiles) {
+    const int m = tile / NT, j = tile - m * NT;
+    const int row0 = m * 16;                    // first expert of the tile; wave row0 / RW, row row0 % RW inside it
+    const unsigned char* ap0 = ring + (row0 / RW) * kDecHalfBytes + ((row0 % RW) + g) * pitch + t * 4;
+    const unsigned char* xrow = xs + min(8 * j + g, n_tok - 1) * pitch + t * 4;
+    const int nks = d / 16, ks0 = part * nks / S, ks1 = (part + 1) * nks / S;
+    // two accumulators (even / odd steps) halve the chain of dependent mma; their sum is the share's product
+    float acc[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
+    int ks = ks0;
+#pragma unroll 4
+    for (; ks + 1 < ks1; ks += 2) {
+      const int kb = ks * 32;
+      const uint32_t a0 = lds32(ap0 + kb), a1 = lds32(ap0 + 8 * pitch + kb), a2 = lds32(ap0 + kb + 16),
+                     a3 = lds32(ap0 + 8 * pitch + kb + 16);
+      const uint32_t b0 = lds32(xrow + kb), b1 = lds32(xrow + kb + 16);
+      const uint32_t c0 = lds32(ap0 + kb + 32), c1 = lds32(ap0 + 8 * pitch + kb + 32), c2 = lds32(ap0 + kb + 48),
+                     c3 = lds32(ap0 + 8 * pitch + kb + 48);
+      const uint32_t d0 = lds32(xrow + kb + 32), d1 = lds32(xrow + kb + 48);
+      mma_bf16_16x8x16(acc, a0, a1, a2, a3, b0, b1);
+      mma_bf16_16x8x16(acc1, c0, c1, c2, c3, d0, d1);
+    }
+    if (ks < ks1) {
+      const int kb = ks * 32;
+      const uint32_t a0 = lds32(ap0 + kb), a1 = lds32(ap0 + 8 * pitch + kb), a2 = lds32(ap0 + kb + 16),
+                     a3 = lds32(ap0 + 8 * pitch + kb + 16);
+      const uint32_t b0 = lds32(xrow + kb), b1 = lds32(xrow + kb + 16);
+      mma_bf16_16x8x16(acc, a0, a1, a2, a3, b0, b1);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) acc[q] += acc1[q];
+    float* rp = red + ((part * n_tiles + tile) * 16 + g) * 8 + 2 * t;
+    *reinterpret_cast<float2*>(rp) = make_float2(acc[0], acc[1]);
+    *reinterpret_cast<float2*>(rp + 8 * 8) = make_float2(acc[2], acc[3]);
+  }
+  if (tid == 0) SWAPMOE_STAMP(0, 12);
+  __syncthreads();
+  if (tid == 0) SWAPMOE_STAMP(0, 13);
+  for (int o = tid; o < n_tiles * 128; o += kDecThreads) {
+    const int tl = o >> 7, r = (o >> 3) & 15, c = o & 7;
+    float sum = 0.f;
+    for (int p = 0; p < S; ++p) sum += red[((p * n_tiles + tl) * 16 + r) * 8 + c];
+    const int m = tl / NT, j = tl - m * NT;
+    const int e = m * 16 + r, tok = 8 * j + c;
+    if (e < E && tok < n_tok) slog[tok * (kMaxE + 1) + e] = sum;
+  }
+  __syncthreads();
+}
+
 template <int NT>
 __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const RouterArgs a, int32_t* status) {
   constexpr int TOK = kRsTok * NT;                          // tokens per CTA
@@ -151,6 +216,13 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
     issue_router_wave(0);
     if (n_rw > 1) issue_router_wave(1);
   }
+  if (warp == 1 && lane == 0) {
+    // The CTA's token rows (one contiguous range) are pulled towards L2 while the kernel in front still runs.
+    // A prefetch only moves what DRAM holds into L2, where any later write of the producer lands too, so it
+    // cannot make the loads after the wait see stale data; it saves them the DRAM latency when x is cold.
+    const uint32_t bytes = (uint32_t)(T * d * 2);
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(x), "r"(bytes) : "memory");
+  }
   pdl_wait();
   pdl_trigger();
   if (tid == 0) SWAPMOE_STAMP(0, 1);
@@ -194,13 +266,20 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
   }
   if (tid == 0) SWAPMOE_STAMP(0, 2);
   bool alive = true;
+  if (n_rw <= 2 && RW % 16 == 0) {
+    // the whole router matrix is resident in the two wave buffers: one pass over all experts
+    for (int w = 0; w < n_rw && alive; ++w) alive = dec_wait_wave(bars, w, R, status, 23);
+    if (tid == 0) SWAPMOE_STAMP(0, 11);
+    if (alive) rs_dots_resident<NT>(ring, E, RW, d, xs, T, red, slog);
+  } else {
 #pragma unroll 1
-  for (int w = 0; w < n_rw; ++w) {
-    if (!dec_wait_wave(bars, w, R, status, 23)) { alive = false; break; }
-    rs_wave_dots<NT>(ring + (w & 1) * kDecHalfBytes, min(RW, E - w * RW), d, xs, T, red, slog + w * RW, kMaxE + 1);
-    if (warp == 0 && w + 2 < n_rw) {
-      ptx::fence_proxy_async();
-      issue_router_wave(w + 2);
+    for (int w = 0; w < n_rw; ++w) {
+      if (!dec_wait_wave(bars, w, R, status, 23)) { alive = false; break; }
+      rs_wave_dots<NT>(ring + (w & 1) * kDecHalfBytes, min(RW, E - w * RW), d, xs, T, red, slog + w * RW, kMaxE + 1);
+      if (warp == 0 && w + 2 < n_rw) {
+        ptx::fence_proxy_async();
+        issue_router_wave(w + 2);
+      }
     }
   }
   if (!alive)
@@ -296,7 +375,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
   if (tid < E) {
     float s = 0.f;
     int n = 0;
-#pragma unroll 1
+#pragma unroll 8
     for (int p = 0; p < P; ++p)
       if (Q->ue[p] == tid) { s += Q->pt[p]; ++n; }
     a.cta_imp[(size_t)blockIdx.x * E + tid] = s;
@@ -306,7 +385,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) router_small_kernel(const Rout
     const int sl = kDecThreads - 1 - tid;                   // the last K threads: slot sums
     int c = 0;
     float m = 0.f;
-#pragma unroll 1
+#pragma unroll 8
     for (int p = 0; p < P; ++p)
       if (Q->sl[p] == sl) { ++c; m += Q->pm[p]; }
     a.cta_hist[(size_t)blockIdx.x * K + sl] = c;

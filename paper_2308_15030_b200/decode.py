@@ -62,10 +62,11 @@ class LayerState:
     last_used: Optional[np.ndarray] = None                 # [K] step at which each slot last served a token (on_demand)
 
 
-def suggest_step_budget(step_seconds: float, pcie_gbytes_per_s: float, expert_bytes: int, share: float = 0.9) -> int:
+def suggest_step_budget(step_seconds: float, pcie_gbytes_per_s: float, expert_bytes: int, share: float = 0.9) -> float:
     """Loads per step that the host link can carry while a step runs (Section 3.4.1: the update
-    traffic must stay below what the link delivers in the time the computation takes)."""
-    return max(1, int(share * step_seconds * pcie_gbytes_per_s * 1e9 / expert_bytes))
+    traffic must stay below what the link delivers in the time the computation takes).  May be a
+    fraction: 0.5 means one load every other step."""
+    return share * step_seconds * pcie_gbytes_per_s * 1e9 / expert_bytes
 
 
 class DecodeStack:
@@ -73,14 +74,18 @@ class DecodeStack:
 
     def __init__(self, layers: Sequence[LayerState], frequency: int = 8, loads_per_step: int = 1,
                  lag: int = 2, compute_stream=None, side_stream=None, time_loads: bool = False,
-                 graph_buffers=None, step_budget: Optional[int] = None, commit: str = "wait",
+                 graph_buffers=None, step_budget: Optional[float] = None, commit: str = "wait",
                  policy: str = "swap", event_factory: Optional[Callable[[], object]] = None,
-                 track_hits: bool = False):
+                 track_hits: bool = False, async_decide: bool = False,
+                 score_alloc: Optional[Callable[[int], object]] = None, max_in_flight: Optional[int] = None):
         import torch
         assert commit in ("wait", "ready") and policy in ("swap", "static_pruning", "on_demand")
         self.layers = list(layers)
         self.frequency, self.loads_per_step, self.lag = int(frequency), int(loads_per_step), int(lag)
-        self.step_budget = None if step_budget is None else int(step_budget)
+        # step_budget: loads per step over all layers; fractions accumulate from step to step (0.5 = one
+        # load every other step), whole budgets do not carry over
+        self.step_budget = None if step_budget is None else float(step_budget)
+        self._bucket = 0.0
         self.commit, self.policy = commit, policy
         self.compute = compute_stream or torch.cuda.current_stream()
         self.side = side_stream or torch.cuda.Stream()
@@ -96,6 +101,23 @@ class DecodeStack:
         self.misses = 0            # on_demand: requested experts that were not resident
         self.blocking_loads = 0    # on_demand: loads the compute stream waited for
         self.requests = 0          # on_demand: (token, expert) requests seen
+        # async_decide: the scores of a decision step are only ENQUEUED for copy-out (pinned buffers, one event);
+        # the top-K choice is made at a later step, once the event has fired - the host never waits for the
+        # device, so the queue of forwards never drains
+        # max_in_flight: the host enqueues step n only once step n - max_in_flight has finished on the device (an
+        # autoregressive decoder cannot run further ahead than its sampler anyway).  Without a bound a host that
+        # is faster than the device queues hundreds of steps, every expert copy - ordered behind the queue - lands
+        # that much later, and the resident sets lag behind the traffic they are meant to follow.
+        self.max_in_flight = max_in_flight
+        self._step_events = []
+        self.host_seconds = 0.0    # host time spent preparing and enqueuing steps (waits for the device excluded)
+        self.throttle_waits = 0    # steps before which the host had to wait for the device (max_in_flight)
+        self._t_step = None
+        self.async_decide = async_decide
+        self.score_alloc = score_alloc or (lambda E: torch.empty((3, E), dtype=torch.float32).pin_memory())
+        self._inflight = None      # (step, event, [pinned score tensors per layer]) of the decision being read
+        self._todo = []            # layers of that decision still to be decided
+        self.decisions_per_step = max(1, -(-len(self.layers) // max(1, min(4, self.frequency - 1))))
         self.track_hits = track_hits
         self.hits = 0              # track_hits: requests of the off-the-shelf gate that met a resident expert ...
         self.asked = 0             # ... out of this many (read at every decision; the table at the decision counts)
@@ -117,6 +139,7 @@ class DecodeStack:
     def step(self, xs: Sequence, outs: Sequence, record: bool = True) -> None:
         """xs[l], outs[l]: device tensors [B, d_model] of layer l for this step."""
         n = self.step_no
+        self._throttle()
         for li, st in enumerate(self.layers):
             self._commit_due(st, n)
             if self.policy == "on_demand":
@@ -125,6 +148,7 @@ class DecodeStack:
             if record:
                 self.trace.append((n, li, st.s2e.copy(), st.phys.copy()))
             st.layer.forward(xs[li], outs[li], stream=self.compute)
+        self._mark_step()
         self._schedule(n)
         self.step_no += 1
 
@@ -145,14 +169,34 @@ class DecodeStack:
                 with torch.cuda.graph(self.graph, capture_error_mode="thread_local"):   # torch's own side stream
                     for li, st in enumerate(self.layers):
                         st.layer.forward(x_buf[li], out_buf[li], stream=None)
+            self._throttle()
             x_buf.copy_(x_step, non_blocking=True)
             for li, st in enumerate(self.layers):
                 self._commit_due(st, n)
                 if record:
                     self.trace.append((n, li, st.s2e.copy(), st.phys.copy()))
             self.graph.replay()
+            self._mark_step()
         self._schedule(n)
         self.step_no += 1
+
+    def _throttle(self) -> None:
+        import time
+        t0 = time.perf_counter()
+        if self._t_step is not None:
+            self.host_seconds += t0 - self._t_step       # host work of the step before (everything but this wait)
+        if self.max_in_flight is not None and len(self._step_events) >= self.max_in_flight:
+            ev = self._step_events.pop(0)
+            if not ev.query():
+                ev.synchronize()
+                self.throttle_waits += 1                   # the device was still busy: the host is ahead
+        self._t_step = time.perf_counter()
+
+    def _mark_step(self) -> None:
+        if self.max_in_flight is not None:
+            ev = self.new_event()
+            ev.record(self.compute)
+            self._step_events.append(ev)
 
     def loader_seconds(self) -> float:
         """Sum of the device-side durations of all copies issued so far (needs time_loads)."""
@@ -162,13 +206,19 @@ class DecodeStack:
     def _schedule(self, n: int) -> None:
         if self.policy != "swap":
             return
-        if (n + 1) % self.frequency == 0:
+        if self.async_decide:
+            self._decide_async(n)
+        elif (n + 1) % self.frequency == 0:
             for li, st in enumerate(self.layers):
                 self._decide(li, st, n)
         # amortised loading: the step's budget is dealt round-robin, starting at a layer that
         # moves on every step so that no layer's queue is starved
         L = len(self.layers)
-        left = self.step_budget if self.step_budget is not None else L * self.loads_per_step
+        if self.step_budget is not None:
+            self._bucket = min(self._bucket + self.step_budget, max(1.0, self.step_budget))
+            left = int(self._bucket + 1e-9)
+        else:
+            left = L * self.loads_per_step
         issued = [0] * L
         progress = True
         while left > 0 and progress:
@@ -180,6 +230,7 @@ class DecodeStack:
                     self._issue_load(st, n)
                     issued[li] += 1
                     left -= 1
+                    self._bucket -= 1.0
                     progress = True
 
     def _commit_due(self, st: LayerState, n: int) -> None:
@@ -205,13 +256,39 @@ class DecodeStack:
         if flipped:
             st.layer.set_resident(st.s2e, st.arena_in, st.arena_out, st.phys, stream=self.compute)
 
-    def _decide(self, li: int, st: LayerState, n: int) -> None:
+    def _decide_async(self, n: int) -> None:
+        if self._inflight is not None and (self._todo or self._inflight[1].query()):
+            # the scores have landed: the layers' decisions are taken a few per step, so that no step has to
+            # wait for the host to work through all of them (the device only has max_in_flight steps queued)
+            n0, _, bufs = self._inflight
+            if not self._todo:
+                self._todo = list(range(len(self.layers)))
+            for li in [self._todo.pop(0) for _ in range(min(len(self._todo), self.decisions_per_step))]:
+                st = self.layers[li]
+                E = st.layer.cfg.E
+                self._decide(li, st, n0, imp=bufs[li][0, :E].numpy().copy(),
+                             cnt=bufs[li][1, :E].numpy().copy() if self.track_hits else None)
+            if not self._todo:
+                self._inflight = None
+        if (n + 1) % self.frequency == 0 and self._inflight is None:
+            if not hasattr(self, "_score_bufs"):
+                self._score_bufs = [self.score_alloc(st.layer.cfg.E) for st in self.layers]
+            kinds = ("eq1", "count") if self.track_hits else ("eq1",)
+            for li, st in enumerate(self.layers):
+                st.layer.read_scores_async(kinds, self._score_bufs[li], reset=True, stream=self.compute)
+            ev = self.new_event()
+            ev.record(self.compute)
+            self._inflight = (n, ev, self._score_bufs)
+
+    def _decide(self, li: int, st: LayerState, n: int, imp=None, cnt=None) -> None:
         K = st.layer.cfg.K
-        imp = st.layer.read_importance(reset=True, stream=self.compute)
+        if imp is None:
+            imp = st.layer.read_importance(reset=True, stream=self.compute)
+            if self.track_hits:
+                cnt = st.layer.read_score("count", reset=True, stream=self.compute)
         top = binding.topk_importance(imp, K)
         self.decisions.append((n, li, imp.copy(), top.copy()))
-        if self.track_hits:
-            cnt = st.layer.read_score("count", reset=True, stream=self.compute)
+        if cnt is not None:
             self.hits += float(cnt[st.s2e].sum())
             self.asked += float(cnt.sum())
         # residents after all pending commits
@@ -245,8 +322,12 @@ class DecodeStack:
         p = _Pending(n + self.lag, slot, expert, phys, ev)
         st.pending.append(p)
         self.loads += 1
-        self.bytes_loaded += st.host_in[expert].numel() * st.host_in.element_size() + \
-            st.host_out[expert].numel() * st.host_out.element_size()
+        if li_bytes := getattr(st, "_expert_bytes", None):
+            self.bytes_loaded += li_bytes
+        else:
+            st._expert_bytes = st.host_in[expert].numel() * st.host_in.element_size() + \
+                st.host_out[expert].numel() * st.host_out.element_size()
+            self.bytes_loaded += st._expert_bytes
         return p
 
     # ---------------------------------------------------------------- comparison policies (Section 4.1)

@@ -3,6 +3,7 @@ copy events (no GPU): asynchronous loading must not block inference (Section 3.2
 per-step load budget is honoured and dealt fairly (amortised loading), and the step budget follows
 the link rate (Section 3.4.1)."""
 import numpy as np
+import torch
 
 from paper_2308_15030_b200 import binding
 from paper_2308_15030_b200.decode import DecodeStack, LayerState, suggest_step_budget
@@ -14,6 +15,9 @@ class FakeEvent:
 
     def query(self):
         return self.done
+
+    def record(self, stream):
+        pass
 
 
 class FakeStream:
@@ -51,6 +55,9 @@ class FakeLayer:
 
     def load_slot_async(self, phys, h_in, h_out, compute, side, ev):
         self.loads.append((phys, ev))
+
+    def read_scores_async(self, kinds, out, reset=False, stream=None):
+        out[0, : self.cfg.E] = torch.from_numpy(self.imp)
 
 
 class FakeHost:
@@ -127,9 +134,20 @@ def test_step_budget_is_global_and_rotates_over_the_layers():
 
 
 def test_budget_from_link_rate():
-    # 0.8 ms per step at 50 GB/s carries 40 MB: two 16.8 MB experts
-    assert suggest_step_budget(0.8e-3, 50.0, 16_777_216) == 2
-    assert suggest_step_budget(1e-5, 50.0, 16_777_216) == 1       # never below one
+    # 0.8 ms per step at 50 GB/s carries 40 MB, 90 % of it for loads: a little over two 16.8 MB experts
+    assert 2.0 <= suggest_step_budget(0.8e-3, 50.0, 16_777_216) < 2.2
+    # a 0.2 ms step carries half an expert: the budget is a fraction, i.e. one load every other step
+    b = suggest_step_budget(0.2e-3, 50.0, 16_777_216)
+    assert 0.5 <= b < 0.6
+    stack, layers, _ = _stack(n_layers=2, K=2, E=8, spare=2, frequency=1, lag=100, step_budget=b, commit="ready")
+    for st in layers:
+        st.layer.imp[:] = [0, 0, 9, 8, 0, 0, 0, 0]
+    per_step = []
+    for _ in range(8):
+        before = stack.loads
+        stack.step([None] * 2, [None] * 2)
+        per_step.append(stack.loads - before)
+    assert max(per_step) == 1 and sum(per_step) == 4 and per_step[0] == 0      # 4 loads wanted, one every other step
 
 
 def test_layers_may_have_different_budgets():
@@ -144,3 +162,30 @@ def test_layers_may_have_different_budgets():
     stack.step([None] * 3, [None] * 3)
     assert stack.loads == 0
     assert [len(d[3]) for d in stack.decisions] == Ks
+
+
+def test_asynchronous_decisions_never_wait_for_the_device():
+    """async_decide: the scores are only enqueued for copy-out at the decision step; the choice is made at the
+    first later step at which the copy's event has fired, with the values of the decision step."""
+    made = []
+
+    def factory():
+        made.append(FakeEvent())
+        return made[-1]
+
+    layers = [LayerState(FakeLayer(2, 6), np.arange(2, dtype=np.int32), np.arange(2, dtype=np.int32), [2],
+                         None, None, FakeHost(), FakeHost())]
+    stack = DecodeStack(layers, frequency=2, lag=0, compute_stream=FakeStream(), side_stream=FakeStream(),
+                        event_factory=factory, commit="ready", async_decide=True,
+                        score_alloc=lambda E: torch.zeros((3, E)))
+    L = layers[0].layer
+    L.imp[:] = [1, 1, 9, 0, 0, 0]
+    stack.step([None], [None])                 # step 0: nothing
+    stack.step([None], [None])                 # step 1: decision step -> copy enqueued, event pending
+    assert len(made) == 1 and not stack.decisions
+    stack.step([None], [None])                 # event not fired yet: still no decision, no load
+    assert not stack.decisions and stack.loads == 0
+    made[0].done = True
+    stack.step([None], [None])                 # fired: the decision of step 1 is taken now, the load goes out
+    assert [d[0] for d in stack.decisions] == [1] and stack.loads == 1
+    assert 2 in stack.decisions[0][3].tolist()

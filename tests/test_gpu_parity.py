@@ -516,3 +516,72 @@ def test_decode_path_default_threshold():
         out = case.run()
         assert (case.layer.launch_count - n0 == 1) == one
         check_against_oracle(case, out)
+
+
+def test_decode_step_prefetch_of_recent_experts_counts_its_hits(monkeypatch):
+    """Decode steps pull the experts served last towards L2 while they route (Section 2.2, activation locality).
+    The same token twice: the second step's slot was predicted; the results stay those of the oracle."""
+    from harness import Case, check_against_oracle
+    monkeypatch.setenv("SWAPMOE_DECODE_PREFETCH", "2")
+    cfg = _cfg(T=2, d=256, f=512, E=16, K=6, zipf_s=1.1, seed=11)
+    case = Case(cfg)
+    case.layer.read_decode_prefetch(reset=True)
+    n0 = case.layer.launch_count
+    out1 = case.run()
+    hits, touched = case.layer.read_decode_prefetch()
+    assert case.layer.launch_count - n0 == 1 and hits == 0 and 1 <= touched <= 2
+    out2 = case.run()
+    hits2, touched2 = case.layer.read_decode_prefetch(reset=True)
+    assert touched2 == 2 * touched and hits2 == touched          # every slot of the repeat had been served just before
+    assert np.array_equal(out1, out2)
+    case.layer.read_importance(reset=True)
+    check_against_oracle(case, case.run())
+
+
+def test_scores_snapshot_without_a_wait():
+    """swapmoe_read_scores_async: one small kernel writes the selected per-expert scores into pinned host memory
+    and zeroes them; the values are those the blocking reads return."""
+    import torch
+    from harness import Case
+    cfg = _cfg(T=300, d=128, f=256, E=24, K=5, k=2, renorm=1, zipf_s=1.1)
+    case = Case(cfg)
+    case.run()
+    ref = {k: case.layer.read_score(k) for k in ("eq1", "count", "eq1_masked")}
+    assert ref["count"].sum() == 300 * 2
+    buf = torch.full((3, cfg.E), -1.0).pin_memory()
+    case.layer.read_scores_async(("eq1", "eq1_masked"), buf, reset=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(buf[0].numpy(), ref["eq1"]) and np.array_equal(buf[2].numpy(), ref["eq1_masked"])
+    assert np.all(buf[1].numpy() == -1.0)                                  # not selected: untouched
+    assert not case.layer.read_score("eq1").any() and not case.layer.read_score("eq1_masked").any()
+    assert np.array_equal(case.layer.read_score("count"), ref["count"])   # not selected: not reset
+
+
+@pytest.mark.parametrize("swap", ["1", "0"])
+def test_fp32_small_slots_swapped_operands(monkeypatch, swap):
+    """fp32 ReLU layers with small slots put the weights on the tensor core's rows and the slot's tokens on its
+    columns (64-token tiles); slots from a handful of rows to more than one tile, GEMM-2 with a sliced
+    contraction.  SWAPMOE_FP32_SWAP=0 runs the same layer on 128-token tiles."""
+    from harness import Case, check_against_oracle
+    monkeypatch.setenv("SWAPMOE_FP32_SWAP", swap)
+    for cfg in (_cfg(T=330, dtype=I.F32, d=256, f=512, E=8, K=5, zipf_s=1.3),
+                _cfg(T=90, dtype=I.F32, d=128, f=384, E=16, K=6, k=2, renorm=1, zipf_s=1.0)):
+        case = Case(cfg)
+        res = check_against_oracle(case, case.run())
+        assert res["out_rel_err"] <= 1e-4
+        cnt = res["oracle"]["count"]
+        assert cnt.max() > 64 or cfg.T < 100
+
+
+@pytest.mark.parametrize("swap", ["1", "0"])
+def test_fp32_small_slots_swapped_operands(monkeypatch, swap):
+    """fp32 ReLU layers with small slots put the weights on the tensor core's rows and the slot's tokens on its
+    columns (64-token tiles); slots from a handful of rows to more than one tile, GEMM-2 with a sliced
+    contraction.  SWAPMOE_FP32_SWAP=0 runs the same layer on 128-token tiles."""
+    from harness import Case, check_against_oracle
+    monkeypatch.setenv("SWAPMOE_FP32_SWAP", swap)
+    for cfg in (_cfg(T=330, dtype=I.F32, d=256, f=512, E=8, K=5, zipf_s=1.3),
+                _cfg(T=90, dtype=I.F32, d=128, f=384, E=16, K=6, k=2, renorm=1, zipf_s=1.0)):
+        case = Case(cfg)
+        res = check_against_oracle(case, case.run())
+        assert res["out_rel_err"] <= 1e-4
