@@ -196,7 +196,7 @@ MIN_REGION_MS = 250.0      # the timed loop is repeated until it covers at least
 
 
 def measure_layer(cfg, steps, warmup, *, rank=0, world=1, local=0, no_graph=False, want_e2e=True,
-                  sampler=None, barrier=None):
+                  sampler=None, barrier=None, min_region_ms=MIN_REGION_MS):
     """Times `steps` forwards of one layer configuration (device-resident inputs), a stage-event pass,
     a warm-cache loop and, if asked, the end-to-end host-buffer path.  Returns a dict of raw figures."""
     import torch
@@ -301,7 +301,7 @@ def measure_layer(cfg, steps, warmup, *, rank=0, world=1, local=0, no_graph=Fals
 
     barrier()
     est = timed(graph, 1)[0]                                      # untimed estimate of one K-step loop
-    reps = int(min(400, max(1, np.ceil(MIN_REGION_MS / max(est, 1e-3)))))
+    reps = int(min(400, max(1, np.ceil(min_region_ms / max(est, 1e-3)))))
     if sampler is not None:
         sampler.mark_begin()
     barrier()
@@ -404,7 +404,7 @@ def run_cuda(args, cfg):
     if rank == 0:
         sampler.start()          # started early: nvidia-smi needs a moment before its first sample
     m = measure_layer(cfg, args.steps, args.warmup, rank=rank, world=world, local=local, no_graph=args.no_graph,
-                      want_e2e=True, sampler=sampler, barrier=barrier)
+                      want_e2e=True, sampler=sampler, barrier=barrier, min_region_ms=args.min_region_ms)
     clocks = sampler.stop() if rank == 0 else None     # sampled over the timed regions (all under load)
 
     from paper_2308_15030_b200.replicas import max_over_ranks
@@ -425,7 +425,7 @@ def run_cuda(args, cfg):
         "scaling": "weak", "vs_baseline": None, "dtype": ent["dtype"], "data": "synthetic",
         "config": {"workload": ent["workload"], "l2": ent["l2"], "launch": ent["launch"],
                    "timing": "median of %d back-to-back repeats of the %d-step loop (>= %.0f ms of device time)"
-                             % (m["reps"], args.steps, MIN_REGION_MS),
+                             % (m["reps"], args.steps, args.min_region_ms),
                    "resident_set": "top-K by Eq.(1) importance of the batch",
                    "touched_slots": ent["touched_slots"], "slot_counts": ent["slot_counts"],
                    "unmasked_hit_rate": ent["unmasked_hit_rate"], "multi_gpu": "replicas only"},
@@ -736,6 +736,8 @@ def main():
                     help="cfg4 diagnostic: swapping arm without expert copies / with copies that are never committed")
     ap.add_argument("--policies", action="store_true",
                     help="cfg4: also run static pruning / on-demand loading / swapping at K = 4, 8, 16 and per-layer K")
+    ap.add_argument("--min-region-ms", type=float, default=MIN_REGION_MS,
+                    help="repeat the timed K-step loop until it covers this much device time (0: once; for profiler runs)")
     ap.add_argument("--no-per-config", action="store_true",
                     help="default workload: skip the short runs of cfg1, cfg3, cfg4, cfg5 that fill `per_config`")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -752,7 +754,7 @@ def main():
     if args.workload == "cfg4":
         print(json.dumps(run_decode(args, cfg)), flush=True)
         return
-    per_config = args.workload == "cfg2" and args.gpus == 1 and not args.no_per_config and args.steps is None
+    per_config = args.workload == "cfg2" and args.gpus == 1 and not args.no_per_config
     args.steps = 2000 if args.steps is None else args.steps
     args.warmup = 50 if args.warmup is None else max(3, args.warmup)
     res = run_cuda(args, cfg)

@@ -79,13 +79,17 @@ __device__ __forceinline__ GateSmem gate_smem_carve(void* base) {
 // valid and of resident experts.  All 256 threads; the caller synchronises afterwards.
 __device__ __forceinline__ void gate_load_tables(const RouterArgs& a, const GateSmem& g) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // (a table entry outside [0, K) - possible only when the caller hands in its own table, as swapmoe_route_static
+  // allows - counts as "not resident")
   for (int e = tid; e < kMaxE; e += kGateThreads) {
-    g.s_e2s[e] = e < a.E ? a.e2s[e] : -1;
+    const int sl = e < a.E ? a.e2s[e] : -1;
+    g.s_e2s[e] = sl < a.K ? sl : -1;
     g.s_enorm[e] = e < a.E ? a.enorm[e] : 0.f;
   }
   // warp w builds word w of the valid-expert mask and of the resident-expert mask
   const int e = warp * 32 + lane;
-  const int sl = e < a.E ? a.e2s[e] : -1;
+  int sl = e < a.E ? a.e2s[e] : -1;
+  if (sl >= a.K) sl = -1;
   const uint32_t wv = __ballot_sync(0xffffffffu, e < a.E), wr = __ballot_sync(0xffffffffu, sl >= 0);
   if (lane == 0) { g.s_mask[warp] = wv; g.s_mask[8 + warp] = wr; g.s_present[warp] = 0u; }
 }
@@ -226,7 +230,12 @@ __device__ __forceinline__ void gate_epilogue(const RouterArgs& a, const GateSme
             g.pe[pl] = -1; g.pt[pl] = 0.f;
           }
         } else {
-          if (token < a.T) {
+          if (token < a.T && e < 0) {
+            // fewer resident experts than top_k (a caller-supplied table: the layer API rules it out): the pair
+            // is routed nowhere instead of indexing the tables with -1
+            a.midx[p] = -1; a.mgate[p] = 0.f; a.slot[p] = -1;
+            g.ps[pl] = -1; g.pm[pl] = 0.f;
+          } else if (token < a.T) {
             const int sl = g.s_e2s[e];
             a.midx[p] = e; a.mgate[p] = gv; a.slot[p] = sl;
             g.ps[pl] = sl; g.pm[pl] = xn * fabsf(gv) * g.s_enorm[e];
