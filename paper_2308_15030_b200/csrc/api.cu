@@ -17,6 +17,7 @@
 #include "gemm_tc.cuh"
 #include "gemm_tc_f32.cuh"
 #include "gemm_tc_pair.cuh"
+#include "gemm_tc_ffn.cuh"
 #include "gemm_tc_small.cuh"
 #include "permute.cuh"
 #include "router_gate.cuh"

@@ -101,10 +101,10 @@ __device__ __forceinline__ void rs_wave_dots(const unsigned char* st, int rows, 
 }
 
 // All logits of the CTA in ONE pass when the router matrix fits the two wave buffers (E <= 2 waves of rows):
-// the output is cut into tiles of 16 experts x 8 tokens (at most 4 x NT of them), a warp owns one tile and a
-// contiguous share of the contraction, and the 16 / tiles shares of a tile are added in order.  Per CTA that is
-// one pair of barriers and a 2-way sum for 64 experts x 16 tokens, where the wave-by-wave form (every wave's
-// contraction split over all 16 warps) pays a 16-way sum and two barriers per wave.
+// a warp owns a tile of 16 experts (all NT token tiles of it: the router-matrix fragments are read once and
+// feed NT mma) and a contiguous share of the contraction; the 16 / tiles shares of a tile are added in order.
+// Per CTA that is one pair of barriers and a 4-way sum for 64 experts x 16 tokens, where the wave-by-wave form
+// (every wave's contraction split over all 16 warps) pays a 16-way sum and two barriers per wave.
 // slog[token * (kMaxE + 1) + expert] receives the logits.
 template <int NT>
 __device__ __forceinline__ void rs_dots_resident(const unsigned char* ring, int E, int RW, int d, const unsigned char* xs,
@@ -112,54 +112,50 @@ __device__ __forceinline__ void rs_dots_resident(const unsigned char* ring, int 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int pitch = d * 2 + kDecRowPad;
   const int MT = (E + 15) >> 4;                 // 16-expert row tiles (<= 4)
-  const int n_tiles = MT * NT;                  // <= 8
   int tiles_p2 = 1;
-  while (tiles_p2 < n_tiles) tiles_p2 <<= 1;
-  const int S = kDecWarps / tiles_p2;           // shares of the contraction per tile
-  const int tile = warp & (tiles_p2 - 1), part = warp / tiles_p2;
-  if (tile < n_tiles) {
-    const int m = tile / NT, j = tile - m * NT;
+  while (tiles_p2 < MT) tiles_p2 <<= 1;
+  const int S = kDecWarps / tiles_p2;           // shares of the contraction per tile (>= 4)
+  const int m = warp & (tiles_p2 - 1), part = warp / tiles_p2;
+  if (m < MT) {
     const int row0 = m * 16;                    // first expert of the tile; wave row0 / RW, row row0 % RW inside it
     const unsigned char* ap0 = ring + (row0 / RW) * kDecHalfBytes + ((row0 % RW) + g) * pitch + t * 4;
-    const unsigned char* xrow = xs + min(8 * j + g, n_tok - 1) * pitch + t * 4;
+    const unsigned char* xrow[NT];
+#pragma unroll
+    for (int j = 0; j < NT; ++j) xrow[j] = xs + min(8 * j + g, n_tok - 1) * pitch + t * 4;
     const int nks = d / 16, ks0 = part * nks / S, ks1 = (part + 1) * nks / S;
-    // two accumulators (even / odd steps) halve the chain of dependent mma; their sum is the share's product
-    float acc[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
-    int ks = ks0;
+    float acc[NT][4];
+#pragma unroll
+    for (int j = 0; j < NT; ++j)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) acc[j][q] = 0.f;
 #pragma unroll 4
-    for (; ks + 1 < ks1; ks += 2) {
+    for (int ks = ks0; ks < ks1; ++ks) {
       const int kb = ks * 32;
       const uint32_t a0 = lds32(ap0 + kb), a1 = lds32(ap0 + 8 * pitch + kb), a2 = lds32(ap0 + kb + 16),
                      a3 = lds32(ap0 + 8 * pitch + kb + 16);
-      const uint32_t b0 = lds32(xrow + kb), b1 = lds32(xrow + kb + 16);
-      const uint32_t c0 = lds32(ap0 + kb + 32), c1 = lds32(ap0 + 8 * pitch + kb + 32), c2 = lds32(ap0 + kb + 48),
-                     c3 = lds32(ap0 + 8 * pitch + kb + 48);
-      const uint32_t d0 = lds32(xrow + kb + 32), d1 = lds32(xrow + kb + 48);
-      mma_bf16_16x8x16(acc, a0, a1, a2, a3, b0, b1);
-      mma_bf16_16x8x16(acc1, c0, c1, c2, c3, d0, d1);
-    }
-    if (ks < ks1) {
-      const int kb = ks * 32;
-      const uint32_t a0 = lds32(ap0 + kb), a1 = lds32(ap0 + 8 * pitch + kb), a2 = lds32(ap0 + kb + 16),
-                     a3 = lds32(ap0 + 8 * pitch + kb + 16);
-      const uint32_t b0 = lds32(xrow + kb), b1 = lds32(xrow + kb + 16);
-      mma_bf16_16x8x16(acc, a0, a1, a2, a3, b0, b1);
+#pragma unroll
+      for (int j = 0; j < NT; ++j) {            // NT independent accumulators: NT chains of dependent mma
+        const uint32_t b0 = lds32(xrow[j] + kb), b1 = lds32(xrow[j] + kb + 16);
+        mma_bf16_16x8x16(acc[j], a0, a1, a2, a3, b0, b1);
+      }
     }
 #pragma unroll
-    for (int q = 0; q < 4; ++q) acc[q] += acc1[q];
-    float* rp = red + ((part * n_tiles + tile) * 16 + g) * 8 + 2 * t;
-    *reinterpret_cast<float2*>(rp) = make_float2(acc[0], acc[1]);
-    *reinterpret_cast<float2*>(rp + 8 * 8) = make_float2(acc[2], acc[3]);
+    for (int j = 0; j < NT; ++j) {
+      float* rp = red + (((part * MT + m) * NT + j) * 16 + g) * 8 + 2 * t;
+      *reinterpret_cast<float2*>(rp) = make_float2(acc[j][0], acc[j][1]);
+      *reinterpret_cast<float2*>(rp + 8 * 8) = make_float2(acc[j][2], acc[j][3]);
+    }
   }
   if (tid == 0) SWAPMOE_STAMP(0, 12);
   __syncthreads();
   if (tid == 0) SWAPMOE_STAMP(0, 13);
+  const int n_tiles = MT * NT;
   for (int o = tid; o < n_tiles * 128; o += kDecThreads) {
-    const int tl = o >> 7, r = (o >> 3) & 15, c = o & 7;
+    const int tl = o >> 7, r = (o >> 3) & 15, c = o & 7;      // tl = m * NT + j
     float sum = 0.f;
     for (int p = 0; p < S; ++p) sum += red[((p * n_tiles + tl) * 16 + r) * 8 + c];
-    const int m = tl / NT, j = tl - m * NT;
-    const int e = m * 16 + r, tok = 8 * j + c;
+    const int mm = tl / NT, j = tl - mm * NT;
+    const int e = mm * 16 + r, tok = 8 * j + c;
     if (e < E && tok < n_tok) slog[tok * (kMaxE + 1) + e] = sum;
   }
   __syncthreads();

@@ -585,3 +585,15 @@ def test_fp32_small_slots_swapped_operands(monkeypatch, swap):
         case = Case(cfg)
         res = check_against_oracle(case, case.run())
         assert res["out_rel_err"] <= 1e-4
+
+
+@pytest.mark.parametrize("k,renorm,T", [(1, 0, 1200), (2, 1, 600)])
+def test_switch_shaped_mid_batch(k, renorm, T):
+    """Switch-shaped layer (d_model 768, d_ff 3072) at a batch of a few row tiles: slots above and below one row
+    tile, ragged tiles, the gate-weighted scatter epilogue (top-1) and the fp32 y epilogue (top-2)."""
+    from harness import Case, check_against_oracle
+    cfg = _cfg(T=T, d=768, f=3072, E=16, K=8, k=k, renorm=renorm, zipf_s=1.2, seed=12)
+    case = Case(cfg)
+    res = check_against_oracle(case, case.run())
+    cnt = res["oracle"]["count"]
+    assert cnt.max() > 128 and cnt.min() < 128
