@@ -17,6 +17,7 @@ exchange step), rank 0 prints the aggregate.
 from __future__ import annotations
 
 import argparse
+import gc
 import json
 import os
 import subprocess
@@ -556,14 +557,16 @@ def run_decode(args, cfg):
             base = dict(host=stack.host_seconds, waits=stack.throttle_waits, loads=stack.loads, bytes=stack.bytes_loaded, stalls=stack.stalls, deferred=stack.deferred,
                         commits=stack.commits, hits=stack.hits, asked=stack.asked, misses=stack.misses,
                         blocking=stack.blocking_loads, requests=stack.requests, n_ev=len(stack.load_events),
-                        launches=sum(st.layer.launch_count for st in stack.layers))
+                        launches=sum(st.layer.launch_count for st in stack.layers), replays=stack.graph_replays)
             if first_timed:
                 sampler.mark_begin()
                 first_timed = False
+            gc.collect(); gc.disable()           # no collector pause inside the timed loop (the scheduler is Python)
             e0.record()
             for s_ in range(steps):
                 stepper(s_)
             e1.record(); torch.cuda.synchronize()
+            gc.enable()
             ms = e0.elapsed_time(e1)
             touched = sum(st.layer.read_touched_slots(reset=True) for st in stack.layers)
             pf = [st.layer.read_decode_prefetch(reset=True) for st in stack.layers]
@@ -574,7 +577,9 @@ def run_decode(args, cfg):
             load_s = sum(a.elapsed_time(b) for a, b in stack.load_events[base["n_ev"]:]) * 1e-3
             nbytes = stack.bytes_loaded - base["bytes"]
             r = {"tokens_per_s": steps * B / (ms * 1e-3), "ms_per_step": ms / steps, "us_per_layer": ms / steps / L * 1e3,
-                 "gpu_launches": sum(st.layer.launch_count for st in stack.layers) - base["launches"],
+                 # eager launches (score snapshots, table updates) + the kernels of every replay of the captured step
+                 "gpu_launches": sum(st.layer.launch_count for st in stack.layers) - base["launches"]
+                 + (stack.graph_replays - base["replays"]) * stack.graph_launches,
                  "touched_slots_per_layer_step": touched / (steps * L),
                  "roofline_us_per_layer": t_roof / (steps * L) * 1e6, "roofline_frac": t_roof * 1e3 / ms,
                  "loads": stack.loads - base["loads"], "loaded_GB": nbytes / 1e9,
@@ -618,9 +623,9 @@ def run_decode(args, cfg):
                                             track_hits=True, async_decide=True, max_in_flight=3)) for fr in args.sweep_frequency}
         if args.sweep_budget and big:
             entry["budget_sweep"] = {
-                str(bu): run_arm(make_stack(frequency=args.frequency, loads_per_step=max(1, -(-bu // L)), step_budget=bu,
+                ("%g" % bu): run_arm(make_stack(frequency=args.frequency, loads_per_step=max(1, int(-(-bu // L))), step_budget=bu,
                                             commit="wait" if args.sweep_commit == "wait" else "ready", track_hits=True,
-                                            async_decide=True))
+                                            async_decide=True, max_in_flight=3))
                 for bu in args.sweep_budget}
         # Section 4.1 baselines as policies over the same kernels, and per-layer budgets (Section 3.3)
         if args.policies and big:
@@ -636,7 +641,7 @@ def run_decode(args, cfg):
             Ks = [8, 12, 16, 24] * (L // 4) + [16] * (L % 4)
             entry["per_layer_K"] = dict(run_arm(make_stack(Ks, frequency=args.frequency, loads_per_step=1,
                                                            step_budget=budget, commit="ready", track_hits=True,
-                                                           async_decide=True)), Ks=Ks)
+                                                           async_decide=True, max_in_flight=3)), Ks=Ks)
         results[str(B)] = entry
     clocks = sampler.stop()
     Bmax = str(max(args.batches))
@@ -728,7 +733,7 @@ def main():
     ap.add_argument("--frequency", type=int, default=8, help="cfg4: steps between two updates of the resident sets")
     ap.add_argument("--sweep-frequency", type=int, nargs="*", default=None,
                     help="cfg4: also run the loop (largest batch) at these update frequencies (steps between updates)")
-    ap.add_argument("--sweep-budget", type=int, nargs="*", default=None,
+    ap.add_argument("--sweep-budget", type=float, nargs="*", default=None,
                     help="cfg4: also run the loop (largest batch) with these numbers of expert loads per step")
     ap.add_argument("--sweep-commit", default="ready", choices=["ready", "wait"],
                     help="cfg4 budget sweep: flip when the copy has landed, or wait for it at the commit step")

@@ -21,6 +21,9 @@
 // overlaps the next item's MMAs), warps 8-11 and 12-15 two converter groups (one per lo slot).  A work item is (row tile, column tile,
 // contraction slice): GEMM-2 has few output tiles and a long contraction, so its slices go to
 // separate copies of y that the combine kernel adds in order (deterministic).
+//
+// The swapped form (small slots: weights on the MMA rows, see kF32Swap* below) splits into bf16 pieces instead and
+// needs half as many MMAs per k-block; its converter rewrites the token rows in place.
 #pragma once
 #include "gemm_tc.cuh"
 
@@ -40,6 +43,24 @@ constexpr int kF32SmemBytes = kF32Stages * kF32StageBytes + kF32LoSlots * kF32BB
 // columns are the tokens of a slot tile (kF32SwapTok of them).
 constexpr int kF32SwapTok = 64;                     // token rows per tile = accumulator columns
 constexpr int kF32TmemAcc = 2 * kF32BN;             // columns of the two accumulator sets
+// The swapped form moves 24 KB per k-block (16 KB of weights, 8 KB of tokens): compact stages, eight of them.
+// Its MMAs are small (128 x 64), and a tcgen05.mma costs about 110 clocks however small it is, so the swapped form
+// is paced by the NUMBER of MMAs.  It therefore splits into bf16 pieces instead of TF32 ones: x = b1 + b2 + (rest
+// below 2^-17 |x|) with b1 = bf16(x), b2 = bf16(x - b1), and the product is b2_a*b1_b + b1_a*b2_b + b1_a*b1_b
+// (the dropped terms are below 2^-16 relative): kind::f16 MMAs cover 16 contraction elements each, so a k-block of
+// 32 takes 6 MMAs where the TF32 split takes 12.  The weights' pieces go to tensor memory (16 + 16 packed columns
+// per slot, four slots), the tokens' pieces replace the fp32 row in place: a 128-byte row of 32 fp32 becomes
+// [32 x b1 | 32 x b2], i.e. a K-major bf16 row of 64, so no second buffer is needed.
+constexpr int kF32SwapBBytes = kF32SwapTok * kF32BK * 4;                 // 8 KB
+constexpr int kF32SwapStageBytes = kF32ABytes + kF32SwapBBytes;          // 24 KB
+constexpr int kF32SwapStages = 8;
+constexpr int kF32SwapASlots = 4;                                        // tensor-memory slots of the weight pieces
+constexpr int kF32SwapASlotCols = kF32BK;                                // 16 columns of b1 pairs + 16 of b2 pairs
+constexpr int kF32SwapASlotBase = 2 * kF32SwapTok;                       // behind the two accumulator sets
+constexpr int kF32SwapTmemCols = 256;
+constexpr int kF32SwapSmemBytes = kF32SwapStages * kF32SwapStageBytes + 2048 + kTcEpiStageBytes;
+static_assert(kF32SwapSmemBytes <= 227 * 1024, "shared memory of the swapped form");
+static_assert(kF32SwapASlotBase + kF32SwapASlots * kF32SwapASlotCols <= kF32SwapTmemCols, "tensor memory of the swapped form");
 constexpr int kF32TmemCols = 512;                   // + 2 slots x (hi 32 + lo 32) columns of A, rounded up to a power of two
 
 // Epilogues of the fp32 path (values continue the bf16 kernels' enum)
@@ -74,6 +95,14 @@ __device__ __forceinline__ void umma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, u
       "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n" ::"r"(tmem_d),
+      "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // 32 consecutive 32-bit columns of this thread's TMEM lane <- registers
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
@@ -88,6 +117,17 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 }  // namespace ptx
+
+// x0, x1 -> (b1 pair, b2 pair): b1 = bf16(x) (round to nearest), b2 = bf16(x - b1); element 0 in the low half.
+__device__ __forceinline__ void split_bf16_pair(uint32_t x0, uint32_t x1, uint32_t* p1, uint32_t* p2) {
+  const float f0 = __uint_as_float(x0), f1 = __uint_as_float(x1);
+  const __nv_bfloat162 b1 = __floats2bfloat162_rn(f0, f1);
+  const uint32_t u1 = *reinterpret_cast<const uint32_t*>(&b1);
+  const float r0 = f0 - __uint_as_float(u1 << 16), r1 = f1 - __uint_as_float(u1 & 0xffff0000u);   // exact
+  const __nv_bfloat162 b2 = __floats2bfloat162_rn(r0, r1);
+  *p1 = u1;
+  *p2 = *reinterpret_cast<const uint32_t*>(&b2);
+}
 
 // Instruction descriptor: tf32 x tf32 -> fp32, both operands K-major, M x N tile.
 __host__ __device__ constexpr uint32_t make_idesc_tf32(int M, int N) {
@@ -131,30 +171,40 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   constexpr int kOutCols = kF32BN / kNB;
   constexpr int kNRows = kSwap ? kF32SwapTok : kF32BN;      // rows of the B operand = accumulator columns
   constexpr int kBBytesK = kNRows * kF32BK * 4;             // bytes of the B operand per k-block
-  constexpr uint32_t kTmemCols = kF32TmemCols;
-  constexpr uint32_t kIdesc = make_idesc_tf32(kTcBM, kNRows);
+  constexpr int kStages = kSwap ? kF32SwapStages : kF32Stages;
+  constexpr int kStageBytes = kSwap ? kF32SwapStageBytes : kF32StageBytes;
+  constexpr int kLoSlots = kSwap ? kF32SwapASlots : kF32LoSlots;      // ring of converted k-blocks
+  constexpr int kLoBytes = kSwap ? 0 : kF32BBytes;                     // (the swapped form converts B in place)
+  constexpr int kAccStride = kNRows;                        // TMEM columns per accumulator set
+  constexpr int kASlotBase = kSwap ? kF32SwapASlotBase : kF32TmemAcc;  // first TMEM column of the A slots
+  constexpr int kASlotCols = kSwap ? kF32SwapASlotCols : 2 * kF32BK;
+  constexpr uint32_t kTmemCols = kSwap ? kF32SwapTmemCols : kF32TmemCols;
+  constexpr uint32_t kIdesc = kSwap ? make_idesc_bf16(kTcBM, kNRows) : make_idesc_tf32(kTcBM, kNRows);
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  unsigned char* raw = smem;                                         // [stages][A 16 KB | B 16 KB]
-  unsigned char* lo = smem + kF32Stages * kF32StageBytes;            // [slots][B 16 KB]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(lo + kF32LoSlots * kF32BBytes);
+  unsigned char* raw = smem;                                         // [stages][A 16 KB | B 16 or 8 KB]
+  unsigned char* lo = smem + kStages * kStageBytes;                  // [slots][B]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(lo + kLoSlots * kLoBytes);
   uint64_t* full = bars;                          // [stages]   TMA -> converters
-  uint64_t* empty = full + kF32Stages;            // [stages]   MMA -> producer
-  uint64_t* conv_done = empty + kF32Stages;       // [slots]    converters -> MMA (128 arrivals)
-  uint64_t* lo_empty = conv_done + kF32LoSlots;   // [slots]    MMA -> converters
-  uint64_t* acc_full = lo_empty + kF32LoSlots;    // [2]
+  uint64_t* empty = full + kStages;               // [stages]   MMA -> producer
+  uint64_t* conv_done = empty + kStages;          // [slots]    converters -> MMA (128 arrivals)
+  uint64_t* lo_empty = conv_done + kLoSlots;      // [slots]    MMA -> converters
+  uint64_t* acc_full = lo_empty + kLoSlots;       // [2]
   uint64_t* acc_empty = acc_full + 2;             // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   unsigned char* epi_stage = reinterpret_cast<unsigned char*>(bars) + 1024;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int kTr = (EPI == kTcEpiF32) ? 3 : 2;           // trace builds: kernel id of the stamps
+  constexpr int kTrKb = 8;                                  // the k-block whose conversion and MMAs are stamped
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kF32Stages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
-    for (int s = 0; s < kF32LoSlots; ++s) { ptx::mbar_init(&conv_done[s], 128); ptx::mbar_init(&lo_empty[s], 1); }
+    SWAPMOE_STAMP(kTr, 0);
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
+    for (int s = 0; s < kLoSlots; ++s) { ptx::mbar_init(&conv_done[s], 128); ptx::mbar_init(&lo_empty[s], 1); }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 128); }
     *abort_flag = 0;
     ptx::fence_barrier_init();
@@ -182,22 +232,24 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       const int4 rawd = __ldcg(reinterpret_cast<const int4*>(a.tiles + rt));
       const TileDesc td = *reinterpret_cast<const TileDesc*>(&rawd);
       const int brow = td.phys * a.b_rows_per_phys + ct * kBoxRows;
-      pre = a.k_blocks < kF32Stages ? a.k_blocks : kF32Stages;
+      pre = a.k_blocks < kStages ? a.k_blocks : kStages;
       for (int kb = 0; kb < pre; ++kb) {
         ptx::mbar_expect_tx(&full[kb], (uint32_t)(kF32ABytes + kBBytesK));
         if (kSwap) {
-          ptx::tma_load_2d(raw + kb * kF32StageBytes, &tmA, &full[kb], (z * a.k_blocks + kb) * kF32BK, brow);
+          ptx::tma_load_2d(raw + kb * kStageBytes, &tmA, &full[kb], (z * a.k_blocks + kb) * kF32BK, brow);
         } else {
 #pragma unroll
           for (int j = 0; j < kNB; ++j)
-            ptx::tma_load_2d(raw + kb * kF32StageBytes + kF32ABytes + j * kBoxRows * kF32BK * 4, &tmB, &full[kb],
+            ptx::tma_load_2d(raw + kb * kStageBytes + kF32ABytes + j * kBoxRows * kF32BK * 4, &tmB, &full[kb],
                              (z * a.k_blocks + kb) * kF32BK, brow + j * a.b_rows_gate);
         }
       }
     }
   }
+  if (threadIdx.x == 0) SWAPMOE_STAMP(kTr, 1);
   pdl_wait();
   pdl_trigger();
+  if (threadIdx.x == 0) SWAPMOE_STAMP(kTr, 2);
   const int n_row_tiles = *a.n_tiles;
   const int per_slice = n_row_tiles * a.n_col_tiles;
   const int total = per_slice * a.n_split;        // item = slice * per_slice + (col tile * n_row_tiles + row tile)
@@ -216,7 +268,7 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         const int kb0 = z * a.k_blocks;
         for (int kb = 0; kb < a.k_blocks; ++kb) {
           const bool early = t == (int)blockIdx.x && kb < pre;   // armed and weights requested above
-          unsigned char* sA = raw + stage * kF32StageBytes;
+          unsigned char* sA = raw + stage * kStageBytes;
           if (!early) {
             ok = bounded_wait(&empty[stage], phase ^ 1u, abort_flag, a.status, 31);
             if (!ok) break;
@@ -235,8 +287,9 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                                  brow + j * a.b_rows_gate);
             }
           }
-          if (++stage == kF32Stages) { stage = 0; phase ^= 1u; }
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
+        SWAPMOE_STAMP(kTr, 3);
       }
       if (!ok) {
         // Give copies that are still in flight time to land before shared memory is released.
@@ -254,14 +307,26 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         ok = bounded_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, a.status, 32);
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * kNRows);
+        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * kAccStride);
         for (int kb = 0; kb < a.k_blocks; ++kb) {
           ok = bounded_wait(&conv_done[slot], slot_phase, abort_flag, a.status, 33);
           if (!ok) break;
           ptx::tc_fence_after();
-          const uint64_t dhb = make_kmajor_sw128_desc(ptx::smem_u32(raw + stage * kF32StageBytes + kF32ABytes));
-          const uint64_t dlb = make_kmajor_sw128_desc(ptx::smem_u32(lo + slot * kF32BBytes));
-          const uint32_t a_hi = tmem_base + (uint32_t)(kF32TmemAcc + slot * 2 * kF32BK), a_lo = a_hi + kF32BK;
+          if (kb == kTrKb && t == (int)blockIdx.x) SWAPMOE_STAMP(kTr, 14);
+          const uint64_t dhb = make_kmajor_sw128_desc(ptx::smem_u32(raw + stage * kStageBytes + kF32ABytes));
+          if constexpr (kSwap) {
+            // B row = [b1 of the 32 elements | b2 of them]: 16 elements = 32 bytes = +2 in the address field;
+            // A slot = [8 columns b1 (k 0-15) | 8 b1 (k 16-31) | 8 b2 | 8 b2]; small terms first
+            const uint32_t a1 = tmem_base + (uint32_t)(kASlotBase + slot * kASlotCols), a2 = a1 + 16;
+            ptx::umma_bf16_ts(tmem_d, a2, dhb, kIdesc, kb > 0 ? 1u : 0u);
+            ptx::umma_bf16_ts(tmem_d, a2 + 8, dhb + 2, kIdesc, 1u);
+            ptx::umma_bf16_ts(tmem_d, a1, dhb + 4, kIdesc, 1u);
+            ptx::umma_bf16_ts(tmem_d, a1 + 8, dhb + 6, kIdesc, 1u);
+            ptx::umma_bf16_ts(tmem_d, a1, dhb, kIdesc, 1u);
+            ptx::umma_bf16_ts(tmem_d, a1 + 8, dhb + 2, kIdesc, 1u);
+          } else {
+          const uint64_t dlb = make_kmajor_sw128_desc(ptx::smem_u32(lo + slot * kLoBytes));
+          const uint32_t a_hi = tmem_base + (uint32_t)(kASlotBase + slot * kASlotCols), a_lo = a_hi + kF32BK;
 #pragma unroll
           for (int k = 0; k < kF32BK / kF32UmmaK; ++k) {
             // 8 fp32 along K: +32 bytes = +2 in the address field of B, +8 columns of A; small terms first
@@ -269,19 +334,22 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             ptx::umma_tf32_ts(tmem_d, a_hi + 8 * k, dlb + (uint64_t)(2 * k), kIdesc, 1u);
             ptx::umma_tf32_ts(tmem_d, a_hi + 8 * k, dhb + (uint64_t)(2 * k), kIdesc, 1u);
           }
+          }
           ptx::umma_commit(&empty[stage]);       // the raw stage may be refilled
           ptx::umma_commit(&lo_empty[slot]);     // the lo slot may be rewritten
-          if (++stage == kF32Stages) stage = 0;
-          if (++slot == kF32LoSlots) { slot = 0; slot_phase ^= 1u; }
+          if (kb == kTrKb && t == (int)blockIdx.x) SWAPMOE_STAMP(kTr, 15);
+          if (++stage == kStages) stage = 0;
+          if (++slot == kLoSlots) { slot = 0; slot_phase ^= 1u; }
         }
         if (!ok) break;
         ptx::umma_commit(&acc_full[acc]);
+        SWAPMOE_STAMP(kTr, 5);
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
   } else if (warp >= 8) {
     // ---------------------------------------------------------------------- converters: hi in place, lo beside
-    // two groups of four warps: group g converts the k-blocks that use lo slot g (every other one), so two
+    // two groups of four warps: group g converts the k-blocks whose lo slot has parity g (every other one), so two
     // conversions are in flight; both groups walk all k-blocks to keep stage and phase counters in step
     const int grp = (warp - 8) >> 2;
     const int ctid = (threadIdx.x - 8 * 32) & 127;   // 0..127 inside the group = row = TMEM lane
@@ -290,18 +358,56 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     bool ok = true;
     for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
       for (int kb = 0; kb < a.k_blocks; ++kb) {
-        if (slot != grp) {
-          if (++stage == kF32Stages) { stage = 0; phase ^= 1u; }
-          if (++slot == kF32LoSlots) { slot = 0; slot_phase ^= 1u; }
+        if ((slot & 1) != grp) {
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (++slot == kLoSlots) { slot = 0; slot_phase ^= 1u; }
           continue;
         }
+        const bool tr = ctid == 0 && kb == kTrKb && t == (int)blockIdx.x;   // kTrKb is even: group 0 converts it
+        if (ctid == 0 && grp == 0 && kb == 0 && t == (int)blockIdx.x) SWAPMOE_STAMP(kTr, 7);
         ok = bounded_wait(&full[stage], phase, abort_flag, a.status, 34);
+        if (ctid == 0 && grp == 0 && kb == 0 && t == (int)blockIdx.x) SWAPMOE_STAMP(kTr, 4);
+        if (tr) SWAPMOE_STAMP(kTr, 8);
         if (ok) ok = bounded_wait(&lo_empty[slot], slot_phase ^ 1u, abort_flag, a.status, 35);
         if (!ok) break;
         ptx::tc_fence_after();
+        if (tr) SWAPMOE_STAMP(kTr, 9);
+        if constexpr (kSwap) {
+          // weights: thread = row (= TMEM lane); 32 values -> 16 packed b1 columns and 16 packed b2 columns
+          const unsigned char* arow = raw + stage * kStageBytes + ctid * 128;
+          uint32_t hm[32];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint4 x = *reinterpret_cast<const uint4*>(arow + ((j ^ (ctid & 7)) << 4));
+            split_bf16_pair(x.x, x.y, &hm[2 * j], &hm[16 + 2 * j]);
+            split_bf16_pair(x.z, x.w, &hm[2 * j + 1], &hm[16 + 2 * j + 1]);
+          }
+          const uint32_t ta = tmem_base + ((uint32_t)((ctid >> 5) * 32) << 16) + (uint32_t)(kASlotBase + slot * kASlotCols);
+          ptx::tmem_st32(ta, hm);
+          if (tr) SWAPMOE_STAMP(kTr, 10);
+          // tokens: the first kF32SwapTok threads own a row each and rewrite it in place as [b1 x 32 | b2 x 32]
+          // (logical 16-byte piece c at physical piece c ^ (row & 7), as the swizzled K-major bf16 row wants it)
+          if (ctid < kF32SwapTok) {
+            unsigned char* brow = raw + stage * kStageBytes + kF32ABytes + ctid * 128;
+            uint32_t p1[16], p2[16];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint4 x = *reinterpret_cast<const uint4*>(brow + ((j ^ (ctid & 7)) << 4));
+              split_bf16_pair(x.x, x.y, &p1[2 * j], &p2[2 * j]);
+              split_bf16_pair(x.z, x.w, &p1[2 * j + 1], &p2[2 * j + 1]);
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              *reinterpret_cast<uint4*>(brow + ((c ^ (ctid & 7)) << 4)) =
+                  make_uint4(p1[4 * c], p1[4 * c + 1], p1[4 * c + 2], p1[4 * c + 3]);
+              *reinterpret_cast<uint4*>(brow + (((4 + c) ^ (ctid & 7)) << 4)) =
+                  make_uint4(p2[4 * c], p2[4 * c + 1], p2[4 * c + 2], p2[4 * c + 3]);
+            }
+          }
+        } else {
         {
           // A: thread = row (= TMEM lane); its 32 values sit in eight 16-byte pieces, piece j at (j ^ (row & 7))
-          const unsigned char* arow = raw + stage * kF32StageBytes + ctid * 128;
+          const unsigned char* arow = raw + stage * kStageBytes + ctid * 128;
           uint32_t h[32], l[32];
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
@@ -313,13 +419,14 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
               l[4 * j + e] = __float_as_uint(__uint_as_float(xs[e]) - __uint_as_float(h[4 * j + e]));
             }
           }
-          const uint32_t ta = tmem_base + ((uint32_t)((ctid >> 5) * 32) << 16) + (uint32_t)(kF32TmemAcc + slot * 2 * kF32BK);
+          const uint32_t ta = tmem_base + ((uint32_t)((ctid >> 5) * 32) << 16) + (uint32_t)(kASlotBase + slot * kASlotCols);
           ptx::tmem_st32(ta, h);
           ptx::tmem_st32(ta + kF32BK, l);
         }
+        if (tr) SWAPMOE_STAMP(kTr, 10);
         // B: elementwise at identical offsets (keeps the swizzled layout): hi in place, lo into the slot
-        uint4* src = reinterpret_cast<uint4*>(raw + stage * kF32StageBytes + kF32ABytes);
-        uint4* dst = reinterpret_cast<uint4*>(lo + slot * kF32BBytes);
+        uint4* src = reinterpret_cast<uint4*>(raw + stage * kStageBytes + kF32ABytes);
+        uint4* dst = reinterpret_cast<uint4*>(lo + slot * kLoBytes);
 #pragma unroll 4
         for (int i = ctid; i < kBBytesK / 16; i += 128) {
           const uint4 x = src[i];
@@ -331,12 +438,16 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           src[i] = h;
           dst[i] = l;
         }
+        }
+        if (tr) SWAPMOE_STAMP(kTr, 11);
         ptx::tmem_st_wait();
+        if (tr) SWAPMOE_STAMP(kTr, 12);
         ptx::tc_fence_before();
         ptx::fence_proxy_async();                // these writes are read by the tensor core (async proxy)
         ptx::mbar_arrive(&conv_done[slot]);
-        if (++stage == kF32Stages) { stage = 0; phase ^= 1u; }
-        if (++slot == kF32LoSlots) { slot = 0; slot_phase ^= 1u; }
+        if (tr) SWAPMOE_STAMP(kTr, 13);
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        if (++slot == kLoSlots) { slot = 0; slot_phase ^= 1u; }
       }
     }
   } else if (warp >= 4) {
@@ -358,7 +469,7 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         ok = bounded_wait(&acc_full[acc], acc_phase, abort_flag, a.status, 36);
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kNRows);
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kAccStride);
 #pragma unroll 1
         for (int c0 = 0; c0 < kNRows; c0 += 32) {
           uint32_t v[32];
@@ -389,6 +500,7 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       }
       ptx::tc_fence_before();
       ptx::mbar_arrive(&acc_empty[acc]);
+      if (r == 0) SWAPMOE_STAMP(kTr, 6);
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }
@@ -451,9 +563,9 @@ inline int32_t tc_f32_init(TcF32State& s, PFN_encodeTiled enc, const swapmoe_con
   s.swap_ok = c.act == SWAPMOE_ACT_RELU;
   if (s.swap_ok &&
       (cudaFuncSetAttribute(tc_gemm_f32_kernel<kTcEpiReluF32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                            kF32SmemBytes) != cudaSuccess ||
+                            kF32SwapSmemBytes) != cudaSuccess ||
        cudaFuncSetAttribute(tc_gemm_f32_kernel<kTcEpiF32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                            kF32SmemBytes) != cudaSuccess))
+                            kF32SwapSmemBytes) != cudaSuccess))
     return SWAPMOE_ERR_CUDA;
   if (cudaFuncSetAttribute(tc_gemm_f32_kernel<kTcEpiReluF32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kF32SmemBytes) != cudaSuccess ||
@@ -499,7 +611,7 @@ inline int32_t tc_ffn_f32(TcF32State& s, const swapmoe_config_t& c, void* h, flo
   int grid = work > s.sm_count ? s.sm_count : (int)work;
   // (swapped form: the weight map is the A operand's, the token map with kF32SwapTok-row boxes the B operand's)
   cudaError_t e = swapped ? launch_kernel(tc_gemm_f32_kernel<kTcEpiReluF32, true>, dim3(grid), dim3(kF32Threads),
-                                          kF32SmemBytes, st, pdl, s.map_win, s.map_xp_tok, g1)
+                                          kF32SwapSmemBytes, st, pdl, s.map_win, s.map_xp_tok, g1)
                   : swiglu ? launch_kernel(tc_gemm_f32_kernel<kTcEpiSwigluF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes,
                                            st, pdl, s.map_xp, s.map_win, g1)
                            : launch_kernel(tc_gemm_f32_kernel<kTcEpiReluF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes,
@@ -525,7 +637,7 @@ inline int32_t tc_ffn_f32(TcF32State& s, const swapmoe_config_t& c, void* h, flo
   g2.early_b = 1;
   work = (long long)max_tiles * n_col2 * split;
   grid = work > s.sm_count ? s.sm_count : (int)work;
-  e = swapped ? launch_kernel(tc_gemm_f32_kernel<kTcEpiF32, true>, dim3(grid), dim3(kF32Threads), kF32SmemBytes, st,
+  e = swapped ? launch_kernel(tc_gemm_f32_kernel<kTcEpiF32, true>, dim3(grid), dim3(kF32Threads), kF32SwapSmemBytes, st,
                               pdl && between == nullptr, s.map_wout, s.map_h_tok, g2)
               : launch_kernel(tc_gemm_f32_kernel<kTcEpiF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes, st,
                               pdl && between == nullptr, s.map_h, s.map_wout, g2);

@@ -128,6 +128,8 @@ class DecodeStack:
         # (step_graph); slot-table flips and expert copies stay outside the graph.
         self.graph_buffers = graph_buffers
         self.graph = None
+        self.graph_launches = 0          # library kernels in the captured step
+        self.graph_replays = 0
         for st in self.layers:
             st.layer.set_resident(st.s2e, st.arena_in, st.arena_out, st.phys, stream=self.compute)
             st.last_used = np.zeros(st.layer.cfg.K, np.int64)
@@ -166,9 +168,11 @@ class DecodeStack:
                     st.layer.read_importance(reset=True, stream=self.compute)
                 self.compute.synchronize()
                 self.graph = torch.cuda.CUDAGraph()
+                l0 = sum(st.layer.launch_count for st in self.layers)
                 with torch.cuda.graph(self.graph, capture_error_mode="thread_local"):   # torch's own side stream
                     for li, st in enumerate(self.layers):
                         st.layer.forward(x_buf[li], out_buf[li], stream=None)
+                self.graph_launches = sum(st.layer.launch_count for st in self.layers) - l0   # kernels per replay
             self._throttle()
             x_buf.copy_(x_step, non_blocking=True)
             for li, st in enumerate(self.layers):
@@ -176,6 +180,7 @@ class DecodeStack:
                 if record:
                     self.trace.append((n, li, st.s2e.copy(), st.phys.copy()))
             self.graph.replay()
+            self.graph_replays += 1
             self._mark_step()
         self._schedule(n)
         self.step_no += 1
