@@ -604,6 +604,9 @@ def run_decode(args, cfg):
 
         # arm 1: scheduler off (no importance reads, no swaps): what the kernels alone allow
         no_swap = run_arm(make_stack(frequency=1 << 30, max_in_flight=3))
+        # the host may run ahead of the device by about 1.5 ms of queued steps (at least 3, at most 8 steps): enough to
+        # ride out a step in which the scheduler decides, short enough for its decisions to be current
+        mif = args.max_in_flight or max(3, min(8, int(1.5e-3 / (no_swap["ms_per_step"] * 1e-3))))
         # arm 2: swapping on.  The step's load budget follows the link: what PCIe carries while a step computes.
         budget = suggest_step_budget(no_swap["ms_per_step"] * 1e-3, pcie_gbs, expert_bytes)
         if args.cfg4_variant == "no_loads":          # diagnostic: decisions only
@@ -611,8 +614,9 @@ def run_decode(args, cfg):
         swap = run_arm(make_stack(frequency=args.frequency, loads_per_step=1, step_budget=budget, commit="ready",
                                   lag=(10 ** 9 if args.cfg4_variant == "no_commits" else 2),
                                   time_loads=(B == max(args.batches)), track_hits=True, async_decide=True,
-                                  max_in_flight=3))
+                                  max_in_flight=mif))
         swap["step_budget"] = budget
+        swap["max_in_flight"] = mif
         swap["slowdown_vs_no_swap"] = swap["us_per_layer"] / no_swap["us_per_layer"]
         entry = {"swap": swap, "no_swap": no_swap}
         big = B == max(args.batches)
@@ -620,12 +624,12 @@ def run_decode(args, cfg):
         if args.sweep_frequency and big:
             entry["frequency_sweep"] = {
                 str(fr): run_arm(make_stack(frequency=fr, loads_per_step=1, step_budget=budget, commit="ready",
-                                            track_hits=True, async_decide=True, max_in_flight=3)) for fr in args.sweep_frequency}
+                                            track_hits=True, async_decide=True, max_in_flight=mif)) for fr in args.sweep_frequency}
         if args.sweep_budget and big:
             entry["budget_sweep"] = {
                 ("%g" % bu): run_arm(make_stack(frequency=args.frequency, loads_per_step=max(1, int(-(-bu // L))), step_budget=bu,
                                             commit="wait" if args.sweep_commit == "wait" else "ready", track_hits=True,
-                                            async_decide=True, max_in_flight=3))
+                                            async_decide=True, max_in_flight=mif))
                 for bu in args.sweep_budget}
         # Section 4.1 baselines as policies over the same kernels, and per-layer budgets (Section 3.3)
         if args.policies and big:
@@ -634,14 +638,14 @@ def run_decode(args, cfg):
                 Ks = [K] * L
                 pol["K=%d" % K] = {
                     "swap": run_arm(make_stack(Ks, frequency=args.frequency, loads_per_step=1, step_budget=budget,
-                                               commit="ready", track_hits=True, async_decide=True, max_in_flight=3)),
+                                               commit="ready", track_hits=True, async_decide=True, max_in_flight=mif)),
                     "static_pruning": run_arm(make_stack(Ks, policy="static_pruning")),
                     "on_demand": run_arm(make_stack(Ks, policy="on_demand", lag=0), graph=False)}
             entry["policies_vs_K"] = pol
             Ks = [8, 12, 16, 24] * (L // 4) + [16] * (L % 4)
             entry["per_layer_K"] = dict(run_arm(make_stack(Ks, frequency=args.frequency, loads_per_step=1,
                                                            step_budget=budget, commit="ready", track_hits=True,
-                                                           async_decide=True, max_in_flight=3)), Ks=Ks)
+                                                           async_decide=True, max_in_flight=mif)), Ks=Ks)
         results[str(B)] = entry
     clocks = sampler.stop()
     Bmax = str(max(args.batches))
@@ -739,6 +743,8 @@ def main():
                     help="cfg4 budget sweep: flip when the copy has landed, or wait for it at the commit step")
     ap.add_argument("--cfg4-variant", default="full", choices=["full", "no_loads", "no_commits"],
                     help="cfg4 diagnostic: swapping arm without expert copies / with copies that are never committed")
+    ap.add_argument("--max-in-flight", type=int, default=0,
+                    help="cfg4: steps the host may run ahead of the device in the swapping arms (0: from the step time)")
     ap.add_argument("--policies", action="store_true",
                     help="cfg4: also run static pruning / on-demand loading / swapping at K = 4, 8, 16 and per-layer K")
     ap.add_argument("--min-region-ms", type=float, default=MIN_REGION_MS,

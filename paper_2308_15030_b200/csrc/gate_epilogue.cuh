@@ -169,6 +169,7 @@ __device__ __forceinline__ void gate_epilogue(const RouterArgs& a, const GateSme
     for (int j = 0; j < kMaxTopK; ++j) { g.cand_v[tid * kMaxTopK + j] = tk.v[j]; g.cand_e[tid * kMaxTopK + j] = tk.e[j]; }
   }
   __syncthreads();
+  if (threadIdx.x == 0) SWAPMOE_STAMP(0, 6);
   // merge the shares of one (token, gate) in ascending expert order: a candidate only displaces
   // an entry it strictly beats, so equal logits keep the lowest expert index
   TopK fin;
@@ -183,6 +184,7 @@ __device__ __forceinline__ void gate_epilogue(const RouterArgs& a, const GateSme
     g.s_m[tl * 2 + (masked ? 1 : 0)] = fin.v[0];
   }
   __syncthreads();
+  if (threadIdx.x == 0) SWAPMOE_STAMP(0, 7);
   {
     const float m = g.s_m[tl * 2 + (masked ? 1 : 0)];
     float den = 0.f;
@@ -203,6 +205,7 @@ __device__ __forceinline__ void gate_epilogue(const RouterArgs& a, const GateSme
     g.part_den[tid] = den;
   }
   __syncthreads();
+  if (threadIdx.x == 0) SWAPMOE_STAMP(0, 8);
   if (part == 0) {
     const float m = fin.v[0];
     float den = 0.f;
@@ -248,6 +251,7 @@ __device__ __forceinline__ void gate_epilogue(const RouterArgs& a, const GateSme
     if (!masked && token < a.T) a.xnorm[token] = xn;
   }
   __syncthreads();
+  if (threadIdx.x == 0) SWAPMOE_STAMP(0, 9);
   // Per-CTA partial sums with a fixed association (lane-strided partials, then the
   // shuffle tree), so the result does not depend on scheduling.  Only experts that some
   // token of this tile selected are visited; the others get an exact zero.
@@ -258,6 +262,7 @@ __device__ __forceinline__ void gate_epilogue(const RouterArgs& a, const GateSme
   }
   for (int sl = tid; sl < a.K; sl += kGateThreads) a.cta_hist[(size_t)blockIdx.x * a.K + sl] = 0;
   __syncthreads();
+  if (threadIdx.x == 0) SWAPMOE_STAMP(0, 10);
   for (int c = 0; c * 32 < E; ++c) {
     uint32_t present = g.s_present[c];
     for (int n = 0; present; ++n) {
@@ -287,7 +292,9 @@ __device__ __forceinline__ void gate_epilogue(const RouterArgs& a, const GateSme
       if (a.cta_mimp) a.cta_mimp[(size_t)blockIdx.x * a.K + sl] = m;
     }
   }
+  if (threadIdx.x == 0) SWAPMOE_STAMP(0, 11);
   finish_router_cta(a.scan, scan_stage, scan_stage_bytes);
+  if (threadIdx.x == 0) SWAPMOE_STAMP(0, 12);
 }
 
 }  // namespace swapmoe

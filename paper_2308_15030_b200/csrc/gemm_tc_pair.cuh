@@ -119,7 +119,10 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const uint32_t rank = ptx::cluster_ctarank();               // 0: issues the MMAs
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
+  constexpr int kTr = (EPI == kTcEpiReluBf16 || EPI == kTcEpiSwigluBf16) ? 2 : 3;   // trace id: GEMM-1 or GEMM-2
+  (void)kTr;
   if (threadIdx.x == 0) {
+    SWAPMOE_STAMP(kTr, 0);
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 8); }
     *abort_flag = 0;
@@ -158,8 +161,10 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
     }
   }
+  if (threadIdx.x == 0) SWAPMOE_STAMP(kTr, 1);
   pdl_wait();      // the activations come from the preceding kernel
   pdl_trigger();
+  if (threadIdx.x == 0) SWAPMOE_STAMP(kTr, 2);
   const int n_row_tiles = *a.n_tiles;
   const int total = n_row_tiles * a.n_col_tiles;
 
@@ -194,6 +199,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (!early) ptx::tma_load_2d_pair(sB + stage * kPairBBytes, &tmB, full_addr, kb * kTcBK, brow);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
+        SWAPMOE_STAMP(kTr, 3);
       }
       if (!ok) {
         // Give copies that are still in flight time to land before shared memory is released.
@@ -216,6 +222,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           ok = bounded_wait(&full[stage], phase, abort_flag, a.status, 13);
           if (!ok) break;
           ptx::tc_fence_after();
+          if (t == pair && kb == 0) SWAPMOE_STAMP(kTr, 4);
           const uint64_t da = make_kmajor_sw128_desc(ptx::smem_u32(sA + stage * kPairABytes));
           const uint64_t db = make_kmajor_sw128_desc(ptx::smem_u32(sB + stage * kPairBBytes));
 #pragma unroll
@@ -226,6 +233,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         if (!ok) break;
         ptx::umma_commit_pair(&acc_full[acc]);    // accumulator complete, in both CTAs
+        SWAPMOE_STAMP(kTr, 5);
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
@@ -264,6 +272,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       __syncwarp();
       // one arrival per warp, on the even CTA's barrier: 8 arrivals hand the buffer back to the MMA issuer
       if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&acc_empty[acc]), 0u));
+      if (r == 0) SWAPMOE_STAMP(kTr, 6);
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }

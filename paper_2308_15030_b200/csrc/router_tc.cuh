@@ -97,6 +97,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   while ((int)tmem_cols < Epad) tmem_cols <<= 1;
 
   if (tid == 0) {
+    SWAPMOE_STAMP(0, 0);
     for (int s = 0; s < n_stages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 5); }
     ptx::mbar_init(acc_full, 1);
     *abort_flag = 0;
@@ -110,6 +111,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   }
   pdl_wait();      // everything above touched only shared memory, TMEM and kernel parameters
   pdl_trigger();
+  if (tid == 0) SWAPMOE_STAMP(0, 1);
   gate_load_tables(a, g);
   ptx::tc_fence_before();
   __syncthreads();
@@ -140,6 +142,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         ok = bounded_wait(&full[stage], phase, abort_flag, status, 12);
         if (!ok) break;
         ptx::tc_fence_after();
+        if (kb == 0) SWAPMOE_STAMP(0, 2);
         const uint64_t da = make_kmajor_sw128_desc(ptx::smem_u32(sA + stage * a_bytes));
         const uint64_t db = make_kmajor_sw128_desc(ptx::smem_u32(sB + stage * b_bytes));
 #pragma unroll
@@ -150,6 +153,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         if (++stage == n_stages) { stage = 0; phase ^= 1u; }
       }
       if (ok) ptx::umma_commit(acc_full);
+      SWAPMOE_STAMP(0, 3);
     }
   } else if (warp >= 4) {
     // ------------------------------------------------ ||x||^2 while the tiles stream through
@@ -187,6 +191,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     // ------------------------------------------------ logits: TMEM lane r -> shared-memory row r
     // (all MMAs have completed once acc_full fires, so the stage buffers are free to reuse)
     if (ok) ok = bounded_wait(acc_full, 0, abort_flag, status, 14);
+    if (tid == 128) SWAPMOE_STAMP(0, 4);
     if (ok && warp_has_rows) {
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -207,6 +212,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, tmem_cols);
   }
+  if (tid == 0) SWAPMOE_STAMP(0, 5);
   const bool failed = *abort_flag != 0;
   // the stage memory is free again: the last CTA stages the scan inputs there
   gate_epilogue(a, g, slog, tok, tok0, failed, smem, stage_area);
