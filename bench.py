@@ -159,9 +159,11 @@ def roofline_objects(cfg, touched, g_ms, ms_step, peaks):
     tc_peak = peaks["bf16_tflops_sustained"] if tc_kind == "sustained" else peaks["bf16_tflops"]
     t_hbm = g_bytes / (peaks["hbm_gbs"] * 1e9)
     t_tc = g_flops / (tc_peak * 1e12) if cfg.dtype == I.BF16 else 0.0
-    # fp32 layers: the grouped GEMM runs on the tensor cores as three TF32 products per fp32 product;
-    # its peak is the measured bf16 figure x the nominal TF32 : bf16 ratio (1.1 : 2.25 PFLOP/s) / 3.
-    tf32x3_peak = peaks["bf16_tflops"] * (1.1 / 2.25) / 3.0
+    # fp32 layers: the grouped GEMM runs on the tensor cores as three reduced-precision products per fp32 product:
+    # bf16 pieces on tcgen05 (peak = the measured bf16 figure / 3), TF32 pieces in the warp-level mma kernels
+    # (SWAPMOE_FP32_TC=0; peak = measured bf16 x the nominal TF32 : bf16 ratio, 1.1 : 2.25 PFLOP/s, / 3).
+    fp32_mma = os.environ.get("SWAPMOE_FP32_TC") == "0"
+    tf32x3_peak = peaks["bf16_tflops"] * ((1.1 / 2.25) if fp32_mma else 1.0) / 3.0
     if cfg.dtype != I.BF16 and t_hbm >= g_flops / (tf32x3_peak * 1e12):
         bound, peak, ach, unit = "hbm", peaks["hbm_gbs"], g_bytes / 2 / (g_ms * 1e-3) / 1e9, "GB/s"
     elif cfg.dtype != I.BF16:
@@ -177,15 +179,16 @@ def roofline_objects(cfg, touched, g_ms, ms_step, peaks):
     traffic, traffic_rec = ncu_traffic(cfg.name)
     if cfg.dtype == I.BF16:
         kernel = "tc_gemm_kernel / tc_gemm_pair_kernel (grouped FFN GEMM on tcgen05, 2 launches per step: GEMM-1+act, GEMM-2)"
-    elif os.environ.get("SWAPMOE_FP32_TC") == "0":
+    elif fp32_mma:
         kernel = "gemm_tf32x3_kernel (split-TF32 warp-level mma, 2 launches per step)"
     else:
-        kernel = "tc_gemm_f32_kernel (split-TF32 on tcgen05, 2 launches per step)"
+        kernel = "tc_gemm_f32_kernel (three products of bf16 pieces on tcgen05, 2 launches per step)"
     roof = {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
             "traffic": traffic, "traffic_source": traffic_rec, "peak_source": peaks["source"], "kernel": kernel,
             "algorithmic_bytes_per_launch": g_bytes / 2, "flops_per_launch": g_flops / 2,
             "avg_launch_ms": g_ms, "tensor_tflops": g_flops / 2 / (g_ms * 1e-3) / 1e12,
-            "tensor_peak_kind": (tc_kind if cfg.dtype == I.BF16 else "bf16 burst x 1.1/2.25 / 3 (TF32 x3)")
+            "tensor_peak_kind": (tc_kind if cfg.dtype == I.BF16 else
+                                 ("bf16 burst x 1.1/2.25 / 3 (TF32 x3)" if fp32_mma else "bf16 burst / 3 (bf16 pieces x3)"))
                                 if bound == "tensor" else None,
             "frac_of_burst_tensor_peak": (ach / peaks["bf16_tflops"]) if bound == "tensor" else None}
     layer = {"t_roof_us": t_roof * 1e6, "frac": t_roof * 1e3 / ms_step,

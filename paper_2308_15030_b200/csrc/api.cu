@@ -85,7 +85,7 @@ struct swapmoe_layer {
   const void* map_x_ptr;
   int32_t map_x_T;
   TcState tc;
-  TcF32State tc32;             // tcgen05 split-TF32 grouped GEMM of fp32 layers (SWAPMOE_FP32_TC=0: warp-level mma)
+  TcF32State tc32;             // tcgen05 grouped GEMM of fp32 layers, bf16-piece split (SWAPMOE_FP32_TC=0: warp-level mma)
   PFN_encodeTiled encode32;
 };
 

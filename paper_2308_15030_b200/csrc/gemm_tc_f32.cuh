@@ -1,67 +1,53 @@
 // Grouped expert GEMM for fp32 layers on the tcgen05 tensor cores (SwapMoE Section 2: the experts'
-// FFN restricted to the resident slots), with fp32-grade accuracy from three TF32 products.
+// FFN restricted to the resident slots), with fp32-grade accuracy from three bf16 products.
 //
-// `kind::tf32` keeps 10 mantissa bits of each operand, which cannot hold the 1e-4 output tolerance
-// over 768-3072-term dot products.  Every operand is therefore split as x = hi + lo with
-// hi = x with its low 13 mantissa bits cleared (exactly a TF32 number) and lo = x - hi (exact in
-// fp32, at most 13 significant bits, so TF32 holds it to 2^-11 relative): the product is
-// lo_a*hi_b + hi_a*lo_b + hi_a*hi_b, accumulated in fp32 in TMEM; the dropped lo*lo term and the
-// rounding of lo are below 2^-20 relative.
+// No tensor-core input type holds fp32's 24 mantissa bits, and a single reduced-precision product cannot hold the
+// 1e-4 output tolerance over 768-3072-term dot products.  Every operand is therefore split as x = b1 + b2 + rest
+// with b1 = bf16(x) (round to nearest), b2 = bf16(x - b1) (the subtraction is exact in fp32) and |rest| below
+// 2^-17 |x|; the product is b2_a*b1_b + b1_a*b2_b + b1_a*b1_b, accumulated in fp32 in TMEM, and the dropped terms
+// are below 2^-16 relative.  (A first version split into TF32 pieces, hi = x with 13 mantissa bits cleared and
+// lo = x - hi: same accuracy, but a kind::tf32 MMA covers 8 contraction elements where a kind::f16 one covers 16,
+// and a tcgen05.mma costs about 110 clocks however small it is - the kernel is paced by the NUMBER of MMAs.)
 //
-// TMA brings the fp32 operands (k-blocks of 32 columns = 128-byte swizzled rows) into a ring of
-// raw stages.  Four converter warps split a stage: the weight half elementwise (which preserves the
-// swizzled layout: hi parts in place, lo parts at the same offsets of one of two "lo" slots); the
-// activation half goes to TENSOR MEMORY: converter thread r owns row r, reads its 32 values and
-// writes hi and lo into 32 + 32 columns of TMEM lane r (`tcgen05.st`), so the MMAs take their A
-// operand from TMEM and read only B from shared memory (with both operands in shared memory a k-block
-// moved 224 KB through it and the kernel was bound by shared-memory bandwidth).  The converters
-// fence and arrive on `conv_done`; one thread then issues the 12 MMAs of the k-block (4 steps of
-// K = 8, three products each) and commits to the barriers that free the raw stage and the slot.  Roles (512 threads): warp 0 TMA producer,
-// warp 1 MMA issuer, warp 2 TMEM allocation, warps 4-7 epilogue (two accumulator sets, so it
-// overlaps the next item's MMAs), warps 8-11 and 12-15 two converter groups (one per lo slot).  A work item is (row tile, column tile,
-// contraction slice): GEMM-2 has few output tiles and a long contraction, so its slices go to
-// separate copies of y that the combine kernel adds in order (deterministic).
-//
-// The swapped form (small slots: weights on the MMA rows, see kF32Swap* below) splits into bf16 pieces instead and
-// needs half as many MMAs per k-block; its converter rewrites the token rows in place.
+// TMA brings the fp32 operands (k-blocks of 32 columns = 128-byte swizzled rows) into a ring of stages.  Two
+// groups of four converter warps take alternate k-blocks.  The A operand goes to TENSOR MEMORY: converter thread r
+// owns row r, reads its 32 values and writes 16 packed b1 pairs and 16 packed b2 pairs into 32 columns of TMEM
+// lane r (`tcgen05.st`), so the MMAs read only B from shared memory.  The B operand is rewritten IN PLACE: a
+// 128-byte row of 32 fp32 becomes [32 x b1 | 32 x b2], which is exactly a swizzled K-major bf16 row of 64, so no
+// second buffer is needed.  The converters fence and arrive on `conv_done`; one thread then issues the 6 MMAs of
+// the k-block (2 steps of K = 16, three products each) and commits to the barriers that free the stage and the
+// TMEM slot.  Roles (512 threads): warp 0 TMA producer, warp 1 MMA issuer, warp 2 TMEM allocation, warps 4-7
+// epilogue (two accumulator sets, so it overlaps the next item's MMAs), warps 8-11 and 12-15 the converter groups.
+// A work item is (row tile, column tile, contraction slice): GEMM-2 has few output tiles and a long contraction, so
+// its slices go to separate copies of y that the combine kernel adds in order (deterministic).
 #pragma once
 #include "gemm_tc.cuh"
 
 namespace swapmoe {
 
 constexpr int kF32BK = 32;                          // fp32 elements per k-block = one 128-byte swizzled row
-constexpr int kF32UmmaK = 8;
-constexpr int kF32BN = 128;                         // accumulator columns per tile
+constexpr int kF32BN = 128;                         // accumulator columns per tile (plain form)
 constexpr int kF32Threads = 512;
-constexpr int kF32ABytes = kTcBM * kF32BK * 4;      // 16 KB
+constexpr int kF32ABytes = kTcBM * kF32BK * 4;      // 16 KB: the operand that goes to tensor memory
+constexpr int kF32ASlots = 4;                       // tensor-memory slots of converted A k-blocks
+constexpr int kF32ASlotCols = kF32BK;               // 16 columns of b1 pairs + 16 of b2 pairs
+// Plain form: A = 128 token rows of a slot tile, B = 128 weight rows; C tile = [128 tokens, 128 outputs].
 constexpr int kF32BBytes = kF32BN * kF32BK * 4;     // 16 KB
 constexpr int kF32StageBytes = kF32ABytes + kF32BBytes;
-constexpr int kF32Stages = 5;                       // raw stages (TMA targets; the B half holds the hi parts after conversion)
-constexpr int kF32LoSlots = 2;                      // lo parts of B in shared memory; hi and lo of A in tensor memory
-constexpr int kF32SmemBytes = kF32Stages * kF32StageBytes + kF32LoSlots * kF32BBytes + 2048 + kTcEpiStageBytes;
+constexpr int kF32Stages = 6;
+constexpr int kF32TmemCols = 512;                   // 2 x 128 accumulator columns + 4 x 32 of A, rounded up
+constexpr int kF32SmemBytes = kF32Stages * kF32StageBytes + 2048 + kTcEpiStageBytes;
 // Swapped form for small slots: the 128 rows of the MMA (and of tensor memory) are WEIGHT rows, the accumulator's
-// columns are the tokens of a slot tile (kF32SwapTok of them).
+// columns are the tokens of a slot tile (kF32SwapTok of them): 24 KB per k-block, eight stages.
 constexpr int kF32SwapTok = 64;                     // token rows per tile = accumulator columns
-constexpr int kF32TmemAcc = 2 * kF32BN;             // columns of the two accumulator sets
-// The swapped form moves 24 KB per k-block (16 KB of weights, 8 KB of tokens): compact stages, eight of them.
-// Its MMAs are small (128 x 64), and a tcgen05.mma costs about 110 clocks however small it is, so the swapped form
-// is paced by the NUMBER of MMAs.  It therefore splits into bf16 pieces instead of TF32 ones: x = b1 + b2 + (rest
-// below 2^-17 |x|) with b1 = bf16(x), b2 = bf16(x - b1), and the product is b2_a*b1_b + b1_a*b2_b + b1_a*b1_b
-// (the dropped terms are below 2^-16 relative): kind::f16 MMAs cover 16 contraction elements each, so a k-block of
-// 32 takes 6 MMAs where the TF32 split takes 12.  The weights' pieces go to tensor memory (16 + 16 packed columns
-// per slot, four slots), the tokens' pieces replace the fp32 row in place: a 128-byte row of 32 fp32 becomes
-// [32 x b1 | 32 x b2], i.e. a K-major bf16 row of 64, so no second buffer is needed.
 constexpr int kF32SwapBBytes = kF32SwapTok * kF32BK * 4;                 // 8 KB
 constexpr int kF32SwapStageBytes = kF32ABytes + kF32SwapBBytes;          // 24 KB
 constexpr int kF32SwapStages = 8;
-constexpr int kF32SwapASlots = 4;                                        // tensor-memory slots of the weight pieces
-constexpr int kF32SwapASlotCols = kF32BK;                                // 16 columns of b1 pairs + 16 of b2 pairs
-constexpr int kF32SwapASlotBase = 2 * kF32SwapTok;                       // behind the two accumulator sets
-constexpr int kF32SwapTmemCols = 256;
+constexpr int kF32SwapTmemCols = 256;               // 2 x 64 accumulator columns + 4 x 32 of A
 constexpr int kF32SwapSmemBytes = kF32SwapStages * kF32SwapStageBytes + 2048 + kTcEpiStageBytes;
-static_assert(kF32SwapSmemBytes <= 227 * 1024, "shared memory of the swapped form");
-static_assert(kF32SwapASlotBase + kF32SwapASlots * kF32SwapASlotCols <= kF32SwapTmemCols, "tensor memory of the swapped form");
-constexpr int kF32TmemCols = 512;                   // + 2 slots x (hi 32 + lo 32) columns of A, rounded up to a power of two
+static_assert(kF32SmemBytes <= 227 * 1024 && kF32SwapSmemBytes <= 227 * 1024, "shared memory per CTA");
+static_assert(2 * kF32BN + kF32ASlots * kF32ASlotCols <= kF32TmemCols, "tensor memory of the plain form");
+static_assert(2 * kF32SwapTok + kF32ASlots * kF32ASlotCols <= kF32SwapTmemCols, "tensor memory of the swapped form");
 
 // Epilogues of the fp32 path (values continue the bf16 kernels' enum)
 enum { kTcEpiReluF32 = 4, kTcEpiSwigluF32 = 5 };
@@ -78,23 +64,8 @@ struct TcF32Args {
 };
 
 namespace ptx {
-__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
-                                          uint32_t accumulate) {
-  asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-      " tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n" ::"r"(tmem_d),
-      "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// A operand from tensor memory (lanes = rows, 32-bit columns = contraction index), B from shared memory.
-__device__ __forceinline__ void umma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
-                                             uint32_t accumulate) {
-  asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-      " tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n}\n" ::"r"(tmem_d),
-      "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
+// A operand from tensor memory (lanes = rows, each 32-bit column = two consecutive bf16 of the contraction), B from
+// shared memory.
 __device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
                                              uint32_t accumulate) {
   asm volatile(
@@ -127,11 +98,6 @@ __device__ __forceinline__ void split_bf16_pair(uint32_t x0, uint32_t x1, uint32
   const __nv_bfloat162 b2 = __floats2bfloat162_rn(r0, r1);
   *p1 = u1;
   *p2 = *reinterpret_cast<const uint32_t*>(&b2);
-}
-
-// Instruction descriptor: tf32 x tf32 -> fp32, both operands K-major, M x N tile.
-__host__ __device__ constexpr uint32_t make_idesc_tf32(int M, int N) {
-  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
 // accumulator columns [c0, c0 + 32) of this thread's TMEM lane -> activation -> eight 16-byte pieces of fp32
@@ -173,25 +139,23 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   constexpr int kBBytesK = kNRows * kF32BK * 4;             // bytes of the B operand per k-block
   constexpr int kStages = kSwap ? kF32SwapStages : kF32Stages;
   constexpr int kStageBytes = kSwap ? kF32SwapStageBytes : kF32StageBytes;
-  constexpr int kLoSlots = kSwap ? kF32SwapASlots : kF32LoSlots;      // ring of converted k-blocks
-  constexpr int kLoBytes = kSwap ? 0 : kF32BBytes;                     // (the swapped form converts B in place)
+  constexpr int kSlots = kF32ASlots;                        // ring of converted k-blocks (TMEM slots of A)
   constexpr int kAccStride = kNRows;                        // TMEM columns per accumulator set
-  constexpr int kASlotBase = kSwap ? kF32SwapASlotBase : kF32TmemAcc;  // first TMEM column of the A slots
-  constexpr int kASlotCols = kSwap ? kF32SwapASlotCols : 2 * kF32BK;
+  constexpr int kASlotBase = 2 * kNRows;                    // first TMEM column of the A slots
+  constexpr int kASlotCols = kF32ASlotCols;
   constexpr uint32_t kTmemCols = kSwap ? kF32SwapTmemCols : kF32TmemCols;
-  constexpr uint32_t kIdesc = kSwap ? make_idesc_bf16(kTcBM, kNRows) : make_idesc_tf32(kTcBM, kNRows);
+  constexpr uint32_t kIdesc = make_idesc_bf16(kTcBM, kNRows);
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   unsigned char* raw = smem;                                         // [stages][A 16 KB | B 16 or 8 KB]
-  unsigned char* lo = smem + kStages * kStageBytes;                  // [slots][B]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(lo + kLoSlots * kLoBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
   uint64_t* full = bars;                          // [stages]   TMA -> converters
   uint64_t* empty = full + kStages;               // [stages]   MMA -> producer
   uint64_t* conv_done = empty + kStages;          // [slots]    converters -> MMA (128 arrivals)
-  uint64_t* lo_empty = conv_done + kLoSlots;      // [slots]    MMA -> converters
-  uint64_t* acc_full = lo_empty + kLoSlots;       // [2]
+  uint64_t* lo_empty = conv_done + kSlots;        // [slots]    MMA -> converters (the TMEM slot is free)
+  uint64_t* acc_full = lo_empty + kSlots;         // [2]
   uint64_t* acc_empty = acc_full + 2;             // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -204,7 +168,7 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   if (threadIdx.x == 0) {
     SWAPMOE_STAMP(kTr, 0);
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
-    for (int s = 0; s < kLoSlots; ++s) { ptx::mbar_init(&conv_done[s], 128); ptx::mbar_init(&lo_empty[s], 1); }
+    for (int s = 0; s < kSlots; ++s) { ptx::mbar_init(&conv_done[s], 128); ptx::mbar_init(&lo_empty[s], 1); }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 128); }
     *abort_flag = 0;
     ptx::fence_barrier_init();
@@ -313,33 +277,21 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           if (!ok) break;
           ptx::tc_fence_after();
           if (kb == kTrKb && t == (int)blockIdx.x) SWAPMOE_STAMP(kTr, 14);
-          const uint64_t dhb = make_kmajor_sw128_desc(ptx::smem_u32(raw + stage * kStageBytes + kF32ABytes));
-          if constexpr (kSwap) {
-            // B row = [b1 of the 32 elements | b2 of them]: 16 elements = 32 bytes = +2 in the address field;
-            // A slot = [8 columns b1 (k 0-15) | 8 b1 (k 16-31) | 8 b2 | 8 b2]; small terms first
-            const uint32_t a1 = tmem_base + (uint32_t)(kASlotBase + slot * kASlotCols), a2 = a1 + 16;
-            ptx::umma_bf16_ts(tmem_d, a2, dhb, kIdesc, kb > 0 ? 1u : 0u);
-            ptx::umma_bf16_ts(tmem_d, a2 + 8, dhb + 2, kIdesc, 1u);
-            ptx::umma_bf16_ts(tmem_d, a1, dhb + 4, kIdesc, 1u);
-            ptx::umma_bf16_ts(tmem_d, a1 + 8, dhb + 6, kIdesc, 1u);
-            ptx::umma_bf16_ts(tmem_d, a1, dhb, kIdesc, 1u);
-            ptx::umma_bf16_ts(tmem_d, a1 + 8, dhb + 2, kIdesc, 1u);
-          } else {
-          const uint64_t dlb = make_kmajor_sw128_desc(ptx::smem_u32(lo + slot * kLoBytes));
-          const uint32_t a_hi = tmem_base + (uint32_t)(kASlotBase + slot * kASlotCols), a_lo = a_hi + kF32BK;
-#pragma unroll
-          for (int k = 0; k < kF32BK / kF32UmmaK; ++k) {
-            // 8 fp32 along K: +32 bytes = +2 in the address field of B, +8 columns of A; small terms first
-            ptx::umma_tf32_ts(tmem_d, a_lo + 8 * k, dhb + (uint64_t)(2 * k), kIdesc, (kb > 0 || k > 0) ? 1u : 0u);
-            ptx::umma_tf32_ts(tmem_d, a_hi + 8 * k, dlb + (uint64_t)(2 * k), kIdesc, 1u);
-            ptx::umma_tf32_ts(tmem_d, a_hi + 8 * k, dhb + (uint64_t)(2 * k), kIdesc, 1u);
-          }
-          }
+          // B row = [b1 of the 32 elements | b2 of them]: 16 elements = 32 bytes = +2 in the address field;
+          // A slot = [8 columns b1 (k 0-15) | 8 b1 (k 16-31) | 8 b2 | 8 b2]; small terms first
+          const uint64_t db = make_kmajor_sw128_desc(ptx::smem_u32(raw + stage * kStageBytes + kF32ABytes));
+          const uint32_t a1 = tmem_base + (uint32_t)(kASlotBase + slot * kASlotCols), a2 = a1 + 16;
+          ptx::umma_bf16_ts(tmem_d, a2, db, kIdesc, kb > 0 ? 1u : 0u);
+          ptx::umma_bf16_ts(tmem_d, a2 + 8, db + 2, kIdesc, 1u);
+          ptx::umma_bf16_ts(tmem_d, a1, db + 4, kIdesc, 1u);
+          ptx::umma_bf16_ts(tmem_d, a1 + 8, db + 6, kIdesc, 1u);
+          ptx::umma_bf16_ts(tmem_d, a1, db, kIdesc, 1u);
+          ptx::umma_bf16_ts(tmem_d, a1 + 8, db + 2, kIdesc, 1u);
           ptx::umma_commit(&empty[stage]);       // the raw stage may be refilled
-          ptx::umma_commit(&lo_empty[slot]);     // the lo slot may be rewritten
+          ptx::umma_commit(&lo_empty[slot]);     // the TMEM slot may be rewritten
           if (kb == kTrKb && t == (int)blockIdx.x) SWAPMOE_STAMP(kTr, 15);
           if (++stage == kStages) stage = 0;
-          if (++slot == kLoSlots) { slot = 0; slot_phase ^= 1u; }
+          if (++slot == kSlots) { slot = 0; slot_phase ^= 1u; }
         }
         if (!ok) break;
         ptx::umma_commit(&acc_full[acc]);
@@ -348,8 +300,8 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       }
     }
   } else if (warp >= 8) {
-    // ---------------------------------------------------------------------- converters: hi in place, lo beside
-    // two groups of four warps: group g converts the k-blocks whose lo slot has parity g (every other one), so two
+    // ---------------------------------------------------------------------- converters
+    // two groups of four warps: group g converts the k-blocks whose slot has parity g (every other one), so two
     // conversions are in flight; both groups walk all k-blocks to keep stage and phase counters in step
     const int grp = (warp - 8) >> 2;
     const int ctid = (threadIdx.x - 8 * 32) & 127;   // 0..127 inside the group = row = TMEM lane
@@ -360,7 +312,7 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       for (int kb = 0; kb < a.k_blocks; ++kb) {
         if ((slot & 1) != grp) {
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
-          if (++slot == kLoSlots) { slot = 0; slot_phase ^= 1u; }
+          if (++slot == kSlots) { slot = 0; slot_phase ^= 1u; }
           continue;
         }
         const bool tr = ctid == 0 && kb == kTrKb && t == (int)blockIdx.x;   // kTrKb is even: group 0 converts it
@@ -372,8 +324,8 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         if (!ok) break;
         ptx::tc_fence_after();
         if (tr) SWAPMOE_STAMP(kTr, 9);
-        if constexpr (kSwap) {
-          // weights: thread = row (= TMEM lane); 32 values -> 16 packed b1 columns and 16 packed b2 columns
+        {
+          // A: thread = row (= TMEM lane); 32 values -> 16 packed b1 columns and 16 packed b2 columns
           const unsigned char* arow = raw + stage * kStageBytes + ctid * 128;
           uint32_t hm[32];
 #pragma unroll
@@ -384,60 +336,26 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
           }
           const uint32_t ta = tmem_base + ((uint32_t)((ctid >> 5) * 32) << 16) + (uint32_t)(kASlotBase + slot * kASlotCols);
           ptx::tmem_st32(ta, hm);
-          if (tr) SWAPMOE_STAMP(kTr, 10);
-          // tokens: the first kF32SwapTok threads own a row each and rewrite it in place as [b1 x 32 | b2 x 32]
-          // (logical 16-byte piece c at physical piece c ^ (row & 7), as the swizzled K-major bf16 row wants it)
-          if (ctid < kF32SwapTok) {
-            unsigned char* brow = raw + stage * kStageBytes + kF32ABytes + ctid * 128;
-            uint32_t p1[16], p2[16];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const uint4 x = *reinterpret_cast<const uint4*>(brow + ((j ^ (ctid & 7)) << 4));
-              split_bf16_pair(x.x, x.y, &p1[2 * j], &p2[2 * j]);
-              split_bf16_pair(x.z, x.w, &p1[2 * j + 1], &p2[2 * j + 1]);
-            }
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              *reinterpret_cast<uint4*>(brow + ((c ^ (ctid & 7)) << 4)) =
-                  make_uint4(p1[4 * c], p1[4 * c + 1], p1[4 * c + 2], p1[4 * c + 3]);
-              *reinterpret_cast<uint4*>(brow + (((4 + c) ^ (ctid & 7)) << 4)) =
-                  make_uint4(p2[4 * c], p2[4 * c + 1], p2[4 * c + 2], p2[4 * c + 3]);
-            }
-          }
-        } else {
-        {
-          // A: thread = row (= TMEM lane); its 32 values sit in eight 16-byte pieces, piece j at (j ^ (row & 7))
-          const unsigned char* arow = raw + stage * kStageBytes + ctid * 128;
-          uint32_t h[32], l[32];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const uint4 x = *reinterpret_cast<const uint4*>(arow + ((j ^ (ctid & 7)) << 4));
-            const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              h[4 * j + e] = xs[e] & 0xffffe000u;
-              l[4 * j + e] = __float_as_uint(__uint_as_float(xs[e]) - __uint_as_float(h[4 * j + e]));
-            }
-          }
-          const uint32_t ta = tmem_base + ((uint32_t)((ctid >> 5) * 32) << 16) + (uint32_t)(kASlotBase + slot * kASlotCols);
-          ptx::tmem_st32(ta, h);
-          ptx::tmem_st32(ta + kF32BK, l);
         }
         if (tr) SWAPMOE_STAMP(kTr, 10);
-        // B: elementwise at identical offsets (keeps the swizzled layout): hi in place, lo into the slot
-        uint4* src = reinterpret_cast<uint4*>(raw + stage * kStageBytes + kF32ABytes);
-        uint4* dst = reinterpret_cast<uint4*>(lo + slot * kLoBytes);
-#pragma unroll 4
-        for (int i = ctid; i < kBBytesK / 16; i += 128) {
-          const uint4 x = src[i];
-          uint4 h, l;
-          h.x = x.x & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(x.x) - __uint_as_float(h.x));
-          h.y = x.y & 0xffffe000u; l.y = __float_as_uint(__uint_as_float(x.y) - __uint_as_float(h.y));
-          h.z = x.z & 0xffffe000u; l.z = __float_as_uint(__uint_as_float(x.z) - __uint_as_float(h.z));
-          h.w = x.w & 0xffffe000u; l.w = __float_as_uint(__uint_as_float(x.w) - __uint_as_float(h.w));
-          src[i] = h;
-          dst[i] = l;
-        }
+        // B: the first kNRows threads own a row each and rewrite it in place as [b1 x 32 | b2 x 32] (logical
+        // 16-byte piece c at physical piece c ^ (row & 7), as the swizzled K-major bf16 row wants it)
+        if (ctid < kNRows) {
+          unsigned char* brow = raw + stage * kStageBytes + kF32ABytes + ctid * 128;
+          uint32_t p1[16], p2[16];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const uint4 x = *reinterpret_cast<const uint4*>(brow + ((j ^ (ctid & 7)) << 4));
+            split_bf16_pair(x.x, x.y, &p1[2 * j], &p2[2 * j]);
+            split_bf16_pair(x.z, x.w, &p1[2 * j + 1], &p2[2 * j + 1]);
+          }
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            *reinterpret_cast<uint4*>(brow + ((c ^ (ctid & 7)) << 4)) =
+                make_uint4(p1[4 * c], p1[4 * c + 1], p1[4 * c + 2], p1[4 * c + 3]);
+            *reinterpret_cast<uint4*>(brow + (((4 + c) ^ (ctid & 7)) << 4)) =
+                make_uint4(p2[4 * c], p2[4 * c + 1], p2[4 * c + 2], p2[4 * c + 3]);
+          }
         }
         if (tr) SWAPMOE_STAMP(kTr, 11);
         ptx::tmem_st_wait();
@@ -447,7 +365,7 @@ tc_gemm_f32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         ptx::mbar_arrive(&conv_done[slot]);
         if (tr) SWAPMOE_STAMP(kTr, 13);
         if (++stage == kStages) { stage = 0; phase ^= 1u; }
-        if (++slot == kLoSlots) { slot = 0; slot_phase ^= 1u; }
+        if (++slot == kSlots) { slot = 0; slot_phase ^= 1u; }
       }
     }
   } else if (warp >= 4) {
