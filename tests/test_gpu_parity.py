@@ -140,8 +140,8 @@ def test_error_codes():
 # ------------------------------------------------------------------ the named configurations
 @pytest.mark.parametrize("path", ["tcgen05", "mma"])
 def test_fp32_gemm_paths(monkeypatch, path):
-    """fp32 layers: split-TF32 on tcgen05 (default) and the warp-level mma form (SWAPMOE_FP32_TC=0) both
-    hold the fp32 tolerance; ReLU top-1 with a sliced GEMM-2 and SwiGLU top-2, slots above and below one
+    """fp32 layers: three products of bf16 pieces on tcgen05 (default) and the warp-level split-TF32 mma form
+    (SWAPMOE_FP32_TC=0) both hold the fp32 tolerance; ReLU top-1 with a sliced GEMM-2 and SwiGLU top-2, slots above and below one
     128-row tile."""
     from harness import Case, check_against_oracle
     if path == "mma":
