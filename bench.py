@@ -326,7 +326,31 @@ def measure_layer(cfg, steps, warmup, *, rank=0, world=1, local=0, no_graph=Fals
     stage_ms = np.array([[evs[i][s].elapsed_time(evs[i][s + 1]) for s in range(nst)] for i in range(n_ev)])
     stage_avg = stage_ms.mean(axis=0)
 
+    # ---- timed region 2b: each grouped GEMM alone, launched back to back over the replicas (so its weights come from
+    # DRAM every time), two events around the loop: the kernel's duration without the launch gaps the events add
+    gemm_alone_ms = None
+    try:
+        n_al = 25 * copies
+        alone = []
+        with torch.cuda.stream(stream):
+            for j in range(copies):                          # every replica's state is that of its own last forward
+                layers[j].forward(d_x[j], d_out[j], stream=stream)
+            for which in (1, 2):
+                for j in range(copies):
+                    layers[j].rerun_gemm(d_out[j], which, stream=stream)
+                ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                ea.record(stream)
+                for i in range(n_al):
+                    layers[i % copies].rerun_gemm(d_out[i % copies], which, stream=stream)
+                eb.record(stream)
+                alone.append((ea, eb))
+        barrier()
+        gemm_alone_ms = [a.elapsed_time(b) / n_al for a, b in alone]
+    except binding.SwapMoEError:
+        gemm_alone_ms = None                                 # paths without a GEMM launch of their own
+
     out = {"ms_total": ms_total, "rep_ms": rep_ms, "reps": reps, "launches": int(launches), "copies": copies,
+           "gemm_alone_ms": gemm_alone_ms,
            "graph": graph is not None, "touched": touched, "count": count, "hit": hit, "warm_ms_total": warm_ms,
            "stage_avg": stage_avg, "stage_ms": stage_ms, "weight_bytes": weight_bytes}
 
@@ -367,8 +391,17 @@ def measure_layer(cfg, steps, warmup, *, rank=0, world=1, local=0, no_graph=Fals
 def layer_entry(cfg, m, steps, peaks, world=1):
     """The figures of one measured configuration, as they go into the JSON line."""
     ms_step = m["ms_total"] / steps
-    g_ms = float(m["stage_avg"][3] + m["stage_avg"][4]) / 2.0          # average duration of one GEMM launch
+    # average duration of one grouped-GEMM launch: each kernel alone, back to back over the replicas; where the path
+    # has no such launch, the stage events of the whole forward (which add a launch gap per stage)
+    g_stage = float(m["stage_avg"][3] + m["stage_avg"][4]) / 2.0
+    alone = m.get("gemm_alone_ms")
+    g_ms = float(sum(alone) / 2.0) if alone else g_stage
     roof, layer = roofline_objects(cfg, m["touched"], g_ms, ms_step, peaks)
+    roof["launch_timing"] = ("each grouped GEMM launched alone, back to back over the %d replicas, events around "
+                             "%d launches" % (m["copies"], 25 * m["copies"])) if alone else "stage events of the whole forward"
+    roof["gemm_alone_us"] = [float(v * 1e3) for v in alone] if alone else None
+    roof["stage_event_avg_launch_ms"] = g_stage
+    roof["frac_by_stage_events"] = roof["frac"] * g_ms / g_stage
     from paper_2308_15030_b200 import binding
     return {
         "workload": workload_string(cfg), "dtype": "bf16" if cfg.dtype == I.BF16 else "f32",

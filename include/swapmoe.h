@@ -175,6 +175,16 @@ int32_t swapmoe_forward_from_logits(swapmoe_layer_t* layer, const void* x_dev,
 int32_t swapmoe_forward_timed(swapmoe_layer_t* layer, const void* x_dev, void* out_dev,
                               int32_t n_tokens, void* stream, void* const* events);
 
+/* Measurement aid: launches ONE of the two grouped GEMMs again (`which` = 1: GEMM-1 + activation, 2: GEMM-2) on the
+ * state the layer's last swapmoe_forward left behind (its routing, permutation, tile list, gathered rows and hidden
+ * activations), on `stream`, so that a caller can time that kernel alone, back to back, with two events around a
+ * loop.  `out_dev` must be the `out_dev` of that forward (GEMM-2 of a top-1 layer writes its rows again, with the
+ * same values).  Nothing else of the path runs: no router, no permutation, no combine kernel; importance is not
+ * touched.  Returns SWAPMOE_ERR_NOT_READY before the first forward and SWAPMOE_ERR_UNSUPPORTED where the last
+ * forward had no GEMM launch of its own to repeat (the one-launch decode kernel, the kernels for up to 64 pairs,
+ * the warp-level mma fallback).  The paper has no counterpart. */
+int32_t swapmoe_debug_rerun_gemm(swapmoe_layer_t* layer, void* out_dev, int32_t which, void* stream);
+
 /* End-to-end form with HOST buffers: copies x_host [n_tokens, d_model] to the
  * device, runs swapmoe_forward, copies the result to out_host, and returns after
  * `stream` has completed.  Pinned host memory makes the copies asynchronous

@@ -30,7 +30,7 @@ TAPS = {
 
 EXPORTS = [
     "swapmoe_create", "swapmoe_destroy", "swapmoe_set_router", "swapmoe_set_resident",
-    "swapmoe_forward", "swapmoe_forward_timed", "swapmoe_forward_from_logits", "swapmoe_forward_host",
+    "swapmoe_forward", "swapmoe_forward_timed", "swapmoe_debug_rerun_gemm", "swapmoe_forward_from_logits", "swapmoe_forward_host",
     "swapmoe_forward_host_async", "swapmoe_host_wait",
     "swapmoe_read_importance", "swapmoe_read_importance_kind", "swapmoe_topk_importance", "swapmoe_load_slot_async",
     "swapmoe_debug_copy", "swapmoe_device_status", "swapmoe_launch_count",
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.swapmoe_set_resident.argtypes = [vp, vp, vp, vp, vp, vp]
         L.swapmoe_forward.argtypes = [vp, vp, vp, i32, vp]
         L.swapmoe_forward_timed.argtypes = [vp, vp, vp, i32, vp, ctypes.POINTER(vp)]
+        L.swapmoe_debug_rerun_gemm.argtypes = [vp, vp, i32, vp]
         L.swapmoe_forward_from_logits.argtypes = [vp, vp, vp, vp, i32, vp]
         L.swapmoe_forward_host.argtypes = [vp, vp, vp, i32, vp]
         L.swapmoe_forward_host_async.argtypes = [vp, vp, vp, i32, vp]
@@ -214,6 +215,11 @@ class Layer:
         arr = (ctypes.c_void_p * (N_STAGES + 1))(*[e.cuda_event for e in events])
         _check(lib().swapmoe_forward_timed(self._h, x.data_ptr(), out.data_ptr(), T,
                                            _stream_ptr(stream), arr), "swapmoe_forward_timed")
+
+    def rerun_gemm(self, out, which: int, stream=None) -> None:
+        """Launches grouped GEMM-1 (which = 1) or GEMM-2 (2) again on the state the last forward left (timing aid)."""
+        _check(lib().swapmoe_debug_rerun_gemm(self._h, out.data_ptr(), int(which), _stream_ptr(stream)),
+               "swapmoe_debug_rerun_gemm")
 
     def forward_from_logits(self, x, logits, out, stream=None) -> None:
         T = int(x.shape[0])

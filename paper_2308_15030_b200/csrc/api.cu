@@ -70,6 +70,7 @@ struct swapmoe_layer {
   int row_group;               // row tiles per scheduling group of the grouped GEMMs (0: automatic; SWAPMOE_ROW_GROUP)
   bool h_valid, y_valid;       // whether the last forward left h / y in the workspace (debug taps)
   int32_t y_split_last;        // copies of y the last forward's GEMM-2 wrote (slices of its contraction)
+  int32_t rerun_gemm;          // 0, or the grouped GEMM swapmoe_debug_rerun_gemm is re-launching (1 / 2)
   int32_t y_copies;            // copies of y in the workspace (slices of a split contraction)
   int32_t sm_count;
   bool use_pdl;                // programmatic dependent launch between the kernels of a forward
@@ -136,7 +137,9 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
                      cudaStream_t st) {
   const swapmoe_config_t& c = L->cfg;
   const bool pdl = L->use_pdl && L->stage_events == nullptr;
+  const int rerun = L->rerun_gemm;          // 1 / 2: only that grouped GEMM, on the state the last forward left
   if (L->decode_path && T <= kDecMaxTokens && T * c.top_k <= L->decode_max_pairs && c.dtype == SWAPMOE_BF16) {
+    if (rerun) return SWAPMOE_ERR_UNSUPPORTED;   // the one-launch kernel has no GEMM launch of its own
     // a handful of tokens: routing, both expert products and the combine in one launch
     DecodeArgs da;
     da.x = static_cast<const bf16*>(x); da.Wr = static_cast<const bf16*>(L->Wr); da.ext_logits = ext_logits;
@@ -231,7 +234,9 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
     if (pf_ctas > 64) pf_ctas = 64;
   }
   mark(L, 0, st);
-  if (small_router) {
+  if (rerun) {
+    // measurement re-run: routing, permutation and tile list are those of the last forward
+  } else if (small_router) {
     if ((rs_nt == 1 ? launch_kernel(router_small_kernel<1>, dim3(n_cta + pf_ctas), dim3(kDecThreads),
                                     router_small_smem_bytes(c.d_model, 1), st, pdl, ra, L->status)
                     : launch_kernel(router_small_kernel<2>, dim3(n_cta + pf_ctas), dim3(kDecThreads),
@@ -257,7 +262,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
         cudaSuccess)
       return SWAPMOE_ERR_CUDA;
   }
-  L->launches++;
+  if (!rerun) L->launches++;
   mark(L, 1, st);   // the slot scan and importance reduction run inside the router's last CTA
 
   // enough permute CTAs to fill the GPU: every row-group of a token tile gets its own CTA
@@ -277,17 +282,21 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   mark(L, 2, st);
   const int groups = groups_planned;
   // own_scan: three extra columns of CTAs, whose first CTAs reduce the three per-expert scores
-  if (launch_kernel(permute_gather_kernel<DT>, dim3(n_cta + (own_scan ? 3 : 0), groups), dim3(kPermThreads), 0, st, pdl, pa) !=
-      cudaSuccess)
-    return SWAPMOE_ERR_CUDA;
-  L->launches++;
+  if (!rerun) {
+    if (launch_kernel(permute_gather_kernel<DT>, dim3(n_cta + (own_scan ? 3 : 0), groups), dim3(kPermThreads), 0, st, pdl,
+                      pa) != cudaSuccess)
+      return SWAPMOE_ERR_CUDA;
+    L->launches++;
+  }
   mark(L, 3, st);
   bool combined = false;
   int y_split = 1;
   if (use_tc) {
     cudaEvent_t mid = L->stage_events ? static_cast<cudaEvent_t>(L->stage_events[4]) : nullptr;
     int32_t rc;
+    L->tc.only = rerun;
     if (L->small_path && n_pairs <= 64 && c.act == SWAPMOE_ACT_RELU) {
+      if (rerun) return SWAPMOE_ERR_UNSUPPORTED;
       rc = tc_ffn_small(L->tc, L->small, c, L->xp, L->h, L->y, out, L->rows_pad_max, L->arena_in, L->arena_out,
                         L->tiles, L->n_tiles, L->row_pair, L->mgate, max_tiles, T, L->status, st, pdl,
                         &L->launches, &combined, mid);
@@ -302,13 +311,17 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
                   max_tiles, mt, T,
                   L->status, st, pdl, &L->launches, &combined, mid, L->row_group);
     }
+    L->tc.only = 0;
     if (rc != SWAPMOE_OK) return rc;
   } else if (use_tc32) {
     cudaEvent_t mid = L->stage_events ? static_cast<cudaEvent_t>(L->stage_events[4]) : nullptr;
+    L->tc32.only = rerun;
     const int32_t rc = tc_ffn_f32(L->tc32, c, L->h, L->y, (long long)L->rows_pad_max * c.d_model, L->y_copies, L->tiles,
                                   L->n_tiles, max_tiles, T, L->status, st, pdl, &L->launches, &y_split, mid, swap32);
+    L->tc32.only = 0;
     if (rc != SWAPMOE_OK) return rc;
   } else {
+    if (rerun) return SWAPMOE_ERR_UNSUPPORTED;
     MmaGemmArgs g1;
     g1.A = L->xp; g1.W = L->arena_in; g1.C = L->h; g1.tiles = L->tiles; g1.n_tiles = L->n_tiles;
     g1.slot_stride = (long long)L->nin * c.d_ff * c.d_model;
@@ -346,6 +359,7 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   ca.n_split = y_split; ca.split_stride = (long long)L->rows_pad_max * c.d_model;
   const long long work = (long long)T * (c.d_model / 8);
   mark(L, 5, st);
+  if (rerun) return check_launch();      // neither the combine kernel nor the taps' validity change
   if (!combined) {
     if (launch_kernel(combine_kernel<DT>, dim3((unsigned)((work + 255) / 256)), dim3(256), 0, st, pdl, ca) !=
         cudaSuccess)
@@ -699,6 +713,15 @@ int32_t swapmoe_forward_timed(swapmoe_layer_t* L, const void* x, void* out, int3
   L->stage_events = events;
   const int32_t rc = forward_checked(L, x, nullptr, out, T, stream);
   L->stage_events = nullptr;
+  return rc;
+}
+
+int32_t swapmoe_debug_rerun_gemm(swapmoe_layer_t* L, void* out, int32_t which, void* stream) {
+  if (!L || !out || (which != 1 && which != 2)) return SWAPMOE_ERR_INVALID_ARG;
+  if (L->last_T <= 0) return SWAPMOE_ERR_NOT_READY;
+  L->rerun_gemm = which;
+  const int32_t rc = forward_checked(L, out, nullptr, out, L->last_T, stream);   // x is not read: no router, no permute
+  L->rerun_gemm = 0;
   return rc;
 }
 

@@ -572,6 +572,7 @@ struct TcState {
   CUtensorMap map_wr;                 // router matrix [E, d], box 64 x Epad
   bool arena_bound;
   bool router_ok;                     // tensor-core router usable (bf16 layer)
+  int only;                           // 0: both grouped GEMMs; 1 / 2: launch only GEMM-1 / GEMM-2 (measurement re-runs)
 };
 
 inline bool tc_supported(const swapmoe_config_t& c) {
@@ -632,6 +633,7 @@ inline int32_t tc_init(TcState& s, const swapmoe_config_t& c, void* xp, void* h,
   s.enabled = false;
   s.arena_bound = false;
   s.router_ok = false;
+  s.only = 0;
   if (c.dtype != SWAPMOE_BF16) return SWAPMOE_OK;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SWAPMOE_ERR_CUDA;

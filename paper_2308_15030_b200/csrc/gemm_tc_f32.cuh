@@ -438,6 +438,7 @@ struct TcF32State {
   CUtensorMap map_win, map_wout;      // weights flattened to 2D; box 32 x 128 (64 for SwiGLU's W1 / W3)
   CUtensorMap map_xp_tok, map_h_tok;  // activations, box 32 x kF32SwapTok (swapped form)
   bool swap_ok;                       // the swapped form is available (ReLU layers)
+  int only;                           // 0: both grouped GEMMs; 1 / 2: launch only GEMM-1 / GEMM-2 (measurement re-runs)
 };
 
 // The driver's tensor-map encoder (nullptr when it cannot be had).
@@ -471,6 +472,7 @@ inline int32_t tc_f32_init(TcF32State& s, PFN_encodeTiled enc, const swapmoe_con
                            int rows_pad, int sm_count) {
   s.enabled = false;
   s.arena_bound = false;
+  s.only = 0;
   s.sm_count = sm_count;
   if (!enc || !tc_f32_supported(c)) return SWAPMOE_OK;
   if (!tc_encode_2d_f32(enc, &s.map_xp, xp, (uint64_t)rows_pad, (uint64_t)c.d_model, kTcBM) ||
@@ -528,14 +530,15 @@ inline int32_t tc_ffn_f32(TcF32State& s, const swapmoe_config_t& c, void* h, flo
   long long work = (long long)max_tiles * g1.n_col_tiles;
   int grid = work > s.sm_count ? s.sm_count : (int)work;
   // (swapped form: the weight map is the A operand's, the token map with kF32SwapTok-row boxes the B operand's)
-  cudaError_t e = swapped ? launch_kernel(tc_gemm_f32_kernel<kTcEpiReluF32, true>, dim3(grid), dim3(kF32Threads),
+  cudaError_t e = s.only == 2 ? cudaSuccess :
+                  swapped ? launch_kernel(tc_gemm_f32_kernel<kTcEpiReluF32, true>, dim3(grid), dim3(kF32Threads),
                                           kF32SwapSmemBytes, st, pdl, s.map_win, s.map_xp_tok, g1)
                   : swiglu ? launch_kernel(tc_gemm_f32_kernel<kTcEpiSwigluF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes,
                                            st, pdl, s.map_xp, s.map_win, g1)
                            : launch_kernel(tc_gemm_f32_kernel<kTcEpiReluF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes,
                                            st, pdl, s.map_xp, s.map_win, g1);
   if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
-  ++*launches;
+  if (s.only != 2) ++*launches;
   if (between) cudaEventRecord(between, st);
 
   // GEMM-2: few output tiles, long contraction: slice it until every SM has an item
@@ -555,6 +558,8 @@ inline int32_t tc_ffn_f32(TcF32State& s, const swapmoe_config_t& c, void* h, flo
   g2.early_b = 1;
   work = (long long)max_tiles * n_col2 * split;
   grid = work > s.sm_count ? s.sm_count : (int)work;
+  *y_split = split;
+  if (s.only == 1) return SWAPMOE_OK;
   e = swapped ? launch_kernel(tc_gemm_f32_kernel<kTcEpiF32, true>, dim3(grid), dim3(kF32Threads), kF32SwapSmemBytes, st,
                               pdl && between == nullptr, s.map_wout, s.map_h_tok, g2)
               : launch_kernel(tc_gemm_f32_kernel<kTcEpiF32>, dim3(grid), dim3(kF32Threads), kF32SmemBytes, st,

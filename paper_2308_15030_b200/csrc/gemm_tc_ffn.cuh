@@ -78,11 +78,14 @@ inline int32_t tc_ffn(TcState& s, const swapmoe_config_t& c, void* h, float* y, 
       {tc_gemm_kernel<256, kTcEpiSwigluBf16>, tc_gemm_kernel<128, kTcEpiSwigluBf16>,
        tc_gemm_kernel<64, kTcEpiSwigluBf16>}};
   static const int smem1[3] = {TcSmem<256>::kBytes, TcSmem<128>::kBytes, TcSmem<64>::kBytes};
-  if (launch_kernel(k1[swiglu ? 1 : 0][i1], dim3(grid), dim3(kTcThreads), smem1[i1], st, pdl, s.map_xp[ia], s.map_win[i1],
-                    g1) != cudaSuccess)
-    return SWAPMOE_ERR_CUDA;
-  ++*launches;
+  if (s.only != 2) {
+    if (launch_kernel(k1[swiglu ? 1 : 0][i1], dim3(grid), dim3(kTcThreads), smem1[i1], st, pdl, s.map_xp[ia], s.map_win[i1],
+                      g1) != cudaSuccess)
+      return SWAPMOE_ERR_CUDA;
+    ++*launches;
+  }
   if (between) cudaEventRecord(between, st);
+  if (s.only == 1) { *combined = scatter; return SWAPMOE_OK; }
 
   // ---- GEMM-2: y = h * W_out^T (or out = gate * y for top-1)
   const int i2 = mt == 2 ? 0 : tc_pick_bn(kBn2Options, 4, c.d_model, row_tiles_est, s.sm_count, a_box_bytes, 32);

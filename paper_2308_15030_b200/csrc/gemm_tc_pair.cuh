@@ -342,14 +342,15 @@ inline int32_t tc_ffn_pair(TcState& s, int n_pairs, const swapmoe_config_t& c, v
   long long work = (long long)max_tiles * g1.n_col_tiles;
   int grid = 2 * (work > n_pairs ? n_pairs : (int)work);
   // weight boxes of 128 rows: kBn1Options[1] for one input matrix, kBn1Options[0] / 2 for SwiGLU's two
-  cudaError_t e =
+  cudaError_t e = s.only == 2 ? cudaSuccess :
       swiglu ? launch_kernel(tc_gemm_pair_kernel<kTcEpiSwigluBf16>, dim3(grid), dim3(kTcThreads), kPairSmemBytes, st, pdl,
                              s.map_xp[0], s.map_win[0], g1)
              : launch_kernel(tc_gemm_pair_kernel<kTcEpiReluBf16>, dim3(grid), dim3(kTcThreads), kPairSmemBytes, st, pdl,
                              s.map_xp[0], s.map_win[1], g1);
   if (e != cudaSuccess) return SWAPMOE_ERR_CUDA;
-  ++*launches;
+  if (s.only != 2) ++*launches;
   if (between) cudaEventRecord(between, st);
+  if (s.only == 1) { *combined = scatter; return SWAPMOE_OK; }
 
   TcGemmArgs g2;
   g2.C = scatter ? out : static_cast<void*>(y);

@@ -587,13 +587,48 @@ def test_fp32_small_slots_swapped_operands(monkeypatch, swap):
         assert res["out_rel_err"] <= 1e-4
 
 
-@pytest.mark.parametrize("k,renorm,T", [(1, 0, 1200), (2, 1, 600)])
-def test_switch_shaped_mid_batch(k, renorm, T):
+@pytest.mark.parametrize("k,renorm,T,zipf_s", [(1, 0, 1200, 1.2), (2, 1, 600, 1.2), (1, 0, 1850, 1.4)])
+def test_switch_shaped_mid_batch(k, renorm, T, zipf_s):
     """Switch-shaped layer (d_model 768, d_ff 3072) at a batch of a few row tiles: slots above and below one row
-    tile, ragged tiles, the gate-weighted scatter epilogue (top-1) and the fp32 y epilogue (top-2)."""
+    tile, ragged tiles, the gate-weighted scatter epilogue (top-1) and the fp32 y epilogue (top-2).  The third case
+    has slots on every side of 128, 256 and 384 rows (one, two, three and four row tiles per slot)."""
     from harness import Case, check_against_oracle
-    cfg = _cfg(T=T, d=768, f=3072, E=16, K=8, k=k, renorm=renorm, zipf_s=1.2, seed=12)
+    cfg = _cfg(T=T, d=768, f=3072, E=16, K=8, k=k, renorm=renorm, zipf_s=zipf_s, seed=12)
     case = Case(cfg)
     res = check_against_oracle(case, case.run())
     cnt = res["oracle"]["count"]
     assert cnt.max() > 128 and cnt.min() < 128
+    if T == 1850:
+        assert cnt.max() > 384 and np.any((cnt > 256) & (cnt <= 384)) and np.any((cnt > 128) & (cnt <= 256))
+
+
+@pytest.mark.parametrize("dtype,T,d,f", [(I.BF16, 900, 256, 512), (I.BF16, 2600, 256, 512), (I.F32, 300, 256, 512)])
+def test_rerun_of_one_grouped_gemm_rewrites_the_same_values(dtype, T, d, f):
+    """The measurement aid that launches one grouped GEMM again (bench.py times the kernels alone with it): after
+    the hidden activations and the output were wiped, GEMM-1 then GEMM-2 (then nothing else for top-1 bf16 layers)
+    bring back exactly what the forward wrote; the one-launch decode path has no GEMM launch to repeat."""
+    import torch
+    from harness import Case, check_against_oracle
+    from paper_2308_15030_b200 import binding
+    case = Case(_cfg(T=T, dtype=dtype, d=d, f=f, E=16, K=6, zipf_s=1.1))
+    out = case.run()
+    check_against_oracle(case, out)
+    h0 = case.layer.tap("h")
+    n0 = case.layer.launch_count
+    case.layer.rerun_gemm(case.d_out, 1)
+    assert case.layer.launch_count - n0 == 1
+    assert np.array_equal(case.layer.tap("h"), h0)
+    if dtype == I.BF16:                       # top-1 bf16: GEMM-2 writes gate * y straight into `out`
+        keep = case.d_out.clone()
+        case.d_out.zero_()
+        case.layer.rerun_gemm(case.d_out, 2)
+        torch.cuda.synchronize()
+        assert torch.equal(case.d_out, keep)
+    else:
+        case.layer.rerun_gemm(case.d_out, 2)  # fp32: the slices of y are written again; the combine kernel is not run
+        assert case.layer.device_status() == (0, 0)
+    small = Case(_cfg(T=2, dtype=I.BF16, d=128, f=256, E=8, K=4))
+    small.run()
+    with pytest.raises(binding.SwapMoEError) as e:
+        small.layer.rerun_gemm(small.d_out, 1)
+    assert e.value.status == -7
