@@ -348,6 +348,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
     R->abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::prefetch_tmap(&tmWo);
+    SWAPMOE_STAMP(0, 0);
   }
   __syncthreads();
   // the router matrix is a constant of the layer: request it before waiting for the predecessor
@@ -361,6 +362,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
   if (warp == kDecWarps - 1 && lane < a.pf_depth) recent_e = __ldcg(a.recent + lane);
   pdl_wait();
   pdl_trigger();
+  if (tid == 0) SWAPMOE_STAMP(0, 1);
   // ------------------------------------------------------------------ routing, in every CTA
   // (integer divisions are kept out of this kernel's once-run paths: each costs dozens of
   // dependent instructions)
@@ -384,6 +386,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
   if (tid < K) R->phys[tid] = a.phys[tid];
   if (tid < kDecMaxTokens) R->tok[tid] = min(tid, T - 1);
   __syncthreads();
+  if (tid == 0) SWAPMOE_STAMP(0, 2);
   if (warp == kDecWarps - 1 && a.pf_depth > 0) {
     // L2 prefetch of the recently served experts that are resident: 16 KB chunks of both matrices, dealt over
     // the CTAs (chunk c of a slot goes to CTA c mod grid), so every SM issues a handful of requests
@@ -438,6 +441,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
     }
   }
   __syncthreads();
+  if (tid == 0) SWAPMOE_STAMP(0, 3);
   if (alive && warp < 2 * kDecMaxTokens && (warp & (kDecMaxTokens - 1)) < T) {
     // gate of token (warp & 7) (Section 2; Fig. 4): warps 0-7 the off-the-shelf gate, 8-15 the masked one
     const int t = warp & (kDecMaxTokens - 1), pass = warp / kDecMaxTokens;
@@ -463,6 +467,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
     }
   }
   __syncthreads();
+  if (tid == 0) SWAPMOE_STAMP(0, 4);
   // slot-sorted pair order (a stable counting sort on the flat pair index), by one warp: lane p
   // holds pair p; its position is (#pairs in lower slots) + (#earlier pairs in its own slot)
   if (warp == 0) {
@@ -493,6 +498,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
     if (lane == 0) R->n_touched = alive ? __popc(leaders) : 0;
   }
   __syncthreads();
+  if (tid == 0) SWAPMOE_STAMP(0, 5);
 
   // -------------------------------------------------------------------- expert work items
   // Waves of an item, in the order they are requested and consumed: the 32 rows of W_in in
@@ -632,6 +638,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
     const bool run_ends = !runs || it + 1 >= my_items || jb + 1 == n_jb || (jb + 1) / kDecGroup != grp;
     const int w = n_rw + v;
     if (!dec_wait_wave(bars, w, R, a.status, 22)) { alive = false; break; }
+    if (tid == 0 && v == 0) SWAPMOE_STAMP(0, 6);
     const unsigned char* st = ring + (w & 1) * kDecHalfBytes;
     if (wi < n_in * n_mats) {
       // ---- RW of the item's 32 hidden units: raw products W1 x (and W3 x), eight pairs at a time
@@ -702,11 +709,13 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
     }
     const bool flush = wi == wpi - 1 && run_ends;
     __syncthreads();                              // the buffer is free; the activations are complete / free
+    if (tid == 0 && v < 3) SWAPMOE_STAMP(0, 7 + v);
     if (warp == 0 && v + 2 < total) {
       ptx::fence_proxy_async();
       issue_item_wave();
     }
     if (!flush) continue;
+    if (tid == 0) SWAPMOE_STAMP(0, 10);
     run_jb = -1;
     // ---- first-step sum: whoever delivers the group's last set of partial rows adds them all.
     // The group's sets: one per item, or with runs one per CTA whose item range meets the group
@@ -725,6 +734,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
       R->last = last;
     }
     __syncthreads();
+    if (tid == 0) SWAPMOE_STAMP(0, 11);
     if (R->last) {
       const int d4 = d / 4;
       // thread (sub, col): sub = tid / 256 adds sets 8 sub .. 8 sub + 7 of 256 float4 columns (all eight
@@ -762,6 +772,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
       }
       __syncthreads();
       if (tid == 0) {
+        SWAPMOE_STAMP(0, 12);
         a.tickets[s * n_groups + grp] = 0u;
         __threadfence();
         const bool last = atomicAdd(&a.tickets[K * n_groups], 1u) == (unsigned)(R->n_touched * n_groups - 1);
@@ -793,10 +804,15 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
           }
         }
         if (tid == 0) a.tickets[K * n_groups] = 0u;
+#ifdef SWAPMOE_TRACE
+        __syncthreads();
+        if (tid == 0) SWAPMOE_STAMP(0, 14);
+#endif
       }
     }
     __syncthreads();     // R->last is reused by the next item
   }
+  if (tid == 0) SWAPMOE_STAMP(0, 15);
   if (!alive && tid == 0) {
     // a wait gave up: let copies that may still be in flight land before the shared memory is released
     const uint64_t t0 = ptx::globaltimer_ns();
