@@ -504,8 +504,9 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_ticket = cv.take<unsigned>(4);
   const size_t o_touched = cv.take<unsigned long long>(2);
   const size_t o_dec_stats = cv.take<unsigned long long>(2), o_dec_recent = cv.take<int32_t>(kDecRecent);
-  const size_t o_tiles = cv.take<TileDesc>(max_tiles);
-  const size_t o_tiles_b = cv.take<TileDesc>(max_tiles), o_ntiles_b = cv.take<int32_t>(4);
+  // (at least 32 entries each: the grouped GEMM's producer warp fetches the first 32 descriptors in one go)
+  const size_t o_tiles = cv.take<TileDesc>(max_tiles < 32 ? 32 : max_tiles);
+  const size_t o_tiles_b = cv.take<TileDesc>(max_tiles < 32 ? 32 : max_tiles), o_ntiles_b = cv.take<int32_t>(4);
   const size_t o_xp = cv.take<char>(rows_pad * c.d_model * L->elem);
   const size_t o_h = cv.take<char>(rows_pad * c.d_ff * L->elem);
   // up to four copies of y for a sliced contraction in the CUDA-core GEMM-2, when they stay small

@@ -400,8 +400,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (is_producer) SWAPMOE_STAMP(kTr, 1);
   pdl_wait();      // the activations come from the preceding kernel
   pdl_trigger();
+  // Which tile comes first depends on the tile count, and its descriptor is a second load behind that one: the
+  // producer's warp fetches the first 32 descriptors together with the count (one per lane; the list's allocation
+  // holds at least 32) and picks the right one by shuffle, so the two round trips overlap.
+  int4 first_raw = make_int4(0, 0, 0, 0);
+  if (warp == 0) first_raw = __ldcg(reinterpret_cast<const int4*>(a.tiles + lane));
   const int n_row_tiles = *a.n_tiles;
   const int total = n_row_tiles * a.n_col_tiles;
+  int first_rt = -1;
+  if (warp == 0 && (int)blockIdx.x < total) {
+    int rt0, ct0;
+    decode_tile((int)blockIdx.x, n_row_tiles, a.n_col_tiles, a.row_group, &rt0, &ct0);
+    first_rt = rt0;
+    const int src = rt0 & 31;
+    first_raw.x = __shfl_sync(0xffffffffu, first_raw.x, src);
+    first_raw.y = __shfl_sync(0xffffffffu, first_raw.y, src);
+    first_raw.z = __shfl_sync(0xffffffffu, first_raw.z, src);
+    first_raw.w = __shfl_sync(0xffffffffu, first_raw.w, src);
+  }
 
   if (warp == 0) {
     if (lane == 0) {
@@ -413,7 +429,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
         int rt, ct;
         decode_tile(t, n_row_tiles, a.n_col_tiles, a.row_group, &rt, &ct);
-        const TileDesc td = a.tiles[rt];
+        const TileDesc td = (t == (int)blockIdx.x && rt == first_rt && rt < 32)
+                                ? *reinterpret_cast<const TileDesc*>(&first_raw) : a.tiles[rt];
         const int brow = td.phys * a.b_rows_per_phys + ct * kBoxRows;
         const int halves = (MT == 2 && td.rows > kTcBM) ? 2 : 1;
         for (int kb = 0; kb < a.k_blocks; ++kb) {
