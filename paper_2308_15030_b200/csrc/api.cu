@@ -71,6 +71,7 @@ struct swapmoe_layer {
   bool h_valid, y_valid;       // whether the last forward left h / y in the workspace (debug taps)
   int32_t y_split_last;        // copies of y the last forward's GEMM-2 wrote (slices of its contraction)
   int32_t rerun_gemm;          // 0, or the grouped GEMM swapmoe_debug_rerun_gemm is re-launching (1 / 2)
+  int32_t permute_groups;      // 0 = automatic, else row groups (CTAs per token tile) of the permute kernel
   int32_t y_copies;            // copies of y in the workspace (slices of a split contraction)
   int32_t sm_count;
   bool use_pdl;                // programmatic dependent launch between the kernels of a forward
@@ -265,10 +266,17 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
   if (!rerun) L->launches++;
   mark(L, 1, st);   // the slot scan and importance reduction run inside the router's last CTA
 
-  // enough permute CTAs to fill the GPU: every row-group of a token tile gets its own CTA
-  int groups_planned = (2 * L->sm_count + n_cta - 1) / n_cta;
+  // Permute CTAs: every row group of a token tile gets its own CTA.  About 1.5 CTAs per SM, more when the rows are
+  // long (at most 96 KB of rows per CTA).  Not more than that: the grouped GEMM's CTAs can only be launched into the
+  // SMs the permute CTAs have left, and launching that grid takes 3-4 us once it can start (8192 tokens of
+  // d_model 768: three groups 137.7 us per forward, two groups 135.3).
+  int groups_planned = (3 * L->sm_count / 2 + n_cta - 1) / n_cta;
   {
+    const long long row_bytes = (long long)n_pairs * c.d_model * L->elem;
+    const int by_bytes = (int)((row_bytes + (long long)n_cta * (96 << 10) - 1) / ((long long)n_cta * (96 << 10)));
+    if (by_bytes > groups_planned) groups_planned = by_bytes;
     const int max_groups = (tok_tile * c.top_k + 7) / 8;
+    if (L->permute_groups > 0) groups_planned = L->permute_groups;
     if (groups_planned > max_groups) groups_planned = max_groups;
     if (groups_planned < 1) groups_planned = 1;
   }
@@ -449,6 +457,8 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   {
     const char* env = std::getenv("SWAPMOE_PDL");      // SWAPMOE_PDL=0 launches every kernel fully serialised
     L->use_pdl = !(env && env[0] == '0');
+    env = std::getenv("SWAPMOE_PERMUTE_GROUPS");        // CTAs per token tile of the permute kernel (0: automatic)
+    L->permute_groups = env ? std::atoi(env) : 0;
     env = std::getenv("SWAPMOE_ROUTER_TOK");            // force the router's token tile (32, 64 or 128)
     L->router_tok = env ? std::atoi(env) : 0;
     if (L->router_tok != 32 && L->router_tok != 64 && L->router_tok != 128) L->router_tok = 0;
