@@ -168,9 +168,12 @@ int32_t swapmoe_forward_from_logits(swapmoe_layer_t* layer, const void* x_dev,
  * SWAPMOE_N_STAGES + 1 caller-owned cudaEvent_t of `events` on `stream` at the
  * stage boundaries (event i before stage i, the last one after the final
  * stage), so a caller can time each kernel of the path with
- * cudaEventElapsedTime.  Stages: 0 router+gate, 1 scan+importance reduce,
- * 2 permute+gather, 3 grouped GEMM-1 (+activation), 4 grouped GEMM-2,
- * 5 combine. */
+ * cudaEventElapsedTime.  Stages: 0 router+gate, 1 scan+importance reduce
+ * (no launch of its own: the scan and the reductions run inside the permute
+ * kernel, so this interval is empty), 2 scan+permute+gather, 3 grouped GEMM-1
+ * (+activation), 4 grouped GEMM-2, 5 combine (empty for top-1 bf16 layers,
+ * whose GEMM-2 writes the gate-weighted rows itself).  The one-launch decode
+ * path records all of its time in stage 0. */
 #define SWAPMOE_N_STAGES 6
 int32_t swapmoe_forward_timed(swapmoe_layer_t* layer, const void* x_dev, void* out_dev,
                               int32_t n_tokens, void* stream, void* const* events);

@@ -17,7 +17,8 @@ from . import build as _build
 
 F32, BF16 = 0, 1
 N_STAGES = 6
-STAGE_NAMES = ("router_gate_scan", "(scan: fused into router)", "permute_gather", "gemm1_act", "gemm2", "combine")
+# stage 1 has had no kernel of its own since the scan moved into the permute kernel: its slot measures an empty interval
+STAGE_NAMES = ("router_gate", "(scan: no kernel of its own)", "scan_permute_gather", "gemm1_act", "gemm2", "combine")
 ACT_RELU, ACT_SWIGLU = 0, 1
 
 TAPS = {

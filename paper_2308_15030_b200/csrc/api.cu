@@ -264,7 +264,8 @@ int32_t forward_impl(swapmoe_layer* L, const void* x, const float* ext_logits, v
       return SWAPMOE_ERR_CUDA;
   }
   if (!rerun) L->launches++;
-  mark(L, 1, st);   // the slot scan and importance reduction run inside the router's last CTA
+  mark(L, 1, st);   // (stage 1, the scan, has no launch of its own: it runs in the permute kernel, or for very large
+                    // grids and swapmoe_route_static in the router's last CTA)
 
   // Permute CTAs: every row group of a token tile gets its own CTA.  About 1.5 CTAs per SM, more when the rows are
   // long (at most 96 KB of rows per CTA).  Not more than that: the grouped GEMM's CTAs can only be launched into the
