@@ -466,7 +466,10 @@ def run_cuda(args, cfg):
                    "resident_set": "top-K by Eq.(1) importance of the batch",
                    "touched_slots": ent["touched_slots"], "slot_counts": ent["slot_counts"],
                    "unmasked_hit_rate": ent["unmasked_hit_rate"], "multi_gpu": "replicas only"},
-        "gpu_launches": ent["gpu_launches"], "repeats": m["reps"], "repeat_ms_min_max": ent["repeat_ms_min_max"],
+        # kernels of this library launched by the K steps of one timed loop (4 per forward for a bf16 top-1 layer),
+        # and over all the repeats of that loop that were timed
+        "gpu_launches": ent["gpu_launches"], "gpu_launches_all_repeats": ent["gpu_launches"] * m["reps"],
+        "repeats": m["reps"], "repeat_ms_min_max": ent["repeat_ms_min_max"],
         "warm_ms_per_step": ent["warm_ms_per_step"],
         "clocks": clocks,
         "e2e": {"value": world * cfg.T * args.steps / (e2e_ms * 1e-3), "unit": UNIT,
