@@ -272,7 +272,9 @@ __device__ __noinline__ bool dec_wait_wave(uint64_t* bars, int w, DecRoute* R, i
 // dst[n * dst_stride + r] = <row r of the wave buffer, token R->tok[n]> for r < rows <= 32,
 // n < nn <= 8.  The contraction is split over the warps in steps of 16; a warp multiplies its
 // steps for both 16-row tiles, the per-warp partial products meet in `red` and are added in warp
-// order.  Rows of the buffer beyond `rows` hold stale data whose products are dropped.
+// order.  Rows of the buffer beyond `rows` hold stale data whose products are dropped; row indices beyond what
+// a wave buffer holds at this row length (fewer than 32 rows from d_model 2048 on) are clamped to its last row,
+// so that no read leaves the buffer.
 __device__ __noinline__ void dec_wave_dots(const unsigned char* st, int rows, int d, const unsigned char* xs,
                                            const DecRoute* R, int nn, float* red, float* dst, int dst_stride) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
@@ -283,16 +285,20 @@ __device__ __noinline__ void dec_wave_dots(const unsigned char* st, int rows, in
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
   const unsigned char* xrow = xs + R->tok[g] * pitch + t * 4;
-  const unsigned char* arow = st + g * pitch + t * 4;
+  const int rmax = decode_rows_per_wave(d) - 1;
+  const unsigned char* ar[2][2];               // rows 16 i + 8 h + g of the buffer
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) ar[i][h] = st + min(16 * i + 8 * h + g, rmax) * pitch + t * 4;
 #pragma unroll 2
   for (int ks = warp; ks < d / 16; ks += kDecWarps) {
     const int kb = ks * 32;                    // byte offset of the step inside a row
     const uint32_t b0 = lds32(xrow + kb), b1 = lds32(xrow + kb + 16);
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const unsigned char* ap = arow + i * 16 * pitch + kb;
-      mma_bf16_16x8x16(acc[i], lds32(ap), lds32(ap + 8 * pitch), lds32(ap + 16), lds32(ap + 8 * pitch + 16), b0, b1);
-    }
+    for (int i = 0; i < 2; ++i)
+      mma_bf16_16x8x16(acc[i], lds32(ar[i][0] + kb), lds32(ar[i][1] + kb), lds32(ar[i][0] + kb + 16),
+                       lds32(ar[i][1] + kb + 16), b0, b1);
   }
 #pragma unroll
   for (int i = 0; i < 2; ++i) {

@@ -62,7 +62,14 @@ __device__ __forceinline__ void rs_wave_dots(const unsigned char* st, int rows, 
     for (int j = 0; j < NT; ++j)
 #pragma unroll
       for (int q = 0; q < 4; ++q) acc[i][j][q] = 0.f;
-  const unsigned char* arow = st + g * pitch + t * 4;
+  // (row indices beyond what a wave buffer holds at this row length are clamped to its last row: their products
+  // are dropped, and no read leaves the buffer)
+  const int rmax = decode_rows_per_wave(d) - 1;
+  const unsigned char* ar[2][2];               // rows 16 i + 8 h + g of the buffer
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) ar[i][h] = st + min(16 * i + 8 * h + g, rmax) * pitch + t * 4;
 #pragma unroll 2
   for (int ks = warp; ks < d / 16; ks += kDecWarps) {
     const int kb = ks * 32;
@@ -75,8 +82,8 @@ __device__ __forceinline__ void rs_wave_dots(const unsigned char* st, int rows, 
     }
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
-      const unsigned char* ap = arow + i * 16 * pitch + kb;
-      const uint32_t a0 = lds32(ap), a1 = lds32(ap + 8 * pitch), a2 = lds32(ap + 16), a3 = lds32(ap + 8 * pitch + 16);
+      const uint32_t a0 = lds32(ar[i][0] + kb), a1 = lds32(ar[i][1] + kb), a2 = lds32(ar[i][0] + kb + 16),
+                     a3 = lds32(ar[i][1] + kb + 16);
 #pragma unroll
       for (int j = 0; j < NT; ++j) mma_bf16_16x8x16(acc[i][j], a0, a1, a2, a3, b0[j], b1[j]);
     }

@@ -47,9 +47,15 @@ __device__ __forceinline__ void rsf_wave_dots(const unsigned char* st, int rows,
   for (int i = 0; i < 2; ++i)
 #pragma unroll
     for (int q = 0; q < 4; ++q) acc[i][q] = 0.f;
-  const float* arow = reinterpret_cast<const float*>(st + g * pitch) + t;
+  // (row indices beyond what a wave buffer holds at this row length - 16 rows at d_model 768, 8 at 2048 - are clamped
+  // to its last row: their products are dropped, and no read leaves the buffer)
+  const int rmax = rsf_rows_per_wave(d) - 1;
+  const float* ar[2][2];                                     // rows 16 i + 8 h + g of the buffer
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) ar[i][h] = reinterpret_cast<const float*>(st + min(16 * i + 8 * h + g, rmax) * pitch) + t;
   const float* xrow = reinterpret_cast<const float*>(xs + min(g, n_tok - 1) * pitch) + t;
-  const int pw = pitch / 4;                                  // words per row
 #pragma unroll 2
   for (int ks = warp; ks < d / 8; ks += kDecWarps) {
     const int k0 = ks * 8;
@@ -58,12 +64,11 @@ __device__ __forceinline__ void rsf_wave_dots(const unsigned char* st, int rows,
     split_tf32(xrow[k0 + 4], bh[1], bl[1]);
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
-      const float* ap = arow + i * 16 * pw + k0;
       uint32_t ah[4], al[4];
-      split_tf32(ap[0], ah[0], al[0]);
-      split_tf32(ap[8 * pw], ah[1], al[1]);
-      split_tf32(ap[4], ah[2], al[2]);
-      split_tf32(ap[8 * pw + 4], ah[3], al[3]);
+      split_tf32(ar[i][0][k0], ah[0], al[0]);
+      split_tf32(ar[i][1][k0], ah[1], al[1]);
+      split_tf32(ar[i][0][k0 + 4], ah[2], al[2]);
+      split_tf32(ar[i][1][k0 + 4], ah[3], al[3]);
       mma_tf32_16x8x8(acc[i], al, bh);
       mma_tf32_16x8x8(acc[i], ah, bl);
       mma_tf32_16x8x8(acc[i], ah, bh);

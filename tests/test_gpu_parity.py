@@ -632,3 +632,21 @@ def test_rerun_of_one_grouped_gemm_rewrites_the_same_values(dtype, T, d, f):
     with pytest.raises(binding.SwapMoEError) as e:
         small.layer.rerun_gemm(small.d_out, 1)
     assert e.value.status == -7
+
+
+@pytest.mark.parametrize("dtype,T,d,f,E,K,act", [
+    (I.F32, 2, 1024, 768, 100, 53, I.ACT_SWIGLU),      # fp32 small-batch router: 16 rows of the router matrix per wave
+    (I.F32, 400, 1024, 256, 64, 21, I.ACT_RELU),
+    (I.F32, 40, 2048, 256, 24, 6, I.ACT_RELU),         # 8 rows per wave
+    (I.BF16, 2, 2048, 512, 40, 8, I.ACT_RELU),         # one-launch decode kernel: 16 rows per wave
+    (I.BF16, 40, 2048, 512, 40, 8, I.ACT_SWIGLU),      # bf16 small-batch router at the same row length
+    (I.BF16, 3, 4096, 512, 8, 4, I.ACT_SWIGLU),        # Mixtral's d_model at decode batch sizes: 8 rows per wave
+])
+def test_long_rows_in_the_wave_buffers(dtype, T, d, f, E, K, act):
+    """From d_model 2048 (bf16) or 768 (fp32) on, a 64.5 KB wave buffer of the small-batch routers and of the
+    one-launch decode kernel holds fewer than 32 matrix rows; the products walk 32 row indices and must stay
+    inside the buffer (a read beyond it left the CTA's shared memory at d_model 1024 in fp32)."""
+    from harness import Case, check_against_oracle
+    case = Case(_cfg(T=T, dtype=dtype, d=d, f=f, E=E, K=K, act=act, zipf_s=1.0, seed=41))
+    check_against_oracle(case, case.run())
+    assert case.layer.device_status() == (0, 0)
