@@ -120,24 +120,38 @@ __global__ void __launch_bounds__(kGateThreads) router_gate_kernel(const RouterA
         }
       }
     };
+    // The tensor core adds into its fp32 accumulators with truncation, so a long chain of accumulating mma drifts
+    // (d_model 4096: 1536 dependent adds, 8e-4 on logits of magnitude 25).  Every 512 contraction elements the
+    // accumulators are therefore added to the logits tile in shared memory with ordinary fp32 adds (each element
+    // has one owner thread) and cleared.
+    // accumulator layout: [0], [1] -> token m0 + g, experts 8 nt + 2 t4, + 1; [2], [3] -> token m0 + g + 8
+    auto flush = [&](bool first) {
+#pragma unroll
+      for (int j = 0; j < EI; ++j) {
+        const int nt = ng + 4 * j;
+        if (nt < NT) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int e = nt * 8 + 2 * t4 + (q & 1);
+            if (e < E) {
+              float* dst = &slog[(m0 + g + (q >> 1) * 8) * (E + 1) + e];
+              *dst = first ? acc[j][q] : *dst + acc[j][q];
+            }
+            acc[j][q] = 0.f;
+          }
+        }
+      }
+    };
     load_chunk(0, 0);
     if (kRouterDK < a.d) load_chunk(kRouterDK, 1);
+    constexpr int kFlushCols = 512;
+    bool first = true;
     for (int c0 = 0; c0 < a.d; c0 += 2 * kRouterDK) {
       stage_and_multiply(0, c0 + 2 * kRouterDK);
       if (c0 + kRouterDK < a.d) stage_and_multiply(1, c0 + 3 * kRouterDK);
+      if ((c0 + 2 * kRouterDK) % kFlushCols == 0 && c0 + 2 * kRouterDK < a.d) { flush(first); first = false; }
     }
-    // accumulator layout: [0], [1] -> token m0 + g, experts 8 nt + 2 t4, + 1; [2], [3] -> token m0 + g + 8
-#pragma unroll
-    for (int j = 0; j < EI; ++j) {
-      const int nt = ng + 4 * j;
-      if (nt < NT) {
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int e = nt * 8 + 2 * t4 + (q & 1);
-          if (e < E) slog[(m0 + g + (q >> 1) * 8) * (E + 1) + e] = acc[j][q];
-        }
-      }
-    }
+    flush(first);
   }
   // ||x||^2 of a row: 8 consecutive lanes hold its partial sums
   sumsq += __shfl_xor_sync(0xffffffffu, sumsq, 1);

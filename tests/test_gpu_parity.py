@@ -650,3 +650,14 @@ def test_long_rows_in_the_wave_buffers(dtype, T, d, f, E, K, act):
     case = Case(_cfg(T=T, dtype=dtype, d=d, f=f, E=E, K=K, act=act, zipf_s=1.0, seed=41))
     check_against_oracle(case, case.run())
     assert case.layer.device_status() == (0, 0)
+
+
+@pytest.mark.parametrize("T,E,k,K", [(64, 31, 2, 29), (511, 2, 2, 2), (1300, 100, 1, 40)])
+def test_fp32_router_long_contraction(T, E, k, K):
+    """fp32 layers of d_model 4096 route through the general fp32 router (the small-batch one does not fit its rows
+    in shared memory).  Its logits must hold 1e-5 of their largest magnitude over a 4096-term contraction: the
+    tensor core truncates when it adds into its fp32 accumulators, so the kernel moves them to ordinary fp32 sums
+    every 512 terms (a single chain of 1536 accumulating mma drifted by 8e-4 on logits of magnitude 25)."""
+    from harness import Case, check_against_oracle
+    case = Case(_cfg(T=T, dtype=I.F32, d=4096, f=128, E=E, k=k, K=K, renorm=1, zipf_s=1.0, seed=43))
+    check_against_oracle(case, case.run())
