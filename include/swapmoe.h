@@ -101,6 +101,13 @@ enum {
  * accumulator.  *out is written only on success.  Errors: INVALID_ARG
  * (null, K < top_k, K > E, sizes out of the limits above), UNSUPPORTED, CUDA,
  * NO_MEMORY (the workspace did not fit).
+ * Reproducibility: a layer object returns the same bits for the same inputs,
+ * tables and weights, call after call and whatever ran before on it (every
+ * reduction has a fixed order).  Two layer objects that differ in max_tokens
+ * may slice GEMM-2's contraction differently where it is sliced at all (fp32
+ * layers, and bf16 layers whose shapes the tcgen05 kernels do not take: the
+ * number of partial copies of y follows the workspace size) and then differ
+ * in the last bit.
  */
 int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg);
 

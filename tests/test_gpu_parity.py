@@ -573,20 +573,6 @@ def test_fp32_small_slots_swapped_operands(monkeypatch, swap):
         assert cnt.max() > 64 or cfg.T < 100
 
 
-@pytest.mark.parametrize("swap", ["1", "0"])
-def test_fp32_small_slots_swapped_operands(monkeypatch, swap):
-    """fp32 ReLU layers with small slots put the weights on the tensor core's rows and the slot's tokens on its
-    columns (64-token tiles); slots from a handful of rows to more than one tile, GEMM-2 with a sliced
-    contraction.  SWAPMOE_FP32_SWAP=0 runs the same layer on 128-token tiles."""
-    from harness import Case, check_against_oracle
-    monkeypatch.setenv("SWAPMOE_FP32_SWAP", swap)
-    for cfg in (_cfg(T=330, dtype=I.F32, d=256, f=512, E=8, K=5, zipf_s=1.3),
-                _cfg(T=90, dtype=I.F32, d=128, f=384, E=16, K=6, k=2, renorm=1, zipf_s=1.0)):
-        case = Case(cfg)
-        res = check_against_oracle(case, case.run())
-        assert res["out_rel_err"] <= 1e-4
-
-
 @pytest.mark.parametrize("k,renorm,T,zipf_s", [(1, 0, 1200, 1.2), (2, 1, 600, 1.2), (1, 0, 1850, 1.4)])
 def test_switch_shaped_mid_batch(k, renorm, T, zipf_s):
     """Switch-shaped layer (d_model 768, d_ff 3072) at a batch of a few row tiles: slots above and below one row
