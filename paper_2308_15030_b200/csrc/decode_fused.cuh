@@ -276,7 +276,8 @@ __device__ __noinline__ bool dec_wait_wave(uint64_t* bars, int w, DecRoute* R, i
 // a wave buffer holds at this row length (fewer than 32 rows from d_model 2048 on) are clamped to its last row,
 // so that no read leaves the buffer.
 __device__ __noinline__ void dec_wave_dots(const unsigned char* st, int rows, int d, const unsigned char* xs,
-                                           const DecRoute* R, int nn, float* red, float* dst, int dst_stride) {
+                                           const DecRoute* R, int nn, float* red, float* dst, int dst_stride,
+                                           int rows_held) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int pitch = d * 2 + kDecRowPad;
   float acc[2][4];
@@ -285,7 +286,7 @@ __device__ __noinline__ void dec_wave_dots(const unsigned char* st, int rows, in
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
   const unsigned char* xrow = xs + R->tok[g] * pitch + t * 4;
-  const int rmax = decode_rows_per_wave(d) - 1;
+  const int rmax = rows_held - 1;              // rows_held = decode_rows_per_wave(d): what a wave buffer holds
   const unsigned char* ar[2][2];               // rows 16 i + 8 h + g of the buffer
 #pragma unroll
   for (int i = 0; i < 2; ++i)
@@ -440,7 +441,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
   for (int w = 0; w < n_rw; ++w) {
     // router wave w holds rows w*RW .. of Wr
     if (!dec_wait_wave(bars, w, R, a.status, 21)) { alive = false; break; }
-    dec_wave_dots(ring + (w & 1) * kDecHalfBytes, min(RW, E - w * RW), d, xs, R, T, red, slog + w * RW, kMaxE + 1);
+    dec_wave_dots(ring + (w & 1) * kDecHalfBytes, min(RW, E - w * RW), d, xs, R, T, red, slog + w * RW, kMaxE + 1, RW);
     if (warp == 0 && w + 2 < n_rw) {               // dec_wave_dots ends with a block barrier: the buffer is free
       ptx::fence_proxy_async();
       issue_rows(w + 2, a.Wr + (size_t)(w + 2) * RW * d, min(RW, E - (w + 2) * RW));
@@ -654,7 +655,7 @@ decode_fused_kernel(const __grid_constant__ CUtensorMap tmWo, const DecodeArgs a
         const int nn = min(8, n_s - nb);
         if (tid < 8) R->tok[tid] = R->tok_at[q0 + nb + min(tid, nn - 1)];
         __syncthreads();
-        dec_wave_dots(st, RW, d, xs, R, nn, red, (mat == 0 ? hraw : hraw3) + nb * kDecJB + rp * RW, kDecJB);
+        dec_wave_dots(st, RW, d, xs, R, nn, red, (mat == 0 ? hraw : hraw3) + nb * kDecJB + rp * RW, kDecJB, RW);
       }
       if (wi == n_in * n_mats - 1) {
         // all 32 units of every pair are in: activation, rounded to bf16 for the second product
