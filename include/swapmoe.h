@@ -153,7 +153,7 @@ int32_t swapmoe_set_resident(swapmoe_layer_t* layer, const int32_t* slot_to_expe
  * enqueued on `stream`; the call does not synchronise and does not allocate.
  * n_tokens = 0 is a valid no-op.  Errors: NOT_READY, TOO_MANY_TOKENS,
  * INVALID_ARG, CUDA (launch failure).
- * Launches: four or five kernels; a bf16 layer given at most six (token,
+ * Launches: four or five kernels; a bf16 layer given at most five (token,
  * expert) pairs (a decode step) runs as a single kernel with the same results
  * and side effects.
  * The router matrix and the arenas must not be written by work enqueued on

@@ -526,9 +526,10 @@ int32_t swapmoe_create(swapmoe_layer_t** out, const swapmoe_config_t* cfg) {
   const size_t o_xs = cv.take<char>(T * c.d_model * L->elem);
   const size_t o_os = cv.take<char>(T * c.d_model * L->elem);
   {
-    // Measured on B200 (d_model 1024, d_ff 4096, top-1): the one-launch path costs about 21 us + 5.5 us
-    // per extra touched slot, the general kernels 42-54 us up to eight tokens: it wins up to six pairs.
-    L->decode_max_pairs = 6;
+    // Measured on B200 (d_model 1024, d_ff 4096, top-1), us per layer for 1 .. 6 tokens: the one-launch path 18.6 /
+    // 23.5 / 29.7 / 33.8 / 38.2 / 42.7, the general kernels 30.5 / 31.8 / 33.0 / 34.1 / 39.2 / 40.5: it wins up to
+    // five pairs.
+    L->decode_max_pairs = 5;
     const char* envt = std::getenv("SWAPMOE_DECODE_MAX_PAIRS");  // 1..32: use the one-launch path up to this many pairs
     if (envt && std::atoi(envt) >= 1 && std::atoi(envt) <= kDecMaxPairs) L->decode_max_pairs = std::atoi(envt);
     const char* env = std::getenv("SWAPMOE_DECODE_PATH");   // SWAPMOE_DECODE_PATH=0: general kernels for tiny batches too

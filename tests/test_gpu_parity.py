@@ -507,10 +507,10 @@ def test_decode_path_external_logits_with_ties(monkeypatch):
 
 
 def test_decode_path_default_threshold():
-    """Without overrides the single-launch path serves up to six (token, expert) pairs, the general
+    """Without overrides the single-launch path serves up to five (token, expert) pairs, the general
     kernels the rest."""
     from harness import Case, check_against_oracle
-    for T, one in ((6, True), (7, False)):
+    for T, one in ((5, True), (6, False)):
         case = Case(_cfg(T=T, d=256, f=512, E=64, K=16, zipf_s=1.1))
         n0 = case.layer.launch_count
         out = case.run()
